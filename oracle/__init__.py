@@ -1,0 +1,241 @@
+"""CPU oracle for the NVFP4 quantize + block-scaled GEMM path.
+
+TEST INFRASTRUCTURE ONLY.  The arithmetic lives in ``nvfp4_oracle.c`` (plain C,
+binary32 steps written one rounding at a time, binary64 for every reference
+quantity); this module compiles it with gcc and exposes it through ctypes on
+numpy arrays.  It shares nothing with the CUDA path and must never be imported
+by the product package.
+
+Functions follow the paper's Appendix B (Eq. 1-5), Appendix C (random Hadamard
+transform), Section 4.3 (2D weight blocks) and Section 4.4 (stochastic
+rounding); each C function cites the passage it restates.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_DIR = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_DIR, "nvfp4_oracle.c")
+_LIB = os.path.join(_DIR, "libnvfp4_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+RNE, SR = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (strict IEEE: no contraction, no fast-math)."""
+    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if force or stale:
+        tmp = f"{_LIB}.{os.getpid()}.tmp"
+        cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
+               "-fno-fast-math", "-fvisibility=hidden", "-o", tmp, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    with _lock:
+        if _lib is None:
+            L = ctypes.CDLL(build())
+            c = ctypes
+            u8p, u16p, u32p = c.POINTER(c.c_uint8), c.POINTER(c.c_uint16), c.POINTER(c.c_uint32)
+            f32p, f64p = c.POINTER(c.c_float), c.POINTER(c.c_double)
+            sig = {
+                "orc_bf16_to_f32": (c.c_float, [c.c_uint16]),
+                "orc_e2m1_decode": (c.c_float, [c.c_uint8]),
+                "orc_e4m3_decode": (c.c_float, [c.c_uint8]),
+                "orc_e4m3_encode_rne": (c.c_uint8, [c.c_float]),
+                "orc_e2m1_encode_rne": (c.c_uint8, [c.c_float]),
+                "orc_e2m1_encode_sr": (c.c_uint8, [c.c_float, c.c_uint8]),
+                "orc_philox4x32_10": (None, [u32p, u32p, u32p]),
+                "orc_sr_draw": (c.c_uint8, [c.c_uint64, c.c_uint64, c.c_uint64]),
+                "orc_hadamard16_entry": (c.c_int, [c.c_int, c.c_int]),
+                "orc_rht16": (None, [f32p, c.c_uint16, f32p]),
+                "orc_global_scale": (None, [c.c_float, f32p, f32p]),
+                "orc_block_scale_byte": (c.c_uint8, [c.c_float, c.c_float]),
+                "orc_block_encode_scale": (c.c_float, [c.c_uint8, c.c_float]),
+                "orc_sf_swizzled_offset": (c.c_int64, [c.c_int64, c.c_int64, c.c_int64]),
+                "orc_quantize": (c.c_int, [u16p, c.c_int64, c.c_int64, c.c_int64, c.c_int, c.c_int,
+                                           c.c_int, c.c_uint16, c.c_int, c.c_uint64, c.c_uint64,
+                                           c.c_float, u8p, u8p, f32p, f32p]),
+                "orc_dequantize": (None, [u8p, u8p, f32p, c.c_int64, c.c_int64, f64p]),
+                "orc_dequantize_local": (None, [u8p, u8p, c.c_int64, c.c_int64, f64p]),
+                "orc_gemm_tn": (None, [f64p, f64p, c.c_int64, c.c_int64, c.c_int64, f64p, f64p]),
+                "orc_gemm_blockscaled": (None, [u8p, u8p, f32p, u8p, u8p, f32p, c.c_int64,
+                                                c.c_int64, c.c_int64, f64p]),
+            }
+            for name, (res, args) in sig.items():
+                fn = getattr(L, name)
+                fn.restype, fn.argtypes = res, args
+            _lib = L
+    return _lib
+
+
+def _p(a, ctype):
+    return a.ctypes.data_as(ctypes.POINTER(ctype))
+
+
+# ---------------------------------------------------------------- scalars ----
+def bf16_to_f32(h: int) -> float:
+    return float(lib().orc_bf16_to_f32(h))
+
+
+def e2m1_decode(code: int) -> float:
+    return float(lib().orc_e2m1_decode(code))
+
+
+def e4m3_decode(byte: int) -> float:
+    return float(lib().orc_e4m3_decode(byte))
+
+
+def e4m3_encode_rne(t: float) -> int:
+    return int(lib().orc_e4m3_encode_rne(np.float32(t)))
+
+
+def e2m1_encode_rne(v: float) -> int:
+    return int(lib().orc_e2m1_encode_rne(np.float32(v)))
+
+
+def e2m1_encode_sr(v: float, u: int) -> int:
+    return int(lib().orc_e2m1_encode_sr(np.float32(v), u))
+
+
+def philox4x32_10(ctr, key):
+    c = np.asarray(ctr, dtype=np.uint32).copy()
+    k = np.asarray(key, dtype=np.uint32).copy()
+    out = np.zeros(4, dtype=np.uint32)
+    lib().orc_philox4x32_10(_p(c, ctypes.c_uint32), _p(k, ctypes.c_uint32), _p(out, ctypes.c_uint32))
+    return out
+
+
+def sr_draw(seed: int, sr_offset: int, e: int) -> int:
+    return int(lib().orc_sr_draw(seed, sr_offset, e))
+
+
+def hadamard16_entry(j: int, k: int) -> int:
+    return int(lib().orc_hadamard16_entry(j, k))
+
+
+def rht16(x, sign_mask: int):
+    xin = np.ascontiguousarray(x, dtype=np.float32)
+    assert xin.shape == (16,)
+    y = np.zeros(16, dtype=np.float32)
+    lib().orc_rht16(_p(xin, ctypes.c_float), sign_mask, _p(y, ctypes.c_float))
+    return y
+
+
+def global_scale(amax: float):
+    e, d = ctypes.c_float(), ctypes.c_float()
+    lib().orc_global_scale(np.float32(amax), ctypes.byref(e), ctypes.byref(d))
+    return np.float32(e.value), np.float32(d.value)
+
+
+def block_scale_byte(amax_b: float, s_enc: float) -> int:
+    return int(lib().orc_block_scale_byte(np.float32(amax_b), np.float32(s_enc)))
+
+
+def block_encode_scale(scale_byte: int, s_dec: float):
+    return np.float32(lib().orc_block_encode_scale(scale_byte, np.float32(s_dec)))
+
+
+def sf_swizzled_offset(r: int, kb: int, n_kb: int) -> int:
+    return int(lib().orc_sf_swizzled_offset(r, kb, n_kb))
+
+
+def sf_unswizzle(swizzled, rows: int, n_kb: int):
+    """Gather a swizzled scale buffer back into the linear [rows][n_kb] layout."""
+    flat = np.asarray(swizzled, dtype=np.uint8).reshape(-1)
+    r = np.arange(rows, dtype=np.int64)[:, None]
+    kb = np.arange(n_kb, dtype=np.int64)[None, :]
+    off = ((r // 128) * (n_kb // 4) + kb // 4) * 512 + (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4
+    return flat[off]
+
+
+# ---------------------------------------------------------------- tensors ----
+class Quantized:
+    """One NVFP4 copy: codes [R][C/2], scales [R][C/16] (linear), global {amax, s_dec}."""
+
+    def __init__(self, codes, scales, glob, rows, cols, y=None):
+        self.codes, self.scales, self.glob = codes, scales, glob
+        self.rows, self.cols, self.y = rows, cols, y
+
+    @property
+    def amax(self):
+        return self.glob[0]
+
+    @property
+    def s_dec(self):
+        return self.glob[1]
+
+
+def quantize(x_bf16_bits, *, colwise=False, block_rows=1, rht=False, sign_mask=0, rounding=RNE,
+             seed=0, sr_offset=0, amax_override=None, return_y=False) -> Quantized:
+    """Quantize one copy of a bf16 tensor given as a 2-D uint16 array of bit patterns."""
+    x = np.asarray(x_bf16_bits)
+    assert x.dtype == np.uint16 and x.ndim == 2
+    ld = x.strides[0] // 2
+    assert x.strides[1] == 2
+    sr, sc = x.shape
+    R, C = (sc, sr) if colwise else (sr, sc)
+    codes = np.zeros((R, C // 2), dtype=np.uint8)
+    scales = np.zeros((R, C // 16), dtype=np.uint8)
+    glob = np.zeros(2, dtype=np.float32)
+    y = np.zeros((R, C), dtype=np.float32) if return_y else None
+    rc = lib().orc_quantize(_p(x, ctypes.c_uint16), sr, sc, ld, int(colwise), block_rows, int(rht),
+                            sign_mask, rounding, seed, sr_offset,
+                            np.float32(-1.0 if amax_override is None else amax_override),
+                            _p(codes, ctypes.c_uint8), _p(scales, ctypes.c_uint8),
+                            _p(glob, ctypes.c_float),
+                            _p(y, ctypes.c_float) if return_y else None)
+    if rc != 0:
+        raise ValueError(f"orc_quantize rejected the shape (rc={rc})")
+    return Quantized(codes, scales, glob, R, C, y)
+
+
+def dequantize(q: Quantized, local_only=False):
+    out = np.zeros((q.rows, q.cols), dtype=np.float64)
+    codes = np.ascontiguousarray(q.codes)
+    scales = np.ascontiguousarray(q.scales)
+    if local_only:
+        lib().orc_dequantize_local(_p(codes, ctypes.c_uint8), _p(scales, ctypes.c_uint8), q.rows,
+                                   q.cols, _p(out, ctypes.c_double))
+    else:
+        g = np.ascontiguousarray(q.glob, dtype=np.float32)
+        lib().orc_dequantize(_p(codes, ctypes.c_uint8), _p(scales, ctypes.c_uint8),
+                             _p(g, ctypes.c_float), q.rows, q.cols, _p(out, ctypes.c_double))
+    return out
+
+
+def gemm_tn(A, B, want_T=True):
+    """D[i,j] = sum_k A[i,k] B[j,k] in binary64 (naive); T = sum |A||B|."""
+    A = np.ascontiguousarray(A, dtype=np.float64)
+    B = np.ascontiguousarray(B, dtype=np.float64)
+    M, K = A.shape
+    N, K2 = B.shape
+    assert K == K2
+    D = np.zeros((M, N), dtype=np.float64)
+    T = np.zeros((M, N), dtype=np.float64) if want_T else None
+    lib().orc_gemm_tn(_p(A, ctypes.c_double), _p(B, ctypes.c_double), M, N, K,
+                      _p(D, ctypes.c_double), _p(T, ctypes.c_double) if want_T else None)
+    return (D, T) if want_T else D
+
+
+def gemm_blockscaled(a: Quantized, b: Quantized):
+    assert a.cols == b.cols
+    D = np.zeros((a.rows, b.rows), dtype=np.float64)
+    ag = np.ascontiguousarray(a.glob, dtype=np.float32)
+    bg = np.ascontiguousarray(b.glob, dtype=np.float32)
+    ac, asf = np.ascontiguousarray(a.codes), np.ascontiguousarray(a.scales)
+    bc, bsf = np.ascontiguousarray(b.codes), np.ascontiguousarray(b.scales)
+    lib().orc_gemm_blockscaled(_p(ac, ctypes.c_uint8), _p(asf, ctypes.c_uint8), _p(ag, ctypes.c_float),
+                               _p(bc, ctypes.c_uint8), _p(bsf, ctypes.c_uint8), _p(bg, ctypes.c_float),
+                               a.rows, b.rows, a.cols, _p(D, ctypes.c_double))
+    return D
