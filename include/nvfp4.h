@@ -1,0 +1,192 @@
+/*
+ * nvfp4.h -- C ABI of the B200 (sm_100a) NVFP4 quantize + block-scaled FP4 GEMM library.
+ *
+ * The calls follow the paper's statement of the problem ("Pretraining Large Language
+ * Models with NVFP4"): a high-precision tensor is converted to E2M1 codes, one E4M3
+ * decode scale per block and one FP32 per-tensor decode scale (Appendix B, Eq. 1-4);
+ * two such tensors are multiplied with block and tensor scales into BF16/FP32
+ * (Eq. 5 and the sentence after it); a linear layer does this three times (Section 4.1,
+ * the compute-flow figure).
+ *
+ * Conventions for every call
+ *   - All data pointers are DEVICE pointers on the current CUDA device and are owned by the
+ *     caller; the library allocates no device memory and keeps no per-call state.  The
+ *     nvfp4_tensor / nvfp4_quant_opts structs themselves live in HOST memory.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the legacy
+ *     default stream).  No call synchronises with the host or copies device data back.
+ *   - Arguments are validated before anything is launched; a non-zero nvfp4_status means
+ *     nothing was enqueued (except NVFP4_ERR_CUDA, which reports a failed launch).
+ *   - Inputs must be finite; the result for NaN/Inf inputs is unspecified.
+ */
+#ifndef NVFP4_H_
+#define NVFP4_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define NVFP4_API __attribute__((visibility("default")))
+#else
+#define NVFP4_API
+#endif
+
+typedef enum nvfp4_status {
+  NVFP4_OK = 0,
+  NVFP4_ERR_NULL = 1,          /* a required pointer is NULL                                  */
+  NVFP4_ERR_SHAPE = 2,         /* a dimension is not a multiple of what the layout needs      */
+  NVFP4_ERR_ALIGN = 3,         /* a pointer or leading dimension is not sufficiently aligned  */
+  NVFP4_ERR_ARG = 4,           /* an option has an unsupported value or combination           */
+  NVFP4_ERR_WORKSPACE = 5,     /* workspace missing or smaller than the *_workspace_bytes()   */
+  NVFP4_ERR_CUDA = 6,          /* a CUDA runtime / driver call failed                         */
+  NVFP4_ERR_TIMEOUT = 7,       /* a bounded device-side wait expired (see device_status)      */
+  NVFP4_ERR_UNIMPLEMENTED = 8
+} nvfp4_status;
+
+enum { NVFP4_ROUND_NEAREST_EVEN = 0, NVFP4_ROUND_STOCHASTIC = 1 };
+enum { NVFP4_SF_LINEAR = 0, NVFP4_SF_SWIZZLED = 1 };
+enum {
+  /* the column-wise copy draws its stochastic-rounding bits from a second stream (bit 63 of
+     sr_offset set) instead of sharing the draw of the same source element with the row-wise copy */
+  NVFP4_SR_INDEPENDENT_COPIES = 1,
+  /* global[0] of each requested copy already holds the tensor amax: skip the reduction pass */
+  NVFP4_AMAX_PROVIDED = 2
+};
+
+/*
+ * One quantized copy of a tensor (Appendix B.3: "the quantized values, the local and global
+ * decode scales are stored in memory").  The copy is a row-major [rows x cols] matrix whose
+ * columns are the dot-product (contraction) dimension of the GEMM that will read it.
+ *   codes : rows * cols/2 bytes; element (r, c) is the E2M1 nibble of byte [r][c/2], even c in
+ *           the low nibble.  E2M1 = sign, 2 exponent bits, 1 mantissa bit (Section 2).
+ *   scales: rows * cols/16 bytes of E4M3 (bias 7, max 448) block decode scales, Eq. 3.
+ *           NVFP4_SF_LINEAR  : byte of (r, kb) at r * cols/16 + kb.
+ *           NVFP4_SF_SWIZZLED: the layout the block-scaled tensor-core instruction reads: 512-byte
+ *             atoms of 128 rows x 4 blocks, atoms ordered along the row's blocks first:
+ *             ((r/128) * (cols/64) + kb/4) * 512 + (r%32) * 16 + ((r%128)/32) * 4 + kb%4.
+ *             Needs rows % 128 == 0 and cols % 64 == 0.
+ *   global: float[2] = { amax of the (transformed) tensor, s_dec = 1 / (6*448/amax) }, Eq. 1.
+ */
+typedef struct nvfp4_tensor {
+  uint8_t* codes;
+  uint8_t* scales;
+  float* global;
+  int64_t rows, cols;
+  int32_t sf_layout;
+  int32_t reserved;
+} nvfp4_tensor;
+
+/*
+ * Quantization recipe (Section 4: 1x16 blocks for activations and gradients, 16x16 blocks for
+ * weights; 16x16 random Hadamard transform on weight-gradient GEMM inputs; stochastic rounding
+ * for gradients, round-to-nearest-even otherwise).
+ */
+typedef struct nvfp4_quant_opts {
+  int32_t block_rows;     /* 1: one scale per 1x16 block; 16: one scale per 16x16 block (Sec. 4.3),  */
+                          /*    replicated to the 16 1x16 blocks it covers in either copy            */
+  int32_t rounding;       /* NVFP4_ROUND_NEAREST_EVEN or NVFP4_ROUND_STOCHASTIC (Sec. 4.4)            */
+  int32_t rht_rowwise;    /* 1: rotate every aligned 16-chunk of each row of the row-wise copy by     */
+  int32_t rht_colwise;    /*    S*H_16 before scaling (Appendix C); same for the column-wise copy     */
+  uint32_t rht_sign_mask; /* low 16 bits: bit j set => the j-th input of a chunk is negated (S_d)     */
+  int32_t flags;          /* NVFP4_SR_INDEPENDENT_COPIES | NVFP4_AMAX_PROVIDED                        */
+  uint64_t seed;          /* Philox4x32-10 key                                                        */
+  uint64_t sr_offset;     /* Philox counter words 2..3; words 0..1 = (row-major source index) >> 4,   */
+                          /* and the element uses byte (index & 15) of the 16 output bytes            */
+} nvfp4_quant_opts;
+
+/*
+ * nvfp4_quantize -- Appendix B (Eq. 1-4) with the recipe options of Section 4.
+ *   x_bf16  : device, bf16 [rows x cols] row-major with leading dimension ld (elements);
+ *             32-byte aligned, ld % 16 == 0, rows % 16 == 0, cols % 16 == 0.
+ *   rowwise : (nullable) receives the copy whose blocks run along the source columns:
+ *             rowwise->rows == rows, rowwise->cols == cols.
+ *   colwise : (nullable) receives the quantized TRANSPOSE (blocks along the source rows,
+ *             Section 4.3: the backward pass contracts over the other dimension):
+ *             colwise->rows == cols, colwise->cols == rows.
+ *   At least one copy must be requested.  With block_rows == 16 both copies hold the same
+ *   quantized values (transposed) and no Hadamard transform is allowed.
+ * Two passes over x: a tensor-amax reduction (in the rotated space for a transformed copy),
+ * then transform + scale + round + pack.  Stochastic rounding rounds up iff
+ * u + 0.5 < 256 * frac, u = the 8-bit Philox draw of the source position, frac = the position of
+ * the scaled value between its two E2M1 neighbours.
+ * Errors: NULL / SHAPE / ALIGN / ARG as described at nvfp4_status; nothing is enqueued on error.
+ */
+NVFP4_API nvfp4_status nvfp4_quantize(const void* x_bf16, int64_t rows, int64_t cols, int64_t ld,
+                                      const nvfp4_quant_opts* opts, const nvfp4_tensor* rowwise,
+                                      const nvfp4_tensor* colwise, void* cuda_stream);
+
+/*
+ * nvfp4_gemm -- Eq. 5: D[i][j] = s_dec^A * s_dec^B * sum_blocks S^A[i,b] S^B[j,b] sum_{k in b} a[i,k] b[j,k]
+ *   A [M x K], B [N x K]: quantized copies whose columns are the contraction dimension, scales in
+ *   the NVFP4_SF_SWIZZLED layout, M % 128 == 0, N % 128 == 0, K % 256 == 0 (K = A->cols = B->cols).
+ *   D: device, row-major [M x N] with leading dimension ldd (elements, >= N, ldd*elemsize % 16 == 0),
+ *   bf16 (round-to-nearest-even) when d_is_fp32 == 0, else fp32.  Partial sums are accumulated in
+ *   FP32 by the tensor cores; the product of the two tensor decode scales is applied once at the end.
+ *   accumulate != 0 adds the product to the existing contents of an fp32 D (gradient accumulation,
+ *   Section 4.1); it is rejected for bf16 outputs.
+ */
+NVFP4_API nvfp4_status nvfp4_gemm(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D,
+                                  int32_t d_is_fp32, int64_t ldd, int32_t accumulate,
+                                  void* cuda_stream);
+
+/*
+ * Linear layer, Section 4.1 (three GEMMs, each quantizing its inputs):
+ *   X [M x K] bf16 (tokens x in-features), W [N x K] bf16, dY [M x N] bf16, all contiguous.
+ *   M, N, K multiples of 256.
+ *
+ * nvfp4_linear_fwd: Y = X W^T (bf16).  Quantizes X row-wise (1x16, RNE) for Fprop and, when
+ *   X_col_saved is given, column-wise with the Hadamard transform for the later Wgrad; quantizes W
+ *   with 16x16 blocks into W_row (Fprop) and W_col_saved (Dgrad) unless w_is_cached != 0, in which
+ *   case W_row must already hold the quantized weight.  opts supplies rht_sign_mask only.
+ *   workspace: device scratch of nvfp4_linear_fwd_workspace_bytes(M, K) for the row-wise copy of X.
+ * nvfp4_linear_bwd: dX = dY W (bf16), dW = dY^T X (fp32).  Quantizes dY with stochastic rounding
+ *   (opts->seed, opts->sr_offset) row-wise for Dgrad and column-wise with the Hadamard transform
+ *   for Wgrad.  dX or dW may be NULL to skip that GEMM.  accumulate_dw != 0 adds into dW.
+ *   workspace: device scratch of nvfp4_linear_bwd_workspace_bytes(M, N) for the two copies of dY.
+ */
+NVFP4_API size_t nvfp4_linear_fwd_workspace_bytes(int64_t M, int64_t K);
+NVFP4_API size_t nvfp4_linear_bwd_workspace_bytes(int64_t M, int64_t N);
+NVFP4_API nvfp4_status nvfp4_linear_fwd(const void* X, const void* W, int64_t M, int64_t N,
+                                        int64_t K, const nvfp4_quant_opts* opts, void* Y_bf16,
+                                        const nvfp4_tensor* X_col_saved, const nvfp4_tensor* W_row,
+                                        const nvfp4_tensor* W_col_saved, int32_t w_is_cached,
+                                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+NVFP4_API nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved,
+                                        const nvfp4_tensor* W_col_saved, int64_t M, int64_t N,
+                                        int64_t K, const nvfp4_quant_opts* opts, void* dX_bf16,
+                                        float* dW_fp32, int32_t accumulate_dw, void* workspace,
+                                        size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Test aids (not on the hot path).
+ * nvfp4_dequantize: out[r][c] = code * fp32(block scale) * s_dec as fp32 (the decode of Section 2).
+ * nvfp4_rht16: the transformed values y = x*(S*H_16) of the row-wise (colwise == 0, out [rows x cols])
+ *   or column-wise (colwise != 0, out [cols x rows]) copy, fp32, as the quantizer sees them.
+ */
+NVFP4_API nvfp4_status nvfp4_dequantize(const nvfp4_tensor* t, float* out, void* cuda_stream);
+NVFP4_API nvfp4_status nvfp4_rht16(const void* x_bf16, int64_t rows, int64_t cols, int64_t ld,
+                                   int32_t colwise, uint32_t sign_mask, float* out,
+                                   void* cuda_stream);
+
+/*
+ * Every device-side wait in the GEMM is bounded; when one expires the kernel records a code in a
+ * device status word and returns.  This call synchronises `cuda_stream`, reads and clears that word
+ * and returns NVFP4_ERR_TIMEOUT (with *detail = the recorded code, if detail != NULL) or NVFP4_OK.
+ */
+NVFP4_API nvfp4_status nvfp4_device_status(void* cuda_stream, uint32_t* detail);
+
+/* Tuning knob: N extent of the GEMM's CTA tile, 128 or 256 (0 = default).  Returns 0, or -1 for any
+ * other value.  Process-wide; results do not depend on it beyond FP32 summation order. */
+NVFP4_API int32_t nvfp4_set_gemm_tile_n(int32_t tile_n);
+
+NVFP4_API const char* nvfp4_status_string(nvfp4_status s);
+/* Number of kernel launches this process has enqueued through the library so far. */
+NVFP4_API uint64_t nvfp4_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NVFP4_H_ */

@@ -159,6 +159,18 @@ def sf_unswizzle(swizzled, rows: int, n_kb: int):
     return flat[off]
 
 
+def sf_swizzle(linear):
+    """Scatter a linear [rows][n_kb] scale array into the swizzled byte order (rows % 128 == 0, n_kb % 4 == 0)."""
+    lin = np.asarray(linear, dtype=np.uint8)
+    rows, n_kb = lin.shape
+    r = np.arange(rows, dtype=np.int64)[:, None]
+    kb = np.arange(n_kb, dtype=np.int64)[None, :]
+    off = ((r // 128) * (n_kb // 4) + kb // 4) * 512 + (r % 32) * 16 + ((r % 128) // 32) * 4 + kb % 4
+    out = np.zeros(rows * n_kb, dtype=np.uint8)
+    out[off.reshape(-1)] = lin.reshape(-1)
+    return out
+
+
 # ---------------------------------------------------------------- tensors ----
 class Quantized:
     """One NVFP4 copy: codes [R][C/2], scales [R][C/16] (linear), global {amax, s_dec}."""

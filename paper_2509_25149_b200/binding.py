@@ -1,0 +1,200 @@
+"""ctypes binding of the C ABI declared in ``include/nvfp4.h``.
+
+Argument marshalling only: every function here passes device pointers of torch tensors (torch is used
+for device memory and streams) straight to the C entry point of the same name.  There is no CPU or
+PyTorch fallback: if the CUDA library is missing and cannot be built, loading fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+OK = 0
+ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
+SF_LINEAR, SF_SWIZZLED = 0, 1
+SR_INDEPENDENT_COPIES, AMAX_PROVIDED = 1, 2
+
+EXPORTED = (
+    "nvfp4_quantize", "nvfp4_gemm", "nvfp4_linear_fwd_workspace_bytes", "nvfp4_linear_bwd_workspace_bytes",
+    "nvfp4_linear_fwd", "nvfp4_linear_bwd", "nvfp4_dequantize", "nvfp4_rht16", "nvfp4_device_status",
+    "nvfp4_set_gemm_tile_n", "nvfp4_status_string", "nvfp4_launch_count",
+)
+
+
+class CTensor(ctypes.Structure):
+    _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("global_", ctypes.c_void_p),
+                ("rows", ctypes.c_int64), ("cols", ctypes.c_int64), ("sf_layout", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+
+class CQuantOpts(ctypes.Structure):
+    _fields_ = [("block_rows", ctypes.c_int32), ("rounding", ctypes.c_int32), ("rht_rowwise", ctypes.c_int32),
+                ("rht_colwise", ctypes.c_int32), ("rht_sign_mask", ctypes.c_uint32), ("flags", ctypes.c_int32),
+                ("seed", ctypes.c_uint64), ("sr_offset", ctypes.c_uint64)]
+
+
+class NVFP4Error(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load (building first if the in-tree library is missing or stale) the C-ABI library."""
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        L = ctypes.CDLL(path)
+        c = ctypes
+        vp, i64, i32, u32 = c.c_void_p, c.c_int64, c.c_int32, c.c_uint32
+        TP, OP = c.POINTER(CTensor), c.POINTER(CQuantOpts)
+        L.nvfp4_quantize.restype, L.nvfp4_quantize.argtypes = i32, [vp, i64, i64, i64, OP, TP, TP, vp]
+        L.nvfp4_gemm.restype, L.nvfp4_gemm.argtypes = i32, [TP, TP, vp, i32, i64, i32, vp]
+        L.nvfp4_linear_fwd_workspace_bytes.restype = c.c_size_t
+        L.nvfp4_linear_fwd_workspace_bytes.argtypes = [i64, i64]
+        L.nvfp4_linear_bwd_workspace_bytes.restype = c.c_size_t
+        L.nvfp4_linear_bwd_workspace_bytes.argtypes = [i64, i64]
+        L.nvfp4_linear_fwd.restype = i32
+        L.nvfp4_linear_fwd.argtypes = [vp, vp, i64, i64, i64, OP, vp, TP, TP, TP, i32, vp, c.c_size_t, vp]
+        L.nvfp4_linear_bwd.restype = i32
+        L.nvfp4_linear_bwd.argtypes = [vp, TP, TP, i64, i64, i64, OP, vp, vp, i32, vp, c.c_size_t, vp]
+        L.nvfp4_dequantize.restype, L.nvfp4_dequantize.argtypes = i32, [TP, vp, vp]
+        L.nvfp4_rht16.restype, L.nvfp4_rht16.argtypes = i32, [vp, i64, i64, i64, i32, u32, vp, vp]
+        L.nvfp4_device_status.restype, L.nvfp4_device_status.argtypes = i32, [vp, c.POINTER(u32)]
+        L.nvfp4_set_gemm_tile_n.restype, L.nvfp4_set_gemm_tile_n.argtypes = i32, [i32]
+        L.nvfp4_status_string.restype, L.nvfp4_status_string.argtypes = c.c_char_p, [i32]
+        L.nvfp4_launch_count.restype, L.nvfp4_launch_count.argtypes = c.c_uint64, []
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().nvfp4_status_string(status).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise NVFP4Error(status, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+@dataclass
+class NVFP4Tensor:
+    """Device buffers of one quantized copy ([rows x cols], cols = contraction dimension)."""
+    codes: torch.Tensor   # uint8 [rows, cols/2]
+    scales: torch.Tensor  # uint8 [rows * cols/16] (linear: viewable as [rows, cols/16])
+    glob: torch.Tensor    # float32 [2] = {amax, s_dec}
+    rows: int
+    cols: int
+    sf_layout: int = SF_SWIZZLED
+
+    def c(self) -> CTensor:
+        return CTensor(self.codes.data_ptr(), self.scales.data_ptr(), self.glob.data_ptr(), self.rows, self.cols,
+                       self.sf_layout, 0)
+
+
+def alloc_tensor(rows: int, cols: int, sf_layout: int = SF_SWIZZLED, device="cuda") -> NVFP4Tensor:
+    return NVFP4Tensor(torch.empty((rows, cols // 2), dtype=torch.uint8, device=device),
+                       torch.empty((rows * cols // 16,), dtype=torch.uint8, device=device),
+                       torch.zeros((2,), dtype=torch.float32, device=device), rows, cols, sf_layout)
+
+
+def quant_opts(block_rows=1, rounding=ROUND_NEAREST_EVEN, rht_rowwise=False, rht_colwise=False, rht_sign_mask=0,
+               flags=0, seed=0, sr_offset=0) -> CQuantOpts:
+    return CQuantOpts(block_rows, rounding, int(rht_rowwise), int(rht_colwise), rht_sign_mask, flags, seed, sr_offset)
+
+
+def _ref(t: Optional[NVFP4Tensor]):
+    return ctypes.byref(t.c()) if t is not None else None
+
+
+def nvfp4_quantize(x: torch.Tensor, opts: CQuantOpts, rowwise: Optional[NVFP4Tensor] = None,
+                   colwise: Optional[NVFP4Tensor] = None) -> None:
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    _check(lib().nvfp4_quantize(x.data_ptr(), x.shape[0], x.shape[1], x.stride(0), ctypes.byref(opts), _ref(rowwise),
+                                _ref(colwise), _stream()), "nvfp4_quantize")
+
+
+def nvfp4_gemm(A: NVFP4Tensor, B: NVFP4Tensor, D: torch.Tensor, accumulate: bool = False) -> None:
+    assert D.is_cuda and D.dim() == 2 and D.stride(1) == 1 and D.dtype in (torch.bfloat16, torch.float32)
+    _check(lib().nvfp4_gemm(_ref(A), _ref(B), D.data_ptr(), int(D.dtype == torch.float32), D.stride(0),
+                            int(accumulate), _stream()), "nvfp4_gemm")
+
+
+def nvfp4_linear_fwd_workspace_bytes(M: int, K: int) -> int:
+    return int(lib().nvfp4_linear_fwd_workspace_bytes(M, K))
+
+
+def nvfp4_linear_bwd_workspace_bytes(M: int, N: int) -> int:
+    return int(lib().nvfp4_linear_bwd_workspace_bytes(M, N))
+
+
+def nvfp4_linear_fwd(X: torch.Tensor, W: Optional[torch.Tensor], opts: CQuantOpts, Y: torch.Tensor,
+                     X_col_saved: Optional[NVFP4Tensor], W_row: NVFP4Tensor, W_col_saved: Optional[NVFP4Tensor],
+                     w_is_cached: bool, workspace: torch.Tensor) -> None:
+    M, K = X.shape
+    N = W_row.rows
+    assert X.is_contiguous() and Y.is_contiguous() and Y.dtype == torch.bfloat16 and tuple(Y.shape) == (M, N)
+    assert W is None or (W.is_contiguous() and tuple(W.shape) == (N, K))
+    _check(lib().nvfp4_linear_fwd(X.data_ptr(), W.data_ptr() if W is not None else None, M, N, K, ctypes.byref(opts),
+                                  Y.data_ptr(), _ref(X_col_saved), _ref(W_row), _ref(W_col_saved), int(w_is_cached),
+                                  workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
+           "nvfp4_linear_fwd")
+
+
+def nvfp4_linear_bwd(dY: torch.Tensor, X_col_saved: Optional[NVFP4Tensor], W_col_saved: Optional[NVFP4Tensor], K: int,
+                     opts: CQuantOpts, dX: Optional[torch.Tensor], dW: Optional[torch.Tensor], accumulate_dw: bool,
+                     workspace: torch.Tensor) -> None:
+    M, N = dY.shape
+    assert dY.is_contiguous()
+    assert dX is None or (dX.is_contiguous() and dX.dtype == torch.bfloat16 and tuple(dX.shape) == (M, K))
+    assert dW is None or (dW.is_contiguous() and dW.dtype == torch.float32 and tuple(dW.shape) == (N, K))
+    _check(lib().nvfp4_linear_bwd(dY.data_ptr(), _ref(X_col_saved), _ref(W_col_saved), M, N, K, ctypes.byref(opts),
+                                  dX.data_ptr() if dX is not None else None,
+                                  dW.data_ptr() if dW is not None else None, int(accumulate_dw),
+                                  workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
+           "nvfp4_linear_bwd")
+
+
+def nvfp4_dequantize(t: NVFP4Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    if out is None:
+        out = torch.empty((t.rows, t.cols), dtype=torch.float32, device=t.codes.device)
+    _check(lib().nvfp4_dequantize(_ref(t), out.data_ptr(), _stream()), "nvfp4_dequantize")
+    return out
+
+
+def nvfp4_rht16(x: torch.Tensor, colwise: bool, sign_mask: int) -> torch.Tensor:
+    R, C = (x.shape[1], x.shape[0]) if colwise else tuple(x.shape)
+    out = torch.empty((R, C), dtype=torch.float32, device=x.device)
+    _check(lib().nvfp4_rht16(x.data_ptr(), x.shape[0], x.shape[1], x.stride(0), int(colwise), sign_mask,
+                             out.data_ptr(), _stream()), "nvfp4_rht16")
+    return out
+
+
+def nvfp4_device_status() -> int:
+    """Synchronises the current stream; raises if a bounded device-side wait expired."""
+    detail = ctypes.c_uint32(0)
+    st = lib().nvfp4_device_status(_stream(), ctypes.byref(detail))
+    if st != OK:
+        raise NVFP4Error(st, f"nvfp4_device_status (code 0x{detail.value:x})")
+    return 0
+
+
+def nvfp4_set_gemm_tile_n(tile_n: int) -> None:
+    if lib().nvfp4_set_gemm_tile_n(tile_n) != 0:
+        raise ValueError("tile_n must be 0, 128 or 256")
+
+
+def nvfp4_launch_count() -> int:
+    return int(lib().nvfp4_launch_count())

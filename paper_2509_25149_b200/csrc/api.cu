@@ -1,0 +1,252 @@
+// C-ABI entry points: argument validation and the stream-ordered composition of the kernels.
+#include <atomic>
+
+#include "common.cuh"
+#include "gemm.h"
+#include "quantize.h"
+
+namespace nvfp4 {
+static std::atomic<uint64_t> g_launches{0};
+static std::atomic<int> g_tile_n{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+}  // namespace nvfp4
+
+using namespace nvfp4;
+
+namespace {
+
+inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+nvfp4_status check_copy(const nvfp4_tensor* t, int64_t rows, int64_t cols) {
+  if (!t->codes || !t->scales || !t->global) return NVFP4_ERR_NULL;
+  if (t->rows != rows || t->cols != cols) return NVFP4_ERR_SHAPE;
+  if (t->sf_layout != NVFP4_SF_LINEAR && t->sf_layout != NVFP4_SF_SWIZZLED) return NVFP4_ERR_ARG;
+  if (t->sf_layout == NVFP4_SF_SWIZZLED && (rows % 128 != 0 || cols % 64 != 0)) return NVFP4_ERR_SHAPE;
+  if (!aligned(t->codes, 16) || !aligned(t->scales, 16) || !aligned(t->global, 8)) return NVFP4_ERR_ALIGN;
+  return NVFP4_OK;
+}
+
+nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld, const nvfp4_quant_opts* o,
+                           const nvfp4_tensor* rowwise, const nvfp4_tensor* colwise, cudaStream_t s) {
+  if (!x || !o) return NVFP4_ERR_NULL;
+  if (!rowwise && !colwise) return NVFP4_ERR_NULL;
+  if (rows <= 0 || cols <= 0 || rows % 16 != 0 || cols % 16 != 0) return NVFP4_ERR_SHAPE;
+  if (ld < cols) return NVFP4_ERR_SHAPE;
+  if (ld % 16 != 0 || !aligned(x, 32)) return NVFP4_ERR_ALIGN;
+  if (o->block_rows != 1 && o->block_rows != 16) return NVFP4_ERR_ARG;
+  if (o->rounding != NVFP4_ROUND_NEAREST_EVEN && o->rounding != NVFP4_ROUND_STOCHASTIC) return NVFP4_ERR_ARG;
+  if ((o->rht_rowwise | o->rht_colwise) & ~1) return NVFP4_ERR_ARG;
+  if (o->block_rows == 16 && (o->rht_rowwise || o->rht_colwise)) return NVFP4_ERR_ARG;
+  if (o->flags & ~(NVFP4_SR_INDEPENDENT_COPIES | NVFP4_AMAX_PROVIDED)) return NVFP4_ERR_ARG;
+  if (rows > (int64_t)1 << 30 || cols > (int64_t)1 << 30 || ((rows + 127) / 128) * ((cols + 127) / 128) > 0x7fffffff)
+    return NVFP4_ERR_SHAPE;
+  nvfp4_status st;
+  if (rowwise && (st = check_copy(rowwise, rows, cols)) != NVFP4_OK) return st;
+  if (colwise && (st = check_copy(colwise, cols, rows)) != NVFP4_OK) return st;
+
+  QuantArgs a{};
+  a.x = static_cast<const uint16_t*>(x);
+  a.rows = rows; a.cols = cols; a.ld = ld;
+  if (rowwise) {
+    a.r_codes = rowwise->codes; a.r_scales = rowwise->scales; a.r_global = rowwise->global;
+    a.r_swz = rowwise->sf_layout == NVFP4_SF_SWIZZLED;
+  }
+  if (colwise) {
+    a.c_codes = colwise->codes; a.c_scales = colwise->scales; a.c_global = colwise->global;
+    a.c_swz = colwise->sf_layout == NVFP4_SF_SWIZZLED;
+  }
+  a.sign_mask = o->rht_sign_mask & 0xffffu;
+  a.seed_lo = (uint32_t)o->seed; a.seed_hi = (uint32_t)(o->seed >> 32);
+  a.off_lo = (uint32_t)o->sr_offset; a.off_hi = (uint32_t)(o->sr_offset >> 32);
+  a.off_hi_col = (o->flags & NVFP4_SR_INDEPENDENT_COPIES) ? (a.off_hi | 0x80000000u) : a.off_hi;
+  a.tiles_r = (int)((rows + 127) / 128);
+  a.tiles_c = (int)((cols + 127) / 128);
+
+  const bool hr = rowwise != nullptr, hc = colwise != nullptr;
+  const bool b2 = o->block_rows == 16, sr = o->rounding == NVFP4_ROUND_STOCHASTIC;
+  if (!(o->flags & NVFP4_AMAX_PROVIDED)) {
+    if (launch_amax(a, hr, hc, o->rht_rowwise != 0, o->rht_colwise != 0, s) != cudaSuccess) return NVFP4_ERR_CUDA;
+  }
+  if (launch_quantize(a, hr, hc, b2, o->rht_rowwise != 0, o->rht_colwise != 0, sr, s) != cudaSuccess)
+    return NVFP4_ERR_CUDA;
+  return NVFP4_OK;
+}
+
+nvfp4_status gemm_impl(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D, int32_t d_is_fp32, int64_t ldd,
+                       int32_t accumulate, cudaStream_t s) {
+  if (!A || !B || !D) return NVFP4_ERR_NULL;
+  if (!A->codes || !A->scales || !A->global || !B->codes || !B->scales || !B->global) return NVFP4_ERR_NULL;
+  if (A->cols != B->cols) return NVFP4_ERR_SHAPE;
+  const int64_t M = A->rows, N = B->rows, K = A->cols;
+  if (M <= 0 || N <= 0 || K <= 0 || M % 128 != 0 || N % 128 != 0 || K % 256 != 0) return NVFP4_ERR_SHAPE;
+  if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff || (M / 128) * (N / 128) > 0x7fffffff) return NVFP4_ERR_SHAPE;
+  if (A->sf_layout != NVFP4_SF_SWIZZLED || B->sf_layout != NVFP4_SF_SWIZZLED) return NVFP4_ERR_ARG;
+  if (accumulate && !d_is_fp32) return NVFP4_ERR_ARG;
+  if (ldd < N) return NVFP4_ERR_SHAPE;
+  const int64_t esz = d_is_fp32 ? 4 : 2;
+  if ((ldd * esz) % 16 != 0 || !aligned(D, 16)) return NVFP4_ERR_ALIGN;
+  if (!aligned(A->codes, 16) || !aligned(B->codes, 16) || !aligned(A->scales, 16) || !aligned(B->scales, 16))
+    return NVFP4_ERR_ALIGN;
+  GemmArgs g{};
+  g.sfa = A->scales; g.sfb = B->scales;
+  g.a_global = A->global; g.b_global = B->global;
+  g.d = D; g.ldd = ldd;
+  g.M = (int)M; g.N = (int)N; g.K = (int)K;
+  g.d_is_fp32 = d_is_fp32 != 0; g.accumulate = accumulate != 0;
+  int tile_n = g_tile_n.load(std::memory_order_relaxed);
+  if (tile_n != 128 && tile_n != 256) tile_n = 256;
+  if (launch_gemm(g, A->codes, B->codes, tile_n, s) != cudaSuccess) return NVFP4_ERR_CUDA;
+  return NVFP4_OK;
+}
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline size_t copy_bytes(int64_t rows, int64_t cols) {
+  return align_up((size_t)(rows * cols / 2), 256) + align_up((size_t)(rows * cols / 16), 256) + 256;
+}
+// carve one swizzled-scale copy [rows x cols] out of a workspace
+nvfp4_tensor carve(uint8_t*& p, int64_t rows, int64_t cols) {
+  nvfp4_tensor t{};
+  t.codes = p;
+  p += align_up((size_t)(rows * cols / 2), 256);
+  t.scales = p;
+  p += align_up((size_t)(rows * cols / 16), 256);
+  t.global = reinterpret_cast<float*>(p);
+  p += 256;
+  t.rows = rows; t.cols = cols; t.sf_layout = NVFP4_SF_SWIZZLED;
+  return t;
+}
+
+}  // namespace
+
+extern "C" {
+
+nvfp4_status nvfp4_quantize(const void* x_bf16, int64_t rows, int64_t cols, int64_t ld, const nvfp4_quant_opts* opts,
+                            const nvfp4_tensor* rowwise, const nvfp4_tensor* colwise, void* cuda_stream) {
+  return quantize_impl(x_bf16, rows, cols, ld, opts, rowwise, colwise, static_cast<cudaStream_t>(cuda_stream));
+}
+
+nvfp4_status nvfp4_gemm(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D, int32_t d_is_fp32, int64_t ldd,
+                        int32_t accumulate, void* cuda_stream) {
+  return gemm_impl(A, B, D, d_is_fp32, ldd, accumulate, static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t nvfp4_linear_fwd_workspace_bytes(int64_t M, int64_t K) { return copy_bytes(M, K); }
+size_t nvfp4_linear_bwd_workspace_bytes(int64_t M, int64_t N) { return 2 * copy_bytes(M, N); }
+
+nvfp4_status nvfp4_linear_fwd(const void* X, const void* W, int64_t M, int64_t N, int64_t K,
+                              const nvfp4_quant_opts* opts, void* Y_bf16, const nvfp4_tensor* X_col_saved,
+                              const nvfp4_tensor* W_row, const nvfp4_tensor* W_col_saved, int32_t w_is_cached,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (!X || !opts || !Y_bf16 || !W_row) return NVFP4_ERR_NULL;
+  if (!w_is_cached && !W) return NVFP4_ERR_NULL;
+  if (M <= 0 || N <= 0 || K <= 0 || M % 256 || N % 256 || K % 256) return NVFP4_ERR_SHAPE;
+  if (!workspace || workspace_bytes < nvfp4_linear_fwd_workspace_bytes(M, K)) return NVFP4_ERR_WORKSPACE;
+  if (!aligned(workspace, 256)) return NVFP4_ERR_ALIGN;
+  nvfp4_status st;
+  if ((st = check_copy(W_row, N, K)) != NVFP4_OK) return st;
+  if (W_col_saved && (st = check_copy(W_col_saved, K, N)) != NVFP4_OK) return st;
+  if (X_col_saved && (st = check_copy(X_col_saved, K, M)) != NVFP4_OK) return st;
+  if (W_row->sf_layout != NVFP4_SF_SWIZZLED) return NVFP4_ERR_ARG;
+
+  if (!w_is_cached) {
+    nvfp4_quant_opts wo{};
+    wo.block_rows = 16;
+    wo.rounding = NVFP4_ROUND_NEAREST_EVEN;
+    if ((st = quantize_impl(W, N, K, K, &wo, W_row, W_col_saved, s)) != NVFP4_OK) return st;
+  }
+  uint8_t* p = static_cast<uint8_t*>(workspace);
+  nvfp4_tensor x_row = carve(p, M, K);
+  nvfp4_quant_opts xo{};
+  xo.block_rows = 1;
+  xo.rounding = NVFP4_ROUND_NEAREST_EVEN;
+  xo.rht_colwise = 1;
+  xo.rht_sign_mask = opts->rht_sign_mask;
+  if ((st = quantize_impl(X, M, K, K, &xo, &x_row, X_col_saved, s)) != NVFP4_OK) return st;
+  return gemm_impl(&x_row, W_row, Y_bf16, 0, N, 0, s);
+}
+
+nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, const nvfp4_tensor* W_col_saved,
+                              int64_t M, int64_t N, int64_t K, const nvfp4_quant_opts* opts, void* dX_bf16,
+                              float* dW_fp32, int32_t accumulate_dw, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream) {
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (!dY || !opts) return NVFP4_ERR_NULL;
+  if (!dX_bf16 && !dW_fp32) return NVFP4_ERR_NULL;
+  if (dX_bf16 && !W_col_saved) return NVFP4_ERR_NULL;
+  if (dW_fp32 && !X_col_saved) return NVFP4_ERR_NULL;
+  if (M <= 0 || N <= 0 || K <= 0 || M % 256 || N % 256 || K % 256) return NVFP4_ERR_SHAPE;
+  if (!workspace || workspace_bytes < nvfp4_linear_bwd_workspace_bytes(M, N)) return NVFP4_ERR_WORKSPACE;
+  if (!aligned(workspace, 256)) return NVFP4_ERR_ALIGN;
+  nvfp4_status st;
+  if (W_col_saved && (st = check_copy(W_col_saved, K, N)) != NVFP4_OK) return st;
+  if (X_col_saved && (st = check_copy(X_col_saved, K, M)) != NVFP4_OK) return st;
+
+  uint8_t* p = static_cast<uint8_t*>(workspace);
+  nvfp4_tensor g_row = carve(p, M, N);
+  nvfp4_tensor g_col = carve(p, N, M);
+  nvfp4_quant_opts go{};
+  go.block_rows = 1;
+  go.rounding = NVFP4_ROUND_STOCHASTIC;
+  go.rht_colwise = 1;
+  go.rht_sign_mask = opts->rht_sign_mask;
+  go.seed = opts->seed;
+  go.sr_offset = opts->sr_offset;
+  go.flags = opts->flags & NVFP4_SR_INDEPENDENT_COPIES;
+  if ((st = quantize_impl(dY, M, N, N, &go, dX_bf16 ? &g_row : nullptr, dW_fp32 ? &g_col : nullptr, s)) != NVFP4_OK)
+    return st;
+  if (dX_bf16 && (st = gemm_impl(&g_row, W_col_saved, dX_bf16, 0, K, 0, s)) != NVFP4_OK) return st;
+  if (dW_fp32 && (st = gemm_impl(&g_col, X_col_saved, dW_fp32, 1, K, accumulate_dw, s)) != NVFP4_OK) return st;
+  return NVFP4_OK;
+}
+
+nvfp4_status nvfp4_dequantize(const nvfp4_tensor* t, float* out, void* cuda_stream) {
+  if (!t || !out || !t->codes || !t->scales || !t->global) return NVFP4_ERR_NULL;
+  nvfp4_status st = check_copy(t, t->rows, t->cols);
+  if (st != NVFP4_OK) return st;
+  if (t->rows <= 0 || t->cols <= 0 || t->cols % 16) return NVFP4_ERR_SHAPE;
+  return launch_dequantize(*t, out, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_rht16(const void* x_bf16, int64_t rows, int64_t cols, int64_t ld, int32_t colwise,
+                         uint32_t sign_mask, float* out, void* cuda_stream) {
+  if (!x_bf16 || !out) return NVFP4_ERR_NULL;
+  if (rows <= 0 || cols <= 0 || ld < cols) return NVFP4_ERR_SHAPE;
+  if ((colwise ? rows : cols) % 16 != 0) return NVFP4_ERR_SHAPE;
+  return launch_rht16(x_bf16, rows, cols, ld, colwise != 0, sign_mask & 0xffffu, out,
+                      static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? NVFP4_OK
+             : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_device_status(void* cuda_stream, uint32_t* detail) {
+  uint32_t code = 0;
+  if (read_device_status(static_cast<cudaStream_t>(cuda_stream), &code) != cudaSuccess) return NVFP4_ERR_CUDA;
+  if (detail) *detail = code;
+  return code ? NVFP4_ERR_TIMEOUT : NVFP4_OK;
+}
+
+int32_t nvfp4_set_gemm_tile_n(int32_t tile_n) {
+  if (tile_n != 0 && tile_n != 128 && tile_n != 256) return -1;
+  g_tile_n.store(tile_n, std::memory_order_relaxed);
+  return 0;
+}
+
+const char* nvfp4_status_string(nvfp4_status s) {
+  switch (s) {
+    case NVFP4_OK: return "ok";
+    case NVFP4_ERR_NULL: return "a required pointer is NULL";
+    case NVFP4_ERR_SHAPE: return "unsupported shape";
+    case NVFP4_ERR_ALIGN: return "insufficient alignment";
+    case NVFP4_ERR_ARG: return "unsupported option";
+    case NVFP4_ERR_WORKSPACE: return "workspace missing or too small";
+    case NVFP4_ERR_CUDA: return "CUDA call failed";
+    case NVFP4_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case NVFP4_ERR_UNIMPLEMENTED: return "not implemented";
+  }
+  return "unknown status";
+}
+
+uint64_t nvfp4_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,117 @@
+// Shared device helpers for the NVFP4 kernels (sm_100a only).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "nvfp4.h"
+
+#if defined(__CUDA_ARCH__) && !defined(__CUDA_ARCH_FEAT_SM100_ALL)
+#error "build with -gencode arch=compute_100a,code=sm_100a"
+#endif
+
+namespace nvfp4 {
+
+// Host-side launch counter (reported by nvfp4_launch_count()).
+void count_launch(int n = 1);
+
+// ---------------------------------------------------------------------------------------------
+// Formats
+// ---------------------------------------------------------------------------------------------
+constexpr float kFltMax = 3.402823466e+38f;
+
+// bf16 pair packed in 32 bits -> two fp32 (exact).
+__device__ __forceinline__ float bf16_lo(uint32_t p) { return __uint_as_float(p << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t p) { return __uint_as_float(p & 0xffff0000u); }
+
+// Eq. 1: s_enc = 6*448/amax (clamped), s_dec = 1/s_enc, IEEE division.
+__device__ __forceinline__ void global_scales(float amax, float& s_enc, float& s_dec) {
+  float e = (amax == 0.0f) ? 1.0f : fminf(__fdiv_rn(2688.0f, amax), kFltMax);
+  s_enc = e;
+  s_dec = __frcp_rn(e);
+}
+
+// Eq. 2-3 and the text after Eq. 3: stored E4M3 byte of a block and the encode scale derived from it.
+__device__ __forceinline__ void block_scales(float amax_b, float s_enc, float s_dec, uint32_t& byte,
+                                             float& s_enc_b) {
+  float t = __fmul_rn(__fdiv_rn(amax_b, 6.0f), s_enc);
+  uint16_t packed;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %1;" : "=h"(packed) : "f"(t));
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(packed));
+  float sf = __half2float(__ushort_as_half((unsigned short)(h2 & 0xffffu)));
+  byte = packed & 0xffu;
+  float d = __fmul_rn(sf, s_dec);
+  s_enc_b = (byte == 0u) ? 0.0f : fminf(__frcp_rn(d), kFltMax);
+}
+
+// Four (lo, hi) pairs -> 8 E2M1 nibbles, element 0 in the lowest nibble (round-to-nearest-even,
+// saturating at +-6).  cvt...e2m1x2 puts its FIRST source in the high nibble.
+__device__ __forceinline__ uint32_t e2m1x8_rne(const float v[8]) {
+  uint32_t r;
+  asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n\t"
+      "mov.b32 %0, {b0, b1, b2, b3};\n\t}"
+      : "=r"(r)
+      : "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]));
+  return r;
+}
+
+// Stochastic rounding of one scaled value to an E2M1 nibble (Section 4.4): neighbours lo <= |v| < hi on
+// the grid {0,.5,1,1.5,2,3,4,6}; round up iff u + 0.5 < 256 * frac.  All steps are exact in fp32.
+__device__ __forceinline__ uint32_t e2m1_sr(float v, uint32_t u) {
+  uint32_t sign = (__float_as_uint(v) >> 28) & 8u;
+  float a = fminf(fabsf(v), 6.0f);
+  float scale = (a < 2.0f) ? 2.0f : ((a < 4.0f) ? 1.0f : 0.5f);
+  uint32_t off = (a < 2.0f) ? 0u : ((a < 4.0f) ? 2u : 4u);
+  float p = a * scale;               // position in units of the local step
+  float fl = floorf(p);
+  float frac = p - fl;
+  uint32_t up = ((float)u + 0.5f < 256.0f * frac) ? 1u : 0u;
+  return sign | ((uint32_t)fl + off + up);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10: counter (g.lo, g.hi, off.lo, off.hi), key (seed.lo, seed.hi) -> 16 random bytes
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+// ---------------------------------------------------------------------------------------------
+// 16-point Walsh-Hadamard butterfly (Sylvester order) on registers; the caller applies the 1/4.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void fwht16(float v[16]) {
+#pragma unroll
+  for (int h = 1; h < 16; h <<= 1) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      if ((i & h) == 0) {
+        float a = v[i], b = v[i | h];
+        v[i] = a + b;
+        v[i | h] = a - b;
+      }
+    }
+  }
+}
+
+// Offset of scale byte (row r, block kb) in the swizzled 128x4 atom layout; n_kb = blocks per row.
+__host__ __device__ __forceinline__ int64_t sf_swizzled_offset(int64_t r, int64_t kb, int64_t n_kb) {
+  return ((r >> 7) * (n_kb >> 2) + (kb >> 2)) * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4 + (kb & 3);
+}
+
+}  // namespace nvfp4

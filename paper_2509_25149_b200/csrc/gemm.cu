@@ -1,0 +1,439 @@
+// Block-scaled NVFP4 GEMM for sm_100a: D[M x N] = alpha * A[M x K] * B[N x K]^T  (Eq. 5 of the paper:
+// per 16-element block partial dot products times the two E4M3 block scales, accumulated in FP32;
+// alpha = s_dec^A * s_dec^B applied once on the result).
+//
+// Persistent, warp-specialised kernel, one CTA per SM:
+//   warp 0   producer: TMA loads of the code tiles (128-byte swizzle) and bulk copies of the scale atoms
+//   warp 1   MMA issuer: tcgen05.cp of the scale atoms into tensor memory, tcgen05.mma
+//            kind::mxf4nvf4.block_scale.scale_vec::4X (M 128, N = BN, K 64 per instruction)
+//   warps 2-5 epilogue: tcgen05.ld of the FP32 accumulator, alpha, conversion, global stores
+// Every wait is bounded: when one expires the kernel records a code in a device status word, every role
+// leaves its loop, tensor memory is released and the kernel returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+#include "gemm.h"
+
+namespace nvfp4 {
+
+__device__ unsigned int g_device_status = 0;  // 0 = fine; else the code of the first wait that expired
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK_BYTES = 128;           // bytes of codes per row per stage = 256 elements of K
+constexpr int BK = 256;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+
+template <int BN>
+struct Cfg {
+  static constexpr int kStages = (BN == 256) ? 4 : 6;
+  static constexpr int kAccStages = (BN == 256) ? 1 : 2;
+  static constexpr int kABytes = BM * BK_BYTES;             // 16 KB
+  static constexpr int kBBytes = BN * BK_BYTES;             // 16 / 32 KB
+  static constexpr int kSfaBytes = 4 * 512;                 // 4 K64-steps x one 128-row atom
+  static constexpr int kSfbBytes = (BN / 128) * 4 * 512;
+  static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  // tensor memory columns
+  static constexpr int kAccCol = 0;
+  static constexpr int kSfCol = kAccStages * BN;            // two buffers of (SFA 16 + SFB 4*BN/32) columns
+  static constexpr int kSfaCols = 16;
+  static constexpr int kSfbCols = 4 * (BN / 32);
+  static constexpr int kSfBufCols = kSfaCols + kSfbCols;
+  static_assert(kSfCol + 2 * kSfBufCols <= 512, "tensor memory budget");
+};
+
+// ------------------------------------------------------------------------------------- PTX ----
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait.  Returns false when the wait expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t code) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (true) {
+    if (mbar_try(bar, parity)) return true;
+    if ((++spins & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = code;
+        atomicCAS(&g_device_status, 0u, code);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,"
+      "%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (sm_100 format: version field = 1).
+//   operands: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart
+//   scale atoms: K-major, no swizzle, 8-row groups of 16-byte rows 128 bytes apart
+__device__ __forceinline__ uint64_t desc_operand(uint32_t saddr) {
+  uint64_t lo = ((saddr >> 4) & 0x3fffu) | (1u << 16);
+  uint64_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+  return lo | (hi << 32);
+}
+__device__ __forceinline__ uint64_t desc_sf(uint32_t saddr) {
+  uint64_t lo = ((saddr >> 4) & 0x3fffu);
+  uint64_t hi = (128u >> 4) | (1u << 14);
+  return lo | (hi << 32);
+}
+
+template <int BN>
+__device__ __forceinline__ constexpr uint32_t instr_desc() {
+  // E2M1 x E2M1 (format id 1 in the mxf4 kinds), K-major both, UE4M3 scales, dense K64
+  return (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (0u << 23) | ((uint32_t)(BM >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------ kernel ----
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+    gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                const GemmArgs g) {
+  using C = Cfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  // barriers live after the stages
+  const uint32_t bar_base = base + C::kStages * C::kStageBytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (C::kStages + s); };
+  auto accf_bar = [&](int s) { return bar_base + 8u * (2 * C::kStages + s); };
+  auto acce_bar = [&](int s) { return bar_base + 8u * (2 * C::kStages + C::kAccStages + s); };
+  volatile uint32_t* tmem_slot =
+      reinterpret_cast<volatile uint32_t*>(base_ptr + C::kStages * C::kStageBytes + 8 * (2 * C::kStages + 2 * C::kAccStages));
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_m = g.M / BM, tiles_n = g.N / BN;
+  const int n_tiles = tiles_m * tiles_n;
+  const int k_blocks = g.K / BK;
+  const int64_t sf_atoms_per_row_group = g.K / 64;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int s = 0; s < C::kAccStages; ++s) {
+      mbar_init(accf_bar(s), 1);
+      mbar_init(acce_bar(s), 4);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer ----
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int m_blk = tile % tiles_m, n_blk = tile / tiles_m;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x100u + stage))) break;
+          const uint32_t st = base + stage * C::kStageBytes;
+          mbar_expect_tx(full_bar(stage), C::kABytes + C::kBBytes + C::kSfaBytes + C::kSfbBytes);
+          tma_load_2d(st, &map_a, kb * BK_BYTES, m_blk * BM, full_bar(stage));
+          tma_load_2d(st + C::kABytes, &map_b, kb * BK_BYTES, n_blk * BN, full_bar(stage));
+          bulk_load(st + C::kABytes + C::kBBytes,
+                    g.sfa + ((int64_t)m_blk * sf_atoms_per_row_group + (int64_t)kb * 4) * 512, C::kSfaBytes,
+                    full_bar(stage));
+#pragma unroll
+          for (int grp = 0; grp < BN / 128; ++grp)
+            bulk_load(st + C::kABytes + C::kBBytes + C::kSfaBytes + grp * 2048,
+                      g.sfb + ((int64_t)(n_blk * (BN / 128) + grp) * sf_atoms_per_row_group + (int64_t)kb * 4) * 512,
+                      2048, full_bar(stage));
+          if (++stage == C::kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer ----
+    if (lane == 0) {
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0, sfbuf = 0;
+      bool ok = true;
+      constexpr uint32_t idesc = instr_desc<BN>();
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        if (!(ok = mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, 0x300u + acc))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem + C::kAccCol + acc * BN;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, 0x200u + stage))) break;
+          tc_fence_after();
+          const uint32_t st = base + stage * C::kStageBytes;
+          const uint32_t sf_t = tmem + C::kSfCol + sfbuf * C::kSfBufCols;
+          // scale atoms -> tensor memory: SFA of K64-step j in columns [4j, 4j+4); SFB of step j in
+          // columns [16 + j*BN/32, ...), 4 columns per 128 rows of B
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            tc_cp_sf(sf_t + j * 4, desc_sf(st + C::kABytes + C::kBBytes + j * 512));
+#pragma unroll
+            for (int grp = 0; grp < BN / 128; ++grp)
+              tc_cp_sf(sf_t + C::kSfaCols + j * (BN / 32) + grp * 4,
+                       desc_sf(st + C::kABytes + C::kBBytes + C::kSfaBytes + grp * 2048 + j * 512));
+          }
+          const uint64_t adesc = desc_operand(st);
+          const uint64_t bdesc = desc_operand(st + C::kABytes);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            // advancing 64 elements of K = 32 bytes inside the 128-byte swizzle span: +2 in the address field
+            tc_mma_nvf4(d_tmem, adesc + 2u * j, bdesc + 2u * j, idesc, sf_t + j * 4,
+                        sf_t + C::kSfaCols + j * (BN / 32), (kb > 0 || j > 0) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));  // frees the stage once the MMAs above have read it
+          sfbuf ^= 1u;
+          if (++stage == C::kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        if (!ok) break;
+        tc_commit(accf_bar(acc));  // accumulator complete
+        if (++acc == C::kAccStages) {
+          acc = 0;
+          acc_phase ^= 1u;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue ----
+    const int quad = warp & 3;  // the 32 tensor-memory lanes this warp may read
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    const float alpha = __fmul_rn(g.a_global[1], g.b_global[1]);
+    for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      const int m_blk = tile % tiles_m, n_blk = tile / tiles_m;
+      ok = mbar_wait(accf_bar(acc), acc_phase, abort_flag, 0x400u + acc);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      tc_fence_after();
+      const int64_t row = (int64_t)m_blk * BM + quad * 32 + lane;
+      const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + C::kAccCol + acc * BN;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tc_ld32(t_row + c * 32, r);
+        tc_wait_ld();
+        const int64_t col = (int64_t)n_blk * BN + c * 32;
+        if (g.d_is_fp32) {
+          float* dst = reinterpret_cast<float*>(g.d) + row * g.ldd + col;
+#pragma unroll
+          for (int v = 0; v < 8; ++v) {
+            float4 o = make_float4(__uint_as_float(r[4 * v]) * alpha, __uint_as_float(r[4 * v + 1]) * alpha,
+                                   __uint_as_float(r[4 * v + 2]) * alpha, __uint_as_float(r[4 * v + 3]) * alpha);
+            if (g.accumulate) {
+              float4 old = *reinterpret_cast<const float4*>(dst + 4 * v);
+              o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+            }
+            *reinterpret_cast<float4*>(dst + 4 * v) = o;
+          }
+        } else {
+          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(g.d) + row * g.ldd + col;
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint32_t p[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * v + 2 * e]) * alpha,
+                                                       __uint_as_float(r[8 * v + 2 * e + 1]) * alpha);
+              p[e] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            *reinterpret_cast<uint4*>(dst + 8 * v) = make_uint4(p[0], p[1], p[2], p[3]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acce_bar(acc));
+      if (++acc == C::kAccStages) {
+        acc = 0;
+        acc_phase ^= 1u;
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown ----
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // give copies that may still be in flight time to land before the shared memory is handed back
+    for (int i = 0; i < 100; ++i) __nanosleep(1000);
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------- host side ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// codes [rows][k_bytes] uint8, box = 128 bytes x box_rows, 128-byte swizzle
+bool make_code_map(CUtensorMap* map, const void* codes, int64_t rows, int64_t k_bytes, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)k_bytes, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)k_bytes};
+  cuuint32_t box[2] = {(cuuint32_t)BK_BYTES, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(codes), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN>
+cudaError_t launch_t(const GemmArgs& g, const void* a_codes, const void* b_codes, int num_sms, cudaStream_t s) {
+  using C = Cfg<BN>;
+  CUtensorMap map_a, map_b;
+  if (!make_code_map(&map_a, a_codes, g.M, g.K / 2, BM) || !make_code_map(&map_b, b_codes, g.N, g.K / 2, BN))
+    return cudaErrorInvalidValue;
+  auto kern = gemm_kernel<BN>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int n_tiles = (g.M / BM) * (g.N / BN);
+  const int grid = n_tiles < num_sms ? n_tiles : num_sms;
+  kern<<<grid, kThreads, C::kSmemBytes, s>>>(map_a, map_b, g);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_codes, int tile_n, cudaStream_t s) {
+  static int num_sms = 0;
+  if (!num_sms) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+  }
+  if (tile_n == 256 && g.N % 256 == 0) return launch_t<256>(g, a_codes, b_codes, num_sms, s);
+  return launch_t<128>(g, a_codes, b_codes, num_sms, s);
+}
+
+cudaError_t read_device_status(cudaStream_t s, uint32_t* code) {
+  cudaError_t e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return e;
+  unsigned int v = 0;
+  e = cudaMemcpyFromSymbol(&v, g_device_status, sizeof(v));
+  if (e != cudaSuccess) return e;
+  if (v) {
+    unsigned int zero = 0;
+    e = cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero));
+  }
+  *code = v;
+  return e;
+}
+
+}  // namespace nvfp4

@@ -1,0 +1,23 @@
+// Internal launch interface of the block-scaled GEMM kernel.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace nvfp4 {
+
+struct GemmArgs {
+  const uint8_t* sfa;     // swizzled scale atoms of A [M x K/16]
+  const uint8_t* sfb;     // swizzled scale atoms of B [N x K/16]
+  const float* a_global;  // {amax, s_dec}
+  const float* b_global;
+  void* d;                // [M x N], bf16 or fp32
+  int64_t ldd;
+  int M, N, K;
+  int d_is_fp32, accumulate;
+};
+
+// tile_n: 128 or 256 (256 needs N % 256 == 0, otherwise 128 is used)
+cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_codes, int tile_n, cudaStream_t s);
+cudaError_t read_device_status(cudaStream_t s, uint32_t* code);
+
+}  // namespace nvfp4

@@ -1,0 +1,605 @@
+// NVFP4 quantizer for sm_100a: tensor-amax reduction (pass 1) and the fused
+// transform + scale + round + pack kernel producing the row-wise and/or the transposed copy (pass 2).
+//
+// Paper: Appendix B (Eq. 1-4), Appendix C (16x16 random Hadamard transform), Section 4.3 (16x16
+// weight blocks, two copies for the two passes), Section 4.4 (stochastic rounding).
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+#include "quantize.h"
+
+namespace nvfp4 {
+
+// ---------------------------------------------------------------------------------------------
+// small PTX helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void ldg256_stream(const void* p, uint32_t (&r)[8]) {
+  asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+                 "=r"(r[7])
+               : "l"(p));
+}
+__device__ __forceinline__ uint4 ldg128_stream(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
+}
+
+__device__ __forceinline__ uint32_t absmax_bf16x2(uint32_t acc, uint32_t v) {
+  __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&acc);
+  uint32_t m = v & 0x7fff7fffu;
+  __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162*>(&m);
+  __nv_bfloat162 r = __hmax2(a, b);
+  return *reinterpret_cast<uint32_t*>(&r);
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// sign word for a bf16 pair whose two elements are inputs j0 and j1 of a Hadamard chunk
+__device__ __forceinline__ uint32_t sign_pair(uint32_t mask, int j0, int j1) {
+  return (((mask >> j0) & 1u) << 15) | (((mask >> j1) & 1u) << 31);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Pass 1: tensor amax (Appendix B.1), plain and / or in the rotated space of a transformed copy.
+// CTA tile 128 rows x 256 columns; a warp owns 16 rows, a lane 8 columns of each of them.
+// ---------------------------------------------------------------------------------------------
+template <bool PLAIN, bool ROT_ROW, bool ROT_COL>
+__global__ void __launch_bounds__(256) amax_kernel(const uint16_t* __restrict__ x, int64_t rows,
+                                                   int64_t cols, int64_t ld, uint32_t sign_mask,
+                                                   int tiles_c, float* __restrict__ out_plain0,
+                                                   float* __restrict__ out_plain1,
+                                                   float* __restrict__ out_rot_row,
+                                                   float* __restrict__ out_rot_col) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t tr = blockIdx.x / tiles_c, tc = blockIdx.x % tiles_c;
+  const int64_t r0 = tr * 128 + warp * 16;
+  const int64_t c0 = tc * 256 + lane * 8;
+  const bool in_range = (r0 < rows) && (c0 < cols);  // rows % 16 == 0, cols % 8 == 0
+
+  uint4 raw[16];
+  if (in_range) {
+    const uint16_t* p = x + r0 * ld + c0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) raw[j] = ldg128_stream(p + j * ld);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) raw[j] = make_uint4(0, 0, 0, 0);
+  }
+
+  float m_plain = 0.f, m_row = 0.f, m_col = 0.f;
+  if (PLAIN) {
+    uint32_t acc = 0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      acc = absmax_bf16x2(acc, raw[j].x);
+      acc = absmax_bf16x2(acc, raw[j].y);
+      acc = absmax_bf16x2(acc, raw[j].z);
+      acc = absmax_bf16x2(acc, raw[j].w);
+    }
+    m_plain = fmaxf(bf16_lo(acc), bf16_hi(acc));
+  }
+  if (ROT_COL) {
+    // chunks run down the 16 rows of the warp's slab: one transform per column
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      float a[16], b[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        uint32_t word = (w == 0) ? raw[j].x : (w == 1) ? raw[j].y : (w == 2) ? raw[j].z : raw[j].w;
+        word ^= sign_pair(sign_mask, j, j);
+        a[j] = bf16_lo(word);
+        b[j] = bf16_hi(word);
+      }
+      fwht16(a);
+      fwht16(b);
+#pragma unroll
+      for (int j = 0; j < 16; ++j) m_col = fmaxf(m_col, fmaxf(fabsf(a[j]), fabsf(b[j])));
+    }
+    m_col *= 0.25f;
+  }
+  if (ROT_ROW) {
+    // a chunk is 16 consecutive columns = the 8 columns of an even lane and of the next odd lane
+    const int half = lane & 1;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      float v[8];
+      const uint32_t w4[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        uint32_t word = w4[k] ^ sign_pair(sign_mask, half * 8 + 2 * k, half * 8 + 2 * k + 1);
+        v[2 * k] = bf16_lo(word);
+        v[2 * k + 1] = bf16_hi(word);
+      }
+#pragma unroll
+      for (int h = 1; h < 8; h <<= 1)
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if ((i & h) == 0) {
+            float a = v[i], b = v[i | h];
+            v[i] = a + b;
+            v[i | h] = a - b;
+          }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        float other = __shfl_xor_sync(0xffffffffu, v[i], 1);
+        float y = half ? (other - v[i]) : (v[i] + other);
+        m_row = fmaxf(m_row, fabsf(y));
+      }
+    }
+    m_row *= 0.25f;
+  }
+
+  __shared__ float red[3][8];
+  m_plain = warp_max(m_plain);
+  m_row = warp_max(m_row);
+  m_col = warp_max(m_col);
+  if (lane == 0) {
+    red[0][warp] = m_plain;
+    red[1][warp] = m_row;
+    red[2][warp] = m_col;
+  }
+  __syncthreads();
+  if (threadIdx.x < 3) {
+    float m = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) m = fmaxf(m, red[threadIdx.x][w]);
+    // non-negative floats order like their bit patterns
+    uint32_t bits = __float_as_uint(m);
+    if (threadIdx.x == 0 && PLAIN) {
+      if (out_plain0) atomicMax(reinterpret_cast<unsigned int*>(out_plain0), bits);
+      if (out_plain1) atomicMax(reinterpret_cast<unsigned int*>(out_plain1), bits);
+    }
+    if (threadIdx.x == 1 && ROT_ROW) atomicMax(reinterpret_cast<unsigned int*>(out_rot_row), bits);
+    if (threadIdx.x == 2 && ROT_COL) atomicMax(reinterpret_cast<unsigned int*>(out_rot_col), bits);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Pass 2: one CTA per 128 x 128 tile of the source.
+//   phase 1  each thread owns four 1x16 chunks (32-byte loads), produces the row-wise copy from
+//            registers and stages the raw tile (and the random bytes) in shared memory;
+//   phase 2  each thread owns 16 rows x 2 columns of the staged tile and produces the transposed copy
+//            into a swizzled staging buffer;
+//   phase 3  staged codes and scale bytes leave with 16-byte stores.
+// Tiles are visited in reverse order so that the end of the tensor, which pass 1 touched last, is read
+// first while it may still sit in L2.
+// ---------------------------------------------------------------------------------------------
+struct QuantSmem {
+  static constexpr int kTile = 0;                    // 128 rows x 256 B of bf16
+  static constexpr int kColCodes = 32768;            // 128 columns x 64 B
+  static constexpr int kSfRow = kColCodes + 8192;    // 1 KB
+  static constexpr int kSfCol = kSfRow + 1024;       // 1 KB
+  static constexpr int kBlkEnc = kSfCol + 1024;      // 64 floats (16x16 mode)
+  static constexpr int kBlkByte = kBlkEnc + 256;     // 64 bytes
+  static constexpr int kRand = kBlkByte + 64;        // 128 rows x 128 B (stochastic rounding only)
+  static constexpr int kBytesNoRand = kRand;
+  static constexpr int kBytesRand = kRand + 16384;
+};
+
+template <bool SR>
+__device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, const uint32_t (&rnd)[4]) {
+  uint2 out;
+  if (!SR) {
+    float v[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(f[i], s_enc_b);
+    const float(&lo)[8] = *reinterpret_cast<const float(*)[8]>(&v[0]);
+    const float(&hi)[8] = *reinterpret_cast<const float(*)[8]>(&v[8]);
+    out.x = e2m1x8_rne(lo);
+    out.y = e2m1x8_rne(hi);
+  } else {
+    uint32_t w0 = 0, w1 = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t u = (rnd[i >> 2] >> (8 * (i & 3))) & 0xffu;
+      w0 |= e2m1_sr(__fmul_rn(f[i], s_enc_b), u) << (4 * i);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      uint32_t u = (rnd[2 + (i >> 2)] >> (8 * (i & 3))) & 0xffu;
+      w1 |= e2m1_sr(__fmul_rn(f[8 + i], s_enc_b), u) << (4 * i);
+    }
+    out.x = w0;
+    out.y = w1;
+  }
+  return out;
+}
+
+__device__ __forceinline__ float amax16(const float (&f)[16]) {
+  float m = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(f[i]));
+  return m;
+}
+
+template <bool HAS_ROW, bool HAS_COL, bool BLOCK2D, bool RHT_ROW, bool RHT_COL, bool SR>
+__global__ void __launch_bounds__(256) quantize_kernel(const QuantArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = (int)(gridDim.x - 1 - blockIdx.x);
+  const int64_t row0 = (int64_t)(tile / a.tiles_c) * 128;
+  const int64_t col0 = (int64_t)(tile % a.tiles_c) * 128;
+  const int64_t n_cb = a.cols >> 4;  // 16-blocks per source row
+  const int64_t n_rb = a.rows >> 4;  // 16-blocks per source column
+
+  float r_senc = 1.f, r_sdec = 1.f, c_senc = 1.f, c_sdec = 1.f;
+  if (HAS_ROW || BLOCK2D) global_scales(HAS_ROW ? a.r_global[0] : a.c_global[0], r_senc, r_sdec);
+  if (HAS_COL) {
+    if (BLOCK2D && HAS_ROW) {
+      c_senc = r_senc;
+      c_sdec = r_sdec;
+    } else {
+      global_scales(a.c_global[0], c_senc, c_sdec);
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    if (HAS_ROW) a.r_global[1] = r_sdec;
+    if (HAS_COL) a.c_global[1] = c_sdec;
+  }
+
+  // ------------------------------------------------------------------ phase 1 ----
+  const int cb = lane & 7;  // chunk column inside the tile
+  uint32_t raw[4][8];
+  bool ok[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = warp * 16 + i * 4 + (lane >> 3);
+    ok[i] = (row0 + r < a.rows) && (col0 + cb * 16 < a.cols);
+    if (ok[i]) {
+      ldg256_stream(a.x + (row0 + r) * a.ld + col0 + cb * 16, raw[i]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) raw[i][k] = 0u;
+    }
+  }
+
+  if (HAS_COL) {
+    // stage the raw tile; halves are written in lane-dependent order so that a quarter warp covers
+    // all 32 banks
+    const int first = (lane >> 2) & 1;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int r = warp * 16 + i * 4 + (lane >> 3);
+      uint8_t* dst = smem + QuantSmem::kTile + r * 256 + cb * 32;
+      uint4 h0 = make_uint4(raw[i][0], raw[i][1], raw[i][2], raw[i][3]);
+      uint4 h1 = make_uint4(raw[i][4], raw[i][5], raw[i][6], raw[i][7]);
+      if (first) {
+        *reinterpret_cast<uint4*>(dst + 16) = h1;
+        *reinterpret_cast<uint4*>(dst) = h0;
+      } else {
+        *reinterpret_cast<uint4*>(dst) = h0;
+        *reinterpret_cast<uint4*>(dst + 16) = h1;
+      }
+    }
+  }
+
+  float blk_amax = 0.f;  // 16x16 mode: running amax of the lane's chunk column over the warp's 16 rows
+  if (BLOCK2D) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t acc = 0;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) acc = absmax_bf16x2(acc, raw[i][k]);
+      blk_amax = fmaxf(blk_amax, fmaxf(bf16_lo(acc), bf16_hi(acc)));
+    }
+    blk_amax = fmaxf(blk_amax, __shfl_xor_sync(0xffffffffu, blk_amax, 8));
+    blk_amax = fmaxf(blk_amax, __shfl_xor_sync(0xffffffffu, blk_amax, 16));
+  }
+  uint32_t blk_byte = 0;
+  float blk_enc = 0.f;
+  if (BLOCK2D) {
+    block_scales(blk_amax, r_senc, r_sdec, blk_byte, blk_enc);
+    if (lane < 8) {
+      reinterpret_cast<float*>(smem + QuantSmem::kBlkEnc)[warp * 8 + cb] = blk_enc;
+      smem[QuantSmem::kBlkByte + warp * 8 + cb] = (uint8_t)blk_byte;
+    }
+  }
+
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = warp * 16 + i * 4 + (lane >> 3);
+    uint32_t rnd[4] = {0u, 0u, 0u, 0u};
+    if (SR) {
+      const uint64_t g = (uint64_t)(row0 + r) * (uint64_t)n_cb + (uint64_t)((col0 >> 4) + cb);
+      uint4 q = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), a.off_lo, a.off_hi, a.seed_lo, a.seed_hi);
+      rnd[0] = q.x; rnd[1] = q.y; rnd[2] = q.z; rnd[3] = q.w;
+      if (HAS_COL) {
+        uint4 qc = q;
+        if (a.off_hi_col != a.off_hi)
+          qc = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), a.off_lo, a.off_hi_col, a.seed_lo, a.seed_hi);
+        *reinterpret_cast<uint4*>(smem + QuantSmem::kRand + r * 128 + cb * 16) = qc;
+      }
+    }
+    if (HAS_ROW) {
+      float f[16];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        uint32_t word = raw[i][k];
+        if (RHT_ROW) word ^= sign_pair(a.sign_mask, 2 * k, 2 * k + 1);
+        f[2 * k] = bf16_lo(word);
+        f[2 * k + 1] = bf16_hi(word);
+      }
+      if (RHT_ROW) {
+        fwht16(f);
+#pragma unroll
+        for (int k = 0; k < 16; ++k) f[k] *= 0.25f;
+      }
+      uint32_t byte;
+      float enc;
+      if (BLOCK2D) {
+        byte = blk_byte;
+        enc = blk_enc;
+      } else {
+        block_scales(amax16(f), r_senc, r_sdec, byte, enc);
+      }
+      uint2 codes = convert16<SR>(f, enc, rnd);
+      if (ok[i])
+        *reinterpret_cast<uint2*>(a.r_codes + (row0 + r) * (a.cols >> 1) + ((col0 + cb * 16) >> 1)) = codes;
+      const int pos = a.r_swz ? ((cb >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (cb & 3)) : (r * 8 + cb);
+      smem[QuantSmem::kSfRow + pos] = (uint8_t)byte;
+    }
+  }
+  __syncthreads();
+
+  // ------------------------------------------------------------------ phase 2 ----
+  if (HAS_COL) {
+    const int q = warp;  // 16-row group inside the tile
+#pragma unroll 1
+    for (int it = 0; it < 2; ++it) {
+      const int cp = lane + 32 * it;  // column pair: tile columns 2cp, 2cp+1
+      float f0[16], f1[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        uint32_t word = *reinterpret_cast<const uint32_t*>(smem + QuantSmem::kTile + (q * 16 + j) * 256 + cp * 4);
+        if (RHT_COL) word ^= sign_pair(a.sign_mask, j, j);
+        f0[j] = bf16_lo(word);
+        f1[j] = bf16_hi(word);
+      }
+      if (RHT_COL) {
+        fwht16(f0);
+        fwht16(f1);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          f0[j] *= 0.25f;
+          f1[j] *= 0.25f;
+        }
+      }
+      uint32_t byte0, byte1;
+      float enc0, enc1;
+      if (BLOCK2D) {
+        enc0 = enc1 = reinterpret_cast<const float*>(smem + QuantSmem::kBlkEnc)[q * 8 + (cp >> 3)];
+        byte0 = byte1 = smem[QuantSmem::kBlkByte + q * 8 + (cp >> 3)];
+      } else {
+        block_scales(amax16(f0), c_senc, c_sdec, byte0, enc0);
+        block_scales(amax16(f1), c_senc, c_sdec, byte1, enc1);
+      }
+      uint32_t rnd0[4] = {0u, 0u, 0u, 0u}, rnd1[4] = {0u, 0u, 0u, 0u};
+      if (SR) {
+        // byte j of rnd0 / rnd1 = draw of source element (row 16q + j, column 2cp / 2cp + 1)
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          uint32_t two = *reinterpret_cast<const uint16_t*>(smem + QuantSmem::kRand + (q * 16 + j) * 128 + cp * 2);
+          rnd0[j >> 2] |= (two & 0xffu) << (8 * (j & 3));
+          rnd1[j >> 2] |= (two >> 8) << (8 * (j & 3));
+        }
+      }
+      uint2 codes0 = convert16<SR>(f0, enc0, rnd0);
+      uint2 codes1 = convert16<SR>(f1, enc1, rnd1);
+      // staging: column c holds eight 8-byte units, unit q stored at (q ^ (c >> 1)) & 7; the column a
+      // lane writes first alternates with bit 3 of the lane so that a half warp covers all banks
+      const int sel = (lane >> 3) & 1;
+#pragma unroll
+      for (int s = 0; s < 2; ++s) {
+        const int odd = s ^ sel;
+        const int c = 2 * cp + odd;
+        uint2 val = odd ? codes1 : codes0;
+        *reinterpret_cast<uint2*>(smem + QuantSmem::kColCodes + c * 64 + (((q ^ (c >> 1)) & 7) << 3)) = val;
+        const uint32_t byte = odd ? byte1 : byte0;
+        const int pos = a.c_swz ? ((q >> 2) * 512 + (c & 31) * 16 + (c >> 5) * 4 + (q & 3)) : (c * 8 + q);
+        smem[QuantSmem::kSfCol + pos] = (uint8_t)byte;
+      }
+    }
+  }
+  __syncthreads();
+
+  // ------------------------------------------------------------------ phase 3 ----
+  if (HAS_COL) {
+    const int64_t pitch = a.rows >> 1;  // bytes per row of the transposed copy
+    const bool vec16 = (a.rows & 31) == 0;
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int unit = threadIdx.x + 256 * k;
+      const int c = unit >> 2, m = unit & 3;  // column, pair of 16-row groups (2m, 2m+1)
+      if (col0 + c >= a.cols) continue;
+      const int x = (c >> 1) & 7;
+      const int base = ((2 * m) ^ x) & 6;
+      uint4 v = *reinterpret_cast<const uint4*>(smem + QuantSmem::kColCodes + c * 64 + base * 8);
+      if (x & 1) v = make_uint4(v.z, v.w, v.x, v.y);
+      uint8_t* dst = a.c_codes + (col0 + c) * pitch + (row0 >> 1) + m * 16;
+      const int64_t rr = row0 + 32 * m;
+      if (rr + 16 < a.rows && vec16) {
+        *reinterpret_cast<uint4*>(dst) = v;
+      } else {
+        if (rr < a.rows) *reinterpret_cast<uint2*>(dst) = make_uint2(v.x, v.y);
+        if (rr + 16 < a.rows) *reinterpret_cast<uint2*>(dst + 8) = make_uint2(v.z, v.w);
+      }
+    }
+  }
+  // scale bytes
+#pragma unroll
+  for (int which = 0; which < 2; ++which) {
+    if (which == 0 && !HAS_ROW) continue;
+    if (which == 1 && !HAS_COL) continue;
+    const uint8_t* src = smem + (which == 0 ? QuantSmem::kSfRow : QuantSmem::kSfCol);
+    uint8_t* dst = which == 0 ? a.r_scales : a.c_scales;
+    const int swz = which == 0 ? a.r_swz : a.c_swz;
+    // the copy's row / block coordinates of this tile
+    const int64_t R0 = which == 0 ? row0 : col0, K0 = which == 0 ? (col0 >> 4) : (row0 >> 4);
+    const int64_t Rn = which == 0 ? a.rows : a.cols, n_kb = which == 0 ? n_cb : n_rb;
+    if (swz) {
+      if (threadIdx.x < 64) {
+        const int atom = threadIdx.x >> 5;
+        if (K0 + atom * 4 < n_kb) {
+          const int64_t off = ((R0 >> 7) * (n_kb >> 2) + (K0 >> 2) + atom) * 512 + (threadIdx.x & 31) * 16;
+          *reinterpret_cast<uint4*>(dst + off) = *reinterpret_cast<const uint4*>(src + threadIdx.x * 16);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int idx = threadIdx.x * 4 + k;
+        const int r = idx >> 3, kb = idx & 7;
+        if (R0 + r < Rn && K0 + kb < n_kb) dst[(R0 + r) * n_kb + K0 + kb] = src[idx];
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Test aids
+// ---------------------------------------------------------------------------------------------
+__global__ void dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
+                                  const float* __restrict__ global, int64_t rows, int64_t cols, int swz,
+                                  float* __restrict__ out) {
+  const int64_t n = rows * cols;
+  const float s_dec = global[1];
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / cols, c = i % cols;
+    const uint32_t byte = codes[r * (cols >> 1) + (c >> 1)];
+    const uint32_t code = (c & 1) ? (byte >> 4) : (byte & 15u);
+    const float mags[8] = {0.f, 0.5f, 1.f, 1.5f, 2.f, 3.f, 4.f, 6.f};
+    float m = mags[code & 7u];
+    if (code & 8u) m = -m;
+    const int64_t so = swz ? sf_swizzled_offset(r, c >> 4, cols >> 4) : (r * (cols >> 4) + (c >> 4));
+    uint16_t sb = scales[so];
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(sb));
+    float sf = __half2float(__ushort_as_half((unsigned short)(h2 & 0xffffu)));
+    out[i] = __fmul_rn(__fmul_rn(m, sf), s_dec);
+  }
+}
+
+__global__ void rht16_kernel(const uint16_t* __restrict__ x, int64_t rows, int64_t cols, int64_t ld,
+                             int colwise, uint32_t mask, float* __restrict__ out) {
+  // one thread per chunk of the requested copy
+  const int64_t R = colwise ? cols : rows, C = colwise ? rows : cols;
+  const int64_t n_chunks = R * (C >> 4);
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n_chunks;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / (C >> 4), kb = i % (C >> 4);
+    float f[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const int64_t sr = colwise ? (kb * 16 + j) : r, sc = colwise ? r : (kb * 16 + j);
+      uint32_t bits = (uint32_t)x[sr * ld + sc] << 16;
+      if ((mask >> j) & 1u) bits ^= 0x80000000u;
+      f[j] = __uint_as_float(bits);
+    }
+    fwht16(f);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) out[r * C + kb * 16 + j] = f[j] * 0.25f;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host launchers
+// ---------------------------------------------------------------------------------------------
+template <bool PLAIN, bool RR, bool RC>
+static cudaError_t launch_amax_t(const QuantArgs& a, float* plain0, float* plain1, float* rot_row,
+                                 float* rot_col, cudaStream_t s) {
+  const int tiles_c = (int)((a.cols + 255) / 256);
+  const int64_t tiles = ((a.rows + 127) / 128) * tiles_c;
+  amax_kernel<PLAIN, RR, RC><<<(unsigned)tiles, 256, 0, s>>>(a.x, a.rows, a.cols, a.ld, a.sign_mask, tiles_c,
+                                                            plain0, plain1, rot_row, rot_col);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_amax(const QuantArgs& a, bool has_row, bool has_col, bool rht_row, bool rht_col,
+                        cudaStream_t s) {
+  cudaError_t e;
+  if (has_row && (e = cudaMemsetAsync(a.r_global, 0, sizeof(float), s)) != cudaSuccess) return e;
+  if (has_col && (e = cudaMemsetAsync(a.c_global, 0, sizeof(float), s)) != cudaSuccess) return e;
+  const bool rr = has_row && rht_row, rc = has_col && rht_col;
+  float* plain0 = (has_row && !rht_row) ? a.r_global : nullptr;
+  float* plain1 = (has_col && !rht_col) ? a.c_global : nullptr;
+  const bool plain = plain0 || plain1;
+  float* rot_row = rr ? a.r_global : nullptr;
+  float* rot_col = rc ? a.c_global : nullptr;
+#define NVFP4_AMAX(P, R, C) \
+  if (plain == P && rr == R && rc == C) return launch_amax_t<P, R, C>(a, plain0, plain1, rot_row, rot_col, s);
+  NVFP4_AMAX(true, false, false)
+  NVFP4_AMAX(true, false, true)
+  NVFP4_AMAX(true, true, false)
+  NVFP4_AMAX(false, true, true)
+  NVFP4_AMAX(false, false, true)
+  NVFP4_AMAX(false, true, false)
+#undef NVFP4_AMAX
+  return cudaErrorInvalidValue;
+}
+
+template <bool HR, bool HC, bool B2, bool RR, bool RC, bool SR>
+static cudaError_t launch_quant_t(const QuantArgs& a, cudaStream_t s) {
+  auto kern = quantize_kernel<HR, HC, B2, RR, RC, SR>;
+  const int smem = (SR && HC) ? QuantSmem::kBytesRand : QuantSmem::kBytesNoRand;
+  static bool configured = false;  // per instantiation; the attribute is per function and idempotent
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, QuantSmem::kBytesRand);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int64_t tiles = (int64_t)a.tiles_r * a.tiles_c;
+  kern<<<(unsigned)tiles, 256, smem, s>>>(a);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_quantize(const QuantArgs& a, bool has_row, bool has_col, bool block2d, bool rht_row,
+                            bool rht_col, bool sr, cudaStream_t s) {
+  rht_row = rht_row && has_row;
+  rht_col = rht_col && has_col;
+#define NVFP4_Q(HR, HC, B2, RR, RC, SRV)                                                           \
+  if (has_row == HR && has_col == HC && block2d == B2 && rht_row == RR && rht_col == RC && sr == SRV) \
+    return launch_quant_t<HR, HC, B2, RR, RC, SRV>(a, s);
+#define NVFP4_Q_COPIES(B2, RR, RC, SRV)      \
+  NVFP4_Q(true, false, B2, RR, false, SRV)   \
+  NVFP4_Q(false, true, B2, false, RC, SRV)   \
+  NVFP4_Q(true, true, B2, RR, RC, SRV)
+  NVFP4_Q_COPIES(true, false, false, false)
+  NVFP4_Q_COPIES(true, false, false, true)
+  NVFP4_Q_COPIES(false, false, false, false)
+  NVFP4_Q_COPIES(false, false, false, true)
+  NVFP4_Q_COPIES(false, false, true, false)
+  NVFP4_Q_COPIES(false, false, true, true)
+  NVFP4_Q_COPIES(false, true, false, false)
+  NVFP4_Q_COPIES(false, true, false, true)
+  NVFP4_Q_COPIES(false, true, true, false)
+  NVFP4_Q_COPIES(false, true, true, true)
+#undef NVFP4_Q_COPIES
+#undef NVFP4_Q
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_dequantize(const nvfp4_tensor& t, float* out, cudaStream_t s) {
+  dequantize_kernel<<<1184, 256, 0, s>>>(t.codes, t.scales, t.global, t.rows, t.cols,
+                                         t.sf_layout == NVFP4_SF_SWIZZLED, out);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rht16(const void* x, int64_t rows, int64_t cols, int64_t ld, int colwise, uint32_t mask,
+                         float* out, cudaStream_t s) {
+  rht16_kernel<<<1184, 256, 0, s>>>(static_cast<const uint16_t*>(x), rows, cols, ld, colwise, mask, out);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace nvfp4

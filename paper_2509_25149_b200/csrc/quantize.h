@@ -1,0 +1,33 @@
+// Internal launch interface of the quantizer kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "nvfp4.h"
+
+namespace nvfp4 {
+
+struct QuantArgs {
+  const uint16_t* x;  // bf16 source [rows x cols], leading dimension ld
+  int64_t rows, cols, ld;
+  uint8_t* r_codes;   // row-wise copy
+  uint8_t* r_scales;
+  float* r_global;
+  uint8_t* c_codes;   // column-wise (transposed) copy
+  uint8_t* c_scales;
+  float* c_global;
+  int r_swz, c_swz;   // 1 = swizzled scale layout
+  uint32_t sign_mask;
+  uint32_t seed_lo, seed_hi, off_lo, off_hi, off_hi_col;
+  int tiles_r, tiles_c;  // 128 x 128 tiles of the source
+};
+
+cudaError_t launch_amax(const QuantArgs& a, bool has_row, bool has_col, bool rht_row, bool rht_col,
+                        cudaStream_t s);
+cudaError_t launch_quantize(const QuantArgs& a, bool has_row, bool has_col, bool block2d, bool rht_row,
+                            bool rht_col, bool sr, cudaStream_t s);
+cudaError_t launch_dequantize(const nvfp4_tensor& t, float* out, cudaStream_t s);
+cudaError_t launch_rht16(const void* x, int64_t rows, int64_t cols, int64_t ld, int colwise, uint32_t mask,
+                         float* out, cudaStream_t s);
+
+}  // namespace nvfp4

@@ -1,0 +1,141 @@
+"""Comparison protocol between the CUDA path (through the C ABI) and the CPU oracle."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2509_25149_b200 import binding as B
+from paper_2509_25149_b200 import synth
+
+E4M3_VALUES = np.array([oracle.e4m3_decode(i) for i in range(0x7F)], dtype=np.float64)
+E4M3_MIDPOINTS = (E4M3_VALUES[1:] + E4M3_VALUES[:-1]) / 2
+E2M1_GRID = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6], dtype=np.float64)
+E2M1_MIDPOINTS = (E2M1_GRID[1:] + E2M1_GRID[:-1]) / 2
+
+
+def unpack(codes: np.ndarray) -> np.ndarray:
+    return np.stack([codes & 15, codes >> 4], axis=-1).reshape(codes.shape[0], -1)
+
+
+def download(t: B.NVFP4Tensor):
+    """GPU copy -> (codes [R][C/2], scales linear [R][C/16], glob[2]) as numpy."""
+    torch.cuda.synchronize()
+    codes = t.codes.cpu().numpy()
+    sc = t.scales.cpu().numpy()
+    if t.sf_layout == B.SF_SWIZZLED:
+        sc = oracle.sf_unswizzle(sc, t.rows, t.cols // 16)
+    else:
+        sc = sc.reshape(t.rows, t.cols // 16)
+    return codes, sc, t.glob.cpu().numpy()
+
+
+def upload(q: oracle.Quantized, device="cuda") -> B.NVFP4Tensor:
+    """Oracle copy -> device tensors in the swizzled scale layout the GEMM reads."""
+    return B.NVFP4Tensor(torch.from_numpy(np.ascontiguousarray(q.codes)).to(device),
+                         torch.from_numpy(oracle.sf_swizzle(q.scales)).to(device),
+                         torch.from_numpy(np.ascontiguousarray(q.glob)).to(device), q.rows, q.cols, B.SF_SWIZZLED)
+
+
+def gpu_quantize(x: torch.Tensor, *, rowwise=True, colwise=False, sf_layout=B.SF_SWIZZLED, **opt):
+    """x: CPU bf16 tensor.  Returns (row copy or None, col copy or None) as device NVFP4Tensors."""
+    xd = x.cuda()
+    R, C = x.shape
+    row = B.alloc_tensor(R, C, sf_layout) if rowwise else None
+    col = B.alloc_tensor(C, R, sf_layout) if colwise else None
+    B.nvfp4_quantize(xd, B.quant_opts(**opt), row, col)
+    torch.cuda.synchronize()
+    return row, col
+
+
+def assert_exact(gpu: B.NVFP4Tensor, ref: oracle.Quantized, what=""):
+    codes, scales, glob = download(gpu)
+    assert glob.view(np.uint32).tolist() == ref.glob.view(np.uint32).tolist(), f"{what}: global {glob} vs {ref.glob}"
+    bad = np.argwhere(scales != ref.scales)
+    assert bad.size == 0, f"{what}: {len(bad)} scale bytes differ, first at {bad[0]}: " \
+                          f"{scales[tuple(bad[0])]:#x} vs {ref.scales[tuple(bad[0])]:#x}"
+    bad = np.argwhere(codes != ref.codes)
+    assert bad.size == 0, f"{what}: {len(bad)} code bytes differ, first at {bad[0]}: " \
+                          f"{codes[tuple(bad[0])]:#x} vs {ref.codes[tuple(bad[0])]:#x}"
+
+
+def assert_rht_close(x_bits: np.ndarray, gpu: B.NVFP4Tensor, y_gpu: np.ndarray, *, colwise, sign_mask, rounding,
+                     seed=0, sr_offset=0, what=""):
+    """Tolerance protocol for transformed copies (the transform is computed in a different order on the GPU):
+    values within 1e-5 of the scale of their dot product; amax within 1e-5; then, with the oracle re-run on the
+    GPU's amax, scale bytes equal except where the pre-rounding scale is within 1e-5 of an E4M3 midpoint, and
+    codes equal except where the pre-rounding value is within 1e-5 of a rounding threshold (an excused code must
+    still be an adjacent grid point).  Excused items must stay below 1e-3 of all elements."""
+    codes, scales, glob = download(gpu)
+    ref0 = oracle.quantize(x_bits, colwise=colwise, rht=True, sign_mask=sign_mask, rounding=rounding, seed=seed,
+                           sr_offset=sr_offset, return_y=True)
+    # (1) transformed values
+    xs = synth.from_bits(x_bits).to(torch.float64).numpy()
+    src = xs.T if colwise else xs
+    l1 = np.abs(src).reshape(src.shape[0], -1, 16).sum(axis=2).repeat(16, axis=1) / 4
+    assert np.all(np.abs(y_gpu.astype(np.float64) - ref0.y) <= 1e-5 * l1 + 1e-30), f"{what}: transformed values"
+    # (2) amax
+    assert abs(float(glob[0]) - float(ref0.amax)) <= 1e-5 * float(ref0.amax), f"{what}: amax"
+    ref = oracle.quantize(x_bits, colwise=colwise, rht=True, sign_mask=sign_mask, rounding=rounding, seed=seed,
+                          sr_offset=sr_offset, amax_override=float(glob[0]), return_y=True)
+    assert glob.view(np.uint32).tolist() == ref.glob.view(np.uint32).tolist(), f"{what}: s_dec from the same amax"
+    s_enc, s_dec = oracle.global_scale(float(glob[0]))
+    # (3) scale bytes
+    R, C = ref.rows, ref.cols
+    amax_b = np.abs(ref.y).reshape(R, C // 16, 16).max(axis=2)
+    t_b = ((amax_b.astype(np.float32) / np.float32(6)) * np.float32(s_enc)).astype(np.float64)
+    nearest_mid = E4M3_MIDPOINTS[np.clip(np.searchsorted(E4M3_MIDPOINTS, t_b), 0, len(E4M3_MIDPOINTS) - 1)]
+    prev_mid = E4M3_MIDPOINTS[np.clip(np.searchsorted(E4M3_MIDPOINTS, t_b) - 1, 0, len(E4M3_MIDPOINTS) - 1)]
+    near = np.minimum(np.abs(t_b - nearest_mid), np.abs(t_b - prev_mid)) <= 1e-5 * np.maximum(t_b, 1e-30)
+    sdiff = scales != ref.scales
+    assert not np.any(sdiff & ~near), f"{what}: {np.count_nonzero(sdiff & ~near)} unexcused scale bytes"
+    assert np.all(np.abs(scales.astype(int) - ref.scales.astype(int))[sdiff] == 1), f"{what}: excused scale not adjacent"
+    # (4) codes in blocks whose scale agrees
+    got, want = unpack(codes), unpack(ref.codes)
+    cdiff = (got != want) & ~np.repeat(sdiff, 16, axis=1)
+    excused = 0
+    for r, c in np.argwhere(cdiff):
+        enc_b = oracle.block_encode_scale(int(ref.scales[r, c // 16]), s_dec)
+        v = float(np.float32(ref.y[r, c]) * enc_b)
+        a = min(abs(v), 6.0)
+        if rounding == oracle.RNE:
+            thr = E2M1_MIDPOINTS
+            step = 0.5 if a < 2 else (1.0 if a < 4 else 2.0)
+        else:
+            sr_, sc_ = (c, r) if colwise else (r, c)
+            u = oracle.sr_draw(seed, sr_offset, sr_ * x_bits.shape[1] + sc_)
+            lo = E2M1_GRID[E2M1_GRID <= a].max()
+            hi = E2M1_GRID[E2M1_GRID > a].min() if a < 6 else 6.0
+            step = max(hi - lo, 0.5)
+            thr = np.array([lo + (hi - lo) * (u + 0.5) / 256])
+        assert np.min(np.abs(thr - a)) <= 1e-5 * max(a, step), f"{what}: code at {(r, c)} differs away from a threshold (v={v})"
+        assert abs(int(got[r, c] & 7) - int(want[r, c] & 7)) <= 1, f"{what}: excused code not adjacent"
+        excused += 1
+    total = R * C
+    n_block_excused = int(np.count_nonzero(sdiff)) * 16
+    assert excused + n_block_excused <= max(1e-3 * total, 16), f"{what}: too many excused items"
+    # blocks with an excused scale: decoded values still within one E2M1 step (in the block's own scale) of y
+    if np.any(sdiff):
+        deq = oracle.dequantize(oracle.Quantized(codes, scales, glob, R, C))
+        sb = np.vectorize(oracle.e4m3_decode)(scales).repeat(16, axis=1) * float(s_dec)
+        m = np.repeat(sdiff, 16, axis=1)
+        assert np.all(np.abs(deq - ref.y)[m] <= 2.0 * sb[m] * (1 + 2.0 ** -3) + 1e-30), f"{what}: excused block decode"
+    return {"excused_codes": excused, "excused_scales": int(np.count_nonzero(sdiff)), "elements": total}
+
+
+def gemm_reference(a: oracle.Quantized, b: oracle.Quantized, rows=None, cols=None):
+    """FP64 product of the decoded operands and its tolerance scale, optionally on a subset of rows / columns."""
+    da, db = oracle.dequantize(a), oracle.dequantize(b)
+    if rows is not None:
+        da = da[rows]
+    if cols is not None:
+        db = db[cols]
+    return oracle.gemm_tn(da, db)
+
+
+def assert_gemm_close(D: np.ndarray, Dref: np.ndarray, T: np.ndarray, bf16_out: bool, what=""):
+    tol = 1e-3 * T + (2.0 ** -9 * np.abs(Dref) if bf16_out else 0.0) + 1e-30
+    err = np.abs(D.astype(np.float64) - Dref)
+    worst = np.unravel_index(np.argmax(err / tol), err.shape)
+    assert np.all(err <= tol), f"{what}: worst at {worst}: got {D[worst]}, want {Dref[worst]}, tol {tol[worst]}"
+    return float((err / np.maximum(T, 1e-300)).max())

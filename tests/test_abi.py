@@ -1,0 +1,76 @@
+"""The C-ABI library builds, loads and exports what include/nvfp4.h declares; argument checks need no GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2509_25149_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "nvfp4.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"NVFP4_API[^;(]*?\b(nvfp4_\w+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    L = B.lib()
+    names = declared_symbols()
+    assert len(names) >= 12 and set(names) == set(B.EXPORTED)
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_struct_layouts_match_the_header():
+    assert ctypes.sizeof(B.CTensor) == 48 and ctypes.sizeof(B.CQuantOpts) == 40
+    assert B.CTensor.rows.offset == 24 and B.CQuantOpts.seed.offset == 24
+
+
+def test_status_strings_and_knobs():
+    assert B.status_string(0) == "ok"
+    assert "NULL" in B.status_string(1) and "shape" in B.status_string(2)
+    B.nvfp4_set_gemm_tile_n(128)
+    B.nvfp4_set_gemm_tile_n(0)
+    with pytest.raises(ValueError):
+        B.nvfp4_set_gemm_tile_n(64)
+    assert B.nvfp4_linear_fwd_workspace_bytes(256, 256) >= 256 * 256 // 2 + 256 * 256 // 16 + 8
+    assert B.nvfp4_linear_bwd_workspace_bytes(256, 512) >= 2 * (256 * 512 // 2 + 256 * 512 // 16 + 8)
+
+
+def test_argument_validation_happens_before_any_launch():
+    L = B.lib()
+    o = B.quant_opts()
+    fake = 0x7F0000000000  # never dereferenced: validation fails first
+    t = B.CTensor(fake, fake, fake, 128, 128, B.SF_SWIZZLED, 0)
+    q = lambda *a: L.nvfp4_quantize(*a)
+    assert q(None, 128, 128, 128, ctypes.byref(o), ctypes.byref(t), None, None) == 1          # NULL input
+    assert q(fake, 128, 128, 128, ctypes.byref(o), None, None, None) == 1                      # no copy requested
+    assert q(fake, 120, 128, 128, ctypes.byref(o), ctypes.byref(t), None, None) == 2           # rows % 16
+    assert q(fake, 128, 128, 64, ctypes.byref(o), ctypes.byref(t), None, None) == 2            # ld < cols
+    assert q(fake + 2, 128, 128, 128, ctypes.byref(o), ctypes.byref(t), None, None) == 3       # alignment
+    bad = B.quant_opts(block_rows=4)
+    assert q(fake, 128, 128, 128, ctypes.byref(bad), ctypes.byref(t), None, None) == 4
+    bad = B.quant_opts(block_rows=16, rht_colwise=True)
+    assert q(fake, 128, 128, 128, ctypes.byref(bad), ctypes.byref(t), None, None) == 4         # no RHT on 2D blocks
+    wrong = B.CTensor(fake, fake, fake, 128, 256, B.SF_SWIZZLED, 0)
+    assert q(fake, 128, 128, 128, ctypes.byref(o), ctypes.byref(wrong), None, None) == 2       # copy shape
+    small = B.CTensor(fake, fake, fake, 64, 128, B.SF_SWIZZLED, 0)
+    assert q(fake, 64, 128, 128, ctypes.byref(o), ctypes.byref(small), None, None) == 2        # swizzled needs 128 rows
+    a = B.CTensor(fake, fake, fake, 128, 256, B.SF_SWIZZLED, 0)
+    b = B.CTensor(fake, fake, fake, 128, 512, B.SF_SWIZZLED, 0)
+    assert L.nvfp4_gemm(ctypes.byref(a), ctypes.byref(b), fake, 0, 128, 0, None) == 2          # K mismatch
+    b = B.CTensor(fake, fake, fake, 128, 256, B.SF_LINEAR, 0)
+    assert L.nvfp4_gemm(ctypes.byref(a), ctypes.byref(b), fake, 0, 128, 0, None) == 4          # needs swizzled scales
+    b = B.CTensor(fake, fake, fake, 128, 256, B.SF_SWIZZLED, 0)
+    assert L.nvfp4_gemm(ctypes.byref(a), ctypes.byref(b), fake, 0, 128, 1, None) == 4          # accumulate into bf16
+    assert L.nvfp4_gemm(ctypes.byref(a), ctypes.byref(b), fake, 0, 64, 0, None) == 2           # ldd < N
+    assert L.nvfp4_gemm(ctypes.byref(a), None, fake, 0, 128, 0, None) == 1
+    assert L.nvfp4_linear_fwd(fake, fake, 256, 256, 256, ctypes.byref(o), fake, None, ctypes.byref(a), None, 0,
+                              None, 0, None) == 5                                              # workspace
+    assert L.nvfp4_linear_fwd(fake, fake, 200, 256, 256, ctypes.byref(o), fake, None, ctypes.byref(a), None, 0,
+                              fake, 1 << 30, None) == 2
+    assert L.nvfp4_linear_bwd(fake, None, None, 256, 256, 256, ctypes.byref(o), None, None, 0, fake, 1 << 30,
+                              None) == 1
