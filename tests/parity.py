@@ -134,7 +134,7 @@ def gemm_reference(a: oracle.Quantized, b: oracle.Quantized, rows=None, cols=Non
 
 
 def assert_gemm_close(D: np.ndarray, Dref: np.ndarray, T: np.ndarray, bf16_out: bool, what=""):
-    tol = 1e-3 * T + (2.0 ** -9 * np.abs(Dref) if bf16_out else 0.0) + 1e-30
+    tol = 1e-3 * T + (2.0 ** -8 * np.abs(Dref) if bf16_out else 0.0) + 1e-30
     err = np.abs(D.astype(np.float64) - Dref)
     worst = np.unravel_index(np.argmax(err / tol), err.shape)
     assert np.all(err <= tol), f"{what}: worst at {worst}: got {D[worst]}, want {Dref[worst]}, tol {tol[worst]}"
