@@ -1,0 +1,402 @@
+"""Benchmark of the NVFP4 linear-layer hot path on B200.
+
+One step = one pass of the whole path over the FFN up-projection of the 12B-class model
+(tokens M = 8192, K = 5120, N = 20480): quantize W (16x16 blocks, both copies), quantize X (row-wise +
+rotated column-wise), Fprop, quantize dY (stochastic rounding, row-wise + rotated column-wise), Dgrad, Wgrad.
+With --gpus N each rank runs the step on its own 8192-token shard (data parallel, weak scaling) and the FP32
+weight gradient is summed across ranks with one NCCL all-reduce.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded slab of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "NVFP4 GEMM TFLOP/s vs FP4 peak; quantize+RHT+SR GB/s vs HBM peak"
+M, N, K = 8192, 20480, 5120
+WORKLOAD = "cfg3_ffn_up_fwd_bwd_M8192_K5120_N20480"
+SLAB = (4096, 2048, 5120)     # tokens, out-features, in-features of the CPU-baseline sample (one run)
+SLAB_REF = (512, 1024, 5120)  # per-step sample of the `--impl reference` arm (many steps)
+
+
+def step_flops(m=M, n=N, k=K) -> float:
+    return 3 * 2.0 * m * n * k
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------ clocks ----
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([t.strip() for t in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+                for nme, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nme)
+            except (ValueError, IndexError):
+                continue
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------ CPU oracle baseline ----
+def oracle_slab_step(prob_slices):
+    """One fwd+bwd of the slab with the CPU oracle, as it stands.  Returns seconds."""
+    import oracle
+    from paper_2509_25149_b200 import synth
+    X, W, dY, mask = prob_slices
+    t0 = time.perf_counter()
+    xb, wb, gb = synth.bits(X), synth.bits(W), synth.bits(dY)
+    w_row = oracle.quantize(wb, block_rows=16)
+    w_col = oracle.quantize(wb, block_rows=16, colwise=True)
+    x_row = oracle.quantize(xb)
+    x_col = oracle.quantize(xb, colwise=True, rht=True, sign_mask=mask)
+    oracle.gemm_tn(oracle.dequantize(x_row), oracle.dequantize(w_row), want_T=False)
+    g_row = oracle.quantize(gb, rounding=oracle.SR)
+    g_col = oracle.quantize(gb, colwise=True, rht=True, sign_mask=mask, rounding=oracle.SR)
+    oracle.gemm_tn(oracle.dequantize(g_row), oracle.dequantize(w_col), want_T=False)
+    oracle.gemm_tn(oracle.dequantize(g_col), oracle.dequantize(x_col), want_T=False)
+    return time.perf_counter() - t0
+
+
+def slab_inputs(slab=SLAB):
+    from paper_2509_25149_b200 import synth
+    ms, ns, ks = slab
+    X = synth.normal_with_outliers_bf16((ms, ks), 0.001, 100.0, 3001, 3004)
+    W = synth.normal_bf16((ns, ks), 0.02, 3002)
+    dY = synth.normal_bf16((ms, ns), 1e-4, 3003)
+    return X, W, dY, synth.DEFAULT_RHT_SIGN_MASK
+
+
+def cpu_baseline(steps=1):
+    import oracle
+    oracle.build()
+    inputs = slab_inputs()
+    times = [oracle_slab_step(inputs) for _ in range(steps)]
+    ms, ns, ks = SLAB
+    t = sum(times) / len(times)
+    return {"value": step_flops(ms, ns, ks) / t / 1e12, "unit": "TFLOP/s", "cores": len(os.sched_getaffinity(0)),
+            "kind": "oracle",
+            "sample": f"fwd+bwd of a {ms}x{ns}x{ks} slab of the workload (tokens 0..{ms - 1}, output features "
+                      f"0..{ns - 1}, all {ks} input features): 7 oracle quantize calls + 3 FP64 GEMMs, {t:.2f} s"}, t
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    inputs = slab_inputs(SLAB_REF)
+    for _ in range(args.warmup):
+        oracle_slab_step(inputs)
+    times = [oracle_slab_step(inputs) for _ in range(args.steps)]
+    ms, ns, ks = SLAB_REF
+    t = sum(times) / len(times)
+    val = step_flops(ms, ns, ks) / t / 1e12
+    cores = len(os.sched_getaffinity(0))
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": f"{ms}x{ns}x{ks} slab per step"},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+                             "sample": f"fwd+bwd of a {ms}x{ns}x{ks} slab of the workload per step"},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ CUDA arm ----
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2509_25149_b200 import binding as B
+    from paper_2509_25149_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B.lib()
+
+    # inputs: rank r owns its own 8192-token shard (different seeds per rank), W is replicated
+    p = synth.config3()
+    if rank > 0:
+        p.X = synth.normal_with_outliers_bf16((M, K), 0.001, 100.0, 3001 + 100 * rank, 3004 + 100 * rank)
+        p.dY = synth.normal_bf16((M, N), 1e-4, 3003 + 100 * rank)
+    hX, hW, hdY = p.X.pin_memory(), p.W.pin_memory(), p.dY.pin_memory()
+    X, W, dY = hX.cuda(), hW.cuda(), hdY.cuda()
+    opts = B.quant_opts(rht_sign_mask=p.rht_sign_mask, seed=0, sr_offset=rank << 32)
+    X_col, W_row, W_col = B.alloc_tensor(K, M), B.alloc_tensor(N, K), B.alloc_tensor(K, N)
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((N, K), dtype=torch.float32, device="cuda")
+    ws_f = torch.empty(B.nvfp4_linear_fwd_workspace_bytes(M, K), dtype=torch.uint8, device="cuda")
+    ws_b = torch.empty(B.nvfp4_linear_bwd_workspace_bytes(M, N), dtype=torch.uint8, device="cuda")
+
+    def step():
+        B.nvfp4_linear_fwd(X, W, opts, Y, X_col, W_row, W_col, False, ws_f)
+        B.nvfp4_linear_bwd(dY, X_col, W_col, K, opts, dX, dW, False, ws_b)
+        if world > 1:
+            dist.all_reduce(dW)  # FP32 sum of the weight gradient across data-parallel replicas
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms: float) -> float:
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    B.nvfp4_device_status()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    # ---- timed region: K steps, device-resident inputs --------------------------------------
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = B.nvfp4_launch_count()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    launches = B.nvfp4_launch_count() - launches0
+    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps)
+    B.nvfp4_device_status()
+
+    # ---- per-kernel pass: the same sequence as separate C-ABI calls with events around each ----
+    x_row = B.alloc_tensor(M, K)
+    g_row, g_col = B.alloc_tensor(M, N), B.alloc_tensor(N, M)
+    w_opts = B.quant_opts(block_rows=16)
+    x_opts = B.quant_opts(rht_colwise=True, rht_sign_mask=p.rht_sign_mask)
+    g_opts = B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True, rht_sign_mask=p.rht_sign_mask, seed=0,
+                          sr_offset=rank << 32)
+    calls = [
+        ("quant_W", lambda: B.nvfp4_quantize(W, w_opts, W_row, W_col)),
+        ("quant_X", lambda: B.nvfp4_quantize(X, x_opts, x_row, X_col)),
+        ("gemm_fprop", lambda: B.nvfp4_gemm(x_row, W_row, Y)),
+        ("quant_dY", lambda: B.nvfp4_quantize(dY, g_opts, g_row, g_col)),
+        ("gemm_dgrad", lambda: B.nvfp4_gemm(g_row, W_col, dX)),
+        ("gemm_wgrad", lambda: B.nvfp4_gemm(g_col, X_col, dW)),
+    ]
+    per = {name: [] for name, _ in calls}
+    for it in range(args.steps + 2):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)]
+        evs[0].record()
+        for i, (_, fn) in enumerate(calls):
+            fn()
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        if it >= 2:
+            for i, (name, _) in enumerate(calls):
+                per[name].append(evs[i].elapsed_time(evs[i + 1]))
+    B.nvfp4_device_status()
+    clocks = sampler.stop() if rank == 0 else None
+    kern_ms = {k: sum(v) / len(v) for k, v in per.items()}
+
+    # ---- end to end: host buffers, copies inside the timed region --------------------------------
+    hY = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    hdX = torch.empty((M, K), dtype=torch.bfloat16).pin_memory()
+    hdW = torch.empty((N, K), dtype=torch.float32).pin_memory()
+
+    def e2e_step():
+        X.copy_(hX, non_blocking=True)
+        W.copy_(hW, non_blocking=True)
+        dY.copy_(hdY, non_blocking=True)
+        step()
+        hY.copy_(Y, non_blocking=True)
+        hdX.copy_(dX, non_blocking=True)
+        hdW.copy_(dW, non_blocking=True)
+
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_step()
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    t1.record()
+    barrier()
+    e2e_ms = max_over_ranks(t0.elapsed_time(t1) / e2e_steps)
+    h2d = sum(t.numel() * t.element_size() for t in (hX, hW, hdY))
+    d2h = sum(t.numel() * t.element_size() for t in (hY, hdX, hdW))
+
+    if rank == 0:
+        peaks = measured_peaks()
+        flops = step_flops()
+        gemm_ms = (kern_ms["gemm_fprop"] + kern_ms["gemm_dgrad"] + kern_ms["gemm_wgrad"]) / 3
+        gemm_tflops = 2.0 * M * N * K / (gemm_ms * 1e-3) / 1e12
+        fp4_peak = 4.0 * peaks["bf16_tflops_sustained"]  # FP4 : BF16 dense = 4 : 1 (nominal ratio)
+        # quantizer: algorithmic bytes = two reads of the bf16 tensor + both copies (codes + scales)
+        q_elems = M * K + N * K + M * N
+        q_bytes = q_elems * (2 + 2 + 2 * (0.5 + 1.0 / 16))
+        q_ms = kern_ms["quant_W"] + kern_ms["quant_X"] + kern_ms["quant_dY"]
+        q_gbs = q_bytes / (q_ms * 1e-3) / 1e9
+        cpu, _ = cpu_baseline(1) if not args.no_cpu_baseline else (None, 0)
+        line = {
+            "metric": METRIC, "value": world * flops / (ms_step * 1e-3) / 1e12, "unit": "TFLOP/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "tokens_per_gpu": M, "in_features": K, "out_features": N,
+                       "parallelism": f"dp{world}", "l2": "inputs (629 MB bf16 per step) exceed the 126 MB L2",
+                       "step": "quantize W (2D), quantize X, Fprop, quantize dY (SR), Dgrad, Wgrad"
+                               + (", FP32 all-reduce of dW" if world > 1 else "")},
+            "gemm_tflops": gemm_tflops, "quant_gbs": q_gbs,
+            "kernel_ms": {k: round(v, 4) for k, v in kern_ms.items()},
+            "roofline": {"bound": "tensor", "kernel": "gemm_kernel (mean of Fprop, Dgrad, Wgrad)",
+                         "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
+                         "frac": gemm_tflops / fp4_peak, "traffic": None,
+                         "peak_source": f"4 x {peaks['source']} sustained bf16 cuBLAS ({peaks['bf16_tflops_sustained']} TFLOP/s)",
+                         "frac_of_burst": gemm_tflops / (4.0 * peaks["bf16_tflops"]),
+                         "frac_of_datasheet_9pf": gemm_tflops / 9000.0},
+            "roofline_quant": {"bound": "hbm", "kernel": "amax_kernel + quantize_kernel (W, X, dY)",
+                               "achieved": q_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                               "frac": q_gbs / peaks["hbm_gbs"], "traffic": None,
+                               "peak_source": f"{peaks['source']} copy bandwidth",
+                               "frac_of_datasheet_8tbs": q_gbs / 8000.0},
+            "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": launches, "clocks": clocks, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------- single-kernel cases (profiling) ----
+CASES = {
+    # name: (kind, rows/M, cols/N, K)
+    "gemm_fprop": ("gemm", 4096, 5120, 5120),      # bf16 output, K = 5120
+    "gemm_wgrad": ("gemm32", 5120, 5120, 4096),    # fp32 output
+    "quant_x": ("qx", 16384, 5120, 0),             # RNE, row-wise + rotated column-wise (168 MB > L2)
+    "quant_dy": ("qdy", 4096, 20480, 0),           # SR, row-wise + rotated column-wise (168 MB > L2)
+    "quant_w": ("qw", 20480, 5120, 0),             # 16x16 blocks, both copies (210 MB > L2)
+}
+
+
+def run_case(args):
+    """Runs ONE kernel family on a reduced shape: the small, self-terminating target for ncu captures."""
+    import torch
+
+    from paper_2509_25149_b200 import binding as B
+    from paper_2509_25149_b200 import synth
+
+    kind, r, c, k = CASES[args.case]
+    torch.cuda.set_device(0)
+    g = torch.Generator(device="cuda").manual_seed(1)
+    mask = synth.DEFAULT_RHT_SIGN_MASK
+    if kind in ("gemm", "gemm32"):
+        a_src = torch.randn((r, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        b_src = (torch.randn((c, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
+        A, Bq = B.alloc_tensor(r, k), B.alloc_tensor(c, k)
+        B.nvfp4_quantize(a_src, B.quant_opts(), A, None)
+        B.nvfp4_quantize(b_src, B.quant_opts(block_rows=16), Bq, None)
+        D = torch.empty((r, c), dtype=torch.float32 if kind == "gemm32" else torch.bfloat16, device="cuda")
+        fn = lambda: B.nvfp4_gemm(A, Bq, D)
+        work, unit = 2.0 * r * c * k / 1e12, "TFLOP/s"
+    else:
+        x = torch.randn((r, c), generator=g, device="cuda", dtype=torch.float32)
+        x = (x * (1e-4 if kind == "qdy" else 0.02 if kind == "qw" else 1.0)).to(torch.bfloat16)
+        row, col = B.alloc_tensor(r, c), B.alloc_tensor(c, r)
+        o = {"qx": B.quant_opts(rht_colwise=True, rht_sign_mask=mask),
+             "qdy": B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True, rht_sign_mask=mask),
+             "qw": B.quant_opts(block_rows=16)}[kind]
+        fn = lambda: B.nvfp4_quantize(x, o, row, col)
+        work, unit = r * c * 5.125 / 1e9, "GB/s"
+    for _ in range(args.warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    B.nvfp4_device_status()
+    ms = e0.elapsed_time(e1) / args.steps
+    print(json.dumps({"case": args.case, "shape": [r, c, k], "ms": ms, "value": work / (ms * 1e-3), "unit": unit}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--case", default=None, choices=sorted(CASES), help="run one kernel on a reduced shape")
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.case:
+        run_case(args)
+    elif args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()
