@@ -93,8 +93,10 @@ nvfp4_status gemm_impl(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D, in
   g.d = D; g.ldd = ldd;
   g.M = (int)M; g.N = (int)N; g.K = (int)K;
   g.d_is_fp32 = d_is_fp32 != 0; g.accumulate = accumulate != 0;
+  // 128 x 256 tiles hold one accumulator (the epilogue is exposed), 128 x 128 tiles two (it overlaps the next
+  // tile's main loop): the wide tile pays off once the main loop is long enough to amortise the epilogue
   int tile_n = g_tile_n.load(std::memory_order_relaxed);
-  if (tile_n != 128 && tile_n != 256) tile_n = 256;
+  if (tile_n != 128 && tile_n != 256) tile_n = (K >= (d_is_fp32 ? 16384 : 8192)) ? 256 : 128;
   if (launch_gemm(g, A->codes, B->codes, tile_n, s) != cudaSuccess) return NVFP4_ERR_CUDA;
   return NVFP4_OK;
 }

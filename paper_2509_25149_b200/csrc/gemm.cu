@@ -4,9 +4,11 @@
 //
 // Persistent, warp-specialised kernel, one CTA per SM:
 //   warp 0   producer: TMA loads of the code tiles (128-byte swizzle) and bulk copies of the scale atoms
-//   warp 1   MMA issuer: tcgen05.cp of the scale atoms into tensor memory, tcgen05.mma
-//            kind::mxf4nvf4.block_scale.scale_vec::4X (M 128, N = BN, K 64 per instruction)
-//   warps 2-5 epilogue: tcgen05.ld of the FP32 accumulator, alpha, conversion, global stores
+//   warp 1   MMA issuer: tcgen05.mma kind::mxf4nvf4.block_scale.scale_vec::4X (M 128, N = BN, K 64 per
+//            instruction), accumulator in tensor memory
+//   warp 2   scale-atom copier: tcgen05.cp of the E4M3 atoms shared -> tensor memory (its own warp because
+//            instruction issue by a single thread, not the tensor pipe, was the bottleneck with both in one)
+//   warps 3-6 epilogue: tcgen05.ld of the FP32 accumulator, alpha, conversion, global stores
 // Every wait is bounded: when one expires the kernel records a code in a device status word, every role
 // leaves its loop, tensor memory is released and the kernel returns.
 #include <cuda.h>
@@ -24,7 +26,7 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK_BYTES = 128;           // bytes of codes per row per stage = 256 elements of K
 constexpr int BK = 256;
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
 constexpr uint32_t kTmemCols = 512;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
@@ -40,11 +42,11 @@ struct Cfg {
   static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
   // tensor memory columns
   static constexpr int kAccCol = 0;
-  static constexpr int kSfCol = kAccStages * BN;            // two buffers of (SFA 16 + SFB 4*BN/32) columns
+  static constexpr int kSfCol = kAccStages * BN;            // one slot of (SFA 16 + SFB 4*BN/32) columns per stage
   static constexpr int kSfaCols = 16;
   static constexpr int kSfbCols = 4 * (BN / 32);
   static constexpr int kSfBufCols = kSfaCols + kSfbCols;
-  static_assert(kSfCol + 2 * kSfBufCols <= 512, "tensor memory budget");
+  static_assert(kSfCol + kStages * kSfBufCols <= 512, "tensor memory budget");
 };
 
 // ------------------------------------------------------------------------------------- PTX ----
@@ -138,18 +140,15 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Shared-memory matrix descriptors (sm_100 format: version field = 1).
+// Shared-memory matrix descriptors (sm_100 format: version field = 1), built from 32-bit halves.
 //   operands: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart
 //   scale atoms: K-major, no swizzle, 8-row groups of 16-byte rows 128 bytes apart
-__device__ __forceinline__ uint64_t desc_operand(uint32_t saddr) {
-  uint64_t lo = ((saddr >> 4) & 0x3fffu) | (1u << 16);
-  uint64_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-  return lo | (hi << 32);
-}
-__device__ __forceinline__ uint64_t desc_sf(uint32_t saddr) {
-  uint64_t lo = ((saddr >> 4) & 0x3fffu);
-  uint64_t hi = (128u >> 4) | (1u << 14);
-  return lo | (hi << 32);
+constexpr uint32_t kDescHiOperand = (1024u >> 4) | (1u << 14) | (2u << 29);
+constexpr uint32_t kDescHiSf = (128u >> 4) | (1u << 14);
+__device__ __forceinline__ uint64_t make_desc(uint32_t lo, uint32_t hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
 }
 
 template <int BN>
@@ -169,12 +168,13 @@ __global__ void __launch_bounds__(kThreads, 1)
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   // barriers live after the stages
   const uint32_t bar_base = base + C::kStages * C::kStageBytes;
-  auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (C::kStages + s); };
-  auto accf_bar = [&](int s) { return bar_base + 8u * (2 * C::kStages + s); };
-  auto acce_bar = [&](int s) { return bar_base + 8u * (2 * C::kStages + C::kAccStages + s); };
-  volatile uint32_t* tmem_slot =
-      reinterpret_cast<volatile uint32_t*>(base_ptr + C::kStages * C::kStageBytes + 8 * (2 * C::kStages + 2 * C::kAccStages));
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };                      // operands + scale atoms landed
+  auto sff_bar = [&](int s) { return bar_base + 8u * (C::kStages + s); };        // scale atoms are in tensor memory
+  auto empty_bar = [&](int s) { return bar_base + 8u * (2 * C::kStages + s); };  // MMAs have consumed the stage
+  auto accf_bar = [&](int s) { return bar_base + 8u * (3 * C::kStages + s); };
+  auto acce_bar = [&](int s) { return bar_base + 8u * (3 * C::kStages + C::kAccStages + s); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(
+      base_ptr + C::kStages * C::kStageBytes + 8 * (3 * C::kStages + 2 * C::kAccStages));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -186,6 +186,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(full_bar(s), 1);
+      mbar_init(sff_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
     for (int s = 0; s < C::kAccStages; ++s) {
@@ -215,20 +216,51 @@ __global__ void __launch_bounds__(kThreads, 1)
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const int m_blk = tile % tiles_m, n_blk = tile / tiles_m;
+        const uint8_t* sfa = g.sfa + (int64_t)m_blk * sf_atoms_per_row_group * 512;
+        const uint8_t* sfb = g.sfb + (int64_t)n_blk * (BN / 128) * sf_atoms_per_row_group * 512;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x100u + stage))) break;
           const uint32_t st = base + stage * C::kStageBytes;
-          mbar_expect_tx(full_bar(stage), C::kABytes + C::kBBytes + C::kSfaBytes + C::kSfbBytes);
+          mbar_expect_tx(full_bar(stage), C::kStageBytes);
           tma_load_2d(st, &map_a, kb * BK_BYTES, m_blk * BM, full_bar(stage));
           tma_load_2d(st + C::kABytes, &map_b, kb * BK_BYTES, n_blk * BN, full_bar(stage));
-          bulk_load(st + C::kABytes + C::kBBytes,
-                    g.sfa + ((int64_t)m_blk * sf_atoms_per_row_group + (int64_t)kb * 4) * 512, C::kSfaBytes,
-                    full_bar(stage));
+          bulk_load(st + C::kABytes + C::kBBytes, sfa + (int64_t)kb * 2048, C::kSfaBytes, full_bar(stage));
 #pragma unroll
           for (int grp = 0; grp < BN / 128; ++grp)
             bulk_load(st + C::kABytes + C::kBBytes + C::kSfaBytes + grp * 2048,
-                      g.sfb + ((int64_t)(n_blk * (BN / 128) + grp) * sf_atoms_per_row_group + (int64_t)kb * 4) * 512,
-                      2048, full_bar(stage));
+                      sfb + ((int64_t)grp * sf_atoms_per_row_group + (int64_t)kb * 4) * 512, 2048, full_bar(stage));
+          if (++stage == C::kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------- scale atoms: shared -> tensor memory ----
+    // SFA of K64-step j goes to columns [4j, 4j+4) of the stage's slot; SFB of step j to
+    // [16 + j*BN/32, ...), 4 columns per 128 rows of B.  The slot of a stage is free again when the
+    // stage's operands are (empty -> producer -> full), so no extra barrier guards it.
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      const uint32_t sf_lo0 = (base + C::kABytes + C::kBBytes) >> 4;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, 0x500u + stage))) break;
+          tc_fence_after();
+          const uint32_t lo = sf_lo0 + stage * (C::kStageBytes >> 4);
+          const uint32_t sf_t = tmem + C::kSfCol + stage * C::kSfBufCols;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            tc_cp_sf(sf_t + j * 4, make_desc(lo + j * 32, kDescHiSf));
+#pragma unroll
+            for (int grp = 0; grp < BN / 128; ++grp)
+              tc_cp_sf(sf_t + C::kSfaCols + j * (BN / 32) + grp * 4,
+                       make_desc(lo + (C::kSfaBytes >> 4) + grp * 128 + j * 32, kDescHiSf));
+          }
+          tc_commit(sff_bar(stage));
           if (++stage == C::kStages) {
             stage = 0;
             phase ^= 1u;
@@ -240,38 +272,28 @@ __global__ void __launch_bounds__(kThreads, 1)
     // ---------------------------------------------------------------- MMA issuer ----
     if (lane == 0) {
       int stage = 0, acc = 0;
-      uint32_t phase = 0, acc_phase = 0, sfbuf = 0;
+      uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
       constexpr uint32_t idesc = instr_desc<BN>();
+      const uint32_t a_lo0 = ((base >> 4) & 0x3fffu) | (1u << 16);
+      const uint32_t b_lo0 = (((base + C::kABytes) >> 4) & 0x3fffu) | (1u << 16);
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         if (!(ok = mbar_wait(acce_bar(acc), acc_phase ^ 1u, abort_flag, 0x300u + acc))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem + C::kAccCol + acc * BN;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, 0x200u + stage))) break;
+          if (!(ok = mbar_wait(sff_bar(stage), phase, abort_flag, 0x200u + stage))) break;
           tc_fence_after();
-          const uint32_t st = base + stage * C::kStageBytes;
-          const uint32_t sf_t = tmem + C::kSfCol + sfbuf * C::kSfBufCols;
-          // scale atoms -> tensor memory: SFA of K64-step j in columns [4j, 4j+4); SFB of step j in
-          // columns [16 + j*BN/32, ...), 4 columns per 128 rows of B
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            tc_cp_sf(sf_t + j * 4, desc_sf(st + C::kABytes + C::kBBytes + j * 512));
-#pragma unroll
-            for (int grp = 0; grp < BN / 128; ++grp)
-              tc_cp_sf(sf_t + C::kSfaCols + j * (BN / 32) + grp * 4,
-                       desc_sf(st + C::kABytes + C::kBBytes + C::kSfaBytes + grp * 2048 + j * 512));
-          }
-          const uint64_t adesc = desc_operand(st);
-          const uint64_t bdesc = desc_operand(st + C::kABytes);
+          const uint32_t a_lo = a_lo0 + stage * (C::kStageBytes >> 4);
+          const uint32_t b_lo = b_lo0 + stage * (C::kStageBytes >> 4);
+          const uint32_t sf_t = tmem + C::kSfCol + stage * C::kSfBufCols;
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             // advancing 64 elements of K = 32 bytes inside the 128-byte swizzle span: +2 in the address field
-            tc_mma_nvf4(d_tmem, adesc + 2u * j, bdesc + 2u * j, idesc, sf_t + j * 4,
-                        sf_t + C::kSfaCols + j * (BN / 32), (kb > 0 || j > 0) ? 1u : 0u);
+            tc_mma_nvf4(d_tmem, make_desc(a_lo + 2 * j, kDescHiOperand), make_desc(b_lo + 2 * j, kDescHiOperand), idesc,
+                        sf_t + j * 4, sf_t + C::kSfaCols + j * (BN / 32), (kb > 0 || j > 0) ? 1u : 0u);
           }
           tc_commit(empty_bar(stage));  // frees the stage once the MMAs above have read it
-          sfbuf ^= 1u;
           if (++stage == C::kStages) {
             stage = 0;
             phase ^= 1u;
@@ -285,7 +307,7 @@ __global__ void __launch_bounds__(kThreads, 1)
         }
       }
     }
-  } else {
+  } else if (warp >= 3) {
     // ------------------------------------------------------------------ epilogue ----
     const int quad = warp & 3;  // the 32 tensor-memory lanes this warp may read
     int acc = 0;
