@@ -61,18 +61,27 @@ __device__ __forceinline__ uint32_t e2m1x8_rne(const float v[8]) {
   return r;
 }
 
-// Stochastic rounding of one scaled value to an E2M1 nibble (Section 4.4): neighbours lo <= |v| < hi on
-// the grid {0,.5,1,1.5,2,3,4,6}; round up iff u + 0.5 < 256 * frac.  All steps are exact in fp32.
-__device__ __forceinline__ uint32_t e2m1_sr(float v, uint32_t u) {
-  uint32_t sign = (__float_as_uint(v) >> 28) & 8u;
-  float a = fminf(fabsf(v), 6.0f);
-  float scale = (a < 2.0f) ? 2.0f : ((a < 4.0f) ? 1.0f : 0.5f);
-  uint32_t off = (a < 2.0f) ? 0u : ((a < 4.0f) ? 2u : 4u);
-  float p = a * scale;               // position in units of the local step
-  float fl = floorf(p);
-  float frac = p - fl;
-  uint32_t up = ((float)u + 0.5f < 256.0f * frac) ? 1u : 0u;
-  return sign | ((uint32_t)fl + off + up);
+// Stochastic rounding of one scaled value to an E2M1 nibble (Section 4.4): neighbours lo <= |v| < hi on the
+// grid {0,.5,1,1.5,2,3,4,6}; round up iff u + 0.5 < 256 * frac, u the element's 8-bit draw.
+//
+// Integer form of that rule.  For 1 <= a <= 6 the binary32 pattern of a is (exponent, one kept mantissa bit,
+// 22 discarded bits m22) and frac = m22 / 2^22, so "round up" <=> m22 > (u << 14) + 2^13 <=> adding
+// D = ((255 - u) << 14) + 0x1FFF carries out of the discarded bits; (bits + D) >> 22 is then
+// 2 * exponent + mantissa bit = code + 252.  Below 1 the grid is uniform (step 0.5): x = a + 1 rounded UP has
+// mantissa ceil(a * 2^23), the comparison with the integer threshold survives the ceiling, and the same carry
+// trick on x gives code + 254.  `nu` is the complemented draw (255 - u) in bits [0, 8).
+__device__ __forceinline__ uint32_t e2m1_sr_bits(float v, uint32_t nu_shifted14) {
+  // nu_shifted14: (255 - u) << 14, other bits zero
+  const float a = fminf(fabsf(v), 6.0f);
+  const bool small = a < 1.0f;
+  const float x = small ? __fadd_ru(a, 1.0f) : a;
+  // + (4 << 22) makes the low three bits of (.. >> 22) equal code for a >= 1 (252 = -4 mod 8 ... 256 - 252);
+  // the small path needs + (2 << 22) instead
+  uint32_t s = __float_as_uint(x) + (nu_shifted14 | 0x01001FFFu);
+  if (small) s -= 0x00800000u;
+  const uint32_t t = s >> 22;
+  // low three bits from t, sign bit (bit 31 of v) into bit 3
+  return (t & 7u) | ((__float_as_uint(v) >> 28) & 8u);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -82,12 +91,11 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
                                                uint32_t k0, uint32_t k1) {
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-    uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
-    uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
-    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0;  // one wide multiply each
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ (k0 + (uint32_t)r * 0x9E3779B9u);
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ (k1 + (uint32_t)r * 0xBB67AE85u);
+    c0 = n0; c1 = (uint32_t)p1; c2 = n2; c3 = (uint32_t)p0;
   }
   return make_uint4(c0, c1, c2, c3);
 }

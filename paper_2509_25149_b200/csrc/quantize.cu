@@ -196,19 +196,19 @@ __device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, 
     out.x = e2m1x8_rne(lo);
     out.y = e2m1x8_rne(hi);
   } else {
-    uint32_t w0 = 0, w1 = 0;
+    // rnd holds the 16 draws, byte i = element i; work with the complemented bytes
+    uint32_t w[2] = {0u, 0u};
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      uint32_t u = (rnd[i >> 2] >> (8 * (i & 3))) & 0xffu;
-      w0 |= e2m1_sr(__fmul_rn(f[i], s_enc_b), u) << (4 * i);
+    for (int i = 0; i < 16; ++i) {
+      const uint32_t nr = ~rnd[i >> 2];
+      const int b = i & 3;
+      // (255 - u) << 14 : move byte b to bits [14, 22)
+      const uint32_t nu14 = (b == 0 ? (nr << 14) : b == 1 ? (nr << 6) : b == 2 ? (nr >> 2) : (nr >> 10)) & 0x003FC000u;
+      const uint32_t nib = e2m1_sr_bits(__fmul_rn(f[i], s_enc_b), nu14);
+      w[i >> 3] = __funnelshift_r(w[i >> 3], nib, 4);  // shifts the new nibble in from the top
     }
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      uint32_t u = (rnd[2 + (i >> 2)] >> (8 * (i & 3))) & 0xffu;
-      w1 |= e2m1_sr(__fmul_rn(f[8 + i], s_enc_b), u) << (4 * i);
-    }
-    out.x = w0;
-    out.y = w1;
+    out.x = w[0];
+    out.y = w[1];
   }
   return out;
 }
