@@ -161,7 +161,7 @@ def run_cuda(args):
     import torch.distributed as dist
 
     from paper_2509_25149_b200 import binding as B
-    from paper_2509_25149_b200 import synth
+    from paper_2509_25149_b200 import dp, synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -180,7 +180,7 @@ def run_cuda(args):
         p.dY = synth.normal_bf16((M, N), 1e-4, 3003 + 100 * rank)
     hX, hW, hdY = p.X.pin_memory(), p.W.pin_memory(), p.dY.pin_memory()
     X, W, dY = hX.cuda(), hW.cuda(), hdY.cuda()
-    opts = B.quant_opts(rht_sign_mask=p.rht_sign_mask, seed=0, sr_offset=rank << 32)
+    opts = B.quant_opts(rht_sign_mask=p.rht_sign_mask, seed=0, sr_offset=dp.rank_sr_offset(rank))
     X_col, W_row, W_col = B.alloc_tensor(K, M), B.alloc_tensor(N, K), B.alloc_tensor(K, N)
     Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
     dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
@@ -191,8 +191,7 @@ def run_cuda(args):
     def step():
         B.nvfp4_linear_fwd(X, W, opts, Y, X_col, W_row, W_col, False, ws_f)
         B.nvfp4_linear_bwd(dY, X_col, W_col, K, opts, dX, dW, False, ws_b)
-        if world > 1:
-            dist.all_reduce(dW)  # FP32 sum of the weight gradient across data-parallel replicas
+        dp.allreduce_weight_grad(dW)  # FP32 sum of the weight gradient across data-parallel replicas (N > 1)
 
     def barrier():
         if world > 1:
@@ -233,7 +232,7 @@ def run_cuda(args):
     w_opts = B.quant_opts(block_rows=16)
     x_opts = B.quant_opts(rht_colwise=True, rht_sign_mask=p.rht_sign_mask)
     g_opts = B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True, rht_sign_mask=p.rht_sign_mask, seed=0,
-                          sr_offset=rank << 32)
+                          sr_offset=dp.rank_sr_offset(rank))
     calls = [
         ("quant_W", lambda: B.nvfp4_quantize(W, w_opts, W_row, W_col)),
         ("quant_X", lambda: B.nvfp4_quantize(X, x_opts, x_row, X_col)),

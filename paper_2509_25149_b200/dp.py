@@ -1,0 +1,30 @@
+"""Data-parallel plumbing of the NVFP4 linear layer (one process per GPU, torch.distributed).
+
+The path shards by tokens: every rank quantizes its own X / dY shard (own per-tensor amax, own stochastic-rounding
+stream) and runs Fprop, Dgrad, Wgrad locally; the single exchange is the FP32 sum of the weight gradient across
+replicas (paper Section 4.1: weight gradients are accumulated in FP32 across data-parallel replicas).
+"""
+from __future__ import annotations
+
+import torch
+import torch.distributed as dist
+
+
+def rank_sr_offset(rank: int, layer: int = 0) -> int:
+    """Philox counter words 2..3 for a rank: the rank in the high word, the layer index in the low word."""
+    assert 0 <= rank < (1 << 31) and 0 <= layer < (1 << 32)
+    return (rank << 32) | layer
+
+
+def token_shard(total_tokens: int, rank: int, world: int) -> tuple[int, int]:
+    """[begin, end) of the rank's tokens; shards are multiples of 256 tokens (the linear layer's granularity)."""
+    assert total_tokens % (256 * world) == 0, "tokens must split into multiples of 256 per rank"
+    per = total_tokens // world
+    return rank * per, (rank + 1) * per
+
+
+def allreduce_weight_grad(dW: torch.Tensor) -> None:
+    """In-place FP32 sum of dW over all ranks (no-op without an initialised process group)."""
+    assert dW.dtype == torch.float32
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(dW, op=dist.ReduceOp.SUM)

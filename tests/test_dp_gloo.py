@@ -1,0 +1,77 @@
+"""World-size-2 check of the data-parallel plumbing on CPU (gloo): token sharding, per-rank SR streams and the
+FP32 all-reduce of the weight gradient.  The per-rank arithmetic is done by the CPU oracle here; the GPU kernels are
+unchanged by data parallelism."""
+import os
+import socket
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import oracle
+from paper_2509_25149_b200 import dp, synth
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _wgrad(X, dY, rank, mask):
+    xq = oracle.quantize(synth.bits(X), colwise=True, rht=True, sign_mask=mask)
+    gq = oracle.quantize(synth.bits(dY), colwise=True, rht=True, sign_mask=mask, rounding=oracle.SR, seed=0,
+                         sr_offset=dp.rank_sr_offset(rank))
+    return oracle.gemm_tn(oracle.dequantize(gq), oracle.dequantize(xq), want_T=False), gq
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        X = synth.normal_bf16((512, 64), 1.0, 1)
+        dY = synth.normal_bf16((512, 48), 1e-3, 2)
+        b, e = dp.token_shard(512, rank, world)
+        dW_local, _ = _wgrad(X[b:e], dY[b:e], rank, synth.DEFAULT_RHT_SIGN_MASK)
+        dW = torch.from_numpy(dW_local.astype(np.float32))
+        dp.allreduce_weight_grad(dW)
+        # replicated weights quantize to identical bytes on every rank (deterministic RNE)
+        W = synth.normal_bf16((48, 64), 0.02, 3)
+        wq = torch.from_numpy(oracle.quantize(synth.bits(W), block_rows=16).codes.copy())
+        gathered = [torch.empty_like(wq) for _ in range(world)]
+        dist.all_gather(gathered, wq)
+        assert all(torch.equal(g, wq) for g in gathered)
+        if rank == 0:
+            np.save(out, dW.numpy())
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_rank_weight_gradient_allreduce(tmp_path):
+    out = str(tmp_path / "dw.npy")
+    mp.spawn(_worker, args=(2, _free_port(), out), nprocs=2, join=True)
+    got = np.load(out)
+    X = synth.normal_bf16((512, 64), 1.0, 1)
+    dY = synth.normal_bf16((512, 48), 1e-3, 2)
+    parts, streams = [], []
+    for r in range(2):
+        b, e = dp.token_shard(512, r, 2)
+        d, gq = _wgrad(X[b:e], dY[b:e], r, synth.DEFAULT_RHT_SIGN_MASK)
+        parts.append(d.astype(np.float32))
+        streams.append(gq)
+    assert np.allclose(got, parts[0] + parts[1], rtol=1e-6, atol=0)
+    exact = dY.double().numpy().T @ X.double().numpy()
+    assert np.linalg.norm(got - exact) / np.linalg.norm(exact) < 0.3
+    # the two ranks draw from different Philox streams
+    assert dp.rank_sr_offset(0) != dp.rank_sr_offset(1)
+    assert oracle.sr_draw(0, dp.rank_sr_offset(0), 5) != oracle.sr_draw(0, dp.rank_sr_offset(1), 5) or \
+        oracle.sr_draw(0, dp.rank_sr_offset(0), 6) != oracle.sr_draw(0, dp.rank_sr_offset(1), 6)
+
+
+def test_token_shard_and_offsets():
+    assert dp.token_shard(8192, 0, 4) == (0, 2048) and dp.token_shard(8192, 3, 4) == (6144, 8192)
+    assert dp.rank_sr_offset(3, 7) == (3 << 32) | 7
+    t = torch.ones(4)
+    dp.allreduce_weight_grad(t)  # no process group: no-op
+    assert torch.equal(t, torch.ones(4))
