@@ -178,8 +178,10 @@ NVFP4_API nvfp4_status nvfp4_rht16(const void* x_bf16, int64_t rows, int64_t col
  */
 NVFP4_API nvfp4_status nvfp4_device_status(void* cuda_stream, uint32_t* detail);
 
-/* Tuning knob: N extent of the GEMM's CTA tile, 128 or 256 (0 = default).  Returns 0, or -1 for any
- * other value.  Process-wide; results do not depend on it beyond FP32 summation order. */
+/* Tuning knob: which GEMM tiling to use.  128 / 256 = one CTA per 128 x 128 / 128 x 256 output tile;
+ * 512 = a CTA pair per 256 x 256 tile (needs M % 256 == 0 and N % 256 == 0, otherwise 128 is used);
+ * 0 = choose by shape.  Returns 0, or -1 for any other value.  Process-wide; results do not depend on it
+ * beyond FP32 summation order. */
 NVFP4_API int32_t nvfp4_set_gemm_tile_n(int32_t tile_n);
 
 NVFP4_API const char* nvfp4_status_string(nvfp4_status s);

@@ -193,7 +193,7 @@ def nvfp4_device_status() -> int:
 
 def nvfp4_set_gemm_tile_n(tile_n: int) -> None:
     if lib().nvfp4_set_gemm_tile_n(tile_n) != 0:
-        raise ValueError("tile_n must be 0, 128 or 256")
+        raise ValueError("tile_n must be 0, 128, 256 or 512")
 
 
 def nvfp4_launch_count() -> int:

@@ -93,10 +93,17 @@ nvfp4_status gemm_impl(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D, in
   g.d = D; g.ldd = ldd;
   g.M = (int)M; g.N = (int)N; g.K = (int)K;
   g.d_is_fp32 = d_is_fp32 != 0; g.accumulate = accumulate != 0;
-  // 128 x 256 tiles hold one accumulator (the epilogue is exposed), 128 x 128 tiles two (it overlaps the next
-  // tile's main loop): the wide tile pays off once the main loop is long enough to amortise the epilogue
+  // CTA pairs on 256 x 256 tiles whenever the shape allows (half the operand traffic per flop, half the
+  // scale-copy and MMA issue work per SM).  Otherwise one CTA per tile: 128 x 256 tiles hold one accumulator
+  // (exposed epilogue), 128 x 128 tiles two (the epilogue overlaps the next tile), so the wide tile pays off
+  // once the main loop is long enough to amortise the epilogue.
   int tile_n = g_tile_n.load(std::memory_order_relaxed);
-  if (tile_n != 128 && tile_n != 256) tile_n = (K >= (d_is_fp32 ? 16384 : 8192)) ? 256 : 128;
+  if (tile_n != 128 && tile_n != 256 && tile_n != 512) {
+    if (M % 256 == 0 && N % 256 == 0)
+      tile_n = 512;
+    else
+      tile_n = (K >= (d_is_fp32 ? 16384 : 8192)) ? 256 : 128;
+  }
   if (launch_gemm(g, A->codes, B->codes, tile_n, s) != cudaSuccess) return NVFP4_ERR_CUDA;
   return NVFP4_OK;
 }
@@ -229,7 +236,7 @@ nvfp4_status nvfp4_device_status(void* cuda_stream, uint32_t* detail) {
 }
 
 int32_t nvfp4_set_gemm_tile_n(int32_t tile_n) {
-  if (tile_n != 0 && tile_n != 128 && tile_n != 256) return -1;
+  if (tile_n != 0 && tile_n != 128 && tile_n != 256 && tile_n != 512) return -1;
   g_tile_n.store(tile_n, std::memory_order_relaxed);
   return 0;
 }

@@ -16,10 +16,37 @@
 
 #include "common.cuh"
 #include "gemm.h"
+#include "tc_ptx.cuh"
+#include "gemm_2cta.cuh"
 
 namespace nvfp4 {
 
-__device__ unsigned int g_device_status = 0;  // 0 = fine; else the code of the first wait that expired
+EncodeTiledFn tensor_map_encoder() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dtype, int elem_bytes, const void* base, uint64_t inner_elems,
+                 uint64_t rows, uint64_t row_pitch_bytes, uint32_t box_inner, uint32_t box_rows, bool swizzle128) {
+  EncodeTiledFn fn = tensor_map_encoder();
+  if (!fn) return false;
+  (void)elem_bytes;
+  cuuint64_t dims[2] = {inner_elems, rows};
+  cuuint64_t strides[1] = {row_pitch_bytes};
+  cuuint32_t box[2] = {box_inner, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, dtype, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 namespace {
 
@@ -28,7 +55,6 @@ constexpr int BK_BYTES = 128;           // bytes of codes per row per stage = 25
 constexpr int BK = 256;
 constexpr int kThreads = 224;
 constexpr uint32_t kTmemCols = 512;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 template <int BN>
 struct Cfg {
@@ -48,114 +74,6 @@ struct Cfg {
   static constexpr int kSfBufCols = kSfaCols + kSfbCols;
   static_assert(kSfCol + kStages * kSfBufCols <= 512, "tensor memory budget");
 };
-
-// ------------------------------------------------------------------------------------- PTX ----
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Bounded wait.  Returns false when the wait expired or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t code) {
-  if (mbar_try(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer_ns();
-  uint32_t spins = 0;
-  while (true) {
-    if (mbar_try(bar, parity)) return true;
-    if ((++spins & 63u) == 0u) {
-      if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
-        *abort_flag = code;
-        atomicCAS(&g_device_status, 0u, code);
-        return false;
-      }
-    }
-  }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
-  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
-}
-__device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %6, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,"
-      "%28,%29,%30,%31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptors (sm_100 format: version field = 1), built from 32-bit halves.
-//   operands: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart
-//   scale atoms: K-major, no swizzle, 8-row groups of 16-byte rows 128 bytes apart
-constexpr uint32_t kDescHiOperand = (1024u >> 4) | (1u << 14) | (2u << 29);
-constexpr uint32_t kDescHiSf = (128u >> 4) | (1u << 14);
-__device__ __forceinline__ uint64_t make_desc(uint32_t lo, uint32_t hi) {
-  uint64_t d;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
-  return d;
-}
-
-template <int BN>
-__device__ __forceinline__ constexpr uint32_t instr_desc() {
-  // E2M1 x E2M1 (format id 1 in the mxf4 kinds), K-major both, UE4M3 scales, dense K64
-  return (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (0u << 23) | ((uint32_t)(BM >> 4) << 24);
-}
 
 // ------------------------------------------------------------------------------------ kernel ----
 template <int BN>
@@ -274,7 +192,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      constexpr uint32_t idesc = instr_desc<BN>();
+      constexpr uint32_t idesc = instr_desc_nvf4(BM, BN);
       const uint32_t a_lo0 = ((base >> 4) & 0x3fffu) | (1u << 16);
       const uint32_t b_lo0 = (((base + C::kABytes) >> 4) & 0x3fffu) | (1u << 16);
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -379,34 +297,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 }
 
 // ------------------------------------------------------------------------------- host side ----
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
 // codes [rows][k_bytes] uint8, box = 128 bytes x box_rows, 128-byte swizzle
 bool make_code_map(CUtensorMap* map, const void* codes, int64_t rows, int64_t k_bytes, int box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)k_bytes, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)k_bytes};
-  cuuint32_t box[2] = {(cuuint32_t)BK_BYTES, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(codes), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return make_map_2d(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, (uint64_t)k_bytes, (uint64_t)rows, (uint64_t)k_bytes,
+                     BK_BYTES, (uint32_t)box_rows, true);
 }
 
 template <int BN>
@@ -429,6 +323,35 @@ cudaError_t launch_t(const GemmArgs& g, const void* a_codes, const void* b_codes
   return cudaGetLastError();
 }
 
+cudaError_t launch_pair(const GemmArgs& g, const void* a_codes, const void* b_codes, int num_sms, cudaStream_t s) {
+  CUtensorMap map_a, map_b, map_sfa, map_sfb, map_d;
+  const uint64_t atoms_a = (uint64_t)(g.M / 128) * (g.K / 64), atoms_b = (uint64_t)(g.N / 128) * (g.K / 64);
+  bool ok = make_code_map(&map_a, a_codes, g.M, g.K / 2, 128) && make_code_map(&map_b, b_codes, g.N, g.K / 2, 128) &&
+            make_map_2d(&map_sfa, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, g.sfa, 128, atoms_a, 512, 128, 4, false) &&
+            make_map_2d(&map_sfb, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, g.sfb, 128, atoms_b, 512, 128, 4, false);
+  if (g.d_is_fp32)
+    ok = ok && make_map_2d(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g.d, (uint64_t)g.N, (uint64_t)g.M,
+                           (uint64_t)g.ldd * 4, 32, 128, true);
+  else
+    ok = ok && make_map_2d(&map_d, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, g.d, (uint64_t)g.N, (uint64_t)g.M,
+                           (uint64_t)g.ldd * 2, 64, 128, true);
+  if (!ok) return cudaErrorInvalidValue;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(pair::gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         pair::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int n_tiles = (g.M / 256) * (g.N / 256);
+  const int max_pairs = num_sms / 2;
+  const int pairs = n_tiles < max_pairs ? n_tiles : max_pairs;
+  pair::Args a{g.M, g.N, g.K, g.a_global, g.b_global, g.d_is_fp32, g.accumulate};
+  pair::gemm_pair_kernel<<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, a);
+  count_launch();
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_codes, int tile_n, cudaStream_t s) {
@@ -440,6 +363,7 @@ cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_co
     e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
   }
+  if (tile_n == 512 && g.M % 256 == 0 && g.N % 256 == 0) return launch_pair(g, a_codes, b_codes, num_sms, s);
   if (tile_n == 256 && g.N % 256 == 0) return launch_t<256>(g, a_codes, b_codes, num_sms, s);
   return launch_t<128>(g, a_codes, b_codes, num_sms, s);
 }

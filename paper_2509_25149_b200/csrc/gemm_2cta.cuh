@@ -1,0 +1,413 @@
+// Block-scaled NVFP4 GEMM on CTA pairs (tcgen05 cta_group::2): a cluster of two CTAs on one TPC computes a
+// 256 x 256 output tile.  Each CTA keeps its own 128 rows of A, HALF of the B tile (128 of its 256 rows) and the
+// accumulator of its 128 output rows in its own tensor memory; the pair's tensor cores exchange the B halves, so
+// every byte of B is fetched from L2 and read from shared memory once per pair.  That halving of the operand
+// traffic per flop is the point: the one-CTA kernel is bound by shared-memory bandwidth, not by the tensor pipe.
+//
+// Roles per CTA (7 warps): 0 TMA producer (both CTAs; every load signals the LEADER's "full" barrier),
+// 1 MMA issuer (leader only; allocates tensor memory in both), 2 scale-atom copier (leader only; cta_group::2
+// copies run in both CTAs from their own shared memory), 3-10 epilogue (both; two groups of four warps, one per
+// 128-column half: tensor memory -> registers -> swizzled staging -> TMA store; the accumulator is released as
+// soon as it has been read).
+// Included by gemm.cu only.
+#pragma once
+
+#include <cuda_bf16.h>
+
+#include "gemm.h"
+#include "tc_ptx.cuh"
+
+namespace nvfp4 {
+namespace pair {
+
+constexpr int kThreads = 448;      // producer, MMA, 2 x 4 epilogue warps, 4 scale-copy warps (2, 11, 12, 13)      // producer, MMA, scale copier, 2 x 4 epilogue warps
+constexpr int kStages = 4;
+constexpr int kABytes = 128 * 128;   // 128 rows x 256 K elements
+constexpr int kBBytes = 128 * 128;   // this CTA's half of the 256-row B tile
+constexpr int kSfaBytes = 4 * 512;   // own 128 rows, four K64 steps
+constexpr int kSfbBytes = 8 * 512;   // all 256 rows of B (both CTAs need them), four K64 steps
+constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 38 KB
+constexpr int kStagingBytes = 4 * 16384;  // two 128 x 128-byte store buffers per epilogue group
+constexpr int kSmemBytes = kStages * kStageBytes + kStagingBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+constexpr uint32_t kTmemCols = 512;
+constexpr int kSfCol = 256;          // after the 256 accumulator columns: one 48-column slot per stage
+constexpr int kSfSlotCols = 48;      // SFA 4 x 4, SFB 4 x 8
+static_assert(kSfCol + kStages * kSfSlotCols <= 512, "tensor memory budget");
+static_assert(kStageBytes % 1024 == 0, "stages must keep the 1024-byte swizzle alignment");
+
+struct Args {
+  int M, N, K;
+  const float* a_global;
+  const float* b_global;
+  int d_is_fp32, accumulate;
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  // default semantics: the explicitly cluster-scoped release form costs ~0.5 us per call on this part, and the
+  // tensor-memory accesses this arrival orders are already fenced with tcgen05.fence::before_thread_sync
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// bounded wait with cluster-scope acquire (the barrier receives arrivals from the peer CTA)
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                  uint32_t code) {
+  if (mbar_try_cluster(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (true) {
+    if (mbar_try_cluster(bar, parity)) return true;
+    if ((++spins & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = code;
+        atomicCAS(&g_device_status, 0u, code);
+        return false;
+      }
+    }
+  }
+}
+
+// pair-aware TMA load: the data lands in this CTA's shared memory, the bytes are counted on `bar`, which may be
+// the peer's barrier (cluster address)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x), "r"(y),
+               "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map),
+               "r"(x), "r"(y), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_all() {
+  asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ void tc2_commit_local(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// arrives on the barrier at the same offset in every CTA of `mask` once all earlier tcgen05 operations of the
+// issuing thread have completed
+__device__ __forceinline__ void tc2_commit_both(uint32_t bar, uint16_t mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask)
+               : "memory");
+}
+__device__ __forceinline__ void tc2_cp_sf(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc2_mma_nvf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
+      : "memory");
+}
+
+// Epilogue helper: 128 accumulator columns of one row per thread (registers) -> alpha, conversion -> 128-byte
+// swizzled rows of a staging buffer -> TMA store (or reduce-add) of 128 x 128-byte boxes.  Two staging buffers
+// alternate; a buffer is rewritten only after the store issued two boxes earlier has finished reading it.
+template <bool FP32>
+__device__ __forceinline__ void store_half(const uint32_t (&r)[128], float alpha, int et, int bar_id, int row_in_tile,
+                                           uint32_t stage_buf, int& buf, const CUtensorMap* map_d, int x0, int row0,
+                                           int accumulate) {
+  constexpr int kChunks = FP32 ? 4 : 2;
+  constexpr int kChunkCols = FP32 ? 32 : 64;
+#pragma unroll
+  for (int c = 0; c < kChunks; ++c) {
+    if (et == 0) bulk_wait_read<1>();
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+    const uint32_t srow = stage_buf + buf * 16384 + row_in_tile * 128;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      uint32_t p[4];
+      if (FP32) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) p[e] = __float_as_uint(__uint_as_float(r[c * 32 + 4 * j + e]) * alpha);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[c * 64 + 8 * j + 2 * e]) * alpha,
+                                                   __uint_as_float(r[c * 64 + 8 * j + 2 * e + 1]) * alpha);
+          p[e] = *reinterpret_cast<uint32_t*>(&h);
+        }
+      }
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(srow + ((j ^ (row_in_tile & 7)) << 4)), "r"(p[0]),
+                   "r"(p[1]), "r"(p[2]), "r"(p[3])
+                   : "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+    if (et == 0) {
+      if (accumulate)
+        tma_reduce_add_2d(map_d, x0 + c * kChunkCols, row0, stage_buf + buf * 16384);
+      else
+        tma_store_2d(map_d, x0 + c * kChunkCols, row0, stage_buf + buf * 16384);
+      bulk_commit();
+    }
+    buf ^= 1;
+  }
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+    gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                     const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
+                     const __grid_constant__ CUtensorMap map_d, const Args g) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t staging = base + kStages * kStageBytes;
+  const uint32_t bar_base = staging + kStagingBytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };                  // used in the leader only
+  auto sff_bar = [&](int s) { return bar_base + 8u * (kStages + s); };       // leader only
+  auto empty_bar = [&](int s) { return bar_base + 8u * (2 * kStages + s); }; // one per CTA
+  const uint32_t accf_bar = bar_base + 8u * (3 * kStages);                   // one per CTA
+  const uint32_t acce_bar = bar_base + 8u * (3 * kStages + 1);               // leader only, 16 arrivals
+  const uint32_t done_bar = bar_base + 8u * (3 * kStages + 2);               // one per CTA, peer arrives
+  volatile uint32_t* tmem_slot =
+      reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + kStagingBytes + 8 * (3 * kStages + 3));
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();  // 0 = leader
+  const bool leader = rank == 0;
+  const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int tiles_m = g.M / 256, tiles_n = g.N / 256;
+  const int n_tiles = tiles_m * tiles_n;
+  const int k_blocks = g.K / 256;
+  const int sf_atoms_k = g.K / 64;  // atoms along K per 128-row group
+  // Tile order: groups of kGroupM row-blocks sweep all column-blocks before the next group starts, so the
+  // group's rows of A and all of B stay in L2 while they are reused.
+  constexpr int kGroupM = 8;
+  auto tile_coords = [&](int tile, int& m_blk, int& n_blk) {
+    const int per_group = kGroupM * tiles_n;
+    const int grp = tile / per_group, in_grp = tile - grp * per_group;
+    const int m0 = grp * kGroupM;
+    const int gm = (tiles_m - m0 < kGroupM) ? (tiles_m - m0) : kGroupM;
+    m_blk = m0 + in_grp % gm;
+    n_blk = in_grp / gm;
+  };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 2);   // one arrive.expect_tx from each CTA's producer
+      mbar_init(sff_bar(s), 4);    // one commit from each scale-copy warp
+      mbar_init(empty_bar(s), 1);
+    }
+    mbar_init(accf_bar, 1);
+    mbar_init(acce_bar, 16);       // eight epilogue warps in each CTA
+    mbar_init(done_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // both CTAs' barriers are initialised before any remote signal
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer ----
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = pair_id; tile < n_tiles && ok; tile += n_pairs) {
+        int m_blk, n_blk;
+        tile_coords(tile, m_blk, n_blk);
+        const int row_a = m_blk * 256 + (int)rank * 128;       // this CTA's A rows
+        const int row_b = n_blk * 256 + (int)rank * 128;       // this CTA's half of the B tile
+        const int atom_a = (m_blk * 2 + (int)rank) * sf_atoms_k;
+        const int atom_b = (n_blk * 2) * sf_atoms_k;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x100u + stage))) break;
+          const uint32_t st = base + stage * kStageBytes;
+          const uint32_t bar = map_to_cta(full_bar(stage), 0);  // the leader's barrier counts both CTAs' bytes
+          mbar_expect_tx_cluster(bar, kStageBytes);
+          tma_load_2d_pair(st, &map_a, kb * 128, row_a, bar);
+          tma_load_2d_pair(st + kABytes, &map_b, kb * 128, row_b, bar);
+          tma_load_2d_pair(st + kABytes + kBBytes, &map_sfa, 0, atom_a + kb * 4, bar);
+          tma_load_2d_pair(st + kABytes + kBBytes + kSfaBytes, &map_sfb, 0, atom_b + kb * 4, bar);
+          tma_load_2d_pair(st + kABytes + kBBytes + kSfaBytes + 2048, &map_sfb, 0, atom_b + sf_atoms_k + kb * 4, bar);
+          if (++stage == kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+    }
+  } else if (warp == 2 || warp >= 11) {
+    // ------------------------------------------- scale atoms: shared -> tensor memory (both CTAs) ----
+    if (leader && lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      const uint32_t sf_lo0 = (base + kABytes + kBBytes) >> 4;
+      for (int tile = pair_id; tile < n_tiles && ok; tile += n_pairs) {
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!(ok = mbar_wait_cluster(full_bar(stage), phase, abort_flag, 0x500u + stage))) break;
+          tc_fence_after();
+          const uint32_t lo = sf_lo0 + stage * (kStageBytes >> 4);
+          const uint32_t sf_t = tmem + kSfCol + stage * kSfSlotCols;
+          {
+            // this warp copies the atoms of K64-step j: SFA (own 128 rows) and both 128-row groups of SFB
+            const int j = (warp == 2) ? 0 : warp - 10;
+            tc2_cp_sf(sf_t + j * 4, make_desc(lo + j * 32, kDescHiSf));
+            tc2_cp_sf(sf_t + 16 + j * 8, make_desc(lo + (kSfaBytes >> 4) + j * 32, kDescHiSf));
+            tc2_cp_sf(sf_t + 16 + j * 8 + 4, make_desc(lo + (kSfaBytes >> 4) + 128 + j * 32, kDescHiSf));
+          }
+          tc2_commit_local(sff_bar(stage));
+          if (++stage == kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer (leader) ----
+    if (leader && lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      constexpr uint32_t idesc = instr_desc_nvf4(256, 256);
+      const uint32_t a_lo0 = ((base >> 4) & 0x3fffu) | (1u << 16);
+      const uint32_t b_lo0 = (((base + kABytes) >> 4) & 0x3fffu) | (1u << 16);
+      for (int tile = pair_id; tile < n_tiles && ok; tile += n_pairs) {
+        if (!(ok = mbar_wait_cluster(acce_bar, acc_phase ^ 1u, abort_flag, 0x300u))) break;
+        tc_fence_after();
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!(ok = mbar_wait(sff_bar(stage), phase, abort_flag, 0x200u + stage))) break;
+          tc_fence_after();
+          const uint32_t a_lo = a_lo0 + stage * (kStageBytes >> 4);
+          const uint32_t b_lo = b_lo0 + stage * (kStageBytes >> 4);
+          const uint32_t sf_t = tmem + kSfCol + stage * kSfSlotCols;
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            tc2_mma_nvf4(tmem, make_desc(a_lo + 2 * j, kDescHiOperand), make_desc(b_lo + 2 * j, kDescHiOperand), idesc,
+                         sf_t + j * 4, sf_t + 16 + j * 8, (kb > 0 || j > 0) ? 1u : 0u);
+          tc2_commit_both(empty_bar(stage), 3);  // both CTAs' stages are free once these MMAs have read them
+          if (++stage == kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        if (!ok) break;
+        tc2_commit_both(accf_bar, 3);  // accumulators of both CTAs complete
+        acc_phase ^= 1u;
+      }
+    }
+  } else if (warp >= 3 && warp <= 10) {
+    // ------------------------------------------------------------------ epilogue ----
+    // Two groups of four warps; group h drains columns [128h, 128h + 128) of the accumulator through its own
+    // pair of staging buffers, so the two halves leave tensor memory concurrently.
+    const int quad = warp & 3;              // tensor-memory lanes this warp may read
+    const int half = (warp - 3) >> 2;       // column half / epilogue group
+    const int et = (threadIdx.x - 96) & 127;  // 0..127 inside the group
+    const int bar_id = 1 + half;
+    uint32_t acc_phase = 0;
+    const float alpha = __fmul_rn(g.a_global[1], g.b_global[1]);
+    const uint32_t acce_leader = map_to_cta(acce_bar, 0);
+    const int row_in_tile = quad * 32 + lane;
+    const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + half * 128;
+    const uint32_t stage_buf = staging + half * 32768;
+    int buf = 0;
+    for (int tile = pair_id; tile < n_tiles; tile += n_pairs) {
+      int m_blk, n_blk;
+      tile_coords(tile, m_blk, n_blk);
+      mbar_wait_cluster(accf_bar, acc_phase, abort_flag, 0x400u);
+      // agree on giving up: a warp that timed out still joins this barrier, then everyone reads the flag
+      asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+      if (*abort_flag) break;
+      tc_fence_after();
+      const int row0 = m_blk * 256 + (int)rank * 128;
+      // read this warp's 32 lanes x 128 columns in one go and hand the accumulator back at once: the MMA issuer
+      // can start the next tile while the values are converted and stored from registers
+      uint32_t r[128];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) tc_ld32(t_row + q * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[q * 32]));
+      tc_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(acce_leader);
+      if (g.d_is_fp32)
+        store_half<true>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, &map_d, n_blk * 256 + half * 128, row0,
+                         g.accumulate);
+      else
+        store_half<false>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, &map_d, n_blk * 256 + half * 128, row0,
+                          g.accumulate);
+      acc_phase ^= 1u;
+    }
+    if (et == 0) bulk_wait_all<0>();  // all stores have left shared memory and are visible
+  }
+
+  // ------------------------------------------------------------------ teardown ----
+  // Neither CTA may leave while the other can still signal its barriers or read its shared memory: each tells
+  // the peer it is done and waits (bounded) for the peer's word.
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    mbar_arrive_cluster(map_to_cta(done_bar, rank ^ 1u));
+    mbar_wait_cluster(done_bar, 0, abort_flag, 0x600u);
+  }
+  __syncthreads();
+  if (*abort_flag) {
+    for (int i = 0; i < 100; ++i) __nanosleep(1000);
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+}  // namespace pair
+}  // namespace nvfp4

@@ -31,17 +31,17 @@ def run_gemm(a, b, fp32, tile_n, accumulate=False, D0=None):
         B.nvfp4_set_gemm_tile_n(0)
 
 
-@pytest.mark.parametrize("tile_n", [128, 256])
+@pytest.mark.parametrize("tile_n", [128, 256, 512])
 def test_exact_all_ones(tile_n):
     # every code 1.0 (nibble 2), every block scale 1.0 (0x38), tensor scales 1: each output = K exactly
-    M, N, K = 128, 256, 512
+    M, N, K = 256, 256, 512
     q = lambda R: oracle.Quantized(np.full((R, K // 2), 0x22, np.uint8), np.full((R, K // 16), 0x38, np.uint8),
                                    np.array([1.0, 1.0], np.float32), R, K)
     D = run_gemm(q(M), q(N), True, tile_n)
     assert np.array_equal(D, np.full((M, N), float(K), np.float32))
 
 
-@pytest.mark.parametrize("tile_n", [128, 256])
+@pytest.mark.parametrize("tile_n", [128, 256, 512])
 def test_exact_small_integers_and_power_of_two_scales(tile_n):
     # codes in {0, +-1, +-2}, power-of-two scales: every partial sum is exact in FP32 in any order
     rng = np.random.default_rng(1)
@@ -60,11 +60,14 @@ def test_exact_small_integers_and_power_of_two_scales(tile_n):
     assert np.array_equal(D.astype(np.float64), Dref)
 
 
-@pytest.mark.parametrize("shape", [(128, 128, 256), (256, 384, 512), (384, 640, 768), (128, 256, 2048)])
-@pytest.mark.parametrize("tile_n", [128, 256])
+@pytest.mark.parametrize("shape", [(128, 128, 256), (256, 384, 512), (384, 640, 768), (128, 256, 2048),
+                                   (256, 256, 256), (512, 768, 1024), (256, 512, 3072)])
+@pytest.mark.parametrize("tile_n", [128, 256, 512])
 @pytest.mark.parametrize("fp32", [False, True])
 def test_against_fp64_product_of_decoded_operands(shape, tile_n, fp32):
     M, N, K = shape
+    if tile_n == 512 and (M % 256 or N % 256):
+        pytest.skip("CTA-pair tiles need M and N to be multiples of 256")
     a, b = operands(M, N, K, 40 + M + N)
     Dref, T = P.gemm_reference(a, b)
     D = run_gemm(a, b, fp32, tile_n)
@@ -79,30 +82,37 @@ def test_many_tiles_per_cta_and_row_identity():
     a.scales[:] = np.clip(a.scales.astype(int) - (np.arange(M)[:, None] // 128 % 4) * 8, 1, 0x7E).astype(np.uint8)
     rows = np.arange(0, M, 37)
     cols = np.arange(0, N, 41)
-    D = run_gemm(a, b, True, 256)
     Dr, Tr = P.gemm_reference(a, b, rows=rows)
-    P.assert_gemm_close(D[rows], Dr, Tr, False, "sampled rows")
     Dc, Tc = P.gemm_reference(a, b, cols=cols)
-    P.assert_gemm_close(D[:, cols], Dc, Tc, False, "sampled cols")
+    for tile_n in (256, 512):
+        D = run_gemm(a, b, True, tile_n)
+        P.assert_gemm_close(D[rows], Dr, Tr, False, f"sampled rows, tile_n={tile_n}")
+        P.assert_gemm_close(D[:, cols], Dc, Tc, False, f"sampled cols, tile_n={tile_n}")
 
 
-def test_accumulate_into_fp32_and_leading_dimension():
-    M, N, K = 128, 256, 256
+@pytest.mark.parametrize("tile_n", [128, 512])
+def test_accumulate_into_fp32_and_leading_dimension(tile_n):
+    M, N, K = 256, 256, 256
     a, b = operands(M, N, K, 3)
     Dref, T = P.gemm_reference(a, b)
     D0 = torch.randn((M, N), dtype=torch.float32, device="cuda")
-    D = run_gemm(a, b, True, 128, accumulate=True, D0=D0)
+    D = run_gemm(a, b, True, tile_n, accumulate=True, D0=D0)
     P.assert_gemm_close(D - D0.cpu().numpy(), Dref, T + np.abs(D0.cpu().numpy()) * 1e-3, False, "accumulate")
     # output embedded in a wider buffer: columns outside [0, N) stay untouched
     A, Bt = P.upload(a), P.upload(b)
     wide = torch.full((M, N + 64), 7.0, dtype=torch.bfloat16, device="cuda")
-    B.nvfp4_gemm(A, Bt, wide[:, :N])
-    B.nvfp4_device_status()
+    B.nvfp4_set_gemm_tile_n(tile_n)
+    try:
+        B.nvfp4_gemm(A, Bt, wide[:, :N])
+        B.nvfp4_device_status()
+    finally:
+        B.nvfp4_set_gemm_tile_n(0)
     assert torch.all(wide[:, N:] == 7.0)
     P.assert_gemm_close(wide[:, :N].float().cpu().numpy(), Dref, T, True, "ldd > N")
 
 
-def test_gemm_is_deterministic():
+@pytest.mark.parametrize("tile_n", [256, 512])
+def test_gemm_is_deterministic(tile_n):
     a, b = operands(256, 256, 1024, 5)
-    D1, D2 = run_gemm(a, b, True, 256), run_gemm(a, b, True, 256)
+    D1, D2 = run_gemm(a, b, True, tile_n), run_gemm(a, b, True, tile_n)
     assert np.array_equal(D1, D2)
