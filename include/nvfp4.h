@@ -161,6 +161,36 @@ NVFP4_API nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_co
                                         size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * nvfp4_linear_fwd_noalloc -- the forward pass for callers that cannot hand over scratch memory.
+ * (The paper has no counterpart: this is a packaging variant of nvfp4_linear_fwd, same arithmetic.)
+ *
+ * Some callers have no way to allocate device memory at the point where they run a layer: code inside a
+ * real-time or inference-server callback that must not call cudaMalloc (it synchronises the device and may
+ * fail under memory pressure), plug-ins that are handed only their input and output buffers, or hosts whose
+ * allocator is owned by another component.  For them the row-wise NVFP4 copy of X, which nvfp4_linear_fwd
+ * keeps in caller-provided workspace, is placed in an array built into the library's device image.
+ *
+ *   - Arguments are those of nvfp4_linear_fwd without `workspace` / `workspace_bytes`; inputs and outputs
+ *     (X, W, Y, the saved copies) are still the caller's.
+ *   - Limit: nvfp4_linear_fwd_workspace_bytes(M, K) must not exceed nvfp4_linear_fwd_noalloc_max_bytes()
+ *     (16 MiB: M * K up to about 29.8 million elements, e.g. 4096 x 5120); larger problems return
+ *     NVFP4_ERR_WORKSPACE and nothing is enqueued.  Every GPU that loads the library carries these 16 MiB
+ *     until the process exits.
+ *   - The call allocates nothing: no cudaMalloc / cudaFree and no allocating library routine.  Its first call
+ *     on a device looks up the array's device address (a host-side query, no allocation) with that device
+ *     current; make that first call before any stream capture begins.
+ *   - All calls share the one array and find the previous call's contents in it; what must start from zero
+ *     (the amax word of the reduction) is cleared by the call itself.  Two calls whose work overlaps on the
+ *     GPU (different streams, or different threads on the same device) race on the array: serialise them.
+ */
+NVFP4_API size_t nvfp4_linear_fwd_noalloc_max_bytes(void);
+NVFP4_API nvfp4_status nvfp4_linear_fwd_noalloc(const void* X, const void* W, int64_t M, int64_t N,
+                                                int64_t K, const nvfp4_quant_opts* opts, void* Y_bf16,
+                                                const nvfp4_tensor* X_col_saved, const nvfp4_tensor* W_row,
+                                                const nvfp4_tensor* W_col_saved, int32_t w_is_cached,
+                                                void* cuda_stream);
+
+/*
  * Test aids (not on the hot path).
  * nvfp4_dequantize: out[r][c] = code * fp32(block scale) * s_dec as fp32 (the decode of Section 2).
  * nvfp4_rht16: the transformed values y = x*(S*H_16) of the row-wise (colwise == 0, out [rows x cols])

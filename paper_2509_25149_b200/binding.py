@@ -23,6 +23,7 @@ EXPORTED = (
     "nvfp4_quantize", "nvfp4_gemm", "nvfp4_linear_fwd_workspace_bytes", "nvfp4_linear_bwd_workspace_bytes",
     "nvfp4_linear_fwd", "nvfp4_linear_bwd", "nvfp4_dequantize", "nvfp4_rht16", "nvfp4_device_status",
     "nvfp4_set_gemm_tile_n", "nvfp4_status_string", "nvfp4_launch_count",
+    "nvfp4_linear_fwd_noalloc", "nvfp4_linear_fwd_noalloc_max_bytes",
 )
 
 
@@ -64,6 +65,9 @@ def lib() -> ctypes.CDLL:
         L.nvfp4_linear_bwd_workspace_bytes.argtypes = [i64, i64]
         L.nvfp4_linear_fwd.restype = i32
         L.nvfp4_linear_fwd.argtypes = [vp, vp, i64, i64, i64, OP, vp, TP, TP, TP, i32, vp, c.c_size_t, vp]
+        L.nvfp4_linear_fwd_noalloc.restype = i32
+        L.nvfp4_linear_fwd_noalloc.argtypes = [vp, vp, i64, i64, i64, OP, vp, TP, TP, TP, i32, vp]
+        L.nvfp4_linear_fwd_noalloc_max_bytes.restype, L.nvfp4_linear_fwd_noalloc_max_bytes.argtypes = c.c_size_t, []
         L.nvfp4_linear_bwd.restype = i32
         L.nvfp4_linear_bwd.argtypes = [vp, TP, TP, i64, i64, i64, OP, vp, vp, i32, vp, c.c_size_t, vp]
         L.nvfp4_dequantize.restype, L.nvfp4_dequantize.argtypes = i32, [TP, vp, vp]
@@ -151,6 +155,25 @@ def nvfp4_linear_fwd(X: torch.Tensor, W: Optional[torch.Tensor], opts: CQuantOpt
                                   Y.data_ptr(), _ref(X_col_saved), _ref(W_row), _ref(W_col_saved), int(w_is_cached),
                                   workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
            "nvfp4_linear_fwd")
+
+
+def nvfp4_linear_fwd_noalloc_max_bytes() -> int:
+    return int(lib().nvfp4_linear_fwd_noalloc_max_bytes())
+
+
+def nvfp4_linear_fwd_noalloc(X: torch.Tensor, W: Optional[torch.Tensor], opts: CQuantOpts, Y: torch.Tensor,
+                             X_col_saved: Optional[NVFP4Tensor], W_row: NVFP4Tensor,
+                             W_col_saved: Optional[NVFP4Tensor], w_is_cached: bool) -> None:
+    """Forward pass for callers that cannot allocate device memory: same as nvfp4_linear_fwd, but the scratch copy
+    of X sits in an array built into the library (16 MiB limit; calls must not overlap on the GPU)."""
+    M, K = X.shape
+    N = W_row.rows
+    assert X.is_contiguous() and Y.is_contiguous() and Y.dtype == torch.bfloat16 and tuple(Y.shape) == (M, N)
+    assert W is None or (W.is_contiguous() and tuple(W.shape) == (N, K))
+    _check(lib().nvfp4_linear_fwd_noalloc(X.data_ptr(), W.data_ptr() if W is not None else None, M, N, K,
+                                          ctypes.byref(opts), Y.data_ptr(), _ref(X_col_saved), _ref(W_row),
+                                          _ref(W_col_saved), int(w_is_cached), _stream()),
+           "nvfp4_linear_fwd_noalloc")
 
 
 def nvfp4_linear_bwd(dY: torch.Tensor, X_col_saved: Optional[NVFP4Tensor], W_col_saved: Optional[NVFP4Tensor], K: int,

@@ -13,6 +13,11 @@ void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_r
 
 using namespace nvfp4;
 
+// Scratch of nvfp4_linear_fwd_noalloc: the row-wise NVFP4 copy of X lives here instead of in caller memory.
+// Every GPU that loads the library holds this array until the process exits.
+#define NVFP4_NOALLOC_SCRATCH_BYTES (16u << 20)
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NVFP4_NOALLOC_SCRATCH_BYTES];
+
 namespace {
 
 inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -209,6 +214,30 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, c
   return NVFP4_OK;
 }
 
+size_t nvfp4_linear_fwd_noalloc_max_bytes(void) { return NVFP4_NOALLOC_SCRATCH_BYTES; }
+
+nvfp4_status nvfp4_linear_fwd_noalloc(const void* X, const void* W, int64_t M, int64_t N, int64_t K,
+                                      const nvfp4_quant_opts* opts, void* Y_bf16, const nvfp4_tensor* X_col_saved,
+                                      const nvfp4_tensor* W_row, const nvfp4_tensor* W_col_saved, int32_t w_is_cached,
+                                      void* cuda_stream) {
+  if (M <= 0 || K <= 0 || M % 256 || K % 256) return NVFP4_ERR_SHAPE;
+  // the request must fit the built-in array: refuse larger problems instead of touching memory we do not own
+  if (nvfp4_linear_fwd_workspace_bytes(M, K) > (size_t)NVFP4_NOALLOC_SCRATCH_BYTES) return NVFP4_ERR_WORKSPACE;
+  // `g_noalloc_scratch` names a host-side handle in host code, not a device address: ask the runtime for the
+  // address once per device (with that device current) and hand that pointer to the kernels.
+  constexpr int kMaxDevices = 64;
+  static void* scratch_of_device[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return NVFP4_ERR_CUDA;
+  if (!scratch_of_device[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return NVFP4_ERR_CUDA;
+    scratch_of_device[dev] = ptr;
+  }
+  return nvfp4_linear_fwd(X, W, M, N, K, opts, Y_bf16, X_col_saved, W_row, W_col_saved, w_is_cached,
+                          scratch_of_device[dev], NVFP4_NOALLOC_SCRATCH_BYTES, cuda_stream);
+}
+
 nvfp4_status nvfp4_dequantize(const nvfp4_tensor* t, float* out, void* cuda_stream) {
   if (!t || !out || !t->codes || !t->scales || !t->global) return NVFP4_ERR_NULL;
   nvfp4_status st = check_copy(t, t->rows, t->cols);
@@ -248,7 +277,7 @@ const char* nvfp4_status_string(nvfp4_status s) {
     case NVFP4_ERR_SHAPE: return "unsupported shape";
     case NVFP4_ERR_ALIGN: return "insufficient alignment";
     case NVFP4_ERR_ARG: return "unsupported option";
-    case NVFP4_ERR_WORKSPACE: return "workspace missing or too small";
+    case NVFP4_ERR_WORKSPACE: return "workspace missing or too small (or the problem exceeds the built-in scratch)";
     case NVFP4_ERR_CUDA: return "CUDA call failed";
     case NVFP4_ERR_TIMEOUT: return "a bounded device-side wait expired";
     case NVFP4_ERR_UNIMPLEMENTED: return "not implemented";
