@@ -324,11 +324,8 @@ cudaError_t launch_t(const GemmArgs& g, const void* a_codes, const void* b_codes
 }
 
 cudaError_t launch_pair(const GemmArgs& g, const void* a_codes, const void* b_codes, int num_sms, cudaStream_t s) {
-  CUtensorMap map_a, map_b, map_sfa, map_sfb, map_d;
-  const uint64_t atoms_a = (uint64_t)(g.M / 128) * (g.K / 64), atoms_b = (uint64_t)(g.N / 128) * (g.K / 64);
-  bool ok = make_code_map(&map_a, a_codes, g.M, g.K / 2, 128) && make_code_map(&map_b, b_codes, g.N, g.K / 2, 128) &&
-            make_map_2d(&map_sfa, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, g.sfa, 128, atoms_a, 512, 128, 4, false) &&
-            make_map_2d(&map_sfb, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, g.sfb, 128, atoms_b, 512, 128, 4, false);
+  CUtensorMap map_a, map_b, map_d;
+  bool ok = make_code_map(&map_a, a_codes, g.M, g.K / 2, 128) && make_code_map(&map_b, b_codes, g.N, g.K / 2, 128);
   if (g.d_is_fp32)
     ok = ok && make_map_2d(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g.d, (uint64_t)g.N, (uint64_t)g.M,
                            (uint64_t)g.ldd * 4, 32, 128, true);
@@ -346,8 +343,8 @@ cudaError_t launch_pair(const GemmArgs& g, const void* a_codes, const void* b_co
   const int n_tiles = (g.M / 256) * (g.N / 256);
   const int max_pairs = num_sms / 2;
   const int pairs = n_tiles < max_pairs ? n_tiles : max_pairs;
-  pair::Args a{g.M, g.N, g.K, g.a_global, g.b_global, g.d_is_fp32, g.accumulate};
-  pair::gemm_pair_kernel<<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, a);
+  pair::Args a{g.M, g.N, g.K, g.sfa, g.sfb, g.a_global, g.b_global, g.d_is_fp32, g.accumulate};
+  pair::gemm_pair_kernel<<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(map_a, map_b, map_d, a);
   count_launch();
   return cudaGetLastError();
 }

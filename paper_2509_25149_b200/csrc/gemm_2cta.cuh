@@ -5,8 +5,8 @@
 // traffic per flop is the point: the one-CTA kernel is bound by shared-memory bandwidth, not by the tensor pipe.
 //
 // Roles per CTA (7 warps): 0 TMA producer (both CTAs; every load signals the LEADER's "full" barrier),
-// 1 MMA issuer (leader only; allocates tensor memory in both), 2 scale-atom copier (leader only; cta_group::2
-// copies run in both CTAs from their own shared memory), 3-10 epilogue (both; two groups of four warps, one per
+// 1 MMA issuer (leader only; allocates tensor memory in both), 2 and 11-13 scale warps (both CTAs; shared memory ->
+// registers -> tensor memory, one warp per 32-lane quadrant), 3-10 epilogue (both; two groups of four warps, one per
 // 128-column half: tensor memory -> registers -> swizzled staging -> TMA store; the accumulator is released as
 // soon as it has been read).
 // Included by gemm.cu only.
@@ -20,7 +20,7 @@
 namespace nvfp4 {
 namespace pair {
 
-constexpr int kThreads = 448;      // producer, MMA, 2 x 4 epilogue warps, 4 scale-copy warps (2, 11, 12, 13)      // producer, MMA, scale copier, 2 x 4 epilogue warps
+constexpr int kThreads = 448;      // producer, MMA, 2 x 4 epilogue warps, 4 scale warps (2, 11, 12, 13)      // producer, MMA, scale copier, 2 x 4 epilogue warps
 constexpr int kStages = 4;
 constexpr int kABytes = 128 * 128;   // 128 rows x 256 K elements
 constexpr int kBBytes = 128 * 128;   // this CTA's half of the 256-row B tile
@@ -37,6 +37,8 @@ static_assert(kStageBytes % 1024 == 0, "stages must keep the 1024-byte swizzle a
 
 struct Args {
   int M, N, K;
+  const uint8_t* sfa;  // swizzled scale atoms of A and B (global memory)
+  const uint8_t* sfb;
   const float* a_global;
   const float* b_global;
   int d_is_fp32, accumulate;
@@ -133,8 +135,19 @@ __device__ __forceinline__ void tc2_commit_both(uint32_t bar, uint16_t mask) {
                ::"r"(bar), "h"(mask)
                : "memory");
 }
-__device__ __forceinline__ void tc2_cp_sf(uint32_t taddr, uint64_t sdesc) {
-  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+// registers -> tensor memory: this warp's 32 lanes x 16 consecutive columns
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+      "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
 }
 __device__ __forceinline__ void tc2_mma_nvf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                              uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
@@ -193,21 +206,21 @@ __device__ __forceinline__ void store_half(const uint32_t (&r)[128], float alpha
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                     const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
                      const __grid_constant__ CUtensorMap map_d, const Args g) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t staging = base + kStages * kStageBytes;
   const uint32_t bar_base = staging + kStagingBytes;
-  auto full_bar = [&](int s) { return bar_base + 8u * s; };                  // used in the leader only
-  auto sff_bar = [&](int s) { return bar_base + 8u * (kStages + s); };       // leader only
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };                  // leader only: both CTAs' operands landed
+  auto sff_bar = [&](int s) { return bar_base + 8u * (kStages + s); };       // leader only: scales of both CTAs in TMEM
   auto empty_bar = [&](int s) { return bar_base + 8u * (2 * kStages + s); }; // one per CTA
-  const uint32_t accf_bar = bar_base + 8u * (3 * kStages);                   // one per CTA
-  const uint32_t acce_bar = bar_base + 8u * (3 * kStages + 1);               // leader only, 16 arrivals
-  const uint32_t done_bar = bar_base + 8u * (3 * kStages + 2);               // one per CTA, peer arrives
+  auto sfl_bar = [&](int s) { return bar_base + 8u * (3 * kStages + s); };   // one per CTA: own scale atoms landed
+  const uint32_t accf_bar = bar_base + 8u * (4 * kStages);                   // one per CTA
+  const uint32_t acce_bar = bar_base + 8u * (4 * kStages + 1);               // leader only, 16 arrivals
+  const uint32_t done_bar = bar_base + 8u * (4 * kStages + 2);               // one per CTA, peer arrives
   volatile uint32_t* tmem_slot =
-      reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + kStagingBytes + 8 * (3 * kStages + 3));
+      reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + kStagingBytes + 8 * (4 * kStages + 3));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -233,8 +246,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(full_bar(s), 2);   // one arrive.expect_tx from each CTA's producer
-      mbar_init(sff_bar(s), 4);    // one commit from each scale-copy warp
+      mbar_init(sff_bar(s), 8);    // four scale warps in each CTA
       mbar_init(empty_bar(s), 1);
+      mbar_init(sfl_bar(s), 1);
     }
     mbar_init(accf_bar, 1);
     mbar_init(acce_bar, 16);       // eight epilogue warps in each CTA
@@ -266,18 +280,21 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
         tile_coords(tile, m_blk, n_blk);
         const int row_a = m_blk * 256 + (int)rank * 128;       // this CTA's A rows
         const int row_b = n_blk * 256 + (int)rank * 128;       // this CTA's half of the B tile
-        const int atom_a = (m_blk * 2 + (int)rank) * sf_atoms_k;
-        const int atom_b = (n_blk * 2) * sf_atoms_k;
+        const uint8_t* sfa = g.sfa + (int64_t)(m_blk * 2 + (int)rank) * sf_atoms_k * 512;  // own 128 rows
+        const uint8_t* sfb = g.sfb + (int64_t)(n_blk * 2) * sf_atoms_k * 512;               // all 256 rows of B
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x100u + stage))) break;
           const uint32_t st = base + stage * kStageBytes;
-          const uint32_t bar = map_to_cta(full_bar(stage), 0);  // the leader's barrier counts both CTAs' bytes
-          mbar_expect_tx_cluster(bar, kStageBytes);
+          const uint32_t bar = map_to_cta(full_bar(stage), 0);  // the leader's barrier counts both CTAs' operands
+          mbar_expect_tx_cluster(bar, kABytes + kBBytes);
           tma_load_2d_pair(st, &map_a, kb * 128, row_a, bar);
           tma_load_2d_pair(st + kABytes, &map_b, kb * 128, row_b, bar);
-          tma_load_2d_pair(st + kABytes + kBBytes, &map_sfa, 0, atom_a + kb * 4, bar);
-          tma_load_2d_pair(st + kABytes + kBBytes + kSfaBytes, &map_sfb, 0, atom_b + kb * 4, bar);
-          tma_load_2d_pair(st + kABytes + kBBytes + kSfaBytes + 2048, &map_sfb, 0, atom_b + sf_atoms_k + kb * 4, bar);
+          // scale atoms: plain bulk copies counted on this CTA's own barrier (its scale warps wait on it)
+          mbar_expect_tx(sfl_bar(stage), kSfaBytes + kSfbBytes);
+          bulk_load(st + kABytes + kBBytes, sfa + (int64_t)kb * 2048, kSfaBytes, sfl_bar(stage));
+          bulk_load(st + kABytes + kBBytes + kSfaBytes, sfb + (int64_t)kb * 2048, 2048, sfl_bar(stage));
+          bulk_load(st + kABytes + kBBytes + kSfaBytes + 2048, sfb + ((int64_t)sf_atoms_k + kb * 4) * 512, 2048,
+                    sfl_bar(stage));
           if (++stage == kStages) {
             stage = 0;
             phase ^= 1u;
@@ -286,32 +303,49 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       }
     }
   } else if (warp == 2 || warp >= 11) {
-    // ------------------------------------------- scale atoms: shared -> tensor memory (both CTAs) ----
-    if (leader && lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
+    // ------------------------------- scale atoms: shared memory -> registers -> tensor memory (both CTAs) ----
+    // One warp per 32-lane quadrant of tensor memory (warps 2, 11, 12, 13 -> quadrants 2, 3, 0, 1).  Lane l of
+    // every quadrant holds row l of each 512-byte atom: columns [4j, 4j+4) of the stage's slot for SFA of K64-step
+    // j, columns [16 + 8j + 4g, ..) for SFB of step j and 128-row group g.  The tensor-memory copy engine
+    // (tcgen05.cp) moves one atom per instruction and was the bottleneck of the main loop; twelve 16-byte loads
+    // and three tcgen05.st per warp do the same work off the critical path.
+    const int quad = warp & 3;
+    int stage = 0;
+    uint32_t phase = 0;
+    const uint32_t sff_leader = map_to_cta(sff_bar(0), 0);
+    for (int tile = pair_id; tile < n_tiles; tile += n_pairs) {
       bool ok = true;
-      const uint32_t sf_lo0 = (base + kABytes + kBBytes) >> 4;
-      for (int tile = pair_id; tile < n_tiles && ok; tile += n_pairs) {
-        for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!(ok = mbar_wait_cluster(full_bar(stage), phase, abort_flag, 0x500u + stage))) break;
-          tc_fence_after();
-          const uint32_t lo = sf_lo0 + stage * (kStageBytes >> 4);
-          const uint32_t sf_t = tmem + kSfCol + stage * kSfSlotCols;
-          {
-            // this warp copies the atoms of K64-step j: SFA (own 128 rows) and both 128-row groups of SFB
-            const int j = (warp == 2) ? 0 : warp - 10;
-            tc2_cp_sf(sf_t + j * 4, make_desc(lo + j * 32, kDescHiSf));
-            tc2_cp_sf(sf_t + 16 + j * 8, make_desc(lo + (kSfaBytes >> 4) + j * 32, kDescHiSf));
-            tc2_cp_sf(sf_t + 16 + j * 8 + 4, make_desc(lo + (kSfaBytes >> 4) + 128 + j * 32, kDescHiSf));
-          }
-          tc2_commit_local(sff_bar(stage));
-          if (++stage == kStages) {
-            stage = 0;
-            phase ^= 1u;
+      for (int kb = 0; kb < k_blocks; ++kb) {
+        ok = mbar_wait(sfl_bar(stage), phase, abort_flag, 0x500u + stage);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        const uint32_t sf_s = base + stage * kStageBytes + kABytes + kBBytes + lane * 16;
+        uint32_t r[48];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint4 a = lds128(sf_s + j * 512);
+          r[4 * j] = a.x; r[4 * j + 1] = a.y; r[4 * j + 2] = a.z; r[4 * j + 3] = a.w;
+#pragma unroll
+          for (int grp = 0; grp < 2; ++grp) {
+            const uint4 b = lds128(sf_s + kSfaBytes + grp * 2048 + j * 512);
+            r[16 + 8 * j + 4 * grp] = b.x; r[16 + 8 * j + 4 * grp + 1] = b.y;
+            r[16 + 8 * j + 4 * grp + 2] = b.z; r[16 + 8 * j + 4 * grp + 3] = b.w;
           }
         }
+        const uint32_t sf_t = tmem + ((uint32_t)(quad * 32) << 16) + kSfCol + stage * kSfSlotCols;
+        tc_st16(sf_t, &r[0]);
+        tc_st16(sf_t + 16, &r[16]);
+        tc_st16(sf_t + 32, &r[32]);
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(sff_leader + 8u * stage);
+        if (++stage == kStages) {
+          stage = 0;
+          phase ^= 1u;
+        }
       }
+      if (!ok) break;
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer (leader) ----
@@ -326,7 +360,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
         if (!(ok = mbar_wait_cluster(acce_bar, acc_phase ^ 1u, abort_flag, 0x300u))) break;
         tc_fence_after();
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!(ok = mbar_wait(sff_bar(stage), phase, abort_flag, 0x200u + stage))) break;
+          if (!(ok = mbar_wait_cluster(full_bar(stage), phase, abort_flag, 0x200u + stage))) break;
+          if (!(ok = mbar_wait_cluster(sff_bar(stage), phase, abort_flag, 0x280u + stage))) break;
           tc_fence_after();
           const uint32_t a_lo = a_lo0 + stage * (kStageBytes >> 4);
           const uint32_t b_lo = b_lo0 + stage * (kStageBytes >> 4);
