@@ -384,7 +384,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", default=None, choices=sorted(CASES), help="run one kernel on a reduced shape")
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")

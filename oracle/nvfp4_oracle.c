@@ -244,7 +244,11 @@ ORC_EXPORT int64_t orc_sf_swizzled_offset(int64_t r, int64_t kb, int64_t n_kb) {
  *             source position the value is stored at)
  * amax_override >= 0: use it instead of the computed tensor amax (used by the
  *             comparison protocol under RHT, where a last-bit difference in
- *             amax must not be smeared over every block)
+ *             amax must not be smeared over every block, and when a slab of
+ *             rows of a larger tensor is quantized on its own)
+ * sr_row0, sr_cols: the tensor is rows [sr_row0, sr_row0 + src_rows) of a
+ *             larger source with sr_cols columns (sr_cols = 0: it is the whole
+ *             source); only the stochastic-rounding draw index depends on it
  * outputs   : codes [R][C/2] (even column in the low nibble), scales [R][C/16]
  *             linear, global = {amax, s_dec}, y_out (nullable) = the values
  *             that were quantized, [R][C] floats.   R x C = shape of the copy.
@@ -254,8 +258,8 @@ ORC_EXPORT int64_t orc_sf_swizzled_offset(int64_t r, int64_t kb, int64_t n_kb) {
 ORC_EXPORT int orc_quantize(const uint16_t* x_bf16, int64_t src_rows, int64_t src_cols, int64_t ld,
                             int colwise, int block_rows, int rht, uint16_t sign_mask,
                             int rounding, uint64_t seed, uint64_t sr_offset,
-                            float amax_override, uint8_t* codes, uint8_t* scales,
-                            float* global, float* y_out) {
+                            float amax_override, int64_t sr_row0, int64_t sr_cols,
+                            uint8_t* codes, uint8_t* scales, float* global, float* y_out) {
   const int64_t R = colwise ? src_cols : src_rows;
   const int64_t C = colwise ? src_rows : src_cols;
   if ((block_rows != 1 && block_rows != 16) || C % 16 || R % block_rows) return -1;
@@ -322,7 +326,7 @@ ORC_EXPORT int orc_quantize(const uint16_t* x_bf16, int64_t src_rows, int64_t sr
           code[j] = orc_e2m1_encode_rne(v);
         } else {
           int64_t sr = colwise ? c : r, sc = colwise ? r : c;
-          uint64_t e = (uint64_t)sr * (uint64_t)src_cols + (uint64_t)sc;
+          uint64_t e = (uint64_t)(sr + sr_row0) * (uint64_t)(sr_cols ? sr_cols : src_cols) + (uint64_t)sc;
           code[j] = orc_e2m1_encode_sr(v, orc_sr_draw(seed, sr_offset, e));
         }
       }

@@ -1,0 +1,125 @@
+"""Parity at the benchmark's full size (cfg 3: M 8192, K 5120, N 20480) in the launch configuration bench.py times:
+nvfp4_linear_fwd / nvfp4_linear_bwd for the GEMM outputs, nvfp4_quantize with the same options for the operand
+copies.  The oracle checks sampled row slabs of every quantized copy and sampled rows / columns of every GEMM."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import parity as P
+from paper_2509_25149_b200 import binding as B
+from paper_2509_25149_b200 import synth
+
+pytestmark = pytest.mark.gpu
+SLABS = (0, 128 * 17, None)  # first, an interior and the last 128-row slab (None = rows - 128)
+
+
+def rotated_amax(x: torch.Tensor, mask: int) -> float:
+    """max |x^T (S H_16)| over the whole tensor, chunks of 16 along the rows (tokens), in float64 (torch matmul)."""
+    H = torch.tensor([[oracle.hadamard16_entry(j, k) for k in range(16)] for j in range(16)], dtype=torch.float64)
+    s = torch.tensor([-1.0 if (mask >> j) & 1 else 1.0 for j in range(16)], dtype=torch.float64)
+    SH = (s[:, None] * H) / 4
+    best = 0.0
+    for r0 in range(0, x.shape[0], 1024):
+        blk = x[r0:r0 + 1024].to(torch.float64).reshape(-1, 16, x.shape[1])       # [chunks, 16, cols]
+        y = torch.einsum("qjc,jk->qkc", blk, SH)
+        best = max(best, float(y.abs().max()))
+    return best
+
+
+def check_copy_slabs(x: torch.Tensor, gpu: B.NVFP4Tensor, *, colwise, block_rows=1, rht=False, mask=0, rounding=0,
+                     seed=0, sr_offset=0, what=""):
+    codes, scales, glob = P.download(gpu)
+    R = x.shape[0]
+    n_bad = n_tot = 0
+    for r0 in SLABS:
+        r0 = R - 128 if r0 is None else r0
+        slab = synth.bits(x[r0:r0 + 128])
+        ref = oracle.quantize(slab, colwise=colwise, block_rows=block_rows, rht=rht, sign_mask=mask, rounding=rounding,
+                              seed=seed, sr_offset=sr_offset, amax_override=float(glob[0]), sr_row0=r0,
+                              sr_cols=x.shape[1])
+        assert glob.view(np.uint32)[1] == ref.glob.view(np.uint32)[1], f"{what}: s_dec"
+        if colwise:
+            got_c, got_s = codes[:, r0 // 2:(r0 + 128) // 2], scales[:, r0 // 16:(r0 + 128) // 16]
+        else:
+            got_c, got_s = codes[r0:r0 + 128], scales[r0:r0 + 128]
+        if not rht:
+            assert np.array_equal(got_s, ref.scales), f"{what}: scale bytes of slab {r0}"
+            assert np.array_equal(got_c, ref.codes), f"{what}: codes of slab {r0}"
+        else:
+            # rotated copies: equal except next to a rounding threshold (butterfly vs float64 summation order)
+            sd = got_s != ref.scales
+            assert np.all(np.abs(got_s.astype(int) - ref.scales.astype(int))[sd] <= 1), f"{what}: scale not adjacent"
+            g, w = P.unpack(got_c), P.unpack(ref.codes)
+            cd = (g != w) & ~np.repeat(sd, 16, axis=1)
+            assert np.all(np.abs((g & 7).astype(int) - (w & 7).astype(int))[cd] <= 1), f"{what}: code not adjacent"
+            n_bad += int(cd.sum()) + 16 * int(sd.sum())
+        n_tot += got_c.size * 2
+    assert n_bad <= 1e-3 * n_tot, f"{what}: {n_bad} of {n_tot} elements differ"
+
+
+def check_gemm_samples(D: torch.Tensor, A: B.NVFP4Tensor, Bt: B.NVFP4Tensor, bf16: bool, what: str, seed: int):
+    rng = np.random.default_rng(seed)
+    rows = np.sort(rng.choice(A.rows, 12, replace=False))
+    cols = np.sort(rng.choice(Bt.rows, 384, replace=False))
+    ac, asc, ag = P.download(A)
+    bc, bsc, bg = P.download(Bt)
+    a = oracle.Quantized(np.ascontiguousarray(ac[rows]), np.ascontiguousarray(asc[rows]), ag, len(rows), A.cols)
+    b = oracle.Quantized(np.ascontiguousarray(bc[cols]), np.ascontiguousarray(bsc[cols]), bg, len(cols), Bt.cols)
+    Dref, T = oracle.gemm_tn(oracle.dequantize(a), oracle.dequantize(b))
+    got = D[torch.from_numpy(rows).cuda()][:, torch.from_numpy(cols).cuda()].float().cpu().numpy()
+    P.assert_gemm_close(got, Dref, T, bf16, what)
+
+
+def test_config3_full_size_forward_and_backward():
+    p = synth.config3()
+    M, N, K = p.M, p.N, p.K
+    mask = p.rht_sign_mask
+    X, W, dY = p.X.cuda(), p.W.cuda(), p.dY.cuda()
+    opts = B.quant_opts(rht_sign_mask=mask, seed=p.sr_seed, sr_offset=p.sr_offset)
+    X_col, W_row, W_col = B.alloc_tensor(K, M), B.alloc_tensor(N, K), B.alloc_tensor(K, N)
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((N, K), dtype=torch.float32, device="cuda")
+    ws_f = torch.empty(B.nvfp4_linear_fwd_workspace_bytes(M, K), dtype=torch.uint8, device="cuda")
+    ws_b = torch.empty(B.nvfp4_linear_bwd_workspace_bytes(M, N), dtype=torch.uint8, device="cuda")
+    B.nvfp4_linear_fwd(X, W, opts, Y, X_col, W_row, W_col, False, ws_f)
+    B.nvfp4_linear_bwd(dY, X_col, W_col, K, opts, dX, dW, False, ws_b)
+    B.nvfp4_device_status()
+
+    # the operand copies the two calls keep in their workspaces, reproduced with the same options
+    X_row = B.alloc_tensor(M, K)
+    X_col2 = B.alloc_tensor(K, M)
+    B.nvfp4_quantize(X, B.quant_opts(rht_colwise=True, rht_sign_mask=mask), X_row, X_col2)
+    g_row, g_col = B.alloc_tensor(M, N), B.alloc_tensor(N, M)
+    B.nvfp4_quantize(dY, B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True, rht_sign_mask=mask,
+                                      seed=p.sr_seed, sr_offset=p.sr_offset), g_row, g_col)
+    torch.cuda.synchronize()
+    assert torch.equal(X_col2.codes, X_col.codes) and torch.equal(X_col2.scales, X_col.scales)  # deterministic
+
+    # ---- quantizer: tensor amax against torch, sampled slabs against the oracle -------------------------------
+    assert float(X_row.glob[0]) == float(p.X.abs().max().float())
+    assert float(W_row.glob[0]) == float(p.W.abs().max().float()) == float(W_col.glob[0])
+    assert float(g_row.glob[0]) == float(p.dY.abs().max().float())
+    for t, src in ((X_col, p.X), (g_col, p.dY)):
+        ref = rotated_amax(src, mask)
+        assert abs(float(t.glob[0]) - ref) <= 1e-5 * ref
+    check_copy_slabs(p.X, X_row, colwise=False, what="X row")
+    check_copy_slabs(p.X, X_col, colwise=True, rht=True, mask=mask, what="X col")
+    check_copy_slabs(p.W, W_row, colwise=False, block_rows=16, what="W row")
+    check_copy_slabs(p.W, W_col, colwise=True, block_rows=16, what="W col")
+    check_copy_slabs(p.dY, g_row, colwise=False, rounding=oracle.SR, seed=p.sr_seed, sr_offset=p.sr_offset, what="dY row")
+    check_copy_slabs(p.dY, g_col, colwise=True, rht=True, mask=mask, rounding=oracle.SR, seed=p.sr_seed,
+                     sr_offset=p.sr_offset, what="dY col")
+
+    # ---- GEMMs: sampled rows x columns against the FP64 product of the decoded operands -----------------------
+    check_gemm_samples(Y, X_row, W_row, True, "Fprop", 1)
+    check_gemm_samples(dX, g_row, W_col, True, "Dgrad", 2)
+    check_gemm_samples(dW, g_col, X_col, False, "Wgrad", 3)
+    # properties that hold at any size: no NaN / Inf, and the layer approximates the unquantized products
+    for t in (Y, dX, dW):
+        assert torch.isfinite(t.float()).all()
+    rows = torch.arange(0, M, 997, device="cuda")
+    exact = X[rows].double() @ W.double().T
+    rel = float((Y[rows].double() - exact).norm() / exact.norm())
+    assert rel < 0.2, rel

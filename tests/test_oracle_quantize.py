@@ -360,3 +360,18 @@ def test_wgrad_rht_pipeline_stays_close_to_the_unquantized_product():
     bad = oracle.quantize(X, colwise=True, rht=False)
     dWbad, _ = oracle.gemm_tn(oracle.dequantize(gq), oracle.dequantize(bad))
     assert np.linalg.norm(dWbad - exact) / np.linalg.norm(exact) > 0.7
+
+
+def test_row_slab_with_given_amax_equals_the_rows_of_the_full_tensor():
+    # used by the full-size GPU tests: a slab of rows, quantized with the full tensor's amax and the slab's
+    # position for the stochastic-rounding index, reproduces the corresponding part of either copy
+    x = _random_bits((64, 48), 21, scale=1e-3)
+    for rounding in (oracle.RNE, oracle.SR):
+        full_r = oracle.quantize(x, rounding=rounding, seed=3, sr_offset=7)
+        full_c = oracle.quantize(x, colwise=True, rounding=rounding, seed=3, sr_offset=7)
+        slab = x[16:48]
+        r = oracle.quantize(slab, rounding=rounding, seed=3, sr_offset=7, amax_override=float(full_r.amax), sr_row0=16, sr_cols=48)
+        c = oracle.quantize(slab, colwise=True, rounding=rounding, seed=3, sr_offset=7, amax_override=float(full_c.amax),
+                            sr_row0=16, sr_cols=48)
+        assert np.array_equal(r.codes, full_r.codes[16:48]) and np.array_equal(r.scales, full_r.scales[16:48])
+        assert np.array_equal(c.codes, full_c.codes[:, 8:24]) and np.array_equal(c.scales, full_c.scales[:, 1:3])
