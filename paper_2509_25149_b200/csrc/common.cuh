@@ -33,9 +33,22 @@ __device__ __forceinline__ void global_scales(float amax, float& s_enc, float& s
 }
 
 // Eq. 2-3 and the text after Eq. 3: stored E4M3 byte of a block and the encode scale derived from it.
+// fl(x / 6) for x >= 0 with three instructions: q = fl(x * fl(1/6)), exact residual r = fma(-6, q, x), corrected
+// q' = fma(r, fl(1/6), q).  x/6 is never closer than ulp/6 to a rounding midpoint (6 * midpoint needs 26 bits), and
+// the correction term is off by only 2^-25 relative, so q' is the correctly rounded quotient whenever the residual is
+// exact, i.e. outside the denormal range (checked exhaustively over whole binades on the host); tiny inputs take the
+// IEEE division.
+__device__ __forceinline__ float div6_rn(float x) {
+  const float c = 0.16666667163372039794921875f;  // fl(1/6)
+  const float q = __fmul_rn(x, c);
+  const float r = __fmaf_rn(-6.0f, q, x);
+  const float fast = __fmaf_rn(r, c, q);
+  return (x != 0.0f && x < 1.0e-30f) ? __fdiv_rn(x, 6.0f) : fast;
+}
+
 __device__ __forceinline__ void block_scales(float amax_b, float s_enc, float s_dec, uint32_t& byte,
                                              float& s_enc_b) {
-  float t = __fmul_rn(__fdiv_rn(amax_b, 6.0f), s_enc);
+  float t = __fmul_rn(div6_rn(amax_b), s_enc);
   uint16_t packed;
   asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %1;" : "=h"(packed) : "f"(t));
   uint32_t h2;

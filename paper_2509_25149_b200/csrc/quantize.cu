@@ -179,13 +179,16 @@ struct QuantSmem {
   static constexpr int kSfCol = kSfRow + 1024;       // 1 KB
   static constexpr int kBlkEnc = kSfCol + 1024;      // 64 floats (16x16 mode)
   static constexpr int kBlkByte = kBlkEnc + 256;     // 64 bytes
-  static constexpr int kRand = kBlkByte + 64;        // 128 rows x 128 B (stochastic rounding only)
+  static constexpr int kGlobalScales = kBlkByte + 64;  // s_enc, s_dec of the row-wise and the column-wise copy
+  static constexpr int kRand = kGlobalScales + 64;   // 128 rows x 128 B (stochastic rounding only)
   static constexpr int kBytesNoRand = kRand;
   static constexpr int kBytesRand = kRand + 16384;
 };
 
-template <bool SR>
-__device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, const uint32_t (&rnd)[4]) {
+// 16 scaled values -> 16 E2M1 nibbles (element 0 in the lowest nibble of .x).  For stochastic rounding `nu14(i)`
+// returns the complemented 8-bit draw of element i placed in bits [14, 22).
+template <bool SR, class Nu14>
+__device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, Nu14 nu14) {
   uint2 out;
   if (!SR) {
     float v[16];
@@ -196,15 +199,10 @@ __device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, 
     out.x = e2m1x8_rne(lo);
     out.y = e2m1x8_rne(hi);
   } else {
-    // rnd holds the 16 draws, byte i = element i; work with the complemented bytes
     uint32_t w[2] = {0u, 0u};
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-      const uint32_t nr = ~rnd[i >> 2];
-      const int b = i & 3;
-      // (255 - u) << 14 : move byte b to bits [14, 22)
-      const uint32_t nu14 = (b == 0 ? (nr << 14) : b == 1 ? (nr << 6) : b == 2 ? (nr >> 2) : (nr >> 10)) & 0x003FC000u;
-      const uint32_t nib = e2m1_sr_bits(__fmul_rn(f[i], s_enc_b), nu14);
+      const uint32_t nib = e2m1_sr_bits(__fmul_rn(f[i], s_enc_b), nu14(i));
       w[i >> 3] = __funnelshift_r(w[i >> 3], nib, 4);  // shifts the new nibble in from the top
     }
     out.x = w[0];
@@ -212,6 +210,24 @@ __device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, 
   }
   return out;
 }
+
+// draws packed four to a word, byte i = element i (the row-wise copy: straight from the Philox output)
+struct Nu14FromWords {
+  const uint32_t (&rnd)[4];
+  __device__ __forceinline__ uint32_t operator()(int i) const {
+    const uint32_t nr = ~rnd[i >> 2];
+    const int b = i & 3;
+    return (b == 0 ? (nr << 14) : b == 1 ? (nr << 6) : b == 2 ? (nr >> 2) : (nr >> 10)) & 0x003FC000u;
+  }
+};
+// draws of two adjacent columns, 16 bits per row (the transposed copy: read back from shared memory)
+template <int COL>
+struct Nu14FromPairs {
+  const uint32_t (&two)[16];
+  __device__ __forceinline__ uint32_t operator()(int i) const {
+    return (COL == 0 ? (~two[i] << 14) : (~two[i] << 6)) & 0x003FC000u;
+  }
+};
 
 __device__ __forceinline__ float amax16(const float (&f)[16]) {
   float m = 0.f;
@@ -230,19 +246,24 @@ __global__ void __launch_bounds__(256) quantize_kernel(const QuantArgs a) {
   const int64_t n_cb = a.cols >> 4;  // 16-blocks per source row
   const int64_t n_rb = a.rows >> 4;  // 16-blocks per source column
 
-  float r_senc = 1.f, r_sdec = 1.f, c_senc = 1.f, c_sdec = 1.f;
-  if (HAS_ROW || BLOCK2D) global_scales(HAS_ROW ? a.r_global[0] : a.c_global[0], r_senc, r_sdec);
-  if (HAS_COL) {
-    if (BLOCK2D && HAS_ROW) {
-      c_senc = r_senc;
-      c_sdec = r_sdec;
-    } else {
-      global_scales(a.c_global[0], c_senc, c_sdec);
+  // Eq. 1 once per CTA (two IEEE divisions per copy), broadcast through shared memory
+  float* g_sc = reinterpret_cast<float*>(smem + QuantSmem::kGlobalScales);
+  if (threadIdx.x == 0) {
+    float re = 1.f, rd = 1.f, ce = 1.f, cd = 1.f;
+    if (HAS_ROW || BLOCK2D) global_scales(HAS_ROW ? a.r_global[0] : a.c_global[0], re, rd);
+    if (HAS_COL) {
+      if (BLOCK2D && HAS_ROW) {
+        ce = re;
+        cd = rd;
+      } else {
+        global_scales(a.c_global[0], ce, cd);
+      }
     }
-  }
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
-    if (HAS_ROW) a.r_global[1] = r_sdec;
-    if (HAS_COL) a.c_global[1] = c_sdec;
+    g_sc[0] = re; g_sc[1] = rd; g_sc[2] = ce; g_sc[3] = cd;
+    if (blockIdx.x == 0) {
+      if (HAS_ROW) a.r_global[1] = rd;
+      if (HAS_COL) a.c_global[1] = cd;
+    }
   }
 
   // ------------------------------------------------------------------ phase 1 ----
@@ -280,6 +301,9 @@ __global__ void __launch_bounds__(256) quantize_kernel(const QuantArgs a) {
       }
     }
   }
+
+  __syncthreads();  // the loads above are in flight; the global scales are in shared memory now
+  const float r_senc = g_sc[0], r_sdec = g_sc[1], c_senc = g_sc[2], c_sdec = g_sc[3];
 
   float blk_amax = 0.f;  // 16x16 mode: running amax of the lane's chunk column over the warp's 16 rows
   if (BLOCK2D) {
@@ -327,20 +351,17 @@ __global__ void __launch_bounds__(256) quantize_kernel(const QuantArgs a) {
         f[2 * k] = bf16_lo(word);
         f[2 * k + 1] = bf16_hi(word);
       }
-      if (RHT_ROW) {
-        fwht16(f);
-#pragma unroll
-        for (int k = 0; k < 16; ++k) f[k] *= 0.25f;
-      }
+      if (RHT_ROW) fwht16(f);  // values are 4 * y: the 1/4 is folded into the amax and the encode scale (exact)
       uint32_t byte;
       float enc;
       if (BLOCK2D) {
         byte = blk_byte;
         enc = blk_enc;
       } else {
-        block_scales(amax16(f), r_senc, r_sdec, byte, enc);
+        block_scales(RHT_ROW ? 0.25f * amax16(f) : amax16(f), r_senc, r_sdec, byte, enc);
+        if (RHT_ROW) enc *= 0.25f;
       }
-      uint2 codes = convert16<SR>(f, enc, rnd);
+      uint2 codes = convert16<SR>(f, enc, Nu14FromWords{rnd});
       if (ok[i])
         *reinterpret_cast<uint2*>(a.r_codes + (row0 + r) * (a.cols >> 1) + ((col0 + cb * 16) >> 1)) = codes;
       const int pos = a.r_swz ? ((cb >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (cb & 3)) : (r * 8 + cb);
@@ -363,14 +384,9 @@ __global__ void __launch_bounds__(256) quantize_kernel(const QuantArgs a) {
         f0[j] = bf16_lo(word);
         f1[j] = bf16_hi(word);
       }
-      if (RHT_COL) {
+      if (RHT_COL) {  // values are 4 * y from here on; the 1/4 is folded into amax and encode scale (exact)
         fwht16(f0);
         fwht16(f1);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          f0[j] *= 0.25f;
-          f1[j] *= 0.25f;
-        }
       }
       uint32_t byte0, byte1;
       float enc0, enc1;
@@ -378,21 +394,24 @@ __global__ void __launch_bounds__(256) quantize_kernel(const QuantArgs a) {
         enc0 = enc1 = reinterpret_cast<const float*>(smem + QuantSmem::kBlkEnc)[q * 8 + (cp >> 3)];
         byte0 = byte1 = smem[QuantSmem::kBlkByte + q * 8 + (cp >> 3)];
       } else {
-        block_scales(amax16(f0), c_senc, c_sdec, byte0, enc0);
-        block_scales(amax16(f1), c_senc, c_sdec, byte1, enc1);
-      }
-      uint32_t rnd0[4] = {0u, 0u, 0u, 0u}, rnd1[4] = {0u, 0u, 0u, 0u};
-      if (SR) {
-        // byte j of rnd0 / rnd1 = draw of source element (row 16q + j, column 2cp / 2cp + 1)
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          uint32_t two = *reinterpret_cast<const uint16_t*>(smem + QuantSmem::kRand + (q * 16 + j) * 128 + cp * 2);
-          rnd0[j >> 2] |= (two & 0xffu) << (8 * (j & 3));
-          rnd1[j >> 2] |= (two >> 8) << (8 * (j & 3));
+        block_scales(RHT_COL ? 0.25f * amax16(f0) : amax16(f0), c_senc, c_sdec, byte0, enc0);
+        block_scales(RHT_COL ? 0.25f * amax16(f1) : amax16(f1), c_senc, c_sdec, byte1, enc1);
+        if (RHT_COL) {
+          enc0 *= 0.25f;
+          enc1 *= 0.25f;
         }
       }
-      uint2 codes0 = convert16<SR>(f0, enc0, rnd0);
-      uint2 codes1 = convert16<SR>(f1, enc1, rnd1);
+      uint32_t two[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) two[j] = 0u;
+      if (SR) {
+        // low / high byte of two[j] = draw of source element (row 16q + j, column 2cp / 2cp + 1)
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          two[j] = *reinterpret_cast<const uint16_t*>(smem + QuantSmem::kRand + (q * 16 + j) * 128 + cp * 2);
+      }
+      uint2 codes0 = convert16<SR>(f0, enc0, Nu14FromPairs<0>{two});
+      uint2 codes1 = convert16<SR>(f1, enc1, Nu14FromPairs<1>{two});
       // staging: column c holds eight 8-byte units, unit q stored at (q ^ (c >> 1)) & 7; the column a
       // lane writes first alternates with bit 3 of the lane so that a half warp covers all banks
       const int sel = (lane >> 3) & 1;
