@@ -21,13 +21,13 @@ namespace nvfp4 {
 namespace pair {
 
 constexpr int kThreads = 448;      // producer, MMA, 2 x 4 epilogue warps, 4 scale warps (2, 11, 12, 13)      // producer, MMA, scale copier, 2 x 4 epilogue warps
-constexpr int kStages = 4;
+constexpr int kStages = 5;
 constexpr int kABytes = 128 * 128;   // 128 rows x 256 K elements
 constexpr int kBBytes = 128 * 128;   // this CTA's half of the 256-row B tile
 constexpr int kSfaBytes = 4 * 512;   // own 128 rows, four K64 steps
 constexpr int kSfbBytes = 8 * 512;   // all 256 rows of B (both CTAs need them), four K64 steps
 constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 38 KB
-constexpr int kStagingBytes = 4 * 16384;  // two 128 x 128-byte store buffers per epilogue group
+constexpr int kStagingBytes = 2 * 16384;  // one 128 x 128-byte store buffer per epilogue group
 constexpr int kSmemBytes = kStages * kStageBytes + kStagingBytes + 1024 /*alignment*/ + 256 /*barriers*/;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSfCol = 256;          // after the 256 accumulator columns: one 48-column slot per stage
@@ -170,9 +170,9 @@ __device__ __forceinline__ void store_half(const uint32_t (&r)[128], float alpha
   constexpr int kChunkCols = FP32 ? 32 : 64;
 #pragma unroll
   for (int c = 0; c < kChunks; ++c) {
-    if (et == 0) bulk_wait_read<1>();
+    if (et == 0) bulk_wait_read<0>();
     asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-    const uint32_t srow = stage_buf + buf * 16384 + row_in_tile * 128;
+    const uint32_t srow = stage_buf + row_in_tile * 128;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       uint32_t p[4];
@@ -195,9 +195,9 @@ __device__ __forceinline__ void store_half(const uint32_t (&r)[128], float alpha
     asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
     if (et == 0) {
       if (accumulate)
-        tma_reduce_add_2d(map_d, x0 + c * kChunkCols, row0, stage_buf + buf * 16384);
+        tma_reduce_add_2d(map_d, x0 + c * kChunkCols, row0, stage_buf);
       else
-        tma_store_2d(map_d, x0 + c * kChunkCols, row0, stage_buf + buf * 16384);
+        tma_store_2d(map_d, x0 + c * kChunkCols, row0, stage_buf);
       bulk_commit();
     }
     buf ^= 1;
@@ -394,7 +394,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     const uint32_t acce_leader = map_to_cta(acce_bar, 0);
     const int row_in_tile = quad * 32 + lane;
     const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + half * 128;
-    const uint32_t stage_buf = staging + half * 32768;
+    const uint32_t stage_buf = staging + half * 16384;
     int buf = 0;
     for (int tile = pair_id; tile < n_tiles; tile += n_pairs) {
       int m_blk, n_blk;
