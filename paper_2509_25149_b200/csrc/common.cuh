@@ -114,6 +114,44 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
 }
 
 // ---------------------------------------------------------------------------------------------
+// Packed FP32 pairs (sm_100: add / sub / mul .f32x2 process two binary32 lanes per instruction, each lane
+// rounded to nearest exactly like the scalar instruction)
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+  float2 r;
+  asm("{.reg .b64 ra, rb, rc; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %5}; add.rn.f32x2 rc, ra, rb; mov.b64 {%0, %1}, rc;}"
+      : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return r;
+}
+__device__ __forceinline__ float2 sub2(float2 a, float2 b) {
+  float2 r;
+  asm("{.reg .b64 ra, rb, rc; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %5}; sub.rn.f32x2 rc, ra, rb; mov.b64 {%0, %1}, rc;}"
+      : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return r;
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+  float2 r;
+  asm("{.reg .b64 ra, rb, rc; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %5}; mul.rn.f32x2 rc, ra, rb; mov.b64 {%0, %1}, rc;}"
+      : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return r;
+}
+
+// 16-point butterfly on sixteen pairs: .x and .y are two independent transforms (two adjacent columns)
+__device__ __forceinline__ void fwht16_pairs(float2 v[16]) {
+#pragma unroll
+  for (int h = 1; h < 16; h <<= 1) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      if ((i & h) == 0) {
+        const float2 a = v[i], b = v[i | h];
+        v[i] = add2(a, b);
+        v[i | h] = sub2(a, b);
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // 16-point Walsh-Hadamard butterfly (Sylvester order) on registers; the caller applies the 1/4.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void fwht16(float v[16]) {

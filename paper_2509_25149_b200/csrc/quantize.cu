@@ -190,10 +190,14 @@ struct QuantSmem {
 template <bool SR, class Nu14>
 __device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, Nu14 nu14) {
   uint2 out;
-  if (!SR) {
-    float v[16];
+  float v[16];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(f[i], s_enc_b);
+  for (int i = 0; i < 16; i += 2) {  // Eq. 4: v = fl(y * s_enc,b), two lanes per instruction
+    const float2 p = mul2(make_float2(f[i], f[i + 1]), make_float2(s_enc_b, s_enc_b));
+    v[i] = p.x;
+    v[i + 1] = p.y;
+  }
+  if (!SR) {
     const float(&lo)[8] = *reinterpret_cast<const float(*)[8]>(&v[0]);
     const float(&hi)[8] = *reinterpret_cast<const float(*)[8]>(&v[8]);
     out.x = e2m1x8_rne(lo);
@@ -202,7 +206,7 @@ __device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, 
     uint32_t w[2] = {0u, 0u};
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-      const uint32_t nib = e2m1_sr_bits(__fmul_rn(f[i], s_enc_b), nu14(i));
+      const uint32_t nib = e2m1_sr_bits(v[i], nu14(i));
       w[i >> 3] = __funnelshift_r(w[i >> 3], nib, 4);  // shifts the new nibble in from the top
     }
     out.x = w[0];
@@ -385,8 +389,15 @@ __global__ void __launch_bounds__(256) quantize_kernel(const QuantArgs a) {
         f1[j] = bf16_hi(word);
       }
       if (RHT_COL) {  // values are 4 * y from here on; the 1/4 is folded into amax and encode scale (exact)
-        fwht16(f0);
-        fwht16(f1);
+        float2 v[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = make_float2(f0[j], f1[j]);
+        fwht16_pairs(v);  // both columns in one pass of packed adds
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          f0[j] = v[j].x;
+          f1[j] = v[j].y;
+        }
       }
       uint32_t byte0, byte1;
       float enc0, enc1;
