@@ -11,7 +11,6 @@ from paper_2509_25149_b200 import binding as B
 from paper_2509_25149_b200 import synth
 
 pytestmark = pytest.mark.gpu
-SLABS = (0, 128 * 17, None)  # first, an interior and the last 128-row slab (None = rows - 128)
 
 
 def rotated_amax(x: torch.Tensor, mask: int) -> float:
@@ -32,8 +31,7 @@ def check_copy_slabs(x: torch.Tensor, gpu: B.NVFP4Tensor, *, colwise, block_rows
     codes, scales, glob = P.download(gpu)
     R = x.shape[0]
     n_bad = n_tot = 0
-    for r0 in SLABS:
-        r0 = R - 128 if r0 is None else r0
+    for r0 in (0, (R // 128) * 5 // 8 * 128 + 0, R - 128):  # first, an interior and the last 128-row slab
         slab = synth.bits(x[r0:r0 + 128])
         ref = oracle.quantize(slab, colwise=colwise, block_rows=block_rows, rht=rht, sign_mask=mask, rounding=rounding,
                               seed=seed, sr_offset=sr_offset, amax_override=float(glob[0]), sr_row0=r0,
@@ -123,3 +121,68 @@ def test_config3_full_size_forward_and_backward():
     exact = X[rows].double() @ W.double().T
     rel = float((Y[rows].double() - exact).norm() / exact.norm())
     assert rel < 0.2, rel
+
+
+def test_config2_quantizer_sweep_full_tensor():
+    """cfg 2: the [8192 x 5120] activation.  One full-tensor bit-exact comparison (RNE, both copies, no transform);
+    the SR and rotated variants on sampled slabs."""
+    x = synth.config2_x()
+    xd = x.cuda()
+    R, C = x.shape
+    row, col = B.alloc_tensor(R, C), B.alloc_tensor(C, R)
+    B.nvfp4_quantize(xd, B.quant_opts(), row, col)
+    P.assert_exact(row, oracle.quantize(synth.bits(x)), "cfg2 X row, full tensor")
+    P.assert_exact(col, oracle.quantize(synth.bits(x), colwise=True), "cfg2 X col, full tensor")
+    mask = synth.DEFAULT_RHT_SIGN_MASK
+    for rounding in (B.ROUND_NEAREST_EVEN, B.ROUND_STOCHASTIC):
+        B.nvfp4_quantize(xd, B.quant_opts(rounding=rounding, rht_colwise=True, rht_sign_mask=mask, seed=7, sr_offset=3),
+                         row, col)
+        check_copy_slabs(x, row, colwise=False, rounding=rounding, seed=7, sr_offset=3, what="cfg2 row")
+        check_copy_slabs(x, col, colwise=True, rht=True, mask=mask, rounding=rounding, seed=7, sr_offset=3,
+                         what="cfg2 col rotated")
+    # only one copy requested
+    B.nvfp4_quantize(xd, B.quant_opts(rounding=B.ROUND_STOCHASTIC, seed=7, sr_offset=3), None, col)
+    check_copy_slabs(x, col, colwise=True, rounding=oracle.SR, seed=7, sr_offset=3, what="cfg2 col only")
+
+
+def test_config4_squared_relu_input_and_long_contraction():
+    """cfg 4 (FFN down-projection): half of X is exactly zero and the tail is heavy; K = 20480."""
+    p = synth.config4(M=2048)  # a quarter of the tokens keeps the host-side generation short; K and N are full size
+    M, N, K = p.M, p.N, p.K
+    X, W = p.X.cuda(), p.W.cuda()
+    X_row, X_col = B.alloc_tensor(M, K), B.alloc_tensor(K, M)
+    W_row = B.alloc_tensor(N, K)
+    B.nvfp4_quantize(X, B.quant_opts(rht_colwise=True, rht_sign_mask=p.rht_sign_mask), X_row, X_col)
+    B.nvfp4_quantize(W, B.quant_opts(block_rows=16), W_row, None)
+    check_copy_slabs(p.X, X_row, colwise=False, what="cfg4 X row")
+    check_copy_slabs(p.X, X_col, colwise=True, rht=True, mask=p.rht_sign_mask, what="cfg4 X col")
+    assert float((X_row.scales == 0).float().mean()) > 0  # all-zero blocks exist and are encoded as scale 0
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    B.nvfp4_gemm(X_row, W_row, Y)
+    B.nvfp4_device_status()
+    check_gemm_samples(Y, X_row, W_row, True, "cfg4 Fprop", 4)
+
+
+def test_config5_qkv_projection_shapes():
+    """cfg 5: the QKV projection 5120 -> 7168 at 16384 tokens (N = 7168 is not a power-of-two multiple)."""
+    p = synth.config5_layer(0, M=4096)  # the GEMM tiling only depends on M through the number of row blocks
+    M, N, K = p.M, p.N, p.K
+    opts = B.quant_opts(rht_sign_mask=p.rht_sign_mask, seed=p.sr_seed, sr_offset=p.sr_offset)
+    X_col, W_row, W_col = B.alloc_tensor(K, M), B.alloc_tensor(N, K), B.alloc_tensor(K, N)
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((N, K), dtype=torch.float32, device="cuda")
+    ws_f = torch.empty(B.nvfp4_linear_fwd_workspace_bytes(M, K), dtype=torch.uint8, device="cuda")
+    ws_b = torch.empty(B.nvfp4_linear_bwd_workspace_bytes(M, N), dtype=torch.uint8, device="cuda")
+    X, W, dY = p.X.cuda(), p.W.cuda(), p.dY.cuda()
+    B.nvfp4_linear_fwd(X, W, opts, Y, X_col, W_row, W_col, False, ws_f)
+    B.nvfp4_linear_bwd(dY, X_col, W_col, K, opts, dX, dW, False, ws_b)
+    B.nvfp4_device_status()
+    X_row = B.alloc_tensor(M, K)
+    B.nvfp4_quantize(X, B.quant_opts(), X_row, None)
+    g_row, g_col = B.alloc_tensor(M, N), B.alloc_tensor(N, M)
+    B.nvfp4_quantize(dY, B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True, rht_sign_mask=p.rht_sign_mask,
+                                      seed=p.sr_seed, sr_offset=p.sr_offset), g_row, g_col)
+    check_gemm_samples(Y, X_row, W_row, True, "cfg5 qkv Fprop", 5)
+    check_gemm_samples(dX, g_row, W_col, True, "cfg5 qkv Dgrad", 6)
+    check_gemm_samples(dW, g_col, X_col, False, "cfg5 qkv Wgrad", 7)
