@@ -380,8 +380,105 @@ def run_case(args):
     print(json.dumps({"case": args.case, "shape": [r, c, k], "ms": ms, "value": work / (ms * 1e-3), "unit": unit}))
 
 
+# ------------------------------------------- other 12B-class configs (extra measurements) ----
+def run_config(args):
+    """Times fwd + bwd of every linear layer of cfg 4 (FFN down) or cfg 5 (all four linears of a block, 16384
+    tokens): per-kernel CUDA-event times and the whole sequence.  Inputs are drawn on the device with the shapes
+    and distributions of the config (timing only; parity for these shapes is covered by the tests)."""
+    import torch
+
+    from paper_2509_25149_b200 import binding as B
+    from paper_2509_25149_b200 import synth
+
+    torch.cuda.set_device(0)
+    gen = torch.Generator(device="cuda").manual_seed(1000 * args.config)
+    layers = {4: [("ffn_down", 8192, 5120, 20480, True)],
+              5: [("qkv", 16384, 7168, 5120, False), ("out_proj", 16384, 5120, 5120, False),
+                  ("ffn_up", 16384, 20480, 5120, False), ("ffn_down", 16384, 5120, 20480, True)]}[args.config]
+    mask = synth.DEFAULT_RHT_SIGN_MASK
+    built = []
+    for li, (name, m, n, k, relu2) in enumerate(layers):
+        x = torch.randn((m, k), generator=gen, device="cuda", dtype=torch.float32)
+        if relu2:
+            x = torch.clamp_min(x, 0).square_()
+        else:
+            x = torch.where(torch.rand((m, k), generator=gen, device="cuda") < 0.001, x * 100.0, x)
+        X = x.to(torch.bfloat16)
+        del x
+        W = (torch.randn((n, k), generator=gen, device="cuda", dtype=torch.float32) * (0.01 if args.config == 4 else 0.02)).to(torch.bfloat16)
+        dY = (torch.randn((m, n), generator=gen, device="cuda", dtype=torch.float32) * 1e-4).to(torch.bfloat16)
+        bufs = dict(X=X, W=W, dY=dY, x_row=B.alloc_tensor(m, k), X_col=B.alloc_tensor(k, m), W_row=B.alloc_tensor(n, k),
+                    W_col=B.alloc_tensor(k, n), g_row=B.alloc_tensor(m, n), g_col=B.alloc_tensor(n, m),
+                    Y=torch.empty((m, n), dtype=torch.bfloat16, device="cuda"),
+                    dX=torch.empty((m, k), dtype=torch.bfloat16, device="cuda"),
+                    dW=torch.empty((n, k), dtype=torch.float32, device="cuda"),
+                    ws_f=torch.empty(B.nvfp4_linear_fwd_workspace_bytes(m, k), dtype=torch.uint8, device="cuda"),
+                    ws_b=torch.empty(B.nvfp4_linear_bwd_workspace_bytes(m, n), dtype=torch.uint8, device="cuda"),
+                    opts=B.quant_opts(rht_sign_mask=mask, seed=0, sr_offset=li))
+        built.append((name, m, n, k, bufs))
+
+    def step():
+        for name, m, n, k, b in built:
+            B.nvfp4_linear_fwd(b["X"], b["W"], b["opts"], b["Y"], b["X_col"], b["W_row"], b["W_col"], False, b["ws_f"])
+        for name, m, n, k, b in reversed(built):
+            B.nvfp4_linear_bwd(b["dY"], b["X_col"], b["W_col"], k, b["opts"], b["dX"], b["dW"], False, b["ws_b"])
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    B.nvfp4_device_status()
+    ms_step = e0.elapsed_time(e1) / args.steps
+
+    out_layers = {}
+    tot_flops = tot_qbytes = tot_gemm_ms = tot_q_ms = 0.0
+    for name, m, n, k, b in built:
+        calls = [
+            ("quant_W", lambda: B.nvfp4_quantize(b["W"], B.quant_opts(block_rows=16), b["W_row"], b["W_col"])),
+            ("quant_X", lambda: B.nvfp4_quantize(b["X"], B.quant_opts(rht_colwise=True, rht_sign_mask=mask), b["x_row"], b["X_col"])),
+            ("gemm_fprop", lambda: B.nvfp4_gemm(b["x_row"], b["W_row"], b["Y"])),
+            ("quant_dY", lambda: B.nvfp4_quantize(b["dY"], B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True,
+                                                                          rht_sign_mask=mask), b["g_row"], b["g_col"])),
+            ("gemm_dgrad", lambda: B.nvfp4_gemm(b["g_row"], b["W_col"], b["dX"])),
+            ("gemm_wgrad", lambda: B.nvfp4_gemm(b["g_col"], b["X_col"], b["dW"])),
+        ]
+        per = {c[0]: [] for c in calls}
+        for it in range(12):
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)]
+            evs[0].record()
+            for i, (_, fn) in enumerate(calls):
+                fn()
+                evs[i + 1].record()
+            torch.cuda.synchronize()
+            if it >= 2:
+                for i, (cn, _) in enumerate(calls):
+                    per[cn].append(evs[i].elapsed_time(evs[i + 1]))
+        km = {c: sum(v) / len(v) for c, v in per.items()}
+        g_ms = km["gemm_fprop"] + km["gemm_dgrad"] + km["gemm_wgrad"]
+        q_ms = km["quant_W"] + km["quant_X"] + km["quant_dY"]
+        q_bytes = (m * k + n * k + m * n) * 5.125
+        out_layers[name] = {"M": m, "N": n, "K": k, "kernel_ms": {c: round(v, 4) for c, v in km.items()},
+                            "gemm_tflops": round(3 * 2.0 * m * n * k / (g_ms * 1e-3) / 1e12, 1),
+                            "quant_gbs": round(q_bytes / (q_ms * 1e-3) / 1e9, 1)}
+        tot_flops += 3 * 2.0 * m * n * k
+        tot_qbytes += q_bytes
+        tot_gemm_ms += g_ms
+        tot_q_ms += q_ms
+    print(json.dumps({"config": args.config, "ms_per_step": ms_step, "value": tot_flops / (ms_step * 1e-3) / 1e12,
+                      "unit": "TFLOP/s", "gemm_tflops": tot_flops / (tot_gemm_ms * 1e-3) / 1e12,
+                      "quant_gbs": tot_qbytes / (tot_q_ms * 1e-3) / 1e9, "layers": out_layers, "steps": args.steps,
+                      "data": "synthetic (device generator)"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--config", type=int, default=3, choices=[3, 4, 5],
+                    help="3 = the benchmark workload (default); 4 / 5 = extra measurements of the other 12B-class configs")
     ap.add_argument("--case", default=None, choices=sorted(CASES), help="run one kernel on a reduced shape")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
@@ -391,6 +488,8 @@ def main():
     args = ap.parse_args()
     if args.case:
         run_case(args)
+    elif args.config != 3:
+        run_config(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
