@@ -82,19 +82,33 @@ __device__ __forceinline__ uint32_t e2m1x8_rne(const float v[8]) {
 // D = ((255 - u) << 14) + 0x1FFF carries out of the discarded bits; (bits + D) >> 22 is then
 // 2 * exponent + mantissa bit = code + 252.  Below 1 the grid is uniform (step 0.5): x = a + 1 rounded UP has
 // mantissa ceil(a * 2^23), the comparison with the integer threshold survives the ceiling, and the same carry
-// trick on x gives code + 254.  `nu` is the complemented draw (255 - u) in bits [0, 8).
-__device__ __forceinline__ uint32_t e2m1_sr_bits(float v, uint32_t nu_shifted14) {
-  // nu_shifted14: (255 - u) << 14, other bits zero
+// trick on x gives code + 254.
+// The kernel evaluates this on the pattern shifted left by 7 (one integer multiply-add, on the FMA pipe): the
+// code then sits in the top three bits of the sum, where a funnel shift collects eight codes into a word.
+//   nu21 : (255 - u) << 21, other bits zero.  Returns s with code = s >> 29 (mod 8), bit 28 is a leftover
+//   fraction bit.
+__device__ __forceinline__ uint32_t e2m1_sr_sum(float v, uint32_t nu21) {
   const float a = fminf(fabsf(v), 6.0f);
   const bool small = a < 1.0f;
   const float x = small ? __fadd_ru(a, 1.0f) : a;
-  // + (4 << 22) makes the low three bits of (.. >> 22) equal code for a >= 1 (252 = -4 mod 8 ... 256 - 252);
-  // the small path needs + (2 << 22) instead
-  uint32_t s = __float_as_uint(x) + (nu_shifted14 | 0x01001FFFu);
-  if (small) s -= 0x00800000u;
-  const uint32_t t = s >> 22;
-  // low three bits from t, sign bit (bit 31 of v) into bit 3
-  return (t & 7u) | ((__float_as_uint(v) >> 28) & 8u);
+  // (pattern + D) << 7 with D = ((255 - u) << 14) + 0x1FFF; + (4 << 29) turns (2 * exponent + mantissa bit) mod 8
+  // into the code for a >= 1, the small path needs + (2 << 29) instead
+  uint32_t s = __float_as_uint(x) * 128u + (nu21 | 0x800FFF80u);
+  if (small) s += 0xC0000000u;
+  return s;
+}
+
+// Eight scaled values -> eight E2M1 nibbles with stochastic rounding, element 0 in the lowest nibble.
+template <class Nu21>
+__device__ __forceinline__ uint32_t e2m1x8_sr(const float* v, Nu21 nu21, int base) {
+  uint32_t codes = 0u, signs = 0u;
+#pragma unroll
+  for (int i = 7; i >= 0; --i) {
+    const uint32_t s = e2m1_sr_sum(v[i], nu21(base + i));
+    codes = __funnelshift_l(s, codes, 4);                      // (codes << 4) | top nibble of s = [code, fraction bit]
+    signs = __funnelshift_l(__float_as_uint(v[i]), signs, 4);  // top nibble of v = [sign, exponent bits]
+  }
+  return ((codes >> 1) & 0x77777777u) | (signs & 0x88888888u);
 }
 
 // ---------------------------------------------------------------------------------------------

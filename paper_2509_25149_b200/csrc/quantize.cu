@@ -186,7 +186,7 @@ struct QuantSmem {
 };
 
 // 16 scaled values -> 16 E2M1 nibbles (element 0 in the lowest nibble of .x).  For stochastic rounding `nu14(i)`
-// returns the complemented 8-bit draw of element i placed in bits [14, 22).
+// returns the complemented 8-bit draw of element i placed in bits [21, 29).
 template <bool SR, class Nu14>
 __device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, Nu14 nu14) {
   uint2 out;
@@ -203,14 +203,8 @@ __device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, 
     out.x = e2m1x8_rne(lo);
     out.y = e2m1x8_rne(hi);
   } else {
-    uint32_t w[2] = {0u, 0u};
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const uint32_t nib = e2m1_sr_bits(v[i], nu14(i));
-      w[i >> 3] = __funnelshift_r(w[i >> 3], nib, 4);  // shifts the new nibble in from the top
-    }
-    out.x = w[0];
-    out.y = w[1];
+    out.x = e2m1x8_sr(&v[0], nu14, 0);
+    out.y = e2m1x8_sr(&v[8], nu14, 8);
   }
   return out;
 }
@@ -221,7 +215,7 @@ struct Nu14FromWords {
   __device__ __forceinline__ uint32_t operator()(int i) const {
     const uint32_t nr = ~rnd[i >> 2];
     const int b = i & 3;
-    return (b == 0 ? (nr << 14) : b == 1 ? (nr << 6) : b == 2 ? (nr >> 2) : (nr >> 10)) & 0x003FC000u;
+    return (b == 0 ? (nr << 21) : b == 1 ? (nr << 13) : b == 2 ? (nr << 5) : (nr >> 3)) & 0x1FE00000u;
   }
 };
 // draws of two adjacent columns, 16 bits per row (the transposed copy: read back from shared memory)
@@ -229,7 +223,7 @@ template <int COL>
 struct Nu14FromPairs {
   const uint32_t (&two)[16];
   __device__ __forceinline__ uint32_t operator()(int i) const {
-    return (COL == 0 ? (~two[i] << 14) : (~two[i] << 6)) & 0x003FC000u;
+    return (COL == 0 ? (~two[i] << 21) : (~two[i] << 13)) & 0x1FE00000u;
   }
 };
 
