@@ -312,7 +312,7 @@ def run_cuda(args):
                          "peak_source": f"4 x {peaks['source']} sustained bf16 cuBLAS ({peaks['bf16_tflops_sustained']} TFLOP/s)",
                          "frac_of_burst": gemm_tflops / (4.0 * peaks["bf16_tflops"]),
                          "frac_of_datasheet_9pf": gemm_tflops / 9000.0},
-            "roofline_quant": {"bound": "hbm", "kernel": "amax_kernel + quantize_kernel (W, X, dY)",
+            "roofline_quant": {"bound": "hbm", "kernel": "amax kernels + quantize_kernel (W, X, dY)",
                                "achieved": q_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                "frac": q_gbs / peaks["hbm_gbs"], "traffic": None,
                                "peak_source": f"{peaks['source']} copy bandwidth",

@@ -163,6 +163,99 @@ __global__ void __launch_bounds__(256) amax_kernel(const uint16_t* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------------------------
+// Pass 1 for a copy transformed down the rows (the transposed copy of a Wgrad operand, Appendix C): the
+// 16-point transform of 8 columns at a time is one bf16 tensor-core product  Y(16x8) = A(16x16) * X(16x8)  with
+// A[k][j] = s_j * h(k, j) (entries +-1, exact in bf16; FP32 accumulation) and the 1/4 applied to the maximum.
+// A lane loads 16 columns of one row; its eight words are fragments of eight 8x8 matrices whose "columns" are an
+// interleaved subset of the 64 columns a quad covers - columns are independent under this transform, so any
+// assignment works - and movmatrix turns each into the k-pair layout the product wants.
+// CTA tile 128 rows x 256 columns; a warp owns 16 rows.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t v) {
+  uint32_t r;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(r) : "r"(v));
+  return r;
+}
+
+template <bool PLAIN>
+__global__ void __launch_bounds__(256) amax_rot_col_kernel(const uint16_t* __restrict__ x, int64_t rows,
+                                                           int64_t cols, int64_t ld, uint32_t sign_mask,
+                                                           int tiles_c, float* __restrict__ out_plain0,
+                                                           float* __restrict__ out_plain1,
+                                                           float* __restrict__ out_rot_col) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int64_t tr = blockIdx.x / tiles_c, tc = blockIdx.x % tiles_c;
+  const int64_t r0 = tr * 128 + warp * 16;
+
+  uint32_t lo[4][8], hi[4][8];  // rows g and g + 8 of the slab, 16 columns each, four 64-column steps
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int64_t c = tc * 256 + q * 64 + t * 16;
+    if (r0 < rows && c < cols) {  // rows % 16 == 0, cols % 16 == 0
+      ldg256_stream(x + (r0 + g) * ld + c, lo[q]);
+      ldg256_stream(x + (r0 + 8 + g) * ld + c, hi[q]);
+    } else {
+#pragma unroll
+      for (int w = 0; w < 8; ++w) lo[q][w] = hi[q][w] = 0u;
+    }
+  }
+
+  // A fragments: entry (k, j) = +-1 as bf16, negative iff popc(k & j) is odd XOR sign bit j
+  auto entry = [&](int k, int j) -> uint32_t {
+    return ((__popc(k & j) ^ (sign_mask >> j)) & 1u) ? 0xBF80u : 0x3F80u;
+  };
+  const uint32_t a0 = entry(g, 2 * t) | (entry(g, 2 * t + 1) << 16);
+  const uint32_t a1 = entry(g + 8, 2 * t) | (entry(g + 8, 2 * t + 1) << 16);
+  const uint32_t a2 = entry(g, 2 * t + 8) | (entry(g, 2 * t + 9) << 16);
+  const uint32_t a3 = entry(g + 8, 2 * t + 8) | (entry(g + 8, 2 * t + 9) << 16);
+
+  float m_col = 0.f;
+  uint32_t acc = 0u;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+      if (PLAIN) {
+        acc = absmax_bf16x2(acc, lo[q][w]);
+        acc = absmax_bf16x2(acc, hi[q][w]);
+      }
+      const uint32_t b0 = movmatrix_trans(lo[q][w]);
+      const uint32_t b1 = movmatrix_trans(hi[q][w]);
+      float d0, d1, d2, d3;
+      asm volatile(
+          "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+          "{%10,%10,%10,%10};"
+          : "=f"(d0), "=f"(d1), "=f"(d2), "=f"(d3)
+          : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+      m_col = fmaxf(fmaxf(m_col, fmaxf(fabsf(d0), fabsf(d1))), fmaxf(fabsf(d2), fabsf(d3)));
+    }
+  }
+  m_col *= 0.25f;
+  float m_plain = PLAIN ? fmaxf(bf16_lo(acc), bf16_hi(acc)) : 0.f;
+
+  __shared__ float red[2][8];
+  m_plain = warp_max(m_plain);
+  m_col = warp_max(m_col);
+  if (lane == 0) {
+    red[0][warp] = m_plain;
+    red[1][warp] = m_col;
+  }
+  __syncthreads();
+  if (threadIdx.x < 2) {
+    float m = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) m = fmaxf(m, red[threadIdx.x][w]);
+    const uint32_t bits = __float_as_uint(m);  // non-negative floats order like their bit patterns
+    if (threadIdx.x == 0 && PLAIN) {
+      if (out_plain0) atomicMax(reinterpret_cast<unsigned int*>(out_plain0), bits);
+      if (out_plain1) atomicMax(reinterpret_cast<unsigned int*>(out_plain1), bits);
+    }
+    if (threadIdx.x == 1) atomicMax(reinterpret_cast<unsigned int*>(out_rot_col), bits);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Pass 2: one CTA per 128 x 128 tile of the source.
 //   phase 1  each thread owns four 1x16 chunks (32-byte loads), produces the row-wise copy from
 //            registers and stages the raw tile (and the random bytes) in shared memory;
@@ -558,6 +651,18 @@ cudaError_t launch_amax(const QuantArgs& a, bool has_row, bool has_col, bool rht
   const bool plain = plain0 || plain1;
   float* rot_row = rr ? a.r_global : nullptr;
   float* rot_col = rc ? a.c_global : nullptr;
+  if (rc && !rr) {  // tensor-core transform for the transposed copy
+    const int tiles_c = (int)((a.cols + 255) / 256);
+    const unsigned tiles = (unsigned)(((a.rows + 127) / 128) * tiles_c);
+    if (plain)
+      amax_rot_col_kernel<true><<<tiles, 256, 0, s>>>(a.x, a.rows, a.cols, a.ld, a.sign_mask, tiles_c, plain0, plain1,
+                                                      rot_col);
+    else
+      amax_rot_col_kernel<false><<<tiles, 256, 0, s>>>(a.x, a.rows, a.cols, a.ld, a.sign_mask, tiles_c, plain0,
+                                                       plain1, rot_col);
+    count_launch();
+    return cudaGetLastError();
+  }
 #define NVFP4_AMAX(P, R, C) \
   if (plain == P && rr == R && rc == C) return launch_amax_t<P, R, C>(a, plain0, plain1, rot_row, rot_col, s);
   NVFP4_AMAX(true, false, false)
