@@ -26,6 +26,10 @@ if ROOT not in sys.path:
 METRIC = "NVFP4 GEMM TFLOP/s vs FP4 peak; quantize+RHT+SR GB/s vs HBM peak"
 M, N, K = 8192, 20480, 5120
 WORKLOAD = "cfg3_ffn_up_fwd_bwd_M8192_K5120_N20480"
+# DRAM bytes (read + write) from a one-pass ncu capture of this workload at full size, cold caches
+# (profiles/dram_traffic_cfg3_step.md): mean of Fprop / Dgrad / Wgrad per launch, and the six quantizer kernels summed.
+GEMM_DRAM_BYTES_PER_LAUNCH = (560.2e6 + 541.5e6 + 655.6e6) / 3
+QUANT_DRAM_BYTES_PER_STEP = 1511.3e6
 SLAB = (4096, 2048, 5120)     # tokens, out-features, in-features of the CPU-baseline sample (one run)
 SLAB_REF = (512, 1024, 5120)  # per-step sample of the `--impl reference` arm (many steps)
 
@@ -308,13 +312,16 @@ def run_cuda(args):
             "kernel_ms": {k: round(v, 4) for k, v in kern_ms.items()},
             "roofline": {"bound": "tensor", "kernel": "gemm_kernel (mean of Fprop, Dgrad, Wgrad)",
                          "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
-                         "frac": gemm_tflops / fp4_peak, "traffic": None,
+                         "frac": gemm_tflops / fp4_peak, "traffic": GEMM_DRAM_BYTES_PER_LAUNCH,
+                         "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum, full-size one-pass "
+                                           "capture, mean of the three GEMMs (profiles/dram_traffic_cfg3_step.md)",
                          "peak_source": f"4 x {peaks['source']} sustained bf16 cuBLAS ({peaks['bf16_tflops_sustained']} TFLOP/s)",
                          "frac_of_burst": gemm_tflops / (4.0 * peaks["bf16_tflops"]),
                          "frac_of_datasheet_9pf": gemm_tflops / 9000.0},
             "roofline_quant": {"bound": "hbm", "kernel": "amax kernels + quantize_kernel (W, X, dY)",
                                "achieved": q_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                               "frac": q_gbs / peaks["hbm_gbs"], "traffic": None,
+                               "frac": q_gbs / peaks["hbm_gbs"], "traffic": QUANT_DRAM_BYTES_PER_STEP,
+                               "algorithmic_bytes": q_bytes,
                                "peak_source": f"{peaks['source']} copy bandwidth",
                                "frac_of_datasheet_8tbs": q_gbs / 8000.0},
             "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
@@ -334,6 +341,7 @@ CASES = {
     "quant_x": ("qx", 16384, 5120, 0),             # RNE, row-wise + rotated column-wise (168 MB > L2)
     "quant_dy": ("qdy", 4096, 20480, 0),           # SR, row-wise + rotated column-wise (168 MB > L2)
     "quant_w": ("qw", 20480, 5120, 0),             # 16x16 blocks, both copies (210 MB > L2)
+    "step": ("step", 8192, 20480, 5120),           # the whole cfg 3 fwd + bwd step, full size: ONE-PASS captures only
 }
 
 
@@ -348,7 +356,23 @@ def run_case(args):
     torch.cuda.set_device(0)
     g = torch.Generator(device="cuda").manual_seed(1)
     mask = synth.DEFAULT_RHT_SIGN_MASK
-    if kind in ("gemm", "gemm32"):
+    if kind == "step":
+        X = torch.randn((r, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        W = (torch.randn((c, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
+        dY = (torch.randn((r, c), generator=g, device="cuda", dtype=torch.float32) * 1e-4).to(torch.bfloat16)
+        Y = torch.empty((r, c), dtype=torch.bfloat16, device="cuda")
+        dX = torch.empty((r, k), dtype=torch.bfloat16, device="cuda")
+        dW = torch.empty((c, k), dtype=torch.float32, device="cuda")
+        X_col, W_row, W_col = B.alloc_tensor(k, r), B.alloc_tensor(c, k), B.alloc_tensor(k, c)
+        ws_f = torch.empty(B.nvfp4_linear_fwd_workspace_bytes(r, k), dtype=torch.uint8, device="cuda")
+        ws_b = torch.empty(B.nvfp4_linear_bwd_workspace_bytes(r, c), dtype=torch.uint8, device="cuda")
+        o = B.quant_opts(rht_sign_mask=mask, seed=0, sr_offset=0)
+
+        def fn():
+            B.nvfp4_linear_fwd(X, W, o, Y, X_col, W_row, W_col, False, ws_f)
+            B.nvfp4_linear_bwd(dY, X_col, W_col, k, o, dX, dW, False, ws_b)
+        work, unit = 3 * 2.0 * r * c * k / 1e12, "TFLOP/s"
+    elif kind in ("gemm", "gemm32"):
         a_src = torch.randn((r, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
         b_src = (torch.randn((c, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
         A, Bq = B.alloc_tensor(r, k), B.alloc_tensor(c, k)

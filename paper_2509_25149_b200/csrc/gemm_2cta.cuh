@@ -4,9 +4,10 @@
 // every byte of B is fetched from L2 and read from shared memory once per pair.  That halving of the operand
 // traffic per flop is the point: the one-CTA kernel is bound by shared-memory bandwidth, not by the tensor pipe.
 //
-// Roles per CTA (7 warps): 0 TMA producer (both CTAs; every load signals the LEADER's "full" barrier),
-// 1 MMA issuer (leader only; allocates tensor memory in both), 2 and 11-13 scale warps (both CTAs; shared memory ->
-// registers -> tensor memory, one warp per 32-lane quadrant), 3-10 epilogue (both; two groups of four warps, one per
+// Roles per CTA (14 warps): 0 TMA producer (both CTAs; every load signals the LEADER's "full" barrier),
+// 1 MMA issuer (leader only; allocates tensor memory in both), 2 and 11-13 scale warps (both CTAs; the A scales go
+// shared memory -> registers -> tensor memory, one warp per 32-lane quadrant; the B scales, identical in both CTAs,
+// go through the tensor-memory copy engine, issued once per pair by the leader's warp 2), 3-10 epilogue (both; two groups of four warps, one per
 // 128-column half: tensor memory -> registers -> swizzled staging -> TMA store; the accumulator is released as
 // soon as it has been read).
 // Included by gemm.cu only.
@@ -20,7 +21,7 @@
 namespace nvfp4 {
 namespace pair {
 
-constexpr int kThreads = 448;      // producer, MMA, 2 x 4 epilogue warps, 4 scale warps (2, 11, 12, 13)      // producer, MMA, scale copier, 2 x 4 epilogue warps
+constexpr int kThreads = 448;      // producer, MMA, 2 x 4 epilogue warps, 4 scale warps (2, 11, 12, 13)
 constexpr int kStages = 5;
 constexpr int kABytes = 128 * 128;   // 128 rows x 256 K elements
 constexpr int kBBytes = 128 * 128;   // this CTA's half of the 256-row B tile
@@ -34,6 +35,11 @@ constexpr int kSfCol = 256;          // after the 256 accumulator columns: one 4
 constexpr int kSfSlotCols = 48;      // SFA 4 x 4, SFB 4 x 8
 static_assert(kSfCol + kStages * kSfSlotCols <= 512, "tensor memory budget");
 static_assert(kStageBytes % 1024 == 0, "stages must keep the 1024-byte swizzle alignment");
+// B row groups (of 128) whose scale atoms take the copy engine (0, 1 or 2); the rest go through registers
+#ifndef NVFP4_PAIR_CP_GROUPS
+#define NVFP4_PAIR_CP_GROUPS 0
+#endif
+constexpr int kCpGroups = NVFP4_PAIR_CP_GROUPS;
 
 struct Args {
   int M, N, K;
@@ -143,6 +149,11 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* r) {
       "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
+// shared memory -> tensor memory of BOTH CTAs of the pair (each reads its own shared memory at the descriptor's
+// address): one 512-byte scale atom, broadcast to the four 32-lane quadrants
+__device__ __forceinline__ void tc2_cp_sf(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
@@ -219,8 +230,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
   const uint32_t accf_bar = bar_base + 8u * (4 * kStages);                   // one per CTA
   const uint32_t acce_bar = bar_base + 8u * (4 * kStages + 1);               // leader only, 16 arrivals
   const uint32_t done_bar = bar_base + 8u * (4 * kStages + 2);               // one per CTA, peer arrives
+  auto sfp_bar = [&](int s) { return bar_base + 8u * (4 * kStages + 3 + s); }; // leader only: the peer's atoms landed
   volatile uint32_t* tmem_slot =
-      reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + kStagingBytes + 8 * (4 * kStages + 3));
+      reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + kStagingBytes + 8 * (5 * kStages + 3));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -246,7 +258,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(full_bar(s), 2);   // one arrive.expect_tx from each CTA's producer
-      mbar_init(sff_bar(s), 8);    // four scale warps in each CTA
+      mbar_init(sff_bar(s), 8 + (kCpGroups > 0 ? 1 : 0));  // four scale warps in each CTA (+ the copy engine)
+      mbar_init(sfp_bar(s), 1);
       mbar_init(empty_bar(s), 1);
       mbar_init(sfl_bar(s), 1);
     }
@@ -313,10 +326,32 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     int stage = 0;
     uint32_t phase = 0;
     const uint32_t sff_leader = map_to_cta(sff_bar(0), 0);
+    const uint32_t sfp_leader = map_to_cta(sfp_bar(0), 0);
+    constexpr int kRegCols = 16 + 16 * (2 - kCpGroups);  // columns of the slot written from registers
     for (int tile = pair_id; tile < n_tiles; tile += n_pairs) {
       bool ok = true;
       for (int kb = 0; kb < k_blocks; ++kb) {
         ok = mbar_wait(sfl_bar(stage), phase, abort_flag, 0x500u + stage);
+        if (kCpGroups > 0 && warp == 2 && lane == 0 && ok) {
+          // B scales of row groups [2 - kCpGroups, 2): one copy per atom into both CTAs' tensor memory, issued by
+          // the leader once the peer's atoms have landed too
+          if (!leader) {
+            mbar_arrive_cluster(sfp_leader + 8u * stage);
+          } else {
+            ok = mbar_wait_cluster(sfp_bar(stage), phase, abort_flag, 0x580u + stage);
+            if (ok) {
+              tc_fence_after();
+              const uint32_t lo = (((base + stage * kStageBytes + kABytes + kBBytes + kSfaBytes) >> 4) & 0x3fffu);
+              const uint32_t sf_b = tmem + kSfCol + stage * kSfSlotCols + 16;
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int grp = 2 - kCpGroups; grp < 2; ++grp)
+                  tc2_cp_sf(sf_b + 8 * j + 4 * grp, make_desc(lo + grp * 128 + j * 32, kDescHiSf));
+              tc2_commit_local(sff_bar(stage));
+            }
+          }
+        }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) break;
         const uint32_t sf_s = base + stage * kStageBytes + kABytes + kBBytes + lane * 16;
@@ -325,17 +360,31 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
         for (int j = 0; j < 4; ++j) {
           const uint4 a = lds128(sf_s + j * 512);
           r[4 * j] = a.x; r[4 * j + 1] = a.y; r[4 * j + 2] = a.z; r[4 * j + 3] = a.w;
-#pragma unroll
-          for (int grp = 0; grp < 2; ++grp) {
-            const uint4 b = lds128(sf_s + kSfaBytes + grp * 2048 + j * 512);
-            r[16 + 8 * j + 4 * grp] = b.x; r[16 + 8 * j + 4 * grp + 1] = b.y;
-            r[16 + 8 * j + 4 * grp + 2] = b.z; r[16 + 8 * j + 4 * grp + 3] = b.w;
-          }
         }
         const uint32_t sf_t = tmem + ((uint32_t)(quad * 32) << 16) + kSfCol + stage * kSfSlotCols;
         tc_st16(sf_t, &r[0]);
-        tc_st16(sf_t + 16, &r[16]);
-        tc_st16(sf_t + 32, &r[32]);
+        if (kCpGroups == 0) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int grp = 0; grp < 2; ++grp) {
+              const uint4 b = lds128(sf_s + kSfaBytes + grp * 2048 + j * 512);
+              r[16 + 8 * j + 4 * grp] = b.x; r[16 + 8 * j + 4 * grp + 1] = b.y;
+              r[16 + 8 * j + 4 * grp + 2] = b.z; r[16 + 8 * j + 4 * grp + 3] = b.w;
+            }
+          tc_st16(sf_t + 16, &r[16]);
+          tc_st16(sf_t + 32, &r[32]);
+        } else if (kCpGroups == 1) {
+          // group 0 from registers: columns 16 + 8j .. 16 + 8j + 3 of each step, written four at a time
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint4 b = lds128(sf_s + kSfaBytes + j * 512);
+            asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sf_t + 16 + 8 * j), "r"(b.x),
+                         "r"(b.y), "r"(b.z), "r"(b.w)
+                         : "memory");
+          }
+        }
+        (void)kRegCols;
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
