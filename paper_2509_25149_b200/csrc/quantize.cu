@@ -265,18 +265,26 @@ __global__ void __launch_bounds__(256) amax_rot_col_kernel(const uint16_t* __res
 // Tiles are visited in reverse order so that the end of the tensor, which pass 1 touched last, is read
 // first while it may still sit in L2.
 // ---------------------------------------------------------------------------------------------
-struct QuantSmem {
-  static constexpr int kTile = 0;                    // 128 rows x 256 B of bf16
-  static constexpr int kColCodes = 32768;            // 128 columns x 64 B
+template <int PITCH>
+struct QuantSmemT {
+  static constexpr int kTile = 0;                    // 128 rows of bf16, kTilePitch bytes apart
+  static constexpr int kTilePitch = PITCH;           // 256, or 256 + 16 for the tensor-core transform: eight
+                                                     // consecutive rows then start in eight different 16-byte bank
+                                                     // groups (conflict-free 8x8 matrix loads)
+  static constexpr int kColCodes = 128 * kTilePitch; // 128 columns x 64 B
   static constexpr int kSfRow = kColCodes + 8192;    // 1 KB
   static constexpr int kSfCol = kSfRow + 1024;       // 1 KB
   static constexpr int kBlkEnc = kSfCol + 1024;      // 64 floats (16x16 mode)
   static constexpr int kBlkByte = kBlkEnc + 256;     // 64 bytes
   static constexpr int kGlobalScales = kBlkByte + 64;  // s_enc, s_dec of the row-wise and the column-wise copy
-  static constexpr int kRand = kGlobalScales + 64;   // 128 rows x 128 B (stochastic rounding only)
+  static constexpr int kRand = kGlobalScales + 64;   // 128 rows x 128 B (stochastic rounding only); the 16-byte
+                                                     // chunk cb of row r sits at slot cb ^ ((r >> 2) & 7)
   static constexpr int kBytesNoRand = kRand;
   static constexpr int kBytesRand = kRand + 16384;
 };
+// the transposed copy with the transform uses the padded pitch
+template <bool HAS_COL, bool BLOCK2D, bool RHT_COL>
+using QuantSmemFor = QuantSmemT<256>;
 
 // 16 scaled values -> 16 E2M1 nibbles (element 0 in the lowest nibble of .x).  For stochastic rounding `nu14(i)`
 // returns the complemented 8-bit draw of element i placed in bits [21, 29).
@@ -328,7 +336,8 @@ __device__ __forceinline__ float amax16(const float (&f)[16]) {
 }
 
 template <bool HAS_ROW, bool HAS_COL, bool BLOCK2D, bool RHT_ROW, bool RHT_COL, bool SR>
-__global__ void __launch_bounds__(256) quantize_kernel(const QuantArgs a) {
+__global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const QuantArgs a) {
+  using QuantSmem = QuantSmemFor<HAS_COL, BLOCK2D, RHT_COL>;
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = (int)(gridDim.x - 1 - blockIdx.x);
@@ -380,7 +389,7 @@ __global__ void __launch_bounds__(256) quantize_kernel(const QuantArgs a) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int r = warp * 16 + i * 4 + (lane >> 3);
-      uint8_t* dst = smem + QuantSmem::kTile + r * 256 + cb * 32;
+      uint8_t* dst = smem + QuantSmem::kTile + r * QuantSmem::kTilePitch + cb * 32;
       uint4 h0 = make_uint4(raw[i][0], raw[i][1], raw[i][2], raw[i][3]);
       uint4 h1 = make_uint4(raw[i][4], raw[i][5], raw[i][6], raw[i][7]);
       if (first) {
@@ -430,7 +439,7 @@ __global__ void __launch_bounds__(256) quantize_kernel(const QuantArgs a) {
         uint4 qc = q;
         if (a.off_hi_col != a.off_hi)
           qc = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), a.off_lo, a.off_hi_col, a.seed_lo, a.seed_hi);
-        *reinterpret_cast<uint4*>(smem + QuantSmem::kRand + r * 128 + cb * 16) = qc;
+        *reinterpret_cast<uint4*>(smem + QuantSmem::kRand + r * 128 + ((cb ^ ((r >> 2) & 7)) << 4)) = qc;
       }
     }
     if (HAS_ROW) {
@@ -470,7 +479,7 @@ __global__ void __launch_bounds__(256) quantize_kernel(const QuantArgs a) {
       float f0[16], f1[16];
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        uint32_t word = *reinterpret_cast<const uint32_t*>(smem + QuantSmem::kTile + (q * 16 + j) * 256 + cp * 4);
+        uint32_t word = *reinterpret_cast<const uint32_t*>(smem + QuantSmem::kTile + (q * 16 + j) * QuantSmem::kTilePitch + cp * 4);
         if (RHT_COL) word ^= sign_pair(a.sign_mask, j, j);
         f0[j] = bf16_lo(word);
         f1[j] = bf16_hi(word);
@@ -506,7 +515,8 @@ __global__ void __launch_bounds__(256) quantize_kernel(const QuantArgs a) {
         // low / high byte of two[j] = draw of source element (row 16q + j, column 2cp / 2cp + 1)
 #pragma unroll
         for (int j = 0; j < 16; ++j)
-          two[j] = *reinterpret_cast<const uint16_t*>(smem + QuantSmem::kRand + (q * 16 + j) * 128 + cp * 2);
+          two[j] = *reinterpret_cast<const uint16_t*>(smem + QuantSmem::kRand + (q * 16 + j) * 128 +
+                                                     (((cp >> 3) ^ ((4 * q + (j >> 2)) & 7)) << 4) + (cp & 7) * 2);
       }
       uint2 codes0 = convert16<SR>(f0, enc0, Nu14FromPairs<0>{two});
       uint2 codes1 = convert16<SR>(f1, enc1, Nu14FromPairs<1>{two});
@@ -678,6 +688,7 @@ cudaError_t launch_amax(const QuantArgs& a, bool has_row, bool has_col, bool rht
 template <bool HR, bool HC, bool B2, bool RR, bool RC, bool SR>
 static cudaError_t launch_quant_t(const QuantArgs& a, cudaStream_t s) {
   auto kern = quantize_kernel<HR, HC, B2, RR, RC, SR>;
+  using QuantSmem = QuantSmemFor<HC, B2, RC>;
   const int smem = (SR && HC) ? QuantSmem::kBytesRand : QuantSmem::kBytesNoRand;
   static bool configured = false;  // per instantiation; the attribute is per function and idempotent
   if (!configured) {
