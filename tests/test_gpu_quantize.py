@@ -126,6 +126,21 @@ def test_degenerate_inputs():
     P.assert_exact(r2, oracle.quantize(synth.bits(wide.cpu())[:, :128]), "amax provided")
 
 
+@pytest.mark.parametrize("scale", [1e-30, 1e-36, 3e-39, 1e30])
+@pytest.mark.parametrize("rounding", [B.ROUND_NEAREST_EVEN, B.ROUND_STOCHASTIC])
+def test_extreme_magnitudes_stay_bit_exact(scale, rounding):
+    """Whole tensors near the ends of the bf16 range: the global encode scale clamps at FLT_MAX (amax below
+    2688 / FLT_MAX), block amaxes are denormal (the exact-division path of amax_b / 6), products land in the
+    denormal range (no flush to zero anywhere), and at the top 2688 / amax is itself tiny."""
+    x = (synth.normal_bf16((128, 256), 1.0, 21).float() * scale).to(torch.bfloat16)
+    x[3, 16:32] = 0.0
+    for block_rows in (1, 16):
+        row, col = P.gpu_quantize(x, colwise=True, block_rows=block_rows, rounding=rounding, seed=5, sr_offset=9)
+        kw = dict(block_rows=block_rows, rounding=rounding, seed=5, sr_offset=9)
+        P.assert_exact(row, oracle.quantize(synth.bits(x), **kw), f"row scale {scale} blocks {block_rows}")
+        P.assert_exact(col, oracle.quantize(synth.bits(x), colwise=True, **kw), f"col scale {scale} blocks {block_rows}")
+
+
 def test_gpu_sr_is_unbiased_over_seeds():
     x = rand_bf16((128, 128), 8, std=1e-3)
     xd = x.cuda()
