@@ -28,3 +28,23 @@ def allreduce_weight_grad(dW: torch.Tensor) -> None:
     assert dW.dtype == torch.float32
     if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
         dist.all_reduce(dW, op=dist.ReduceOp.SUM)
+
+
+def weight_grad_shard(n_rows: int, rank: int, world: int) -> tuple[int, int]:
+    """[begin, end) of the rows of dW a rank owns when the optimizer state is sharded (rows split evenly)."""
+    assert n_rows % world == 0, "output features must split evenly across ranks"
+    per = n_rows // world
+    return rank * per, (rank + 1) * per
+
+
+def reduce_scatter_weight_grad(dW: torch.Tensor, out: torch.Tensor) -> None:
+    """FP32 sum of dW over all ranks, each rank receiving only its own row shard (`weight_grad_shard`) in `out`:
+    the exchange for a sharded optimizer, half the bytes of the all-reduce.  Without a process group `out` is a
+    copy of dW."""
+    assert dW.dtype == torch.float32 and out.dtype == torch.float32 and dW.is_contiguous() and out.is_contiguous()
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        assert out.numel() * dist.get_world_size() == dW.numel()
+        dist.reduce_scatter_tensor(out, dW, op=dist.ReduceOp.SUM)
+    else:
+        assert out.numel() == dW.numel()
+        out.copy_(dW.view_as(out))

@@ -35,7 +35,11 @@ def _worker(rank, world, port, out):
         b, e = dp.token_shard(512, rank, world)
         dW_local, _ = _wgrad(X[b:e], dY[b:e], rank, synth.DEFAULT_RHT_SIGN_MASK)
         dW = torch.from_numpy(dW_local.astype(np.float32))
+        shard = torch.empty((48 // world, 64), dtype=torch.float32)
+        dp.reduce_scatter_weight_grad(dW.clone(), shard)
         dp.allreduce_weight_grad(dW)
+        b0, e0 = dp.weight_grad_shard(48, rank, world)
+        assert torch.equal(shard, dW[b0:e0]), "reduce-scatter shard differs from the rows of the all-reduced dW"
         # replicated weights quantize to identical bytes on every rank (deterministic RNE)
         W = synth.normal_bf16((48, 64), 0.02, 3)
         wq = torch.from_numpy(oracle.quantize(synth.bits(W), block_rows=16).codes.copy())
@@ -75,3 +79,6 @@ def test_token_shard_and_offsets():
     t = torch.ones(4)
     dp.allreduce_weight_grad(t)  # no process group: no-op
     assert torch.equal(t, torch.ones(4))
+    o = torch.empty(4)
+    dp.reduce_scatter_weight_grad(t, o)
+    assert torch.equal(o, t) and dp.weight_grad_shard(20480, 1, 8) == (2560, 5120)
