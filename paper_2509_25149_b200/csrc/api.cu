@@ -77,8 +77,9 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
   return NVFP4_OK;
 }
 
-nvfp4_status gemm_impl(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D, int32_t d_is_fp32, int64_t ldd,
-                       int32_t accumulate, cudaStream_t s) {
+// argument checks of one GEMM and its launch description
+nvfp4_status gemm_prepare(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D, int32_t d_is_fp32, int64_t ldd,
+                          int32_t accumulate, GemmArgs& g) {
   if (!A || !B || !D) return NVFP4_ERR_NULL;
   if (!A->codes || !A->scales || !A->global || !B->codes || !B->scales || !B->global) return NVFP4_ERR_NULL;
   if (A->cols != B->cols) return NVFP4_ERR_SHAPE;
@@ -92,12 +93,18 @@ nvfp4_status gemm_impl(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D, in
   if ((ldd * esz) % 16 != 0 || !aligned(D, 16)) return NVFP4_ERR_ALIGN;
   if (!aligned(A->codes, 16) || !aligned(B->codes, 16) || !aligned(A->scales, 16) || !aligned(B->scales, 16))
     return NVFP4_ERR_ALIGN;
-  GemmArgs g{};
+  g = GemmArgs{};
   g.sfa = A->scales; g.sfb = B->scales;
   g.a_global = A->global; g.b_global = B->global;
   g.d = D; g.ldd = ldd;
   g.M = (int)M; g.N = (int)N; g.K = (int)K;
   g.d_is_fp32 = d_is_fp32 != 0; g.accumulate = accumulate != 0;
+  return NVFP4_OK;
+}
+
+int gemm_tile(const GemmArgs& g) {
+  const int M = g.M, N = g.N, K = g.K;
+  const int d_is_fp32 = g.d_is_fp32;
   // CTA pairs on 256 x 256 tiles whenever the shape allows (half the operand traffic per flop, half the
   // scale-copy and MMA issue work per SM).  Otherwise one CTA per tile: 128 x 256 tiles hold one accumulator
   // (exposed epilogue), 128 x 128 tiles two (the epilogue overlaps the next tile), so the wide tile pays off
@@ -109,7 +116,15 @@ nvfp4_status gemm_impl(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D, in
     else
       tile_n = (K >= (d_is_fp32 ? 16384 : 8192)) ? 256 : 128;
   }
-  if (launch_gemm(g, A->codes, B->codes, tile_n, s) != cudaSuccess) return NVFP4_ERR_CUDA;
+  return tile_n;
+}
+
+nvfp4_status gemm_impl(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D, int32_t d_is_fp32, int64_t ldd,
+                       int32_t accumulate, cudaStream_t s) {
+  GemmArgs g;
+  nvfp4_status st = gemm_prepare(A, B, D, d_is_fp32, ldd, accumulate, g);
+  if (st != NVFP4_OK) return st;
+  if (launch_gemm(g, A->codes, B->codes, gemm_tile(g), s) != cudaSuccess) return NVFP4_ERR_CUDA;
   return NVFP4_OK;
 }
 
@@ -209,6 +224,20 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, c
   go.flags = opts->flags & NVFP4_SR_INDEPENDENT_COPIES;
   if ((st = quantize_impl(dY, M, N, N, &go, dX_bf16 ? &g_row : nullptr, dW_fp32 ? &g_col : nullptr, s)) != NVFP4_OK)
     return st;
+  if (dX_bf16 && dW_fp32) {
+    // Dgrad and Wgrad are independent: when both run on CTA pairs they share one launch, the longer contraction
+    // first, so the partial last round of one is filled with tiles of the other
+    GemmArgs gd, gw;
+    if ((st = gemm_prepare(&g_row, W_col_saved, dX_bf16, 0, K, 0, gd)) != NVFP4_OK) return st;
+    if ((st = gemm_prepare(&g_col, X_col_saved, dW_fp32, 1, K, accumulate_dw, gw)) != NVFP4_OK) return st;
+    if (gemm_tile(gd) == 512 && gemm_tile(gw) == 512) {
+      const bool dgrad_first = gd.K >= gw.K;
+      const cudaError_t e = dgrad_first
+                                ? launch_gemm_two(gd, g_row.codes, W_col_saved->codes, gw, g_col.codes, X_col_saved->codes, s)
+                                : launch_gemm_two(gw, g_col.codes, X_col_saved->codes, gd, g_row.codes, W_col_saved->codes, s);
+      return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+    }
+  }
   if (dX_bf16 && (st = gemm_impl(&g_row, W_col_saved, dX_bf16, 0, K, 0, s)) != NVFP4_OK) return st;
   if (dW_fp32 && (st = gemm_impl(&g_col, X_col_saved, dW_fp32, 1, K, accumulate_dw, s)) != NVFP4_OK) return st;
   return NVFP4_OK;

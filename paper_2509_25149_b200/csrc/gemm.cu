@@ -323,16 +323,32 @@ cudaError_t launch_t(const GemmArgs& g, const void* a_codes, const void* b_codes
   return cudaGetLastError();
 }
 
-cudaError_t launch_pair(const GemmArgs& g, const void* a_codes, const void* b_codes, int num_sms, cudaStream_t s) {
-  CUtensorMap map_a, map_b, map_d;
-  bool ok = make_code_map(&map_a, a_codes, g.M, g.K / 2, 128) && make_code_map(&map_b, b_codes, g.N, g.K / 2, 128);
+bool make_pair_maps(const GemmArgs& g, const void* a_codes, const void* b_codes, CUtensorMap* map_a, CUtensorMap* map_b,
+                    CUtensorMap* map_d) {
+  bool ok = make_code_map(map_a, a_codes, g.M, g.K / 2, 128) && make_code_map(map_b, b_codes, g.N, g.K / 2, 128);
   if (g.d_is_fp32)
-    ok = ok && make_map_2d(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g.d, (uint64_t)g.N, (uint64_t)g.M,
+    ok = ok && make_map_2d(map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g.d, (uint64_t)g.N, (uint64_t)g.M,
                            (uint64_t)g.ldd * 4, 32, 128, true);
   else
-    ok = ok && make_map_2d(&map_d, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, g.d, (uint64_t)g.N, (uint64_t)g.M,
+    ok = ok && make_map_2d(map_d, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, g.d, (uint64_t)g.N, (uint64_t)g.M,
                            (uint64_t)g.ldd * 2, 64, 128, true);
-  if (!ok) return cudaErrorInvalidValue;
+  return ok;
+}
+
+pair::Problem pair_problem(const GemmArgs& g) {
+  return pair::Problem{g.M, g.N, g.K, g.sfa, g.sfb, g.a_global, g.b_global, g.d_is_fp32, g.accumulate};
+}
+
+// g1 == nullptr: one problem
+cudaError_t launch_pair(const GemmArgs& g0, const void* a0, const void* b0, const GemmArgs* g1, const void* a1,
+                        const void* b1, int num_sms, cudaStream_t s) {
+  CUtensorMap m[6];
+  if (!make_pair_maps(g0, a0, b0, &m[0], &m[1], &m[2])) return cudaErrorInvalidValue;
+  if (g1) {
+    if (!make_pair_maps(*g1, a1, b1, &m[3], &m[4], &m[5])) return cudaErrorInvalidValue;
+  } else {
+    m[3] = m[0]; m[4] = m[1]; m[5] = m[2];
+  }
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(pair::gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -340,18 +356,19 @@ cudaError_t launch_pair(const GemmArgs& g, const void* a_codes, const void* b_co
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  const int n_tiles = (g.M / 256) * (g.N / 256);
+  pair::Args a{};
+  a.p[0] = pair_problem(g0);
+  a.p[1] = pair_problem(g1 ? *g1 : g0);
+  a.n_tiles0 = (g0.M / 256) * (g0.N / 256);
+  a.n_tiles = a.n_tiles0 + (g1 ? (g1->M / 256) * (g1->N / 256) : 0);
   const int max_pairs = num_sms / 2;
-  const int pairs = n_tiles < max_pairs ? n_tiles : max_pairs;
-  pair::Args a{g.M, g.N, g.K, g.sfa, g.sfb, g.a_global, g.b_global, g.d_is_fp32, g.accumulate};
-  pair::gemm_pair_kernel<<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(map_a, map_b, map_d, a);
+  const int pairs = a.n_tiles < max_pairs ? a.n_tiles : max_pairs;
+  pair::gemm_pair_kernel<<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5], a);
   count_launch();
   return cudaGetLastError();
 }
 
-}  // namespace
-
-cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_codes, int tile_n, cudaStream_t s) {
+cudaError_t sm_count(int* n) {
   static int num_sms = 0;
   if (!num_sms) {
     int dev = 0;
@@ -360,9 +377,28 @@ cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_co
     e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
   }
-  if (tile_n == 512 && g.M % 256 == 0 && g.N % 256 == 0) return launch_pair(g, a_codes, b_codes, num_sms, s);
+  *n = num_sms;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_codes, int tile_n, cudaStream_t s) {
+  int num_sms = 0;
+  cudaError_t e = sm_count(&num_sms);
+  if (e != cudaSuccess) return e;
+  if (tile_n == 512 && g.M % 256 == 0 && g.N % 256 == 0)
+    return launch_pair(g, a_codes, b_codes, nullptr, nullptr, nullptr, num_sms, s);
   if (tile_n == 256 && g.N % 256 == 0) return launch_t<256>(g, a_codes, b_codes, num_sms, s);
   return launch_t<128>(g, a_codes, b_codes, num_sms, s);
+}
+
+cudaError_t launch_gemm_two(const GemmArgs& g0, const void* a0, const void* b0, const GemmArgs& g1, const void* a1,
+                            const void* b1, cudaStream_t s) {
+  int num_sms = 0;
+  cudaError_t e = sm_count(&num_sms);
+  if (e != cudaSuccess) return e;
+  return launch_pair(g0, a0, b0, &g1, a1, b1, num_sms, s);
 }
 
 cudaError_t read_device_status(cudaStream_t s, uint32_t* code) {

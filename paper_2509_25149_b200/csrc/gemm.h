@@ -18,6 +18,10 @@ struct GemmArgs {
 
 // tile_n: 128 or 256 (256 needs N % 256 == 0, otherwise 128 is used)
 cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_codes, int tile_n, cudaStream_t s);
+// Two independent GEMMs in one launch of the CTA-pair kernel (all of M, N multiples of 256, K of 256): the tiles of
+// g0 are worked through first, then those of g1, on one persistent grid.
+cudaError_t launch_gemm_two(const GemmArgs& g0, const void* a0, const void* b0, const GemmArgs& g1, const void* a1,
+                            const void* b1, cudaStream_t s);
 cudaError_t read_device_status(cudaStream_t s, uint32_t* code);
 
 }  // namespace nvfp4

@@ -5,9 +5,8 @@
 // traffic per flop is the point: the one-CTA kernel is bound by shared-memory bandwidth, not by the tensor pipe.
 //
 // Roles per CTA (14 warps): 0 TMA producer (both CTAs; every load signals the LEADER's "full" barrier),
-// 1 MMA issuer (leader only; allocates tensor memory in both), 2 and 11-13 scale warps (both CTAs; the A scales go
-// shared memory -> registers -> tensor memory, one warp per 32-lane quadrant; the B scales, identical in both CTAs,
-// go through the tensor-memory copy engine, issued once per pair by the leader's warp 2), 3-10 epilogue (both; two groups of four warps, one per
+// 1 MMA issuer (leader only; allocates tensor memory in both), 2 and 11-13 scale warps (both CTAs; shared memory ->
+// registers -> tensor memory, one warp per 32-lane quadrant), 3-10 epilogue (both; two groups of four warps, one per
 // 128-column half: tensor memory -> registers -> swizzled staging -> TMA store; the accumulator is released as
 // soon as it has been read).
 // Included by gemm.cu only.
@@ -35,19 +34,22 @@ constexpr int kSfCol = 256;          // after the 256 accumulator columns: one 4
 constexpr int kSfSlotCols = 48;      // SFA 4 x 4, SFB 4 x 8
 static_assert(kSfCol + kStages * kSfSlotCols <= 512, "tensor memory budget");
 static_assert(kStageBytes % 1024 == 0, "stages must keep the 1024-byte swizzle alignment");
-// B row groups (of 128) whose scale atoms take the copy engine (0, 1 or 2); the rest go through registers
-#ifndef NVFP4_PAIR_CP_GROUPS
-#define NVFP4_PAIR_CP_GROUPS 0
-#endif
-constexpr int kCpGroups = NVFP4_PAIR_CP_GROUPS;
 
-struct Args {
+struct Problem {
   int M, N, K;
   const uint8_t* sfa;  // swizzled scale atoms of A and B (global memory)
   const uint8_t* sfb;
   const float* a_global;
   const float* b_global;
   int d_is_fp32, accumulate;
+};
+// One launch works through the tiles of up to two independent GEMMs (problem 0 first): Dgrad and Wgrad of a
+// linear layer share no output, so their tiles can fill the same persistent grid and the partial last round of
+// the first problem is not paid twice.
+struct Args {
+  Problem p[2];
+  int n_tiles0;  // tiles of problem 0
+  int n_tiles;   // tiles of both problems
 };
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -149,11 +151,6 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* r) {
       "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
-// shared memory -> tensor memory of BOTH CTAs of the pair (each reads its own shared memory at the descriptor's
-// address): one 512-byte scale atom, broadcast to the four 32-lane quadrants
-__device__ __forceinline__ void tc2_cp_sf(uint32_t taddr, uint64_t sdesc) {
-  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
-}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
@@ -216,8 +213,10 @@ __device__ __forceinline__ void store_half(const uint32_t (&r)[128], float alpha
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-    gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                     const __grid_constant__ CUtensorMap map_d, const Args g) {
+    gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_b0,
+                     const __grid_constant__ CUtensorMap map_d0, const __grid_constant__ CUtensorMap map_a1,
+                     const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_d1,
+                     const __grid_constant__ Args g) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -230,23 +229,22 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
   const uint32_t accf_bar = bar_base + 8u * (4 * kStages);                   // one per CTA
   const uint32_t acce_bar = bar_base + 8u * (4 * kStages + 1);               // leader only, 16 arrivals
   const uint32_t done_bar = bar_base + 8u * (4 * kStages + 2);               // one per CTA, peer arrives
-  auto sfp_bar = [&](int s) { return bar_base + 8u * (4 * kStages + 3 + s); }; // leader only: the peer's atoms landed
   volatile uint32_t* tmem_slot =
-      reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + kStagingBytes + 8 * (5 * kStages + 3));
+      reinterpret_cast<volatile uint32_t*>(base_ptr + kStages * kStageBytes + kStagingBytes + 8 * (4 * kStages + 3));
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();  // 0 = leader
   const bool leader = rank == 0;
   const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int tiles_m = g.M / 256, tiles_n = g.N / 256;
-  const int n_tiles = tiles_m * tiles_n;
-  const int k_blocks = g.K / 256;
-  const int sf_atoms_k = g.K / 64;  // atoms along K per 128-row group
-  // Tile order: groups of kGroupM row-blocks sweep all column-blocks before the next group starts, so the
-  // group's rows of A and all of B stay in L2 while they are reused.
+  const int n_tiles = g.n_tiles;
+  // Tile order inside a problem: groups of kGroupM row-blocks sweep all column-blocks before the next group
+  // starts, so the group's rows of A and all of B stay in L2 while they are reused.
   constexpr int kGroupM = 8;
-  auto tile_coords = [&](int tile, int& m_blk, int& n_blk) {
+  auto tile_coords = [&](int tile, int& prob, int& m_blk, int& n_blk) {
+    prob = tile >= g.n_tiles0 ? 1 : 0;
+    if (prob) tile -= g.n_tiles0;
+    const int tiles_m = g.p[prob].M / 256, tiles_n = g.p[prob].N / 256;
     const int per_group = kGroupM * tiles_n;
     const int grp = tile / per_group, in_grp = tile - grp * per_group;
     const int m0 = grp * kGroupM;
@@ -254,12 +252,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     m_blk = m0 + in_grp % gm;
     n_blk = in_grp / gm;
   };
+  auto k_blocks_of = [&](int tile) { return g.p[tile >= g.n_tiles0 ? 1 : 0].K / 256; };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(full_bar(s), 2);   // one arrive.expect_tx from each CTA's producer
-      mbar_init(sff_bar(s), 8 + (kCpGroups > 0 ? 1 : 0));  // four scale warps in each CTA (+ the copy engine)
-      mbar_init(sfp_bar(s), 1);
+      mbar_init(sff_bar(s), 8);    // four scale warps in each CTA
       mbar_init(empty_bar(s), 1);
       mbar_init(sfl_bar(s), 1);
     }
@@ -289,19 +287,24 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = pair_id; tile < n_tiles && ok; tile += n_pairs) {
-        int m_blk, n_blk;
-        tile_coords(tile, m_blk, n_blk);
+        int prob, m_blk, n_blk;
+        tile_coords(tile, prob, m_blk, n_blk);
+        const Problem& pr = g.p[prob];
+        const CUtensorMap* map_a = prob ? &map_a1 : &map_a0;
+        const CUtensorMap* map_b = prob ? &map_b1 : &map_b0;
+        const int k_blocks = pr.K / 256;
+        const int sf_atoms_k = pr.K / 64;  // atoms along K per 128-row group
         const int row_a = m_blk * 256 + (int)rank * 128;       // this CTA's A rows
         const int row_b = n_blk * 256 + (int)rank * 128;       // this CTA's half of the B tile
-        const uint8_t* sfa = g.sfa + (int64_t)(m_blk * 2 + (int)rank) * sf_atoms_k * 512;  // own 128 rows
-        const uint8_t* sfb = g.sfb + (int64_t)(n_blk * 2) * sf_atoms_k * 512;               // all 256 rows of B
+        const uint8_t* sfa = pr.sfa + (int64_t)(m_blk * 2 + (int)rank) * sf_atoms_k * 512;  // own 128 rows
+        const uint8_t* sfb = pr.sfb + (int64_t)(n_blk * 2) * sf_atoms_k * 512;               // all 256 rows of B
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x100u + stage))) break;
           const uint32_t st = base + stage * kStageBytes;
           const uint32_t bar = map_to_cta(full_bar(stage), 0);  // the leader's barrier counts both CTAs' operands
           mbar_expect_tx_cluster(bar, kABytes + kBBytes);
-          tma_load_2d_pair(st, &map_a, kb * 128, row_a, bar);
-          tma_load_2d_pair(st + kABytes, &map_b, kb * 128, row_b, bar);
+          tma_load_2d_pair(st, map_a, kb * 128, row_a, bar);
+          tma_load_2d_pair(st + kABytes, map_b, kb * 128, row_b, bar);
           // scale atoms: plain bulk copies counted on this CTA's own barrier (its scale warps wait on it)
           mbar_expect_tx(sfl_bar(stage), kSfaBytes + kSfbBytes);
           bulk_load(st + kABytes + kBBytes, sfa + (int64_t)kb * 2048, kSfaBytes, sfl_bar(stage));
@@ -326,32 +329,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     int stage = 0;
     uint32_t phase = 0;
     const uint32_t sff_leader = map_to_cta(sff_bar(0), 0);
-    const uint32_t sfp_leader = map_to_cta(sfp_bar(0), 0);
-    constexpr int kRegCols = 16 + 16 * (2 - kCpGroups);  // columns of the slot written from registers
     for (int tile = pair_id; tile < n_tiles; tile += n_pairs) {
       bool ok = true;
+      const int k_blocks = k_blocks_of(tile);
       for (int kb = 0; kb < k_blocks; ++kb) {
         ok = mbar_wait(sfl_bar(stage), phase, abort_flag, 0x500u + stage);
-        if (kCpGroups > 0 && warp == 2 && lane == 0 && ok) {
-          // B scales of row groups [2 - kCpGroups, 2): one copy per atom into both CTAs' tensor memory, issued by
-          // the leader once the peer's atoms have landed too
-          if (!leader) {
-            mbar_arrive_cluster(sfp_leader + 8u * stage);
-          } else {
-            ok = mbar_wait_cluster(sfp_bar(stage), phase, abort_flag, 0x580u + stage);
-            if (ok) {
-              tc_fence_after();
-              const uint32_t lo = (((base + stage * kStageBytes + kABytes + kBBytes + kSfaBytes) >> 4) & 0x3fffu);
-              const uint32_t sf_b = tmem + kSfCol + stage * kSfSlotCols + 16;
-#pragma unroll
-              for (int j = 0; j < 4; ++j)
-#pragma unroll
-                for (int grp = 2 - kCpGroups; grp < 2; ++grp)
-                  tc2_cp_sf(sf_b + 8 * j + 4 * grp, make_desc(lo + grp * 128 + j * 32, kDescHiSf));
-              tc2_commit_local(sff_bar(stage));
-            }
-          }
-        }
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) break;
         const uint32_t sf_s = base + stage * kStageBytes + kABytes + kBBytes + lane * 16;
@@ -363,28 +345,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
         }
         const uint32_t sf_t = tmem + ((uint32_t)(quad * 32) << 16) + kSfCol + stage * kSfSlotCols;
         tc_st16(sf_t, &r[0]);
-        if (kCpGroups == 0) {
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
+        for (int j = 0; j < 4; ++j)
 #pragma unroll
-            for (int grp = 0; grp < 2; ++grp) {
-              const uint4 b = lds128(sf_s + kSfaBytes + grp * 2048 + j * 512);
-              r[16 + 8 * j + 4 * grp] = b.x; r[16 + 8 * j + 4 * grp + 1] = b.y;
-              r[16 + 8 * j + 4 * grp + 2] = b.z; r[16 + 8 * j + 4 * grp + 3] = b.w;
-            }
-          tc_st16(sf_t + 16, &r[16]);
-          tc_st16(sf_t + 32, &r[32]);
-        } else if (kCpGroups == 1) {
-          // group 0 from registers: columns 16 + 8j .. 16 + 8j + 3 of each step, written four at a time
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint4 b = lds128(sf_s + kSfaBytes + j * 512);
-            asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1,%2,%3,%4};" ::"r"(sf_t + 16 + 8 * j), "r"(b.x),
-                         "r"(b.y), "r"(b.z), "r"(b.w)
-                         : "memory");
+          for (int grp = 0; grp < 2; ++grp) {
+            const uint4 b = lds128(sf_s + kSfaBytes + grp * 2048 + j * 512);
+            r[16 + 8 * j + 4 * grp] = b.x; r[16 + 8 * j + 4 * grp + 1] = b.y;
+            r[16 + 8 * j + 4 * grp + 2] = b.z; r[16 + 8 * j + 4 * grp + 3] = b.w;
           }
-        }
-        (void)kRegCols;
+        tc_st16(sf_t + 16, &r[16]);
+        tc_st16(sf_t + 32, &r[32]);
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -408,6 +378,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       for (int tile = pair_id; tile < n_tiles && ok; tile += n_pairs) {
         if (!(ok = mbar_wait_cluster(acce_bar, acc_phase ^ 1u, abort_flag, 0x300u))) break;
         tc_fence_after();
+        const int k_blocks = k_blocks_of(tile);
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!(ok = mbar_wait_cluster(full_bar(stage), phase, abort_flag, 0x200u + stage))) break;
           if (!(ok = mbar_wait_cluster(sff_bar(stage), phase, abort_flag, 0x280u + stage))) break;
@@ -439,15 +410,19 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     const int et = (threadIdx.x - 96) & 127;  // 0..127 inside the group
     const int bar_id = 1 + half;
     uint32_t acc_phase = 0;
-    const float alpha = __fmul_rn(g.a_global[1], g.b_global[1]);
+    const float alpha0 = __fmul_rn(g.p[0].a_global[1], g.p[0].b_global[1]);
+    const float alpha1 = __fmul_rn(g.p[1].a_global[1], g.p[1].b_global[1]);
     const uint32_t acce_leader = map_to_cta(acce_bar, 0);
     const int row_in_tile = quad * 32 + lane;
     const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + half * 128;
     const uint32_t stage_buf = staging + half * 16384;
     int buf = 0;
     for (int tile = pair_id; tile < n_tiles; tile += n_pairs) {
-      int m_blk, n_blk;
-      tile_coords(tile, m_blk, n_blk);
+      int prob, m_blk, n_blk;
+      tile_coords(tile, prob, m_blk, n_blk);
+      const CUtensorMap* map_d = prob ? &map_d1 : &map_d0;
+      const float alpha = prob ? alpha1 : alpha0;
+      const int d_is_fp32 = g.p[prob].d_is_fp32, accumulate = g.p[prob].accumulate;
       mbar_wait_cluster(accf_bar, acc_phase, abort_flag, 0x400u);
       // agree on giving up: a warp that timed out still joins this barrier, then everyone reads the flag
       asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
@@ -463,12 +438,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(acce_leader);
-      if (g.d_is_fp32)
-        store_half<true>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, &map_d, n_blk * 256 + half * 128, row0,
-                         g.accumulate);
+      if (d_is_fp32)
+        store_half<true>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, map_d, n_blk * 256 + half * 128, row0,
+                         accumulate);
       else
-        store_half<false>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, &map_d, n_blk * 256 + half * 128, row0,
-                          g.accumulate);
+        store_half<false>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, map_d, n_blk * 256 + half * 128, row0,
+                          accumulate);
       acc_phase ^= 1u;
     }
     if (et == 0) bulk_wait_all<0>();  // all stores have left shared memory and are visible
