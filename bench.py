@@ -192,10 +192,25 @@ def run_cuda(args):
     ws_f = torch.empty(B.nvfp4_linear_fwd_workspace_bytes(M, K), dtype=torch.uint8, device="cuda")
     ws_b = torch.empty(B.nvfp4_linear_bwd_workspace_bytes(M, N), dtype=torch.uint8, device="cuda")
 
+    # N > 1: the FP32 all-reduce of dW runs beside the next step's kernels; two dW buffers alternate and a buffer
+    # is rewritten only after its own exchange has finished (every step's exchange is inside the timed region, the
+    # last one is waited for before the closing event)
+    dWs = [dW, torch.empty_like(dW)] if world > 1 else [dW]
+    pending = [None] * len(dWs)
+    counter = [0]
+
     def step():
+        i = counter[0] % len(dWs)
+        counter[0] += 1
+        dp.wait_weight_grad(pending[i])
         B.nvfp4_linear_fwd(X, W, opts, Y, X_col, W_row, W_col, False, ws_f)
-        B.nvfp4_linear_bwd(dY, X_col, W_col, K, opts, dX, dW, False, ws_b)
-        dp.allreduce_weight_grad(dW)  # FP32 sum of the weight gradient across data-parallel replicas (N > 1)
+        B.nvfp4_linear_bwd(dY, X_col, W_col, K, opts, dX, dWs[i], False, ws_b)
+        pending[i] = dp.allreduce_weight_grad(dWs[i], async_op=True)  # None at N = 1
+
+    def drain():
+        for j in range(len(pending)):
+            dp.wait_weight_grad(pending[j])
+            pending[j] = None
 
     def barrier():
         if world > 1:
@@ -211,6 +226,7 @@ def run_cuda(args):
 
     for _ in range(max(args.warmup, 3)):
         step()
+    drain()
     B.nvfp4_device_status()
 
     sampler = ClockSampler(local)
@@ -224,6 +240,7 @@ def run_cuda(args):
     e0.record()
     for _ in range(args.steps):
         step()
+    drain()
     e1.record()
     barrier()
     launches = B.nvfp4_launch_count() - launches0
@@ -265,22 +282,53 @@ def run_cuda(args):
     hdX = torch.empty((M, K), dtype=torch.bfloat16).pin_memory()
     hdW = torch.empty((N, K), dtype=torch.float32).pin_memory()
 
-    def e2e_step():
-        X.copy_(hX, non_blocking=True)
-        W.copy_(hW, non_blocking=True)
-        dY.copy_(hdY, non_blocking=True)
-        step()
-        hY.copy_(Y, non_blocking=True)
-        hdX.copy_(dX, non_blocking=True)
-        hdW.copy_(dW, non_blocking=True)
+    # Copies and kernels of neighbouring steps overlap: inputs and outputs are double-buffered on the device, the
+    # host->device copies of step i+1 and the device->host copies of step i-1 run on their own streams beside the
+    # kernels of step i.  Every step still moves all of its inputs and all of its results.
+    drain()
+    cur = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ins = [(X, W, dY), (torch.empty_like(X), torch.empty_like(W), torch.empty_like(dY))]
+    outs = [(Y, dX, dW), (torch.empty_like(Y), torch.empty_like(dX), torch.empty_like(dW))]
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_comp = [torch.cuda.Event() for _ in range(2)]
+    ev_out = [torch.cuda.Event() for _ in range(2)]
 
-    e2e_steps = max(2, min(args.steps, 5))
-    e2e_step()
+    def e2e_step(i):
+        b = i & 1
+        Xb, Wb, dYb = ins[b]
+        Yb, dXb, dWb = outs[b]
+        with torch.cuda.stream(s_in):
+            s_in.wait_event(ev_comp[b])  # step i-2 has consumed this input buffer
+            Xb.copy_(hX, non_blocking=True)
+            Wb.copy_(hW, non_blocking=True)
+            dYb.copy_(hdY, non_blocking=True)
+            ev_in[b].record(s_in)
+        cur.wait_event(ev_in[b])
+        cur.wait_event(ev_out[b])        # the results of step i-2 have left this output buffer
+        B.nvfp4_linear_fwd(Xb, Wb, opts, Yb, X_col, W_row, W_col, False, ws_f)
+        B.nvfp4_linear_bwd(dYb, X_col, W_col, K, opts, dXb, dWb, False, ws_b)
+        dp.allreduce_weight_grad(dWb)
+        ev_comp[b].record(cur)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_comp[b])
+            hY.copy_(Yb, non_blocking=True)
+            hdX.copy_(dXb, non_blocking=True)
+            hdW.copy_(dWb, non_blocking=True)
+            ev_out[b].record(s_out)
+
+    e2e_steps = max(4, min(args.steps, 10))
+    e2e_step(0)
+    e2e_step(1)
+    cur.wait_stream(s_in)
+    cur.wait_stream(s_out)
     barrier()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
-    for _ in range(e2e_steps):
-        e2e_step()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    cur.wait_stream(s_in)
+    cur.wait_stream(s_out)
     t1.record()
     barrier()
     e2e_ms = max_over_ranks(t0.elapsed_time(t1) / e2e_steps)
@@ -325,7 +373,8 @@ def run_cuda(args):
                                "peak_source": f"{peaks['source']} copy bandwidth",
                                "frac_of_datasheet_8tbs": q_gbs / 8000.0},
             "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
+                    "overlap": "copies of neighbouring steps overlap the kernels (double-buffered)"},
             "gpu_launches": launches, "clocks": clocks, "cpu_baseline": cpu,
         }
         print(json.dumps(line))

@@ -23,11 +23,23 @@ def token_shard(total_tokens: int, rank: int, world: int) -> tuple[int, int]:
     return rank * per, (rank + 1) * per
 
 
-def allreduce_weight_grad(dW: torch.Tensor) -> None:
-    """In-place FP32 sum of dW over all ranks (no-op without an initialised process group)."""
+def allreduce_weight_grad(dW: torch.Tensor, async_op: bool = False):
+    """In-place FP32 sum of dW over all ranks (no-op without an initialised process group).
+
+    async_op=True returns the collective's work handle (None without a process group): the exchange then runs
+    beside the next layer's / next step's kernels, and the caller waits on the handle before dW is read or
+    overwritten (`wait_weight_grad`)."""
     assert dW.dtype == torch.float32
     if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
-        dist.all_reduce(dW, op=dist.ReduceOp.SUM)
+        return dist.all_reduce(dW, op=dist.ReduceOp.SUM, async_op=async_op) if async_op else \
+            dist.all_reduce(dW, op=dist.ReduceOp.SUM)
+    return None
+
+
+def wait_weight_grad(work) -> None:
+    """Blocks the current stream (NCCL) or the caller (gloo) until an asynchronous exchange has finished."""
+    if work is not None:
+        work.wait()
 
 
 def weight_grad_shard(n_rows: int, rank: int, world: int) -> tuple[int, int]:

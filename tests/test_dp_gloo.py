@@ -37,7 +37,11 @@ def _worker(rank, world, port, out):
         dW = torch.from_numpy(dW_local.astype(np.float32))
         shard = torch.empty((48 // world, 64), dtype=torch.float32)
         dp.reduce_scatter_weight_grad(dW.clone(), shard)
-        dp.allreduce_weight_grad(dW)
+        ref = dW.clone()
+        dp.allreduce_weight_grad(ref)
+        work = dp.allreduce_weight_grad(dW, async_op=True)  # the overlapped form used by the bench at N > 1
+        dp.wait_weight_grad(work)
+        assert torch.equal(ref, dW), "asynchronous all-reduce differs from the blocking one"
         b0, e0 = dp.weight_grad_shard(48, rank, world)
         assert torch.equal(shard, dW[b0:e0]), "reduce-scatter shard differs from the rows of the all-reduced dW"
         # replicated weights quantize to identical bytes on every rank (deterministic RNE)
@@ -78,6 +82,8 @@ def test_token_shard_and_offsets():
     assert dp.rank_sr_offset(3, 7) == (3 << 32) | 7
     t = torch.ones(4)
     dp.allreduce_weight_grad(t)  # no process group: no-op
+    assert dp.allreduce_weight_grad(t, async_op=True) is None
+    dp.wait_weight_grad(None)
     assert torch.equal(t, torch.ones(4))
     o = torch.empty(4)
     dp.reduce_scatter_weight_grad(t, o)
