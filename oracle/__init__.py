@@ -71,6 +71,15 @@ def lib():
                 "orc_gemm_tn": (None, [f64p, f64p, c.c_int64, c.c_int64, c.c_int64, f64p, f64p]),
                 "orc_gemm_blockscaled": (None, [u8p, u8p, f32p, u8p, u8p, f32p, c.c_int64,
                                                 c.c_int64, c.c_int64, f64p]),
+                "orc_ue8m0_decode": (c.c_float, [c.c_uint8]),
+                "orc_mx_block_scale_byte": (c.c_uint8, [c.c_float]),
+                "orc_mx_block_encode_scale": (c.c_float, [c.c_uint8]),
+                "orc_hadamard32_entry": (c.c_int, [c.c_int, c.c_int]),
+                "orc_rht32": (None, [f32p, c.c_uint32, f32p]),
+                "orc_quantize_mx": (c.c_int, [u16p, c.c_int64, c.c_int64, c.c_int64, c.c_int, c.c_int,
+                                              c.c_int, c.c_uint32, c.c_int, c.c_uint64, c.c_uint64,
+                                              c.c_int64, c.c_int64, u8p, u8p, f32p]),
+                "orc_dequantize_mx": (None, [u8p, u8p, c.c_int64, c.c_int64, f64p]),
             }
             for name, (res, args) in sig.items():
                 fn = getattr(L, name)
@@ -254,3 +263,64 @@ def gemm_blockscaled(a: Quantized, b: Quantized):
                                _p(bc, ctypes.c_uint8), _p(bsf, ctypes.c_uint8), _p(bg, ctypes.c_float),
                                a.rows, b.rows, a.cols, _p(D, ctypes.c_double))
     return D
+
+
+# ----------------------------------------------------------------- MXFP4 ----
+def ue8m0_decode(b: int) -> float:
+    return float(lib().orc_ue8m0_decode(b))
+
+
+def mx_block_scale_byte(amax_b: float) -> int:
+    return int(lib().orc_mx_block_scale_byte(np.float32(amax_b)))
+
+
+def mx_block_encode_scale(b: int):
+    return np.float32(lib().orc_mx_block_encode_scale(b))
+
+
+def hadamard32_entry(j: int, k: int) -> int:
+    return int(lib().orc_hadamard32_entry(j, k))
+
+
+def rht32(x, sign_mask: int):
+    xin = np.ascontiguousarray(x, dtype=np.float32)
+    assert xin.shape == (32,)
+    y = np.zeros(32, dtype=np.float32)
+    lib().orc_rht32(_p(xin, ctypes.c_float), sign_mask, _p(y, ctypes.c_float))
+    return y
+
+
+class QuantizedMX:
+    """One MXFP4 copy: codes [R][C/2], UE8M0 scales [R][C/32] (linear); no tensor-level scale."""
+
+    def __init__(self, codes, scales, rows, cols, y=None):
+        self.codes, self.scales = codes, scales
+        self.rows, self.cols, self.y = rows, cols, y
+
+
+def quantize_mx(x_bf16_bits, *, colwise=False, block_rows=1, rht=False, sign_mask=0, rounding=RNE, seed=0,
+                sr_offset=0, return_y=False, sr_row0=0, sr_cols=0) -> QuantizedMX:
+    """MXFP4 quantization of one copy of a bf16 tensor given as a 2-D uint16 array of bit patterns."""
+    x = np.asarray(x_bf16_bits)
+    assert x.dtype == np.uint16 and x.ndim == 2 and x.strides[1] == 2
+    ld = x.strides[0] // 2
+    sr, sc = x.shape
+    R, C = (sc, sr) if colwise else (sr, sc)
+    codes = np.zeros((R, C // 2), dtype=np.uint8)
+    scales = np.zeros((R, max(C // 32, 1)), dtype=np.uint8)
+    y = np.zeros((R, C), dtype=np.float32) if return_y else None
+    rc = lib().orc_quantize_mx(_p(x, ctypes.c_uint16), sr, sc, ld, int(colwise), block_rows, int(rht), sign_mask,
+                               rounding, seed, sr_offset, sr_row0, sr_cols, _p(codes, ctypes.c_uint8),
+                               _p(scales, ctypes.c_uint8), _p(y, ctypes.c_float) if return_y else None)
+    if rc != 0:
+        raise ValueError(f"orc_quantize_mx rejected the shape (rc={rc})")
+    return QuantizedMX(codes, scales, R, C, y)
+
+
+def dequantize_mx(q: QuantizedMX):
+    out = np.zeros((q.rows, q.cols), dtype=np.float64)
+    codes = np.ascontiguousarray(q.codes)
+    scales = np.ascontiguousarray(q.scales)
+    lib().orc_dequantize_mx(_p(codes, ctypes.c_uint8), _p(scales, ctypes.c_uint8), q.rows, q.cols,
+                            _p(out, ctypes.c_double))
+    return out

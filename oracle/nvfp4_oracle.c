@@ -4,7 +4,8 @@
  * A plain, slow, step-by-step restatement of the NVFP4 quantization procedure
  * (paper Appendix B, Eq. 1-5), the tiled random Hadamard transform (Appendix C),
  * stochastic rounding (Section 4.4) and the block-scaled GEMM (Eq. 5 plus the
- * sentence after it).  It shares no code, table or constant generator with the
+ * sentence after it); at the end, the same for MXFP4, the comparison format
+ * (Section 2, Section 5, Appendix B.4).  It shares no code, table or constant generator with the
  * CUDA path.  Only tests, the smoke check and the CPU-baseline legs of the
  * benchmark may build or call it.
  *
@@ -406,5 +407,134 @@ ORC_EXPORT void orc_gemm_blockscaled(const uint8_t* a_codes, const uint8_t* a_sc
                (double)orc_e4m3_decode(b_scales[j * (K / 16) + kb]) * part;
       }
       D[i * N + j] = acc * (double)a_global[1] * (double)b_global[1];
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* MXFP4, the comparison format (Section 2, Section 5, Appendix B.4):         */
+/* E2M1 elements, one UE8M0 (power-of-two) scale per 32 contiguous elements,  */
+/* no tensor-level scale.                                                     */
+/* ------------------------------------------------------------------------- */
+
+/* UE8M0: byte b encodes 2^(b - 127), b = 0..254 (0xFF is NaN, never produced). */
+ORC_EXPORT float orc_ue8m0_decode(uint8_t b) { return ldexpf(1.0f, (int)b - 127); }
+
+/* Appendix B.4: the decode scale amax_b / 6 is rounded UP to a power of two so
+ * that the scaled block never exceeds 6: the smallest e with 6 * 2^e >= amax_b,
+ * found by search.  A zero block gets the smallest scale (byte 0); e is clamped
+ * to what the byte can hold. */
+ORC_EXPORT uint8_t orc_mx_block_scale_byte(float amax_b) {
+  if (amax_b == 0.0f) return 0;
+  int e = -160;
+  while (ldexp(6.0, e) < (double)amax_b) ++e;
+  int b = e + 127;
+  if (b < 0) b = 0;
+  if (b > 254) b = 254;
+  return (uint8_t)b;
+}
+
+/* encode scale = 1 / decode scale = 2^(127 - b), exact */
+ORC_EXPORT float orc_mx_block_encode_scale(uint8_t b) { return ldexpf(1.0f, 127 - (int)b); }
+
+/* +-1 Sylvester matrix of order 32 = H_2 (x) H_16 */
+ORC_EXPORT int orc_hadamard32_entry(int j, int k) {
+  int top = ((j >> 4) & (k >> 4) & 1) ? -1 : 1;
+  return top * orc_hadamard16_entry(j & 15, k & 15);
+}
+
+/* Section 5: transform size d = 32 for MXFP4, aligned with its block size.
+ * y_k = (1/sqrt(32)) * sum_j s_j x_j h(j,k); the whole expression is evaluated
+ * in binary64 and rounded once to binary32. */
+ORC_EXPORT void orc_rht32(const float x[32], uint32_t sign_mask, float y[32]) {
+  const double norm = 1.0 / sqrt(32.0);
+  for (int k = 0; k < 32; ++k) {
+    double acc = 0.0;
+    for (int j = 0; j < 32; ++j) {
+      double s = ((sign_mask >> j) & 1u) ? -1.0 : 1.0;
+      acc += s * (double)x[j] * (double)orc_hadamard32_entry(j, k);
+    }
+    y[k] = (float)(norm * acc);
+  }
+}
+
+/*
+ * MXFP4 quantization of one copy; arguments as orc_quantize, except:
+ * block_rows: 1 = 1x32 blocks along the copy's columns; 32 = 32x32 blocks
+ *             (the 2D weight scaling of Section 4.3 at this format's block size)
+ * rht       : x * (S * H_32) on every aligned 32-chunk
+ * outputs   : codes [R][C/2], scales [R][C/32] UE8M0 bytes (linear layout),
+ *             y_out (nullable).  There is no tensor-level scale.
+ * returns -1 when C is not a multiple of 32 (or R not of block_rows).
+ */
+ORC_EXPORT int orc_quantize_mx(const uint16_t* x_bf16, int64_t src_rows, int64_t src_cols, int64_t ld,
+                               int colwise, int block_rows, int rht, uint32_t sign_mask, int rounding,
+                               uint64_t seed, uint64_t sr_offset, int64_t sr_row0, int64_t sr_cols,
+                               uint8_t* codes, uint8_t* scales, float* y_out) {
+  const int64_t R = colwise ? src_cols : src_rows;
+  const int64_t C = colwise ? src_rows : src_cols;
+  if ((block_rows != 1 && block_rows != 32) || C % 32 || R % block_rows) return -1;
+  float* y = (float*)malloc(sizeof(float) * (size_t)(R * C));
+  if (!y) return -2;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < R; ++r)
+    for (int64_t c = 0; c < C; ++c) {
+      int64_t sr = colwise ? c : r, sc = colwise ? r : c;
+      y[r * C + c] = orc_bf16_to_f32(x_bf16[sr * ld + sc]);
+    }
+  if (rht) {
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < R; ++r)
+      for (int64_t c0 = 0; c0 < C; c0 += 32) {
+        float t[32];
+        orc_rht32(&y[r * C + c0], sign_mask, t);
+        memcpy(&y[r * C + c0], t, sizeof t);
+      }
+  }
+  const int64_t nkb = C / 32;
+#pragma omp parallel for schedule(static)
+  for (int64_t rb = 0; rb < R / block_rows; ++rb)
+    for (int64_t kb = 0; kb < nkb; ++kb) {
+      float amax_b = 0.0f;
+      for (int64_t i = 0; i < block_rows; ++i)
+        for (int64_t j = 0; j < 32; ++j) {
+          float a = fabsf(y[(rb * block_rows + i) * C + kb * 32 + j]);
+          if (a > amax_b) amax_b = a;
+        }
+      uint8_t sb = orc_mx_block_scale_byte(amax_b);
+      for (int64_t i = 0; i < block_rows; ++i) scales[(rb * block_rows + i) * nkb + kb] = sb;
+    }
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < R; ++r)
+    for (int64_t kb = 0; kb < nkb; ++kb) {
+      const float s_enc_b = orc_mx_block_encode_scale(scales[r * nkb + kb]);
+      uint8_t code[32];
+      for (int64_t j = 0; j < 32; ++j) {
+        int64_t c = kb * 32 + j;
+        float v = y[r * C + c] * s_enc_b;
+        if (rounding == 0) {
+          code[j] = orc_e2m1_encode_rne(v);
+        } else {
+          int64_t sr = colwise ? c : r, sc = colwise ? r : c;
+          uint64_t e = (uint64_t)(sr + sr_row0) * (uint64_t)(sr_cols ? sr_cols : src_cols) + (uint64_t)sc;
+          code[j] = orc_e2m1_encode_sr(v, orc_sr_draw(seed, sr_offset, e));
+        }
+      }
+      for (int64_t j = 0; j < 32; j += 2)
+        codes[r * (C / 2) + (kb * 32 + j) / 2] = (uint8_t)(code[j] | (code[j + 1] << 4));
+    }
+  if (y_out) memcpy(y_out, y, sizeof(float) * (size_t)(R * C));
+  free(y);
+  return 0;
+}
+
+/* Decode: x^ = (+-magnitude) * 2^(scale byte - 127), exact in binary64. */
+ORC_EXPORT void orc_dequantize_mx(const uint8_t* codes, const uint8_t* scales, int64_t R, int64_t C,
+                                  double* out) {
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < R; ++r)
+    for (int64_t c = 0; c < C; ++c) {
+      uint8_t byte = codes[r * (C / 2) + c / 2];
+      uint8_t code = (c & 1) ? (byte >> 4) : (byte & 15);
+      out[r * C + c] = (double)orc_e2m1_decode(code) * ldexp(1.0, (int)scales[r * (C / 32) + c / 32] - 127);
     }
 }
