@@ -48,6 +48,12 @@ typedef enum nvfp4_status {
 
 enum { NVFP4_ROUND_NEAREST_EVEN = 0, NVFP4_ROUND_STOCHASTIC = 1 };
 enum { NVFP4_SF_LINEAR = 0, NVFP4_SF_SWIZZLED = 1 };
+/* Element / scale format of a copy.  NVFP4 is the paper's format (Section 2, Appendix B).  MXFP4 is the
+   format the paper compares against (Section 2, Section 5, Appendix B.4): E2M1 elements with one UE8M0
+   power-of-two scale per 32 elements, the decode scale amax_b / 6 rounded UP to a power of two, no
+   tensor-level scale (global = {0, 1}), transform size 32 on the weight-gradient operands, 32x32 blocks
+   for weights. */
+enum { NVFP4_FORMAT_NVFP4 = 0, NVFP4_FORMAT_MXFP4 = 1 };
 enum {
   /* the column-wise copy draws its stochastic-rounding bits from a second stream (bit 63 of
      sr_offset set) instead of sharing the draw of the same source element with the row-wise copy */
@@ -76,7 +82,9 @@ typedef struct nvfp4_tensor {
   float* global;
   int64_t rows, cols;
   int32_t sf_layout;
-  int32_t reserved;
+  int32_t format;   /* NVFP4_FORMAT_NVFP4 (0) or NVFP4_FORMAT_MXFP4; MXFP4: scales hold rows * cols/32 UE8M0
+                       bytes (byte b = 2^(b-127)), same two layouts with 32-element blocks (swizzled needs
+                       cols % 128 == 0), global is written as {0, 1} and not used */
 } nvfp4_tensor;
 
 /*
@@ -87,10 +95,12 @@ typedef struct nvfp4_tensor {
 typedef struct nvfp4_quant_opts {
   int32_t block_rows;     /* 1: one scale per 1x16 block; 16: one scale per 16x16 block (Sec. 4.3),  */
                           /*    replicated to the 16 1x16 blocks it covers in either copy            */
+                          /*    (MXFP4 outputs: 1 or 32, blocks of 1x32 / 32x32)                      */
   int32_t rounding;       /* NVFP4_ROUND_NEAREST_EVEN or NVFP4_ROUND_STOCHASTIC (Sec. 4.4)            */
   int32_t rht_rowwise;    /* 1: rotate every aligned 16-chunk of each row of the row-wise copy by     */
   int32_t rht_colwise;    /*    S*H_16 before scaling (Appendix C); same for the column-wise copy     */
-  uint32_t rht_sign_mask; /* low 16 bits: bit j set => the j-th input of a chunk is negated (S_d)     */
+  uint32_t rht_sign_mask; /* low 16 bits: bit j set => the j-th input of a chunk is negated (S_d);    */
+                          /* MXFP4 outputs use all 32 bits (transform size 32, Section 5)             */
   int32_t flags;          /* NVFP4_SR_INDEPENDENT_COPIES | NVFP4_AMAX_PROVIDED                        */
   uint64_t seed;          /* Philox4x32-10 key                                                        */
   uint64_t sr_offset;     /* Philox counter words 2..3; words 0..1 = (row-major source index) >> 4,   */
@@ -127,6 +137,8 @@ NVFP4_API nvfp4_status nvfp4_quantize(const void* x_bf16, int64_t rows, int64_t 
  *   FP32 by the tensor cores; the product of the two tensor decode scales is applied once at the end.
  *   accumulate != 0 adds the product to the existing contents of an fp32 D (gradient accumulation,
  *   Section 4.1); it is rejected for bf16 outputs.
+ *   Both operands must have the same format.  MXFP4 operands (no tensor-level scale, the block scales
+ *   are powers of two) need M % 256 == 0 and N % 256 == 0; other shapes return NVFP4_ERR_UNIMPLEMENTED.
  */
 NVFP4_API nvfp4_status nvfp4_gemm(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D,
                                   int32_t d_is_fp32, int64_t ldd, int32_t accumulate,

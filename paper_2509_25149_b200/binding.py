@@ -18,6 +18,7 @@ OK = 0
 ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
 SF_LINEAR, SF_SWIZZLED = 0, 1
 SR_INDEPENDENT_COPIES, AMAX_PROVIDED = 1, 2
+FORMAT_NVFP4, FORMAT_MXFP4 = 0, 1
 
 EXPORTED = (
     "nvfp4_quantize", "nvfp4_gemm", "nvfp4_linear_fwd_workspace_bytes", "nvfp4_linear_bwd_workspace_bytes",
@@ -30,7 +31,7 @@ EXPORTED = (
 class CTensor(ctypes.Structure):
     _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("global_", ctypes.c_void_p),
                 ("rows", ctypes.c_int64), ("cols", ctypes.c_int64), ("sf_layout", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("format", ctypes.c_int32)]
 
 
 class CQuantOpts(ctypes.Structure):
@@ -102,16 +103,22 @@ class NVFP4Tensor:
     rows: int
     cols: int
     sf_layout: int = SF_SWIZZLED
+    format: int = FORMAT_NVFP4  # FORMAT_MXFP4: scales are rows * cols/32 UE8M0 bytes, glob unused ({0, 1})
 
     def c(self) -> CTensor:
         return CTensor(self.codes.data_ptr(), self.scales.data_ptr(), self.glob.data_ptr(), self.rows, self.cols,
-                       self.sf_layout, 0)
+                       self.sf_layout, self.format)
 
 
-def alloc_tensor(rows: int, cols: int, sf_layout: int = SF_SWIZZLED, device="cuda") -> NVFP4Tensor:
+def alloc_tensor(rows: int, cols: int, sf_layout: int = SF_SWIZZLED, device="cuda",
+                 format: int = FORMAT_NVFP4) -> NVFP4Tensor:
+    block = 32 if format == FORMAT_MXFP4 else 16
+    glob = torch.zeros((2,), dtype=torch.float32, device=device)
+    if format == FORMAT_MXFP4:
+        glob[1] = 1.0
     return NVFP4Tensor(torch.empty((rows, cols // 2), dtype=torch.uint8, device=device),
-                       torch.empty((rows * cols // 16,), dtype=torch.uint8, device=device),
-                       torch.zeros((2,), dtype=torch.float32, device=device), rows, cols, sf_layout)
+                       torch.empty((rows * cols // block,), dtype=torch.uint8, device=device),
+                       glob, rows, cols, sf_layout, format)
 
 
 def quant_opts(block_rows=1, rounding=ROUND_NEAREST_EVEN, rht_rowwise=False, rht_colwise=False, rht_sign_mask=0,

@@ -26,7 +26,9 @@ nvfp4_status check_copy(const nvfp4_tensor* t, int64_t rows, int64_t cols) {
   if (!t->codes || !t->scales || !t->global) return NVFP4_ERR_NULL;
   if (t->rows != rows || t->cols != cols) return NVFP4_ERR_SHAPE;
   if (t->sf_layout != NVFP4_SF_LINEAR && t->sf_layout != NVFP4_SF_SWIZZLED) return NVFP4_ERR_ARG;
-  if (t->sf_layout == NVFP4_SF_SWIZZLED && (rows % 128 != 0 || cols % 64 != 0)) return NVFP4_ERR_SHAPE;
+  if (t->format != NVFP4_FORMAT_NVFP4 && t->format != NVFP4_FORMAT_MXFP4) return NVFP4_ERR_ARG;
+  const int64_t atom_cols = t->format == NVFP4_FORMAT_MXFP4 ? 128 : 64;  // four blocks of 32 / 16 elements
+  if (t->sf_layout == NVFP4_SF_SWIZZLED && (rows % 128 != 0 || cols % atom_cols != 0)) return NVFP4_ERR_SHAPE;
   if (!aligned(t->codes, 16) || !aligned(t->scales, 16) || !aligned(t->global, 8)) return NVFP4_ERR_ALIGN;
   return NVFP4_OK;
 }
@@ -87,6 +89,9 @@ nvfp4_status gemm_prepare(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D,
   if (M <= 0 || N <= 0 || K <= 0 || M % 128 != 0 || N % 128 != 0 || K % 256 != 0) return NVFP4_ERR_SHAPE;
   if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff || (M / 128) * (N / 128) > 0x7fffffff) return NVFP4_ERR_SHAPE;
   if (A->sf_layout != NVFP4_SF_SWIZZLED || B->sf_layout != NVFP4_SF_SWIZZLED) return NVFP4_ERR_ARG;
+  if (A->format != B->format) return NVFP4_ERR_ARG;
+  if (A->format != NVFP4_FORMAT_NVFP4 && A->format != NVFP4_FORMAT_MXFP4) return NVFP4_ERR_ARG;
+  if (A->format == NVFP4_FORMAT_MXFP4 && (M % 256 != 0 || N % 256 != 0)) return NVFP4_ERR_UNIMPLEMENTED;
   if (accumulate && !d_is_fp32) return NVFP4_ERR_ARG;
   if (ldd < N) return NVFP4_ERR_SHAPE;
   const int64_t esz = d_is_fp32 ? 4 : 2;
@@ -99,6 +104,7 @@ nvfp4_status gemm_prepare(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D,
   g.d = D; g.ldd = ldd;
   g.M = (int)M; g.N = (int)N; g.K = (int)K;
   g.d_is_fp32 = d_is_fp32 != 0; g.accumulate = accumulate != 0;
+  g.mx = A->format == NVFP4_FORMAT_MXFP4;
   return NVFP4_OK;
 }
 
@@ -110,6 +116,7 @@ int gemm_tile(const GemmArgs& g) {
   // (exposed epilogue), 128 x 128 tiles two (the epilogue overlaps the next tile), so the wide tile pays off
   // once the main loop is long enough to amortise the epilogue.
   int tile_n = g_tile_n.load(std::memory_order_relaxed);
+  if (g.mx) return 512;  // MXFP4 runs on the CTA-pair kernel only
   if (tile_n != 128 && tile_n != 256 && tile_n != 512) {
     if (M % 256 == 0 && N % 256 == 0)
       tile_n = 512;

@@ -349,10 +349,14 @@ cudaError_t launch_pair(const GemmArgs& g0, const void* a0, const void* b0, cons
   } else {
     m[3] = m[0]; m[4] = m[1]; m[5] = m[2];
   }
+  if (g1 && g1->mx != g0.mx) return cudaErrorInvalidValue;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(pair::gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(pair::gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          pair::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(pair::gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             pair::kSmemBytes);
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -363,7 +367,10 @@ cudaError_t launch_pair(const GemmArgs& g0, const void* a0, const void* b0, cons
   a.n_tiles = a.n_tiles0 + (g1 ? (g1->M / 256) * (g1->N / 256) : 0);
   const int max_pairs = num_sms / 2;
   const int pairs = a.n_tiles < max_pairs ? a.n_tiles : max_pairs;
-  pair::gemm_pair_kernel<<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5], a);
+  if (g0.mx)
+    pair::gemm_pair_kernel<true><<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5], a);
+  else
+    pair::gemm_pair_kernel<false><<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5], a);
   count_launch();
   return cudaGetLastError();
 }
@@ -387,7 +394,8 @@ cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_co
   int num_sms = 0;
   cudaError_t e = sm_count(&num_sms);
   if (e != cudaSuccess) return e;
-  if (tile_n == 512 && g.M % 256 == 0 && g.N % 256 == 0)
+  if (g.mx && !(g.M % 256 == 0 && g.N % 256 == 0)) return cudaErrorNotSupported;
+  if ((tile_n == 512 || g.mx) && g.M % 256 == 0 && g.N % 256 == 0)
     return launch_pair(g, a_codes, b_codes, nullptr, nullptr, nullptr, num_sms, s);
   if (tile_n == 256 && g.N % 256 == 0) return launch_t<256>(g, a_codes, b_codes, num_sms, s);
   return launch_t<128>(g, a_codes, b_codes, num_sms, s);

@@ -14,6 +14,7 @@ struct GemmArgs {
   int64_t ldd;
   int M, N, K;
   int d_is_fp32, accumulate;
+  int mx;                 // operands are MXFP4 (UE8M0 scale per 32 elements) instead of NVFP4
 };
 
 // tile_n: 128 or 256 (256 needs N % 256 == 0, otherwise 128 is used)

@@ -167,6 +167,16 @@ __device__ __forceinline__ void tc2_mma_nvf4(uint32_t d_tmem, uint64_t adesc, ui
       : "memory");
 }
 
+__device__ __forceinline__ void tc2_mma_mxf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
+      : "memory");
+}
+
 // Epilogue helper: 128 accumulator columns of one row per thread (registers) -> alpha, conversion -> 128-byte
 // swizzled rows of a staging buffer -> TMA store (or reduce-add) of 128 x 128-byte boxes.  Two staging buffers
 // alternate; a buffer is rewritten only after the store issued two boxes earlier has finished reading it.
@@ -212,6 +222,10 @@ __device__ __forceinline__ void store_half(const uint32_t (&r)[128], float alpha
   }
 }
 
+// MX = false: NVFP4 (E4M3 scale per 16 elements: one 512-byte atom per 128 rows and K = 64).
+// MX = true : MXFP4 (UE8M0 scale per 32 elements: one atom per 128 rows and K = 128, so half the atoms, the same
+//             slots in shared and tensor memory half used, and the byte pair picked by the instruction descriptor).
+template <bool MX>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_b0,
                      const __grid_constant__ CUtensorMap map_d0, const __grid_constant__ CUtensorMap map_a1,
@@ -293,7 +307,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
         const CUtensorMap* map_a = prob ? &map_a1 : &map_a0;
         const CUtensorMap* map_b = prob ? &map_b1 : &map_b0;
         const int k_blocks = pr.K / 256;
-        const int sf_atoms_k = pr.K / 64;  // atoms along K per 128-row group
+        const int sf_atoms_k = pr.K / (MX ? 128 : 64);  // atoms along K per 128-row group
+        constexpr int kAtomsKb = MX ? 2 : 4;              // atoms per 256-deep k-block and 128-row group
         const int row_a = m_blk * 256 + (int)rank * 128;       // this CTA's A rows
         const int row_b = n_blk * 256 + (int)rank * 128;       // this CTA's half of the B tile
         const uint8_t* sfa = pr.sfa + (int64_t)(m_blk * 2 + (int)rank) * sf_atoms_k * 512;  // own 128 rows
@@ -306,11 +321,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
           tma_load_2d_pair(st, map_a, kb * 128, row_a, bar);
           tma_load_2d_pair(st + kABytes, map_b, kb * 128, row_b, bar);
           // scale atoms: plain bulk copies counted on this CTA's own barrier (its scale warps wait on it)
-          mbar_expect_tx(sfl_bar(stage), kSfaBytes + kSfbBytes);
-          bulk_load(st + kABytes + kBBytes, sfa + (int64_t)kb * 2048, kSfaBytes, sfl_bar(stage));
-          bulk_load(st + kABytes + kBBytes + kSfaBytes, sfb + (int64_t)kb * 2048, 2048, sfl_bar(stage));
-          bulk_load(st + kABytes + kBBytes + kSfaBytes + 2048, sfb + ((int64_t)sf_atoms_k + kb * 4) * 512, 2048,
+          mbar_expect_tx(sfl_bar(stage), 3 * kAtomsKb * 512);
+          bulk_load(st + kABytes + kBBytes, sfa + (int64_t)kb * kAtomsKb * 512, kAtomsKb * 512, sfl_bar(stage));
+          bulk_load(st + kABytes + kBBytes + kSfaBytes, sfb + (int64_t)kb * kAtomsKb * 512, kAtomsKb * 512,
                     sfl_bar(stage));
+          bulk_load(st + kABytes + kBBytes + kSfaBytes + 2048, sfb + ((int64_t)sf_atoms_k + kb * kAtomsKb) * 512,
+                    kAtomsKb * 512, sfl_bar(stage));
           if (++stage == kStages) {
             stage = 0;
             phase ^= 1u;
@@ -338,23 +354,31 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
         if (!ok) break;
         const uint32_t sf_s = base + stage * kStageBytes + kABytes + kBBytes + lane * 16;
         uint32_t r[48];
+        constexpr int kAtomsKb = MX ? 2 : 4;  // atoms per k-block and 128-row group
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < kAtomsKb; ++j) {
           const uint4 a = lds128(sf_s + j * 512);
           r[4 * j] = a.x; r[4 * j + 1] = a.y; r[4 * j + 2] = a.z; r[4 * j + 3] = a.w;
         }
         const uint32_t sf_t = tmem + ((uint32_t)(quad * 32) << 16) + kSfCol + stage * kSfSlotCols;
-        tc_st16(sf_t, &r[0]);
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
+        for (int j = 0; j < kAtomsKb; ++j)
 #pragma unroll
           for (int grp = 0; grp < 2; ++grp) {
             const uint4 b = lds128(sf_s + kSfaBytes + grp * 2048 + j * 512);
             r[16 + 8 * j + 4 * grp] = b.x; r[16 + 8 * j + 4 * grp + 1] = b.y;
             r[16 + 8 * j + 4 * grp + 2] = b.z; r[16 + 8 * j + 4 * grp + 3] = b.w;
           }
-        tc_st16(sf_t + 16, &r[16]);
-        tc_st16(sf_t + 32, &r[32]);
+        if (MX) {
+          asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(sf_t), "r"(r[0]),
+                       "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                       : "memory");
+          tc_st16(sf_t + 16, &r[16]);
+        } else {
+          tc_st16(sf_t, &r[0]);
+          tc_st16(sf_t + 16, &r[16]);
+          tc_st16(sf_t + 32, &r[32]);
+        }
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -373,6 +397,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
       constexpr uint32_t idesc = instr_desc_nvf4(256, 256);
+      constexpr uint32_t idesc_mx[2] = {instr_desc_mxf4(256, 256, 0), instr_desc_mxf4(256, 256, 2)};
       const uint32_t a_lo0 = ((base >> 4) & 0x3fffu) | (1u << 16);
       const uint32_t b_lo0 = (((base + kABytes) >> 4) & 0x3fffu) | (1u << 16);
       for (int tile = pair_id; tile < n_tiles && ok; tile += n_pairs) {
@@ -387,9 +412,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
           const uint32_t b_lo = b_lo0 + stage * (kStageBytes >> 4);
           const uint32_t sf_t = tmem + kSfCol + stage * kSfSlotCols;
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
-            tc2_mma_nvf4(tmem, make_desc(a_lo + 2 * j, kDescHiOperand), make_desc(b_lo + 2 * j, kDescHiOperand), idesc,
-                         sf_t + j * 4, sf_t + 16 + j * 8, (kb > 0 || j > 0) ? 1u : 0u);
+          for (int j = 0; j < 4; ++j) {
+            if (MX)  // one atom (4 columns) serves two K = 64 steps: bytes 0-1, then bytes 2-3
+              tc2_mma_mxf4(tmem, make_desc(a_lo + 2 * j, kDescHiOperand), make_desc(b_lo + 2 * j, kDescHiOperand),
+                           idesc_mx[j & 1], sf_t + (j >> 1) * 4, sf_t + 16 + (j >> 1) * 8, (kb > 0 || j > 0) ? 1u : 0u);
+            else
+              tc2_mma_nvf4(tmem, make_desc(a_lo + 2 * j, kDescHiOperand), make_desc(b_lo + 2 * j, kDescHiOperand), idesc,
+                           sf_t + j * 4, sf_t + 16 + j * 8, (kb > 0 || j > 0) ? 1u : 0u);
+          }
           tc2_commit_both(empty_bar(stage), 3);  // both CTAs' stages are free once these MMAs have read them
           if (++stage == kStages) {
             stage = 0;

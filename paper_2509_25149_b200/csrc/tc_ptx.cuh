@@ -120,6 +120,13 @@ __host__ __device__ constexpr uint32_t instr_desc_nvf4(int m, int n) {
   return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (0u << 23) | ((uint32_t)(m >> 4) << 24);
 }
 
+// Same for MXFP4 (kind::mxf4, scale_vec::2X): UE8M0 scales (bit 23), two scale bytes per row and K = 64 step, taken
+// from bytes [sf_id, sf_id + 2) of the 32-bit tensor-memory column (A: bits 29-30, B: bits 4-5).
+__host__ __device__ constexpr uint32_t instr_desc_mxf4(int m, int n, uint32_t sf_id) {
+  return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(m >> 4) << 24) |
+         (sf_id << 29) | (sf_id << 4);
+}
+
 // ---- host-side tensor-map encoder (driver entry point fetched through the runtime) ----
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
