@@ -40,10 +40,17 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
   if (rows <= 0 || cols <= 0 || rows % 16 != 0 || cols % 16 != 0) return NVFP4_ERR_SHAPE;
   if (ld < cols) return NVFP4_ERR_SHAPE;
   if (ld % 16 != 0 || !aligned(x, 32)) return NVFP4_ERR_ALIGN;
-  if (o->block_rows != 1 && o->block_rows != 16) return NVFP4_ERR_ARG;
+  const int32_t fmt = rowwise ? rowwise->format : colwise->format;
+  if (fmt != NVFP4_FORMAT_NVFP4 && fmt != NVFP4_FORMAT_MXFP4) return NVFP4_ERR_ARG;
+  if (rowwise && colwise && rowwise->format != colwise->format) return NVFP4_ERR_ARG;
+  const bool mx = fmt == NVFP4_FORMAT_MXFP4;
+  const int32_t blk = mx ? 32 : 16;  // block length along the contraction dimension, and the 2D block size
+  if (mx && (rows % 32 != 0 || cols % 32 != 0)) return NVFP4_ERR_SHAPE;
+  if (o->block_rows != 1 && o->block_rows != blk) return NVFP4_ERR_ARG;
   if (o->rounding != NVFP4_ROUND_NEAREST_EVEN && o->rounding != NVFP4_ROUND_STOCHASTIC) return NVFP4_ERR_ARG;
   if ((o->rht_rowwise | o->rht_colwise) & ~1) return NVFP4_ERR_ARG;
-  if (o->block_rows == 16 && (o->rht_rowwise || o->rht_colwise)) return NVFP4_ERR_ARG;
+  if (o->block_rows == blk && (o->rht_rowwise || o->rht_colwise)) return NVFP4_ERR_ARG;
+  if (mx && o->rht_rowwise) return NVFP4_ERR_UNIMPLEMENTED;  // the recipe transforms the transposed copies only
   if (o->flags & ~(NVFP4_SR_INDEPENDENT_COPIES | NVFP4_AMAX_PROVIDED)) return NVFP4_ERR_ARG;
   if (rows > (int64_t)1 << 30 || cols > (int64_t)1 << 30 || ((rows + 127) / 128) * ((cols + 127) / 128) > 0x7fffffff)
     return NVFP4_ERR_SHAPE;
@@ -62,7 +69,7 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
     a.c_codes = colwise->codes; a.c_scales = colwise->scales; a.c_global = colwise->global;
     a.c_swz = colwise->sf_layout == NVFP4_SF_SWIZZLED;
   }
-  a.sign_mask = o->rht_sign_mask & 0xffffu;
+  a.sign_mask = mx ? o->rht_sign_mask : (o->rht_sign_mask & 0xffffu);
   a.seed_lo = (uint32_t)o->seed; a.seed_hi = (uint32_t)(o->seed >> 32);
   a.off_lo = (uint32_t)o->sr_offset; a.off_hi = (uint32_t)(o->sr_offset >> 32);
   a.off_hi_col = (o->flags & NVFP4_SR_INDEPENDENT_COPIES) ? (a.off_hi | 0x80000000u) : a.off_hi;
@@ -70,7 +77,9 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
   a.tiles_c = (int)((cols + 127) / 128);
 
   const bool hr = rowwise != nullptr, hc = colwise != nullptr;
-  const bool b2 = o->block_rows == 16, sr = o->rounding == NVFP4_ROUND_STOCHASTIC;
+  const bool b2 = o->block_rows == blk, sr = o->rounding == NVFP4_ROUND_STOCHASTIC;
+  if (mx)  // no tensor-level scale, hence no amax pass
+    return launch_quantize_mx(a, hr, hc, b2, o->rht_colwise != 0, sr, s) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
   if (!(o->flags & NVFP4_AMAX_PROVIDED)) {
     if (launch_amax(a, hr, hc, o->rht_rowwise != 0, o->rht_colwise != 0, s) != cudaSuccess) return NVFP4_ERR_CUDA;
   }
@@ -278,7 +287,7 @@ nvfp4_status nvfp4_dequantize(const nvfp4_tensor* t, float* out, void* cuda_stre
   if (!t || !out || !t->codes || !t->scales || !t->global) return NVFP4_ERR_NULL;
   nvfp4_status st = check_copy(t, t->rows, t->cols);
   if (st != NVFP4_OK) return st;
-  if (t->rows <= 0 || t->cols <= 0 || t->cols % 16) return NVFP4_ERR_SHAPE;
+  if (t->rows <= 0 || t->cols <= 0 || t->cols % (t->format == NVFP4_FORMAT_MXFP4 ? 32 : 16)) return NVFP4_ERR_SHAPE;
   return launch_dequantize(*t, out, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 

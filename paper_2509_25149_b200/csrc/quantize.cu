@@ -8,44 +8,9 @@
 
 #include "common.cuh"
 #include "quantize.h"
+#include "quantize_common.cuh"
 
 namespace nvfp4 {
-
-// ---------------------------------------------------------------------------------------------
-// small PTX helpers
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void ldg256_stream(const void* p, uint32_t (&r)[8]) {
-  asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-                 "=r"(r[7])
-               : "l"(p));
-}
-__device__ __forceinline__ uint4 ldg128_stream(const void* p) {
-  uint4 r;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-               : "l"(p));
-  return r;
-}
-
-__device__ __forceinline__ uint32_t absmax_bf16x2(uint32_t acc, uint32_t v) {
-  __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&acc);
-  uint32_t m = v & 0x7fff7fffu;
-  __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162*>(&m);
-  __nv_bfloat162 r = __hmax2(a, b);
-  return *reinterpret_cast<uint32_t*>(&r);
-}
-
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  return v;
-}
-
-// sign word for a bf16 pair whose two elements are inputs j0 and j1 of a Hadamard chunk
-__device__ __forceinline__ uint32_t sign_pair(uint32_t mask, int j0, int j1) {
-  return (((mask >> j0) & 1u) << 15) | (((mask >> j1) & 1u) << 31);
-}
 
 // ---------------------------------------------------------------------------------------------
 // Pass 1: tensor amax (Appendix B.1), plain and / or in the rotated space of a transformed copy.
@@ -285,55 +250,6 @@ struct QuantSmemT {
 // the transposed copy with the transform uses the padded pitch
 template <bool HAS_COL, bool BLOCK2D, bool RHT_COL>
 using QuantSmemFor = QuantSmemT<256>;
-
-// 16 scaled values -> 16 E2M1 nibbles (element 0 in the lowest nibble of .x).  For stochastic rounding `nu14(i)`
-// returns the complemented 8-bit draw of element i placed in bits [21, 29).
-template <bool SR, class Nu14>
-__device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, Nu14 nu14) {
-  uint2 out;
-  float v[16];
-#pragma unroll
-  for (int i = 0; i < 16; i += 2) {  // Eq. 4: v = fl(y * s_enc,b), two lanes per instruction
-    const float2 p = mul2(make_float2(f[i], f[i + 1]), make_float2(s_enc_b, s_enc_b));
-    v[i] = p.x;
-    v[i + 1] = p.y;
-  }
-  if (!SR) {
-    const float(&lo)[8] = *reinterpret_cast<const float(*)[8]>(&v[0]);
-    const float(&hi)[8] = *reinterpret_cast<const float(*)[8]>(&v[8]);
-    out.x = e2m1x8_rne(lo);
-    out.y = e2m1x8_rne(hi);
-  } else {
-    out.x = e2m1x8_sr(&v[0], nu14, 0);
-    out.y = e2m1x8_sr(&v[8], nu14, 8);
-  }
-  return out;
-}
-
-// draws packed four to a word, byte i = element i (the row-wise copy: straight from the Philox output)
-struct Nu14FromWords {
-  const uint32_t (&rnd)[4];
-  __device__ __forceinline__ uint32_t operator()(int i) const {
-    const uint32_t nr = ~rnd[i >> 2];
-    const int b = i & 3;
-    return (b == 0 ? (nr << 21) : b == 1 ? (nr << 13) : b == 2 ? (nr << 5) : (nr >> 3)) & 0x1FE00000u;
-  }
-};
-// draws of two adjacent columns, 16 bits per row (the transposed copy: read back from shared memory)
-template <int COL>
-struct Nu14FromPairs {
-  const uint32_t (&two)[16];
-  __device__ __forceinline__ uint32_t operator()(int i) const {
-    return (COL == 0 ? (~two[i] << 21) : (~two[i] << 13)) & 0x1FE00000u;
-  }
-};
-
-__device__ __forceinline__ float amax16(const float (&f)[16]) {
-  float m = 0.f;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(f[i]));
-  return m;
-}
 
 template <bool HAS_ROW, bool HAS_COL, bool BLOCK2D, bool RHT_ROW, bool RHT_COL, bool SR>
 __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const QuantArgs a) {
@@ -595,7 +511,7 @@ __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const Qu
 // ---------------------------------------------------------------------------------------------
 __global__ void dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
                                   const float* __restrict__ global, int64_t rows, int64_t cols, int swz,
-                                  float* __restrict__ out) {
+                                  int mx, float* __restrict__ out) {
   const int64_t n = rows * cols;
   const float s_dec = global[1];
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
@@ -605,11 +521,17 @@ __global__ void dequantize_kernel(const uint8_t* __restrict__ codes, const uint8
     const float mags[8] = {0.f, 0.5f, 1.f, 1.5f, 2.f, 3.f, 4.f, 6.f};
     float m = mags[code & 7u];
     if (code & 8u) m = -m;
-    const int64_t so = swz ? sf_swizzled_offset(r, c >> 4, cols >> 4) : (r * (cols >> 4) + (c >> 4));
+    const int sh = mx ? 5 : 4;  // block length 32 (UE8M0 scale) or 16 (E4M3 scale)
+    const int64_t so = swz ? sf_swizzled_offset(r, c >> sh, cols >> sh) : (r * (cols >> sh) + (c >> sh));
     uint16_t sb = scales[so];
-    uint32_t h2;
-    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(sb));
-    float sf = __half2float(__ushort_as_half((unsigned short)(h2 & 0xffffu)));
+    float sf;
+    if (mx) {
+      sf = sb == 0 ? __uint_as_float(0x00400000u) : __uint_as_float((uint32_t)sb << 23);  // 2^(byte - 127)
+    } else {
+      uint32_t h2;
+      asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(sb));
+      sf = __half2float(__ushort_as_half((unsigned short)(h2 & 0xffffu)));
+    }
     out[i] = __fmul_rn(__fmul_rn(m, sf), s_dec);
   }
 }
@@ -730,7 +652,7 @@ cudaError_t launch_quantize(const QuantArgs& a, bool has_row, bool has_col, bool
 
 cudaError_t launch_dequantize(const nvfp4_tensor& t, float* out, cudaStream_t s) {
   dequantize_kernel<<<1184, 256, 0, s>>>(t.codes, t.scales, t.global, t.rows, t.cols,
-                                         t.sf_layout == NVFP4_SF_SWIZZLED, out);
+                                         t.sf_layout == NVFP4_SF_SWIZZLED, t.format == NVFP4_FORMAT_MXFP4, out);
   count_launch();
   return cudaGetLastError();
 }

@@ -26,6 +26,9 @@ cudaError_t launch_amax(const QuantArgs& a, bool has_row, bool has_col, bool rht
                         cudaStream_t s);
 cudaError_t launch_quantize(const QuantArgs& a, bool has_row, bool has_col, bool block2d, bool rht_row,
                             bool rht_col, bool sr, cudaStream_t s);
+// MXFP4 outputs (quantize_mx.cu): one pass, no tensor-level scale
+cudaError_t launch_quantize_mx(const QuantArgs& a, bool has_row, bool has_col, bool block2d, bool rht_col, bool sr,
+                               cudaStream_t s);
 cudaError_t launch_dequantize(const nvfp4_tensor& t, float* out, cudaStream_t s);
 cudaError_t launch_rht16(const void* x, int64_t rows, int64_t cols, int64_t ld, int colwise, uint32_t mask,
                          float* out, cudaStream_t s);

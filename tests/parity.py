@@ -139,3 +139,77 @@ def assert_gemm_close(D: np.ndarray, Dref: np.ndarray, T: np.ndarray, bf16_out: 
     worst = np.unravel_index(np.argmax(err / tol), err.shape)
     assert np.all(err <= tol), f"{what}: worst at {worst}: got {D[worst]}, want {Dref[worst]}, tol {tol[worst]}"
     return float((err / np.maximum(T, 1e-300)).max())
+
+
+# ------------------------------------------------------------------ MXFP4 (comparison format) ----
+def download_mx(t: B.NVFP4Tensor):
+    """GPU MXFP4 copy -> (codes [R][C/2], UE8M0 scales linear [R][C/32]) as numpy."""
+    torch.cuda.synchronize()
+    codes = t.codes.cpu().numpy()
+    sc = t.scales.cpu().numpy()
+    sc = oracle.sf_unswizzle(sc, t.rows, t.cols // 32) if t.sf_layout == B.SF_SWIZZLED else sc.reshape(t.rows, t.cols // 32)
+    g = t.glob.cpu().numpy()
+    assert g.tolist() == [0.0, 1.0], "an MXFP4 copy has no tensor-level scale"
+    return codes, sc
+
+
+def gpu_quantize_mx(x: torch.Tensor, *, rowwise=True, colwise=False, sf_layout=B.SF_SWIZZLED, **opt):
+    xd = x.cuda()
+    R, C = x.shape
+    row = B.alloc_tensor(R, C, sf_layout, format=B.FORMAT_MXFP4) if rowwise else None
+    col = B.alloc_tensor(C, R, sf_layout, format=B.FORMAT_MXFP4) if colwise else None
+    B.nvfp4_quantize(xd, B.quant_opts(**opt), row, col)
+    torch.cuda.synchronize()
+    return row, col
+
+
+def assert_exact_mx(gpu: B.NVFP4Tensor, ref: oracle.QuantizedMX, what=""):
+    codes, scales = download_mx(gpu)
+    bad = np.argwhere(scales != ref.scales)
+    assert bad.size == 0, f"{what}: {len(bad)} scale bytes differ, first at {bad[0]}: " \
+                          f"{scales[tuple(bad[0])]} vs {ref.scales[tuple(bad[0])]}"
+    bad = np.argwhere(codes != ref.codes)
+    assert bad.size == 0, f"{what}: {len(bad)} code bytes differ, first at {bad[0]}: " \
+                          f"{codes[tuple(bad[0])]:#x} vs {ref.codes[tuple(bad[0])]:#x}"
+
+
+def assert_mx_rht_close(x_bits: np.ndarray, gpu: B.NVFP4Tensor, *, colwise, sign_mask, rounding, seed=0, sr_offset=0,
+                        what=""):
+    """Tolerance protocol for transformed MXFP4 copies (the GPU sums in FP32 and multiplies by fl(1/sqrt(32)), the
+    oracle rounds the exact value once): scale bytes equal except where amax_b / 6 is within 1e-5 of a power of two
+    (an excused byte is adjacent); codes, in blocks whose scale agrees, equal except where the scaled value is
+    within 1e-5 of a rounding threshold (an excused code is an adjacent grid point).  Excused items must stay below
+    1e-3 of all elements."""
+    codes, scales = download_mx(gpu)
+    ref = oracle.quantize_mx(x_bits, colwise=colwise, rht=True, sign_mask=sign_mask, rounding=rounding, seed=seed,
+                             sr_offset=sr_offset, return_y=True)
+    R, C = ref.rows, ref.cols
+    amax_b = np.abs(ref.y.astype(np.float64)).reshape(R, C // 32, 32).max(axis=2)
+    t = amax_b / 6.0
+    with np.errstate(divide="ignore"):
+        frac = np.where(t > 0, t / 2.0 ** np.floor(np.log2(np.maximum(t, 1e-300))), 1.5)  # in [1, 2)
+    near = (frac - 1.0 <= 1e-5) | (2.0 - frac <= 2e-5)
+    sdiff = scales != ref.scales
+    assert not np.any(sdiff & ~near), f"{what}: {np.count_nonzero(sdiff & ~near)} unexcused scale bytes"
+    assert np.all(np.abs(scales.astype(int) - ref.scales.astype(int))[sdiff] == 1), f"{what}: excused scale not adjacent"
+    got, want = unpack(codes), unpack(ref.codes)
+    cdiff = (got != want) & ~np.repeat(sdiff, 32, axis=1)
+    excused = 0
+    for r, c in np.argwhere(cdiff):
+        v = float(np.float32(ref.y[r, c]) * oracle.mx_block_encode_scale(int(ref.scales[r, c // 32])))
+        a = min(abs(v), 6.0)
+        if rounding == oracle.RNE:
+            thr = E2M1_MIDPOINTS
+            step = 0.5 if a < 2 else (1.0 if a < 4 else 2.0)
+        else:
+            sr_, sc_ = (c, r) if colwise else (r, c)
+            u = oracle.sr_draw(seed, sr_offset, sr_ * x_bits.shape[1] + sc_)
+            lo = E2M1_GRID[E2M1_GRID <= a].max()
+            hi = E2M1_GRID[E2M1_GRID > a].min() if a < 6 else 6.0
+            step = max(hi - lo, 0.5)
+            thr = np.array([lo + (hi - lo) * (u + 0.5) / 256])
+        assert np.min(np.abs(thr - a)) <= 1e-5 * max(a, step), f"{what}: code at {(r, c)} differs away from a threshold (v={v})"
+        assert abs(int(got[r, c] & 7) - int(want[r, c] & 7)) <= 1, f"{what}: excused code not adjacent"
+        excused += 1
+    assert excused + int(np.count_nonzero(sdiff)) * 32 <= max(1e-3 * R * C, 32), f"{what}: too many excused items"
+    return {"excused_codes": excused, "excused_scales": int(np.count_nonzero(sdiff)), "elements": R * C}

@@ -69,3 +69,95 @@ def test_gemm_rejects_mixed_formats_and_ragged_mx_shapes():
     with pytest.raises(B.NVFP4Error) as e:
         B.nvfp4_gemm(n, m, torch.empty((256, 256), dtype=torch.float32, device="cuda"))
     assert e.value.status == 4
+
+
+# ------------------------------------------------------------------------------- quantizer ----
+MASK32 = 0xA5C373E5
+
+
+@pytest.mark.parametrize("shape", [(128, 128), (256, 384), (512, 1024), (32, 32), (160, 224), (96, 416)])
+@pytest.mark.parametrize("which", ["row", "col", "both"])
+@pytest.mark.parametrize("rounding", [B.ROUND_NEAREST_EVEN, B.ROUND_STOCHASTIC])
+def test_quantize_1x32_is_bit_exact(shape, which, rounding):
+    x = synth.normal_with_outliers_bf16(shape, 0.01, 50.0, 41, 42)
+    layout = B.SF_SWIZZLED if shape[0] % 128 == 0 and shape[1] % 128 == 0 else B.SF_LINEAR
+    row, col = P.gpu_quantize_mx(x, rowwise=which != "col", colwise=which != "row", sf_layout=layout,
+                                 rounding=rounding, seed=7, sr_offset=3)
+    kw = dict(rounding=rounding, seed=7, sr_offset=3)
+    if row is not None:
+        P.assert_exact_mx(row, oracle.quantize_mx(synth.bits(x), **kw), f"row {shape}")
+    if col is not None:
+        P.assert_exact_mx(col, oracle.quantize_mx(synth.bits(x), colwise=True, **kw), f"col {shape}")
+
+
+@pytest.mark.parametrize("shape", [(128, 128), (256, 384), (160, 224)])
+@pytest.mark.parametrize("rounding", [B.ROUND_NEAREST_EVEN, B.ROUND_STOCHASTIC])
+def test_quantize_32x32_weights_bit_exact_and_consistent(shape, rounding):
+    w = synth.normal_bf16(shape, 0.02, 43)
+    layout = B.SF_SWIZZLED if shape[0] % 128 == 0 and shape[1] % 128 == 0 else B.SF_LINEAR
+    row, col = P.gpu_quantize_mx(w, colwise=True, sf_layout=layout, block_rows=32, rounding=rounding, seed=1)
+    kw = dict(block_rows=32, rounding=rounding, seed=1)
+    P.assert_exact_mx(row, oracle.quantize_mx(synth.bits(w), **kw), "2d row")
+    P.assert_exact_mx(col, oracle.quantize_mx(synth.bits(w), colwise=True, **kw), "2d col")
+    if rounding == B.ROUND_NEAREST_EVEN:
+        rc, _ = P.download_mx(row)
+        cc, _ = P.download_mx(col)
+        assert np.array_equal(P.unpack(rc), P.unpack(cc).T), "the transposed copy holds the same codes"
+
+
+@pytest.mark.parametrize("shape", [(128, 128), (256, 384), (160, 224)])
+@pytest.mark.parametrize("rounding", [B.ROUND_NEAREST_EVEN, B.ROUND_STOCHASTIC])
+def test_quantize_rht32_copy_follows_the_tolerance_protocol(shape, rounding):
+    x = synth.normal_with_outliers_bf16(shape, 0.01, 50.0, 45, 46)
+    layout = B.SF_SWIZZLED if shape[0] % 128 == 0 and shape[1] % 128 == 0 else B.SF_LINEAR
+    row, col = P.gpu_quantize_mx(x, colwise=True, sf_layout=layout, rounding=rounding, rht_colwise=True,
+                                 rht_sign_mask=MASK32, seed=2, sr_offset=5)
+    P.assert_exact_mx(row, oracle.quantize_mx(synth.bits(x), rounding=rounding, seed=2, sr_offset=5), "row beside rht col")
+    st = P.assert_mx_rht_close(synth.bits(x), col, colwise=True, sign_mask=MASK32, rounding=rounding, seed=2,
+                               sr_offset=5, what=f"rht col {shape}")
+    assert st["excused_codes"] + st["excused_scales"] <= max(1e-3 * st["elements"], 32)
+
+
+def test_quantize_degenerate_and_rejected_inputs():
+    z = torch.zeros((128, 128), dtype=torch.bfloat16)
+    row, col = P.gpu_quantize_mx(z, colwise=True)
+    P.assert_exact_mx(row, oracle.quantize_mx(synth.bits(z)), "zeros row")
+    P.assert_exact_mx(col, oracle.quantize_mx(synth.bits(z), colwise=True), "zeros col")
+    for scale in (1e-36, 3e-39, 1e30):
+        x = (synth.normal_bf16((128, 128), 1.0, 21).float() * scale).to(torch.bfloat16)
+        row, col = P.gpu_quantize_mx(x, colwise=True)
+        P.assert_exact_mx(row, oracle.quantize_mx(synth.bits(x)), f"row scale {scale}")
+        P.assert_exact_mx(col, oracle.quantize_mx(synth.bits(x), colwise=True), f"col scale {scale}")
+    x = synth.normal_bf16((48, 64), 1.0, 1).cuda()  # 48 rows: not a multiple of 32
+    with pytest.raises(B.NVFP4Error) as e:
+        B.nvfp4_quantize(x, B.quant_opts(), B.alloc_tensor(48, 64, B.SF_LINEAR, format=B.FORMAT_MXFP4), None)
+    assert e.value.status == 2
+    x = synth.normal_bf16((64, 64), 1.0, 1).cuda()
+    with pytest.raises(B.NVFP4Error) as e:  # 16x16 blocks belong to the other format
+        B.nvfp4_quantize(x, B.quant_opts(block_rows=16), B.alloc_tensor(64, 64, B.SF_LINEAR, format=B.FORMAT_MXFP4), None)
+    assert e.value.status == 4
+    with pytest.raises(B.NVFP4Error) as e:  # the two copies must share a format
+        B.nvfp4_quantize(x, B.quant_opts(), B.alloc_tensor(64, 64, B.SF_LINEAR, format=B.FORMAT_MXFP4),
+                         B.alloc_tensor(64, 64, B.SF_LINEAR))
+    assert e.value.status == 4
+
+
+def test_quantize_then_gemm_matches_the_oracle_pipeline():
+    """Wgrad-like use: both operands transposed copies with the 32-point transform, gradients stochastically rounded."""
+    M, N, K = 512, 256, 256  # tokens, out features, in features
+    X = synth.normal_with_outliers_bf16((M, K), 0.01, 50.0, 51, 52)
+    dY = synth.normal_bf16((M, N), 1e-3, 53)
+    _, x_col = P.gpu_quantize_mx(X, rowwise=False, colwise=True, rht_colwise=True, rht_sign_mask=MASK32)
+    _, g_col = P.gpu_quantize_mx(dY, rowwise=False, colwise=True, rht_colwise=True, rht_sign_mask=MASK32,
+                                 rounding=B.ROUND_STOCHASTIC, seed=4)
+    dW = torch.empty((N, K), dtype=torch.float32, device="cuda")
+    B.nvfp4_gemm(g_col, x_col, dW)
+    B.nvfp4_device_status()
+    # reference: the FP64 product of what the GPU stored (decoded by the oracle)
+    gc, gs = P.download_mx(g_col)
+    xc, xs = P.download_mx(x_col)
+    Dref, T = oracle.gemm_tn(oracle.dequantize_mx(oracle.QuantizedMX(gc, gs, N, M)),
+                             oracle.dequantize_mx(oracle.QuantizedMX(xc, xs, K, M)))
+    P.assert_gemm_close(dW.cpu().numpy(), Dref, T, False, "mx wgrad")
+    exact = dY.double().numpy().T @ X.double().numpy()
+    assert np.linalg.norm(dW.cpu().numpy() - exact) / np.linalg.norm(exact) < 0.35  # the transform cancels
