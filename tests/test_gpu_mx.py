@@ -153,11 +153,12 @@ def test_quantize_then_gemm_matches_the_oracle_pipeline():
     dW = torch.empty((N, K), dtype=torch.float32, device="cuda")
     B.nvfp4_gemm(g_col, x_col, dW)
     B.nvfp4_device_status()
-    # reference: the FP64 product of what the GPU stored (decoded by the oracle)
-    gc, gs = P.download_mx(g_col)
-    xc, xs = P.download_mx(x_col)
-    Dref, T = oracle.gemm_tn(oracle.dequantize_mx(oracle.QuantizedMX(gc, gs, N, M)),
-                             oracle.dequantize_mx(oracle.QuantizedMX(xc, xs, K, M)))
-    P.assert_gemm_close(dW.cpu().numpy(), Dref, T, False, "mx wgrad")
+    # reference: the oracle's own pipeline; the few codes the tolerance protocol may excuse move single products
+    x_ref = oracle.quantize_mx(synth.bits(X), colwise=True, rht=True, sign_mask=MASK32)
+    g_ref = oracle.quantize_mx(synth.bits(dY), colwise=True, rht=True, sign_mask=MASK32, rounding=oracle.SR, seed=4)
+    Dref, T = oracle.gemm_tn(oracle.dequantize_mx(g_ref), oracle.dequantize_mx(x_ref))
+    err = np.abs(dW.cpu().numpy() - Dref)
+    assert np.count_nonzero(err > 1e-3 * T) <= 1e-3 * err.size
+    assert np.all(err <= 2e-2 * T)
     exact = dY.double().numpy().T @ X.double().numpy()
     assert np.linalg.norm(dW.cpu().numpy() - exact) / np.linalg.norm(exact) < 0.35  # the transform cancels
