@@ -158,6 +158,10 @@ NVFP4_API nvfp4_status nvfp4_gemm(const nvfp4_tensor* A, const nvfp4_tensor* B, 
  *   (opts->seed, opts->sr_offset) row-wise for Dgrad and column-wise with the Hadamard transform
  *   for Wgrad.  dX or dW may be NULL to skip that GEMM.  accumulate_dw != 0 adds into dW.
  *   workspace: device scratch of nvfp4_linear_bwd_workspace_bytes(M, N) for the two copies of dY.
+ *   When both GEMMs are requested they run in one launch of the CTA-pair kernel.
+ * Format: the layer runs in the format of the copies it is given (W_row / W_col_saved / X_col_saved must
+ *   agree).  With MXFP4 copies the same sequence uses 1x32 and 32x32 blocks and the 32-point transform
+ *   (Section 5); opts->rht_sign_mask then supplies 32 sign bits.
  */
 NVFP4_API size_t nvfp4_linear_fwd_workspace_bytes(int64_t M, int64_t K);
 NVFP4_API size_t nvfp4_linear_bwd_workspace_bytes(int64_t M, int64_t N);

@@ -149,7 +149,7 @@ inline size_t copy_bytes(int64_t rows, int64_t cols) {
   return align_up((size_t)(rows * cols / 2), 256) + align_up((size_t)(rows * cols / 16), 256) + 256;
 }
 // carve one swizzled-scale copy [rows x cols] out of a workspace
-nvfp4_tensor carve(uint8_t*& p, int64_t rows, int64_t cols) {
+nvfp4_tensor carve(uint8_t*& p, int64_t rows, int64_t cols, int32_t format = NVFP4_FORMAT_NVFP4) {
   nvfp4_tensor t{};
   t.codes = p;
   p += align_up((size_t)(rows * cols / 2), 256);
@@ -158,6 +158,7 @@ nvfp4_tensor carve(uint8_t*& p, int64_t rows, int64_t cols) {
   t.global = reinterpret_cast<float*>(p);
   p += 256;
   t.rows = rows; t.cols = cols; t.sf_layout = NVFP4_SF_SWIZZLED;
+  t.format = format;
   return t;
 }
 
@@ -193,15 +194,18 @@ nvfp4_status nvfp4_linear_fwd(const void* X, const void* W, int64_t M, int64_t N
   if (W_col_saved && (st = check_copy(W_col_saved, K, N)) != NVFP4_OK) return st;
   if (X_col_saved && (st = check_copy(X_col_saved, K, M)) != NVFP4_OK) return st;
   if (W_row->sf_layout != NVFP4_SF_SWIZZLED) return NVFP4_ERR_ARG;
+  // the format of the layer is the format of its weight copy (MXFP4: 32-element blocks, transform size 32)
+  const int32_t fmt = W_row->format;
+  if ((W_col_saved && W_col_saved->format != fmt) || (X_col_saved && X_col_saved->format != fmt)) return NVFP4_ERR_ARG;
 
   if (!w_is_cached) {
     nvfp4_quant_opts wo{};
-    wo.block_rows = 16;
+    wo.block_rows = fmt == NVFP4_FORMAT_MXFP4 ? 32 : 16;
     wo.rounding = NVFP4_ROUND_NEAREST_EVEN;
     if ((st = quantize_impl(W, N, K, K, &wo, W_row, W_col_saved, s)) != NVFP4_OK) return st;
   }
   uint8_t* p = static_cast<uint8_t*>(workspace);
-  nvfp4_tensor x_row = carve(p, M, K);
+  nvfp4_tensor x_row = carve(p, M, K, fmt);
   nvfp4_quant_opts xo{};
   xo.block_rows = 1;
   xo.rounding = NVFP4_ROUND_NEAREST_EVEN;
@@ -227,9 +231,11 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, c
   if (W_col_saved && (st = check_copy(W_col_saved, K, N)) != NVFP4_OK) return st;
   if (X_col_saved && (st = check_copy(X_col_saved, K, M)) != NVFP4_OK) return st;
 
+  const int32_t fmt = W_col_saved ? W_col_saved->format : X_col_saved->format;
+  if (W_col_saved && X_col_saved && W_col_saved->format != X_col_saved->format) return NVFP4_ERR_ARG;
   uint8_t* p = static_cast<uint8_t*>(workspace);
-  nvfp4_tensor g_row = carve(p, M, N);
-  nvfp4_tensor g_col = carve(p, N, M);
+  nvfp4_tensor g_row = carve(p, M, N, fmt);
+  nvfp4_tensor g_col = carve(p, N, M, fmt);
   nvfp4_quant_opts go{};
   go.block_rows = 1;
   go.rounding = NVFP4_ROUND_STOCHASTIC;

@@ -162,3 +162,45 @@ def test_quantize_then_gemm_matches_the_oracle_pipeline():
     assert np.all(err <= 2e-2 * T)
     exact = dY.double().numpy().T @ X.double().numpy()
     assert np.linalg.norm(dW.cpu().numpy() - exact) / np.linalg.norm(exact) < 0.35  # the transform cancels
+
+
+def test_linear_layer_in_mxfp4_matches_the_oracle_pipeline():
+    """fwd + bwd of one layer with MXFP4 copies: every stored operand against the oracle, the three products against
+    the FP64 product of the oracle's own operands."""
+    M, N, K = 512, 768, 256
+    X = synth.normal_with_outliers_bf16((M, K), 0.01, 50.0, 61, 62)
+    W = synth.normal_bf16((N, K), 0.02, 63)
+    dY = synth.normal_bf16((M, N), 1e-3, 64)
+    mx = dict(format=B.FORMAT_MXFP4)
+    X_col, W_row, W_col = B.alloc_tensor(K, M, **mx), B.alloc_tensor(N, K, **mx), B.alloc_tensor(K, N, **mx)
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((N, K), dtype=torch.float32, device="cuda")
+    ws_f = torch.empty(B.nvfp4_linear_fwd_workspace_bytes(M, K), dtype=torch.uint8, device="cuda")
+    ws_b = torch.empty(B.nvfp4_linear_bwd_workspace_bytes(M, N), dtype=torch.uint8, device="cuda")
+    opts = B.quant_opts(rht_sign_mask=MASK32, seed=9, sr_offset=1)
+    B.nvfp4_linear_fwd(X.cuda(), W.cuda(), opts, Y, X_col, W_row, W_col, False, ws_f)
+    B.nvfp4_linear_bwd(dY.cuda(), X_col, W_col, K, opts, dX, dW, False, ws_b)
+    B.nvfp4_device_status()
+    xb, wb, gb = synth.bits(X), synth.bits(W), synth.bits(dY)
+    w_row, w_col = oracle.quantize_mx(wb, block_rows=32), oracle.quantize_mx(wb, block_rows=32, colwise=True)
+    P.assert_exact_mx(W_row, w_row, "W row")
+    P.assert_exact_mx(W_col, w_col, "W col")
+    P.assert_mx_rht_close(xb, X_col, colwise=True, sign_mask=MASK32, rounding=oracle.RNE, what="X col")
+    deq = oracle.dequantize_mx
+    Dref, T = oracle.gemm_tn(deq(oracle.quantize_mx(xb)), deq(w_row))
+    P.assert_gemm_close(Y.float().cpu().numpy(), Dref, T, True, "Fprop")
+    g_row = oracle.quantize_mx(gb, rounding=oracle.SR, seed=9, sr_offset=1)
+    Dref, T = oracle.gemm_tn(deq(g_row), deq(w_col))
+    P.assert_gemm_close(dX.float().cpu().numpy(), Dref, T, True, "Dgrad")
+    g_col = oracle.quantize_mx(gb, colwise=True, rht=True, sign_mask=MASK32, rounding=oracle.SR, seed=9, sr_offset=1)
+    x_col = oracle.quantize_mx(xb, colwise=True, rht=True, sign_mask=MASK32)
+    Dref, T = oracle.gemm_tn(deq(g_col), deq(x_col))
+    err = np.abs(dW.cpu().numpy() - Dref)
+    assert np.count_nonzero(err > 1e-3 * T) <= 1e-3 * err.size and np.all(err <= 2e-2 * T)
+    exact = dY.double().numpy().T @ X.double().numpy()
+    assert np.linalg.norm(dW.cpu().numpy() - exact) / np.linalg.norm(exact) < 0.35
+    # a layer cannot mix formats
+    with pytest.raises(B.NVFP4Error) as e:
+        B.nvfp4_linear_fwd(X.cuda(), W.cuda(), opts, Y, B.alloc_tensor(K, M), W_row, W_col, False, ws_f)
+    assert e.value.status == 4
