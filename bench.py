@@ -184,8 +184,13 @@ def run_cuda(args):
         p.dY = synth.normal_bf16((M, N), 1e-4, 3003 + 100 * rank)
     hX, hW, hdY = p.X.pin_memory(), p.W.pin_memory(), p.dY.pin_memory()
     X, W, dY = hX.cuda(), hW.cuda(), hdY.cuda()
-    opts = B.quant_opts(rht_sign_mask=p.rht_sign_mask, seed=0, sr_offset=dp.rank_sr_offset(rank))
-    X_col, W_row, W_col = B.alloc_tensor(K, M), B.alloc_tensor(N, K), B.alloc_tensor(K, N)
+    # --format mxfp4: the same step in the paper's comparison format (extra measurement; the default is NVFP4)
+    mx = args.format == "mxfp4"
+    fmt = B.FORMAT_MXFP4 if mx else B.FORMAT_NVFP4
+    sign_mask = (p.rht_sign_mask | (0xA5C3 << 16)) if mx else p.rht_sign_mask  # 32 sign bits for the 32-point transform
+    alloc = lambda r, c: B.alloc_tensor(r, c, format=fmt)
+    opts = B.quant_opts(rht_sign_mask=sign_mask, seed=0, sr_offset=dp.rank_sr_offset(rank))
+    X_col, W_row, W_col = alloc(K, M), alloc(N, K), alloc(K, N)
     Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
     dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
     dW = torch.empty((N, K), dtype=torch.float32, device="cuda")
@@ -248,11 +253,11 @@ def run_cuda(args):
     B.nvfp4_device_status()
 
     # ---- per-kernel pass: the same sequence as separate C-ABI calls with events around each ----
-    x_row = B.alloc_tensor(M, K)
-    g_row, g_col = B.alloc_tensor(M, N), B.alloc_tensor(N, M)
-    w_opts = B.quant_opts(block_rows=16)
-    x_opts = B.quant_opts(rht_colwise=True, rht_sign_mask=p.rht_sign_mask)
-    g_opts = B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True, rht_sign_mask=p.rht_sign_mask, seed=0,
+    x_row = alloc(M, K)
+    g_row, g_col = alloc(M, N), alloc(N, M)
+    w_opts = B.quant_opts(block_rows=32 if mx else 16)
+    x_opts = B.quant_opts(rht_colwise=True, rht_sign_mask=sign_mask)
+    g_opts = B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True, rht_sign_mask=sign_mask, seed=0,
                           sr_offset=dp.rank_sr_offset(rank))
     calls = [
         ("quant_W", lambda: B.nvfp4_quantize(W, w_opts, W_row, W_col)),
@@ -343,16 +348,18 @@ def run_cuda(args):
         fp4_peak = 4.0 * peaks["bf16_tflops_sustained"]  # FP4 : BF16 dense = 4 : 1 (nominal ratio)
         # quantizer: algorithmic bytes = two reads of the bf16 tensor + both copies (codes + scales)
         q_elems = M * K + N * K + M * N
-        q_bytes = q_elems * (2 + 2 + 2 * (0.5 + 1.0 / 16))
+        # (MXFP4 has no tensor-level scale, hence one read, and one scale byte per 32 elements)
+        q_bytes = q_elems * ((2 + 2 * (0.5 + 1.0 / 32)) if mx else (2 + 2 + 2 * (0.5 + 1.0 / 16)))
         q_ms = kern_ms["quant_W"] + kern_ms["quant_X"] + kern_ms["quant_dY"]
         q_gbs = q_bytes / (q_ms * 1e-3) / 1e9
-        cpu, _ = cpu_baseline(1) if not args.no_cpu_baseline else (None, 0)
+        cpu, _ = cpu_baseline(1) if not (args.no_cpu_baseline or mx) else (None, 0)
         line = {
             "metric": METRIC, "value": world * flops / (ms_step * 1e-3) / 1e12, "unit": "TFLOP/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1",
             "data": "synthetic",
-            "config": {"workload": WORKLOAD, "tokens_per_gpu": M, "in_features": K, "out_features": N,
+            "config": {"workload": WORKLOAD + ("_mxfp4" if mx else ""), "tokens_per_gpu": M, "in_features": K,
+                       "out_features": N,
                        "parallelism": f"dp{world}", "l2": "inputs (629 MB bf16 per step) exceed the 126 MB L2",
                        "step": "quantize W (2D), quantize X, Fprop, quantize dY (SR), Dgrad, Wgrad"
                                + (", FP32 all-reduce of dW" if world > 1 else "")},
@@ -360,7 +367,7 @@ def run_cuda(args):
             "kernel_ms": {k: round(v, 4) for k, v in kern_ms.items()},
             "roofline": {"bound": "tensor", "kernel": "gemm_kernel (mean of Fprop, Dgrad, Wgrad)",
                          "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
-                         "frac": gemm_tflops / fp4_peak, "traffic": GEMM_DRAM_BYTES_PER_LAUNCH,
+                         "frac": gemm_tflops / fp4_peak, "traffic": None if mx else GEMM_DRAM_BYTES_PER_LAUNCH,
                          "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum, full-size one-pass "
                                            "capture, mean of the three GEMMs (profiles/dram_traffic_cfg3_step.md)",
                          "peak_source": f"4 x {peaks['source']} sustained bf16 cuBLAS ({peaks['bf16_tflops_sustained']} TFLOP/s)",
@@ -368,7 +375,7 @@ def run_cuda(args):
                          "frac_of_datasheet_9pf": gemm_tflops / 9000.0},
             "roofline_quant": {"bound": "hbm", "kernel": "amax kernels + quantize_kernel (W, X, dY)",
                                "achieved": q_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                               "frac": q_gbs / peaks["hbm_gbs"], "traffic": QUANT_DRAM_BYTES_PER_STEP,
+                               "frac": q_gbs / peaks["hbm_gbs"], "traffic": None if mx else QUANT_DRAM_BYTES_PER_STEP,
                                "algorithmic_bytes": q_bytes,
                                "peak_source": f"{peaks['source']} copy bandwidth",
                                "frac_of_datasheet_8tbs": q_gbs / 8000.0},
@@ -558,6 +565,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--format", default="nvfp4", choices=["nvfp4", "mxfp4"],
+                    help="mxfp4: run the step in the paper's comparison format (extra measurement)")
     args = ap.parse_args()
     if args.case:
         run_case(args)
