@@ -55,7 +55,7 @@ constexpr float kInvSqrt32 = 0.176776695296636893f;  // fl(1 / sqrt(32))
 //   phase 2  each thread owns 32 rows x 2 columns of the staged tile and produces the transposed copy;
 //   phase 3  staged codes and scale bytes leave with 16-byte stores.
 template <bool HAS_ROW, bool HAS_COL, bool BLOCK2D, bool RHT_COL, bool SR>
-__global__ void __launch_bounds__(256, 2) quantize_mx_kernel(const QuantArgs a) {
+__global__ void __launch_bounds__(256, RHT_COL ? 2 : 3) quantize_mx_kernel(const QuantArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = (int)blockIdx.x;
