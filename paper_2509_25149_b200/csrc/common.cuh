@@ -80,22 +80,21 @@ __device__ __forceinline__ uint32_t e2m1x8_rne(const float v[8]) {
 // Integer form of that rule.  For 1 <= a <= 6 the binary32 pattern of a is (exponent, one kept mantissa bit,
 // 22 discarded bits m22) and frac = m22 / 2^22, so "round up" <=> m22 > (u << 14) + 2^13 <=> adding
 // D = ((255 - u) << 14) + 0x1FFF carries out of the discarded bits; (bits + D) >> 22 is then
-// 2 * exponent + mantissa bit = code + 252.  Below 1 the grid is uniform (step 0.5): x = a + 1 rounded UP has
-// mantissa ceil(a * 2^23), the comparison with the integer threshold survives the ceiling, and the same carry
-// trick on x gives code + 254.
-// The kernel evaluates this on the pattern shifted left by 7 (one integer multiply-add, on the FMA pipe): the
-// code then sits in the top three bits of the sum, where a funnel shift collects eight codes into a word.
+// 2 * exponent + mantissa bit = code + 252.  Below 1 the grid is uniform (step 0.5) and the value is first mapped
+// to x = a / 2 + 1/2 in [1/2, 1), rounded UP: there the kept bit and the 22 discarded bits of x hold the same
+// (code, frac) as above with the same offset 252, the thresholds are representable at x's spacing so the ceiling
+// preserves the strict comparison, and a carry up to 3/4 or 1 lands on the right code.  Because a / 2 + 1/2 > a
+// exactly when a < 1 (and rounding up cannot pass the representable a), the choice between the two forms is a max.
+// The kernel evaluates the sum on the pattern shifted left by 7 (one integer multiply-add, on the FMA pipe): the
+// code then sits in the top three bits, where a funnel shift collects eight codes into a word.
 //   nu21 : (255 - u) << 21, other bits zero.  Returns s with code = s >> 29 (mod 8), bit 28 is a leftover
 //   fraction bit.
 __device__ __forceinline__ uint32_t e2m1_sr_sum(float v, uint32_t nu21) {
   const float a = fminf(fabsf(v), 6.0f);
-  const bool small = a < 1.0f;
-  const float x = small ? __fadd_ru(a, 1.0f) : a;
+  const float x = fmaxf(a, __fmaf_ru(a, 0.5f, 0.5f));
   // (pattern + D) << 7 with D = ((255 - u) << 14) + 0x1FFF; + (4 << 29) turns (2 * exponent + mantissa bit) mod 8
-  // into the code for a >= 1, the small path needs + (2 << 29) instead
-  uint32_t s = __float_as_uint(x) * 128u + (nu21 | 0x800FFF80u);
-  if (small) s += 0xC0000000u;
-  return s;
+  // into the code
+  return __float_as_uint(x) * 128u + (nu21 | 0x800FFF80u);
 }
 
 // Eight scaled values -> eight E2M1 nibbles with stochastic rounding, element 0 in the lowest nibble.
