@@ -397,6 +397,9 @@ CASES = {
     "quant_x": ("qx", 16384, 5120, 0),             # RNE, row-wise + rotated column-wise (168 MB > L2)
     "quant_dy": ("qdy", 4096, 20480, 0),           # SR, row-wise + rotated column-wise (168 MB > L2)
     "quant_w": ("qw", 20480, 5120, 0),             # 16x16 blocks, both copies (210 MB > L2)
+    "quant_dy_mx": ("qdy_mx", 4096, 20480, 0),      # MXFP4: SR, row-wise + rotated column-wise, one pass
+    "quant_w_mx": ("qw_mx", 20480, 5120, 0),        # MXFP4: 32x32 blocks, both copies
+    "gemm_fprop_mx": ("gemm_mx", 4096, 5120, 5120), # MXFP4 operands, bf16 output
     "step": ("step", 8192, 20480, 5120),           # the whole cfg 3 fwd + bwd step, full size: ONE-PASS captures only
 }
 
@@ -428,6 +431,23 @@ def run_case(args):
             B.nvfp4_linear_fwd(X, W, o, Y, X_col, W_row, W_col, False, ws_f)
             B.nvfp4_linear_bwd(dY, X_col, W_col, k, o, dX, dW, False, ws_b)
         work, unit = 3 * 2.0 * r * c * k / 1e12, "TFLOP/s"
+    elif kind == "gemm_mx":
+        a_src = torch.randn((r, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        b_src = (torch.randn((c, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
+        A, Bq = B.alloc_tensor(r, k, format=B.FORMAT_MXFP4), B.alloc_tensor(c, k, format=B.FORMAT_MXFP4)
+        B.nvfp4_quantize(a_src, B.quant_opts(), A, None)
+        B.nvfp4_quantize(b_src, B.quant_opts(block_rows=32), Bq, None)
+        D = torch.empty((r, c), dtype=torch.bfloat16, device="cuda")
+        fn = lambda: B.nvfp4_gemm(A, Bq, D)
+        work, unit = 2.0 * r * c * k / 1e12, "TFLOP/s"
+    elif kind in ("qdy_mx", "qw_mx"):
+        x = torch.randn((r, c), generator=g, device="cuda", dtype=torch.float32)
+        x = (x * (1e-4 if kind == "qdy_mx" else 0.02)).to(torch.bfloat16)
+        row, col = B.alloc_tensor(r, c, format=B.FORMAT_MXFP4), B.alloc_tensor(c, r, format=B.FORMAT_MXFP4)
+        o = (B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True, rht_sign_mask=0xA5C373E5)
+             if kind == "qdy_mx" else B.quant_opts(block_rows=32))
+        fn = lambda: B.nvfp4_quantize(x, o, row, col)
+        work, unit = r * c * 3.0625 / 1e9, "GB/s"
     elif kind in ("gemm", "gemm32"):
         a_src = torch.randn((r, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
         b_src = (torch.randn((c, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
