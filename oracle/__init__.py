@@ -65,7 +65,7 @@ def lib():
                 "orc_sf_swizzled_offset": (c.c_int64, [c.c_int64, c.c_int64, c.c_int64]),
                 "orc_quantize": (c.c_int, [u16p, c.c_int64, c.c_int64, c.c_int64, c.c_int, c.c_int,
                                            c.c_int, c.c_uint16, c.c_int, c.c_uint64, c.c_uint64,
-                                           c.c_float, c.c_int64, c.c_int64, u8p, u8p, f32p, f32p]),
+                                           c.c_float, c.c_int64, c.c_int64, c.c_int64, u8p, u8p, f32p, f32p]),
                 "orc_dequantize": (None, [u8p, u8p, f32p, c.c_int64, c.c_int64, f64p]),
                 "orc_dequantize_local": (None, [u8p, u8p, c.c_int64, c.c_int64, f64p]),
                 "orc_gemm_tn": (None, [f64p, f64p, c.c_int64, c.c_int64, c.c_int64, f64p, f64p]),
@@ -78,7 +78,7 @@ def lib():
                 "orc_rht32": (None, [f32p, c.c_uint32, f32p]),
                 "orc_quantize_mx": (c.c_int, [u16p, c.c_int64, c.c_int64, c.c_int64, c.c_int, c.c_int,
                                               c.c_int, c.c_uint32, c.c_int, c.c_uint64, c.c_uint64,
-                                              c.c_int64, c.c_int64, u8p, u8p, f32p]),
+                                              c.c_int64, c.c_int64, c.c_int64, u8p, u8p, f32p]),
                 "orc_dequantize_mx": (None, [u8p, u8p, c.c_int64, c.c_int64, f64p]),
             }
             for name, (res, args) in sig.items():
@@ -198,11 +198,11 @@ class Quantized:
 
 
 def quantize(x_bf16_bits, *, colwise=False, block_rows=1, rht=False, sign_mask=0, rounding=RNE,
-             seed=0, sr_offset=0, amax_override=None, return_y=False, sr_row0=0, sr_cols=0) -> Quantized:
+             seed=0, sr_offset=0, amax_override=None, return_y=False, sr_row0=0, sr_cols=0, sr_col0=0) -> Quantized:
     """Quantize one copy of a bf16 tensor given as a 2-D uint16 array of bit patterns.
 
-    sr_row0 / sr_cols: the array is a slab of rows starting at sr_row0 of a larger source with sr_cols columns
-    (only the index of the stochastic-rounding draws depends on it)."""
+    sr_row0 / sr_col0 / sr_cols: the array is the block starting at (sr_row0, sr_col0) of a larger source with
+    sr_cols columns (only the index of the stochastic-rounding draws depends on it)."""
     x = np.asarray(x_bf16_bits)
     assert x.dtype == np.uint16 and x.ndim == 2
     ld = x.strides[0] // 2
@@ -215,7 +215,7 @@ def quantize(x_bf16_bits, *, colwise=False, block_rows=1, rht=False, sign_mask=0
     y = np.zeros((R, C), dtype=np.float32) if return_y else None
     rc = lib().orc_quantize(_p(x, ctypes.c_uint16), sr, sc, ld, int(colwise), block_rows, int(rht),
                             sign_mask, rounding, seed, sr_offset,
-                            np.float32(-1.0 if amax_override is None else amax_override), sr_row0, sr_cols,
+                            np.float32(-1.0 if amax_override is None else amax_override), sr_row0, sr_cols, sr_col0,
                             _p(codes, ctypes.c_uint8), _p(scales, ctypes.c_uint8),
                             _p(glob, ctypes.c_float),
                             _p(y, ctypes.c_float) if return_y else None)
@@ -299,7 +299,7 @@ class QuantizedMX:
 
 
 def quantize_mx(x_bf16_bits, *, colwise=False, block_rows=1, rht=False, sign_mask=0, rounding=RNE, seed=0,
-                sr_offset=0, return_y=False, sr_row0=0, sr_cols=0) -> QuantizedMX:
+                sr_offset=0, return_y=False, sr_row0=0, sr_cols=0, sr_col0=0) -> QuantizedMX:
     """MXFP4 quantization of one copy of a bf16 tensor given as a 2-D uint16 array of bit patterns."""
     x = np.asarray(x_bf16_bits)
     assert x.dtype == np.uint16 and x.ndim == 2 and x.strides[1] == 2
@@ -310,7 +310,7 @@ def quantize_mx(x_bf16_bits, *, colwise=False, block_rows=1, rht=False, sign_mas
     scales = np.zeros((R, max(C // 32, 1)), dtype=np.uint8)
     y = np.zeros((R, C), dtype=np.float32) if return_y else None
     rc = lib().orc_quantize_mx(_p(x, ctypes.c_uint16), sr, sc, ld, int(colwise), block_rows, int(rht), sign_mask,
-                               rounding, seed, sr_offset, sr_row0, sr_cols, _p(codes, ctypes.c_uint8),
+                               rounding, seed, sr_offset, sr_row0, sr_cols, sr_col0, _p(codes, ctypes.c_uint8),
                                _p(scales, ctypes.c_uint8), _p(y, ctypes.c_float) if return_y else None)
     if rc != 0:
         raise ValueError(f"orc_quantize_mx rejected the shape (rc={rc})")

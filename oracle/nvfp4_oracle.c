@@ -247,9 +247,10 @@ ORC_EXPORT int64_t orc_sf_swizzled_offset(int64_t r, int64_t kb, int64_t n_kb) {
  *             comparison protocol under RHT, where a last-bit difference in
  *             amax must not be smeared over every block, and when a slab of
  *             rows of a larger tensor is quantized on its own)
- * sr_row0, sr_cols: the tensor is rows [sr_row0, sr_row0 + src_rows) of a
- *             larger source with sr_cols columns (sr_cols = 0: it is the whole
- *             source); only the stochastic-rounding draw index depends on it
+ * sr_row0, sr_cols, sr_col0: the tensor is the block of rows [sr_row0, sr_row0 +
+ *             src_rows) and columns [sr_col0, sr_col0 + src_cols) of a larger
+ *             source with sr_cols columns (sr_cols = 0: it is the whole source);
+ *             only the stochastic-rounding draw index depends on it
  * outputs   : codes [R][C/2] (even column in the low nibble), scales [R][C/16]
  *             linear, global = {amax, s_dec}, y_out (nullable) = the values
  *             that were quantized, [R][C] floats.   R x C = shape of the copy.
@@ -259,7 +260,7 @@ ORC_EXPORT int64_t orc_sf_swizzled_offset(int64_t r, int64_t kb, int64_t n_kb) {
 ORC_EXPORT int orc_quantize(const uint16_t* x_bf16, int64_t src_rows, int64_t src_cols, int64_t ld,
                             int colwise, int block_rows, int rht, uint16_t sign_mask,
                             int rounding, uint64_t seed, uint64_t sr_offset,
-                            float amax_override, int64_t sr_row0, int64_t sr_cols,
+                            float amax_override, int64_t sr_row0, int64_t sr_cols, int64_t sr_col0,
                             uint8_t* codes, uint8_t* scales, float* global, float* y_out) {
   const int64_t R = colwise ? src_cols : src_rows;
   const int64_t C = colwise ? src_rows : src_cols;
@@ -327,7 +328,7 @@ ORC_EXPORT int orc_quantize(const uint16_t* x_bf16, int64_t src_rows, int64_t sr
           code[j] = orc_e2m1_encode_rne(v);
         } else {
           int64_t sr = colwise ? c : r, sc = colwise ? r : c;
-          uint64_t e = (uint64_t)(sr + sr_row0) * (uint64_t)(sr_cols ? sr_cols : src_cols) + (uint64_t)sc;
+          uint64_t e = (uint64_t)(sr + sr_row0) * (uint64_t)(sr_cols ? sr_cols : src_cols) + (uint64_t)(sc + sr_col0);
           code[j] = orc_e2m1_encode_sr(v, orc_sr_draw(seed, sr_offset, e));
         }
       }
@@ -469,7 +470,7 @@ ORC_EXPORT void orc_rht32(const float x[32], uint32_t sign_mask, float y[32]) {
 ORC_EXPORT int orc_quantize_mx(const uint16_t* x_bf16, int64_t src_rows, int64_t src_cols, int64_t ld,
                                int colwise, int block_rows, int rht, uint32_t sign_mask, int rounding,
                                uint64_t seed, uint64_t sr_offset, int64_t sr_row0, int64_t sr_cols,
-                               uint8_t* codes, uint8_t* scales, float* y_out) {
+                               int64_t sr_col0, uint8_t* codes, uint8_t* scales, float* y_out) {
   const int64_t R = colwise ? src_cols : src_rows;
   const int64_t C = colwise ? src_rows : src_cols;
   if ((block_rows != 1 && block_rows != 32) || C % 32 || R % block_rows) return -1;
@@ -515,7 +516,7 @@ ORC_EXPORT int orc_quantize_mx(const uint16_t* x_bf16, int64_t src_rows, int64_t
           code[j] = orc_e2m1_encode_rne(v);
         } else {
           int64_t sr = colwise ? c : r, sc = colwise ? r : c;
-          uint64_t e = (uint64_t)(sr + sr_row0) * (uint64_t)(sr_cols ? sr_cols : src_cols) + (uint64_t)sc;
+          uint64_t e = (uint64_t)(sr + sr_row0) * (uint64_t)(sr_cols ? sr_cols : src_cols) + (uint64_t)(sc + sr_col0);
           code[j] = orc_e2m1_encode_sr(v, orc_sr_draw(seed, sr_offset, e));
         }
       }

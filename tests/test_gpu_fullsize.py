@@ -56,17 +56,53 @@ def check_copy_slabs(x: torch.Tensor, gpu: B.NVFP4Tensor, *, colwise, block_rows
     assert n_bad <= 1e-3 * n_tot, f"{what}: {n_bad} of {n_tot} elements differ"
 
 
-def check_gemm_samples(D: torch.Tensor, A: B.NVFP4Tensor, Bt: B.NVFP4Tensor, bf16: bool, what: str, seed: int):
+class Operand:
+    """How an operand copy was made from its source, so that the oracle can remake any of its rows."""
+
+    def __init__(self, gpu: B.NVFP4Tensor, src: torch.Tensor, *, colwise, block_rows=1, rht=False, mask=0, rounding=0,
+                 seed=0, sr_offset=0):
+        self.gpu, self.src = gpu, src
+        self.kw = dict(colwise=colwise, block_rows=block_rows, rht=rht, sign_mask=mask, rounding=rounding, seed=seed,
+                       sr_offset=sr_offset)
+        self.colwise = colwise
+
+    def oracle_rows(self, rows):
+        """The sampled rows of the copy, quantized by the oracle from the source (groups of 16 rows of the copy;
+        the tensor amax is the GPU's, as the comparison protocol prescribes)."""
+        amax = float(self.gpu.glob[0])
+        src_bits = synth.bits(self.src)
+        n_cols = self.gpu.cols
+        codes = np.zeros((len(rows), n_cols // 2), np.uint8)
+        scales = np.zeros((len(rows), n_cols // 16), np.uint8)
+        glob = None
+        for i, r in enumerate(rows):
+            g0 = (int(r) // 16) * 16
+            if self.colwise:
+                q = oracle.quantize(src_bits[:, g0:g0 + 16], amax_override=amax, sr_cols=self.src.shape[1], sr_col0=g0,
+                                    **self.kw)
+            else:
+                q = oracle.quantize(src_bits[g0:g0 + 16], amax_override=amax, sr_cols=self.src.shape[1], sr_row0=g0,
+                                    **self.kw)
+            codes[i], scales[i], glob = q.codes[int(r) - g0], q.scales[int(r) - g0], q.glob
+        return oracle.Quantized(codes, scales, glob, len(rows), n_cols)
+
+
+def check_gemm_samples(D: torch.Tensor, A: Operand, Bt: Operand, bf16: bool, what: str, seed: int):
+    """Sampled rows x columns of a full-size product against the FP64 product of operand rows the ORACLE made from
+    the sources.  Operands with the transform may differ from the GPU's in the few codes the protocol excuses, so
+    for them a handful of outputs may exceed the bound by the size of one moved product."""
     rng = np.random.default_rng(seed)
-    rows = np.sort(rng.choice(A.rows, 12, replace=False))
-    cols = np.sort(rng.choice(Bt.rows, 384, replace=False))
-    ac, asc, ag = P.download(A)
-    bc, bsc, bg = P.download(Bt)
-    a = oracle.Quantized(np.ascontiguousarray(ac[rows]), np.ascontiguousarray(asc[rows]), ag, len(rows), A.cols)
-    b = oracle.Quantized(np.ascontiguousarray(bc[cols]), np.ascontiguousarray(bsc[cols]), bg, len(cols), Bt.cols)
+    rows = np.sort(rng.choice(A.gpu.rows, 12, replace=False))
+    cols = np.sort(rng.choice(Bt.gpu.rows, 384, replace=False))
+    a, b = A.oracle_rows(rows), Bt.oracle_rows(cols)
     Dref, T = oracle.gemm_tn(oracle.dequantize(a), oracle.dequantize(b))
     got = D[torch.from_numpy(rows).cuda()][:, torch.from_numpy(cols).cuda()].float().cpu().numpy()
-    P.assert_gemm_close(got, Dref, T, bf16, what)
+    if A.kw["rht"] or Bt.kw["rht"]:
+        err = np.abs(got - Dref)
+        assert np.count_nonzero(err > 1e-3 * T + 1e-30) <= 1e-3 * err.size, what
+        assert np.all(err <= 2e-2 * T + 1e-30), what
+    else:
+        P.assert_gemm_close(got, Dref, T, bf16, what)
 
 
 def test_config3_full_size_forward_and_backward():
@@ -111,9 +147,14 @@ def test_config3_full_size_forward_and_backward():
                      sr_offset=p.sr_offset, what="dY col")
 
     # ---- GEMMs: sampled rows x columns against the FP64 product of the decoded operands -----------------------
-    check_gemm_samples(Y, X_row, W_row, True, "Fprop", 1)
-    check_gemm_samples(dX, g_row, W_col, True, "Dgrad", 2)
-    check_gemm_samples(dW, g_col, X_col, False, "Wgrad", 3)
+    sr = dict(rounding=oracle.SR, seed=p.sr_seed, sr_offset=p.sr_offset)
+    o_x_row, o_x_col = Operand(X_row, p.X, colwise=False), Operand(X_col, p.X, colwise=True, rht=True, mask=mask)
+    o_w_row = Operand(W_row, p.W, colwise=False, block_rows=16)
+    o_w_col = Operand(W_col, p.W, colwise=True, block_rows=16)
+    o_g_row, o_g_col = Operand(g_row, p.dY, colwise=False, **sr), Operand(g_col, p.dY, colwise=True, rht=True, mask=mask, **sr)
+    check_gemm_samples(Y, o_x_row, o_w_row, True, "Fprop", 1)
+    check_gemm_samples(dX, o_g_row, o_w_col, True, "Dgrad", 2)
+    check_gemm_samples(dW, o_g_col, o_x_col, False, "Wgrad", 3)
     # properties that hold at any size: no NaN / Inf, and the layer approximates the unquantized products
     for t in (Y, dX, dW):
         assert torch.isfinite(t.float()).all()
@@ -160,7 +201,8 @@ def test_config4_squared_relu_input_and_long_contraction():
     Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
     B.nvfp4_gemm(X_row, W_row, Y)
     B.nvfp4_device_status()
-    check_gemm_samples(Y, X_row, W_row, True, "cfg4 Fprop", 4)
+    check_gemm_samples(Y, Operand(X_row, p.X, colwise=False), Operand(W_row, p.W, colwise=False, block_rows=16), True,
+                       "cfg4 Fprop", 4)
 
 
 def test_config5_qkv_projection_shapes():
@@ -183,6 +225,11 @@ def test_config5_qkv_projection_shapes():
     g_row, g_col = B.alloc_tensor(M, N), B.alloc_tensor(N, M)
     B.nvfp4_quantize(dY, B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True, rht_sign_mask=p.rht_sign_mask,
                                       seed=p.sr_seed, sr_offset=p.sr_offset), g_row, g_col)
-    check_gemm_samples(Y, X_row, W_row, True, "cfg5 qkv Fprop", 5)
-    check_gemm_samples(dX, g_row, W_col, True, "cfg5 qkv Dgrad", 6)
-    check_gemm_samples(dW, g_col, X_col, False, "cfg5 qkv Wgrad", 7)
+    mask = p.rht_sign_mask
+    sr = dict(rounding=oracle.SR, seed=p.sr_seed, sr_offset=p.sr_offset)
+    check_gemm_samples(Y, Operand(X_row, p.X, colwise=False), Operand(W_row, p.W, colwise=False, block_rows=16), True,
+                       "cfg5 qkv Fprop", 5)
+    check_gemm_samples(dX, Operand(g_row, p.dY, colwise=False, **sr), Operand(W_col, p.W, colwise=True, block_rows=16),
+                       True, "cfg5 qkv Dgrad", 6)
+    check_gemm_samples(dW, Operand(g_col, p.dY, colwise=True, rht=True, mask=mask, **sr),
+                       Operand(X_col, p.X, colwise=True, rht=True, mask=mask), False, "cfg5 qkv Wgrad", 7)

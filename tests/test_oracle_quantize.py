@@ -375,3 +375,22 @@ def test_row_slab_with_given_amax_equals_the_rows_of_the_full_tensor():
                             sr_row0=16, sr_cols=48)
         assert np.array_equal(r.codes, full_r.codes[16:48]) and np.array_equal(r.scales, full_r.scales[16:48])
         assert np.array_equal(c.codes, full_c.codes[:, 8:24]) and np.array_equal(c.scales, full_c.scales[:, 1:3])
+
+
+def test_column_slab_with_given_amax_equals_the_rows_of_the_transposed_copy():
+    # also used by the full-size GPU tests: 16 source columns (a strided view), quantized with the full tensor's
+    # amax and the slab's column offset for the draw index, reproduce 16 rows of the transposed copy and the
+    # corresponding columns of the row-wise copy
+    x = _random_bits((64, 48), 22, scale=1e-3)
+    for rounding in (oracle.RNE, oracle.SR):
+        for rht in (False, True):
+            full_c = oracle.quantize(x, colwise=True, rht=rht, sign_mask=0x73E5, rounding=rounding, seed=3, sr_offset=7)
+            slab = x[:, 16:32]
+            assert slab.strides[0] == 96
+            c = oracle.quantize(slab, colwise=True, rht=rht, sign_mask=0x73E5, rounding=rounding, seed=3, sr_offset=7,
+                                amax_override=float(full_c.amax), sr_cols=48, sr_col0=16)
+            assert np.array_equal(c.codes, full_c.codes[16:32]) and np.array_equal(c.scales, full_c.scales[16:32])
+        full_r = oracle.quantize(x, block_rows=16, rounding=rounding, seed=3, sr_offset=7)
+        r = oracle.quantize(x[:, 16:32], block_rows=16, rounding=rounding, seed=3, sr_offset=7,
+                            amax_override=float(full_r.amax), sr_cols=48, sr_col0=16)
+        assert np.array_equal(r.codes, full_r.codes[:, 8:16]) and np.array_equal(r.scales, full_r.scales[:, 1:2])
