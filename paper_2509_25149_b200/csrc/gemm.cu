@@ -11,6 +11,9 @@
 //   warps 3-6 epilogue: tcgen05.ld of the FP32 accumulator, alpha, conversion, global stores
 // Every wait is bounded: when one expires the kernel records a code in a device status word, every role
 // leaves its loop, tensor memory is released and the kernel returns.
+//
+// This file holds the one-CTA kernel (shapes with M or N not a multiple of 256), the tensor-map helpers and the
+// launchers of both kernels; the CTA-pair kernel that carries the large shapes is in gemm_2cta.cuh.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
