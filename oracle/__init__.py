@@ -66,6 +66,9 @@ def lib():
                 "orc_quantize": (c.c_int, [u16p, c.c_int64, c.c_int64, c.c_int64, c.c_int, c.c_int,
                                            c.c_int, c.c_uint16, c.c_int, c.c_uint64, c.c_uint64,
                                            c.c_float, c.c_int64, c.c_int64, c.c_int64, u8p, u8p, f32p, f32p]),
+                "orc_quantize_f32": (c.c_int, [f32p, c.c_int64, c.c_int64, c.c_int64, c.c_int, c.c_int,
+                                               c.c_int, c.c_uint16, c.c_int, c.c_uint64, c.c_uint64,
+                                               c.c_float, c.c_int64, c.c_int64, c.c_int64, u8p, u8p, f32p, f32p]),
                 "orc_dequantize": (None, [u8p, u8p, f32p, c.c_int64, c.c_int64, f64p]),
                 "orc_dequantize_local": (None, [u8p, u8p, c.c_int64, c.c_int64, f64p]),
                 "orc_gemm_tn": (None, [f64p, f64p, c.c_int64, c.c_int64, c.c_int64, f64p, f64p]),
@@ -199,26 +202,28 @@ class Quantized:
 
 def quantize(x_bf16_bits, *, colwise=False, block_rows=1, rht=False, sign_mask=0, rounding=RNE,
              seed=0, sr_offset=0, amax_override=None, return_y=False, sr_row0=0, sr_cols=0, sr_col0=0) -> Quantized:
-    """Quantize one copy of a bf16 tensor given as a 2-D uint16 array of bit patterns.
+    """Quantize one copy of a bf16 tensor given as a 2-D uint16 array of bit patterns (or of a binary32 tensor given
+    as a float32 array).
 
     sr_row0 / sr_col0 / sr_cols: the array is the block starting at (sr_row0, sr_col0) of a larger source with
     sr_cols columns (only the index of the stochastic-rounding draws depends on it)."""
     x = np.asarray(x_bf16_bits)
-    assert x.dtype == np.uint16 and x.ndim == 2
-    ld = x.strides[0] // 2
-    assert x.strides[1] == 2
+    f32 = x.dtype == np.float32  # a binary32 source instead of bf16 bit patterns
+    assert (x.dtype == np.uint16 or f32) and x.ndim == 2
+    esz = 4 if f32 else 2
+    ld = x.strides[0] // esz
+    assert x.strides[1] == esz
     sr, sc = x.shape
     R, C = (sc, sr) if colwise else (sr, sc)
     codes = np.zeros((R, C // 2), dtype=np.uint8)
     scales = np.zeros((R, C // 16), dtype=np.uint8)
     glob = np.zeros(2, dtype=np.float32)
     y = np.zeros((R, C), dtype=np.float32) if return_y else None
-    rc = lib().orc_quantize(_p(x, ctypes.c_uint16), sr, sc, ld, int(colwise), block_rows, int(rht),
-                            sign_mask, rounding, seed, sr_offset,
-                            np.float32(-1.0 if amax_override is None else amax_override), sr_row0, sr_cols, sr_col0,
-                            _p(codes, ctypes.c_uint8), _p(scales, ctypes.c_uint8),
-                            _p(glob, ctypes.c_float),
-                            _p(y, ctypes.c_float) if return_y else None)
+    fn, src = (lib().orc_quantize_f32, _p(x, ctypes.c_float)) if f32 else (lib().orc_quantize, _p(x, ctypes.c_uint16))
+    rc = fn(src, sr, sc, ld, int(colwise), block_rows, int(rht), sign_mask, rounding, seed, sr_offset,
+            np.float32(-1.0 if amax_override is None else amax_override), sr_row0, sr_cols, sr_col0,
+            _p(codes, ctypes.c_uint8), _p(scales, ctypes.c_uint8), _p(glob, ctypes.c_float),
+            _p(y, ctypes.c_float) if return_y else None)
     if rc != 0:
         raise ValueError(f"orc_quantize rejected the shape (rc={rc})")
     return Quantized(codes, scales, glob, R, C, y)

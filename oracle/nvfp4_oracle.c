@@ -257,11 +257,11 @@ ORC_EXPORT int64_t orc_sf_swizzled_offset(int64_t r, int64_t kb, int64_t n_kb) {
  * returns 0, or -1 when the copy's contraction length is not a multiple of 16
  * (or its row count not a multiple of block_rows).
  */
-ORC_EXPORT int orc_quantize(const uint16_t* x_bf16, int64_t src_rows, int64_t src_cols, int64_t ld,
-                            int colwise, int block_rows, int rht, uint16_t sign_mask,
-                            int rounding, uint64_t seed, uint64_t sr_offset,
-                            float amax_override, int64_t sr_row0, int64_t sr_cols, int64_t sr_col0,
-                            uint8_t* codes, uint8_t* scales, float* global, float* y_out) {
+static int quantize_source(const uint16_t* x_bf16, const float* x_f32, int64_t src_rows, int64_t src_cols,
+                           int64_t ld, int colwise, int block_rows, int rht, uint16_t sign_mask,
+                           int rounding, uint64_t seed, uint64_t sr_offset,
+                           float amax_override, int64_t sr_row0, int64_t sr_cols, int64_t sr_col0,
+                           uint8_t* codes, uint8_t* scales, float* global, float* y_out) {
   const int64_t R = colwise ? src_cols : src_rows;
   const int64_t C = colwise ? src_rows : src_cols;
   if ((block_rows != 1 && block_rows != 16) || C % 16 || R % block_rows) return -1;
@@ -273,7 +273,7 @@ ORC_EXPORT int orc_quantize(const uint16_t* x_bf16, int64_t src_rows, int64_t sr
   for (int64_t r = 0; r < R; ++r)
     for (int64_t c = 0; c < C; ++c) {
       int64_t sr = colwise ? c : r, sc = colwise ? r : c;
-      y[r * C + c] = orc_bf16_to_f32(x_bf16[sr * ld + sc]);
+      y[r * C + c] = x_f32 ? x_f32[sr * ld + sc] : orc_bf16_to_f32(x_bf16[sr * ld + sc]);
     }
 
   /* Appendix C: rotate every aligned chunk of 16 along the contraction dim */
@@ -339,6 +339,26 @@ ORC_EXPORT int orc_quantize(const uint16_t* x_bf16, int64_t src_rows, int64_t sr
   if (y_out) memcpy(y_out, y, sizeof(float) * (size_t)(R * C));
   free(y);
   return 0;
+}
+
+ORC_EXPORT int orc_quantize(const uint16_t* x_bf16, int64_t src_rows, int64_t src_cols, int64_t ld,
+                            int colwise, int block_rows, int rht, uint16_t sign_mask,
+                            int rounding, uint64_t seed, uint64_t sr_offset,
+                            float amax_override, int64_t sr_row0, int64_t sr_cols, int64_t sr_col0,
+                            uint8_t* codes, uint8_t* scales, float* global, float* y_out) {
+  return quantize_source(x_bf16, NULL, src_rows, src_cols, ld, colwise, block_rows, rht, sign_mask, rounding, seed,
+                         sr_offset, amax_override, sr_row0, sr_cols, sr_col0, codes, scales, global, y_out);
+}
+
+/* The same procedure from a binary32 source (Appendix B: "from higher precision (FP32 or BF16)"): only step one,
+ * reading the element, differs. */
+ORC_EXPORT int orc_quantize_f32(const float* x_f32, int64_t src_rows, int64_t src_cols, int64_t ld,
+                                int colwise, int block_rows, int rht, uint16_t sign_mask,
+                                int rounding, uint64_t seed, uint64_t sr_offset,
+                                float amax_override, int64_t sr_row0, int64_t sr_cols, int64_t sr_col0,
+                                uint8_t* codes, uint8_t* scales, float* global, float* y_out) {
+  return quantize_source(NULL, x_f32, src_rows, src_cols, ld, colwise, block_rows, rht, sign_mask, rounding, seed,
+                         sr_offset, amax_override, sr_row0, sr_cols, sr_col0, codes, scales, global, y_out);
 }
 
 /* Decode: x^ = (+-magnitude) * fp32(block scale) * s_dec, in binary64 (exact:

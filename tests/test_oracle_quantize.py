@@ -394,3 +394,29 @@ def test_column_slab_with_given_amax_equals_the_rows_of_the_transposed_copy():
         r = oracle.quantize(x[:, 16:32], block_rows=16, rounding=rounding, seed=3, sr_offset=7,
                             amax_override=float(full_r.amax), sr_cols=48, sr_col0=16)
         assert np.array_equal(r.codes, full_r.codes[:, 8:16]) and np.array_equal(r.scales, full_r.scales[:, 1:2])
+
+
+def test_binary32_source_follows_the_same_procedure():
+    """Appendix B converts "from higher precision (FP32 or BF16)": a binary32 source differs only in how the
+    element is read."""
+    x = _random_bits((32, 64), 31, scale=1.0)
+    xf = synth.from_bits(x).float().numpy()
+    for kw in (dict(), dict(colwise=True), dict(block_rows=16), dict(rounding=oracle.SR, seed=5),
+               dict(colwise=True, rht=True, sign_mask=0x73E5)):
+        a, b = oracle.quantize(x, **kw), oracle.quantize(xf, **kw)  # values exact in bf16: identical results
+        assert np.array_equal(a.codes, b.codes) and np.array_equal(a.scales, b.scales)
+        assert a.glob.view(np.uint32).tolist() == b.glob.view(np.uint32).tolist()
+    # a hand-worked block that bf16 could not hold: amax 2688 * (1 + 2^-20) -> s_enc = fl(2688 / amax) < 1
+    blk = np.zeros((1, 16), dtype=np.float32)
+    blk[0, :4] = [2688.0 * (1 + 2.0 ** -20), 1344.0, -448.0 * (1 + 2.0 ** -12), 3.0000002]
+    q = oracle.quantize(blk)
+    assert float(q.amax) == float(np.float32(2688.0 * (1 + 2.0 ** -20)))
+    s_enc = np.float32(2688.0) / q.amax
+    assert s_enc < 1 and float(q.s_dec) == float(np.float32(1.0) / s_enc)
+    assert q.scales[0, 0] == 0x7E  # the block holding the tensor amax gets 448
+    codes = [(q.codes[0, i // 2] >> (4 * (i & 1))) & 15 for i in range(4)]
+    # v = x * fl(1 / (448 * s_dec)): 6 (amax), 3 (half of it), -1 - a little (rounds to -1), ~0.0067 (rounds to 0)
+    assert [oracle.e2m1_decode(c) for c in codes] == [6.0, 3.0, -1.0, 0.0]
+    # low mantissa bits matter: the same block rounded to bf16 first gives a different tensor amax
+    qb = oracle.quantize(synth.bits(torch.from_numpy(blk).to(torch.bfloat16)))
+    assert float(qb.amax) != float(q.amax)
