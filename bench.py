@@ -400,6 +400,7 @@ CASES = {
     "quant_dy_mx": ("qdy_mx", 4096, 20480, 0),      # MXFP4: SR, row-wise + rotated column-wise, one pass
     "quant_w_mx": ("qw_mx", 20480, 5120, 0),        # MXFP4: 32x32 blocks, both copies
     "gemm_fprop_mx": ("gemm_mx", 4096, 5120, 5120), # MXFP4 operands, bf16 output
+    "quant_w_f32": ("qw_f32", 20480, 5120, 0),      # 16x16 blocks, both copies, from a binary32 source (419 MB)
     "step": ("step", 8192, 20480, 5120),           # the whole cfg 3 fwd + bwd step, full size: ONE-PASS captures only
 }
 
@@ -448,6 +449,12 @@ def run_case(args):
              if kind == "qdy_mx" else B.quant_opts(block_rows=32))
         fn = lambda: B.nvfp4_quantize(x, o, row, col)
         work, unit = r * c * 3.0625 / 1e9, "GB/s"
+    elif kind == "qw_f32":
+        x = torch.randn((r, c), generator=g, device="cuda", dtype=torch.float32) * 0.02
+        row, col = B.alloc_tensor(r, c), B.alloc_tensor(c, r)
+        o = B.quant_opts(block_rows=16)
+        fn = lambda: B.nvfp4_quantize(x, o, row, col)
+        work, unit = r * c * (4 + 4 + 1.125) / 1e9, "GB/s"
     elif kind in ("gemm", "gemm32"):
         a_src = torch.randn((r, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
         b_src = (torch.randn((c, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)

@@ -59,7 +59,10 @@ enum {
      sr_offset set) instead of sharing the draw of the same source element with the row-wise copy */
   NVFP4_SR_INDEPENDENT_COPIES = 1,
   /* global[0] of each requested copy already holds the tensor amax: skip the reduction pass */
-  NVFP4_AMAX_PROVIDED = 2
+  NVFP4_AMAX_PROVIDED = 2,
+  /* the source is binary32 instead of bf16 (Appendix B: "from higher precision (FP32 or BF16)"), e.g. weights
+     quantized from their FP32 master copy.  NVFP4 outputs without the Hadamard transform only; ld counts floats */
+  NVFP4_INPUT_FP32 = 4
 };
 
 /*
@@ -101,7 +104,7 @@ typedef struct nvfp4_quant_opts {
   int32_t rht_colwise;    /*    S*H_16 before scaling (Appendix C); same for the column-wise copy     */
   uint32_t rht_sign_mask; /* low 16 bits: bit j set => the j-th input of a chunk is negated (S_d);    */
                           /* MXFP4 outputs use all 32 bits (transform size 32, Section 5)             */
-  int32_t flags;          /* NVFP4_SR_INDEPENDENT_COPIES | NVFP4_AMAX_PROVIDED                        */
+  int32_t flags;          /* NVFP4_SR_INDEPENDENT_COPIES | NVFP4_AMAX_PROVIDED | NVFP4_INPUT_FP32     */
   uint64_t seed;          /* Philox4x32-10 key                                                        */
   uint64_t sr_offset;     /* Philox counter words 2..3; words 0..1 = (row-major source index) >> 4,   */
                           /* and the element uses byte (index & 15) of the 16 output bytes            */
@@ -111,6 +114,7 @@ typedef struct nvfp4_quant_opts {
  * nvfp4_quantize -- Appendix B (Eq. 1-4) with the recipe options of Section 4.
  *   x_bf16  : device, bf16 [rows x cols] row-major with leading dimension ld (elements);
  *             32-byte aligned, ld % 16 == 0, rows % 16 == 0, cols % 16 == 0.
+ *             With NVFP4_INPUT_FP32 in opts->flags the same for a binary32 array.
  *   rowwise : (nullable) receives the copy whose blocks run along the source columns:
  *             rowwise->rows == rows, rowwise->cols == cols.
  *   colwise : (nullable) receives the quantized TRANSPOSE (blocks along the source rows,

@@ -51,7 +51,9 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
   if ((o->rht_rowwise | o->rht_colwise) & ~1) return NVFP4_ERR_ARG;
   if (o->block_rows == blk && (o->rht_rowwise || o->rht_colwise)) return NVFP4_ERR_ARG;
   if (mx && o->rht_rowwise) return NVFP4_ERR_UNIMPLEMENTED;  // the recipe transforms the transposed copies only
-  if (o->flags & ~(NVFP4_SR_INDEPENDENT_COPIES | NVFP4_AMAX_PROVIDED)) return NVFP4_ERR_ARG;
+  if (o->flags & ~(NVFP4_SR_INDEPENDENT_COPIES | NVFP4_AMAX_PROVIDED | NVFP4_INPUT_FP32)) return NVFP4_ERR_ARG;
+  const bool f32 = (o->flags & NVFP4_INPUT_FP32) != 0;
+  if (f32 && (mx || o->rht_rowwise || o->rht_colwise)) return NVFP4_ERR_UNIMPLEMENTED;
   if (rows > (int64_t)1 << 30 || cols > (int64_t)1 << 30 || ((rows + 127) / 128) * ((cols + 127) / 128) > 0x7fffffff)
     return NVFP4_ERR_SHAPE;
   nvfp4_status st;
@@ -80,6 +82,10 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
   const bool b2 = o->block_rows == blk, sr = o->rounding == NVFP4_ROUND_STOCHASTIC;
   if (mx)  // no tensor-level scale, hence no amax pass
     return launch_quantize_mx(a, hr, hc, b2, o->rht_colwise != 0, sr, s) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+  if (f32) {
+    if (!(o->flags & NVFP4_AMAX_PROVIDED) && launch_amax_f32(a, hr, hc, s) != cudaSuccess) return NVFP4_ERR_CUDA;
+    return launch_quantize_f32(a, hr, hc, b2, sr, s) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+  }
   if (!(o->flags & NVFP4_AMAX_PROVIDED)) {
     if (launch_amax(a, hr, hc, o->rht_rowwise != 0, o->rht_colwise != 0, s) != cudaSuccess) return NVFP4_ERR_CUDA;
   }

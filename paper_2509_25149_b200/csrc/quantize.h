@@ -8,7 +8,7 @@
 namespace nvfp4 {
 
 struct QuantArgs {
-  const uint16_t* x;  // bf16 source [rows x cols], leading dimension ld
+  const uint16_t* x;  // bf16 source [rows x cols], leading dimension ld (binary32 when the f32 launchers are used)
   int64_t rows, cols, ld;
   uint8_t* r_codes;   // row-wise copy
   uint8_t* r_scales;
@@ -29,6 +29,9 @@ cudaError_t launch_quantize(const QuantArgs& a, bool has_row, bool has_col, bool
 // MXFP4 outputs (quantize_mx.cu): one pass, no tensor-level scale
 cudaError_t launch_quantize_mx(const QuantArgs& a, bool has_row, bool has_col, bool block2d, bool rht_col, bool sr,
                                cudaStream_t s);
+// binary32 source (quantize_f32.cu): plain amax pass and the quantize pass, no transform
+cudaError_t launch_amax_f32(const QuantArgs& a, bool has_row, bool has_col, cudaStream_t s);
+cudaError_t launch_quantize_f32(const QuantArgs& a, bool has_row, bool has_col, bool block2d, bool sr, cudaStream_t s);
 cudaError_t launch_dequantize(const nvfp4_tensor& t, float* out, cudaStream_t s);
 cudaError_t launch_rht16(const void* x, int64_t rows, int64_t cols, int64_t ld, int colwise, uint32_t mask,
                          float* out, cudaStream_t s);

@@ -182,3 +182,26 @@ def test_config1_tensors_all_roles():
     P.assert_rht_close(synth.bits(p.dY), col, B.nvfp4_rht16(p.dY.cuda(), True, p.rht_sign_mask).cpu().numpy(),
                        colwise=True, sign_mask=p.rht_sign_mask, rounding=oracle.SR, seed=p.sr_seed,
                        sr_offset=p.sr_offset, what="cfg1 dY col")
+
+
+@pytest.mark.parametrize("shape", [(128, 128), (256, 384), (144, 208)])
+@pytest.mark.parametrize("block_rows", [1, 16])
+@pytest.mark.parametrize("rounding", [B.ROUND_NEAREST_EVEN, B.ROUND_STOCHASTIC])
+def test_binary32_source_is_bit_exact(shape, block_rows, rounding):
+    """Appendix B: the source may be FP32 (e.g. master weights).  Values with full 24-bit mantissas."""
+    g = torch.Generator().manual_seed(77)
+    x = torch.randn(shape, generator=g, dtype=torch.float32) * 0.02
+    x[3, 5] = 1.2345678  # the amax, not representable in bf16
+    layout = B.SF_SWIZZLED if shape[0] % 128 == 0 and shape[1] % 128 == 0 else B.SF_LINEAR
+    R, C = shape
+    row, col = B.alloc_tensor(R, C, layout), B.alloc_tensor(C, R, layout)
+    B.nvfp4_quantize(x.cuda(), B.quant_opts(block_rows=block_rows, rounding=rounding, seed=11, sr_offset=2), row, col)
+    kw = dict(block_rows=block_rows, rounding=rounding, seed=11, sr_offset=2)
+    P.assert_exact(row, oracle.quantize(x.numpy(), **kw), "f32 row")
+    P.assert_exact(col, oracle.quantize(x.numpy(), colwise=True, **kw), "f32 col")
+    only = B.alloc_tensor(C, R, layout)
+    B.nvfp4_quantize(x.cuda(), B.quant_opts(block_rows=block_rows, rounding=rounding, seed=11, sr_offset=2), None, only)
+    P.assert_exact(only, oracle.quantize(x.numpy(), colwise=True, **kw), "f32 col only")
+    with pytest.raises(B.NVFP4Error) as e:  # no transform on a binary32 source
+        B.nvfp4_quantize(x.cuda(), B.quant_opts(rht_colwise=True, rht_sign_mask=MASK), row, col)
+    assert e.value.status == 8
