@@ -73,6 +73,10 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
   }
   a.sign_mask = mx ? o->rht_sign_mask : (o->rht_sign_mask & 0xffffu);
   a.seed_lo = (uint32_t)o->seed; a.seed_hi = (uint32_t)(o->seed >> 32);
+  for (uint32_t r = 0; r < 10; ++r) {  // Philox key schedule
+    a.rk[2 * r] = a.seed_lo + r * 0x9E3779B9u;
+    a.rk[2 * r + 1] = a.seed_hi + r * 0xBB67AE85u;
+  }
   a.off_lo = (uint32_t)o->sr_offset; a.off_hi = (uint32_t)(o->sr_offset >> 32);
   a.off_hi_col = (o->flags & NVFP4_SR_INDEPENDENT_COPIES) ? (a.off_hi | 0x80000000u) : a.off_hi;
   a.tiles_r = (int)((rows + 127) / 128);

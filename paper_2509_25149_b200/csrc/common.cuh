@@ -113,14 +113,16 @@ __device__ __forceinline__ uint32_t e2m1x8_sr(const float* v, Nu21 nu21, int bas
 // ---------------------------------------------------------------------------------------------
 // Philox4x32-10: counter (g.lo, g.hi, off.lo, off.hi), key (seed.lo, seed.hi) -> 16 random bytes
 // ---------------------------------------------------------------------------------------------
+// rk: the ten round keys, (k0 + r * 0x9E3779B9, k1 + r * 0xBB67AE85) for r = 0..9, computed once on the host and
+// read from the kernel's parameter bank
 __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                               uint32_t k0, uint32_t k1) {
+                                               const uint32_t (&rk)[20]) {
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
     const uint64_t p0 = (uint64_t)0xD2511F53u * c0;  // one wide multiply each
     const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
-    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ (k0 + (uint32_t)r * 0x9E3779B9u);
-    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ (k1 + (uint32_t)r * 0xBB67AE85u);
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk[2 * r];
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk[2 * r + 1];
     c0 = n0; c1 = (uint32_t)p1; c2 = n2; c3 = (uint32_t)p0;
   }
   return make_uint4(c0, c1, c2, c3);

@@ -19,6 +19,7 @@ struct QuantArgs {
   int r_swz, c_swz;   // 1 = swizzled scale layout
   uint32_t sign_mask;
   uint32_t seed_lo, seed_hi, off_lo, off_hi, off_hi_col;
+  uint32_t rk[20];       // Philox round keys (seed_lo + r * W0, seed_hi + r * W1), r = 0..9, filled by the host
   int tiles_r, tiles_c;  // 128 x 128 tiles of the source
 };
 

@@ -141,12 +141,12 @@ __global__ void __launch_bounds__(256, 2) quantize_f32_kernel(const QuantArgs a)
     uint32_t rnd[4] = {0u, 0u, 0u, 0u};
     if (SR) {
       const uint64_t g = (uint64_t)(row0 + r) * (uint64_t)n_cb + (uint64_t)((col0 >> 4) + cb);
-      uint4 q = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), a.off_lo, a.off_hi, a.seed_lo, a.seed_hi);
+      uint4 q = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), a.off_lo, a.off_hi, a.rk);
       rnd[0] = q.x; rnd[1] = q.y; rnd[2] = q.z; rnd[3] = q.w;
       if (HAS_COL) {
         uint4 qc = q;
         if (a.off_hi_col != a.off_hi)
-          qc = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), a.off_lo, a.off_hi_col, a.seed_lo, a.seed_hi);
+          qc = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), a.off_lo, a.off_hi_col, a.rk);
         *reinterpret_cast<uint4*>(smem + F32Smem::kRand + r * 128 + ((cb ^ ((r >> 2) & 7)) << 4)) = qc;
       }
     }
