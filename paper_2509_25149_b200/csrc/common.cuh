@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "nvfp4.h"
 
 #if defined(__CUDA_ARCH__) && !defined(__CUDA_ARCH_FEAT_SM100_ALL)
@@ -15,6 +17,18 @@ namespace nvfp4 {
 
 // Host-side launch counter (reported by nvfp4_launch_count()).
 void count_launch(int n = 1);
+
+// One-time, per-device configuration of a call site (function attributes are per device): `seen` holds one bit per
+// device ordinal.  Returns true when the current device still has to be configured; the caller marks it afterwards.
+// Devices beyond ordinal 63 are configured on every call (the attribute calls are idempotent).
+inline bool device_needs_config(const std::atomic<uint64_t>& seen, int* dev) {
+  *dev = -1;
+  if (cudaGetDevice(dev) != cudaSuccess || *dev < 0 || *dev >= 64) return true;
+  return (seen.load(std::memory_order_acquire) & (1ull << *dev)) == 0;
+}
+inline void device_configured(std::atomic<uint64_t>& seen, int dev) {
+  if (dev >= 0 && dev < 64) seen.fetch_or(1ull << dev, std::memory_order_release);
+}
 
 // ---------------------------------------------------------------------------------------------
 // Formats

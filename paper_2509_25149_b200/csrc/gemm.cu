@@ -313,11 +313,12 @@ cudaError_t launch_t(const GemmArgs& g, const void* a_codes, const void* b_codes
   if (!make_code_map(&map_a, a_codes, g.M, g.K / 2, BM) || !make_code_map(&map_b, b_codes, g.N, g.K / 2, BN))
     return cudaErrorInvalidValue;
   auto kern = gemm_kernel<BN>;
-  static bool configured = false;
-  if (!configured) {
+  static std::atomic<uint64_t> configured{0};  // per call site (template instantiation) and device
+  int dev;
+  if (device_needs_config(configured, &dev)) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     if (e != cudaSuccess) return e;
-    configured = true;
+    device_configured(configured, dev);
   }
   const int n_tiles = (g.M / BM) * (g.N / BN);
   const int grid = n_tiles < num_sms ? n_tiles : num_sms;
@@ -353,15 +354,16 @@ cudaError_t launch_pair(const GemmArgs& g0, const void* a0, const void* b0, cons
     m[3] = m[0]; m[4] = m[1]; m[5] = m[2];
   }
   if (g1 && g1->mx != g0.mx) return cudaErrorInvalidValue;
-  static bool configured = false;
-  if (!configured) {
+  static std::atomic<uint64_t> configured{0};  // per call site (template instantiation) and device
+  int dev;
+  if (device_needs_config(configured, &dev)) {
     cudaError_t e = cudaFuncSetAttribute(pair::gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          pair::kSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(pair::gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              pair::kSmemBytes);
     if (e != cudaSuccess) return e;
-    configured = true;
+    device_configured(configured, dev);
   }
   pair::Args a{};
   a.p[0] = pair_problem(g0);
@@ -379,15 +381,17 @@ cudaError_t launch_pair(const GemmArgs& g0, const void* a0, const void* b0, cons
 }
 
 cudaError_t sm_count(int* n) {
-  static int num_sms = 0;
-  if (!num_sms) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+  static std::atomic<int> cache[64] = {};  // per device ordinal
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  int v = (dev >= 0 && dev < 64) ? cache[dev].load(std::memory_order_relaxed) : 0;
+  if (!v) {
+    e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) cache[dev].store(v, std::memory_order_relaxed);
   }
-  *n = num_sms;
+  *n = v;
   return cudaSuccess;
 }
 

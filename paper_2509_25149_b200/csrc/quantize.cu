@@ -612,11 +612,12 @@ static cudaError_t launch_quant_t(const QuantArgs& a, cudaStream_t s) {
   auto kern = quantize_kernel<HR, HC, B2, RR, RC, SR>;
   using QuantSmem = QuantSmemFor<HC, B2, RC>;
   const int smem = (SR && HC) ? QuantSmem::kBytesRand : QuantSmem::kBytesNoRand;
-  static bool configured = false;  // per instantiation; the attribute is per function and idempotent
-  if (!configured) {
+  static std::atomic<uint64_t> configured{0};  // per call site (template instantiation) and device
+  int dev;
+  if (device_needs_config(configured, &dev)) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, QuantSmem::kBytesRand);
     if (e != cudaSuccess) return e;
-    configured = true;
+    device_configured(configured, dev);
   }
   const int64_t tiles = (int64_t)a.tiles_r * a.tiles_c;
   kern<<<(unsigned)tiles, 256, smem, s>>>(a);

@@ -284,11 +284,12 @@ template <bool HR, bool HC, bool B2, bool SR>
 static cudaError_t launch_f32_t(const QuantArgs& a, cudaStream_t s) {
   auto kern = quantize_f32_kernel<HR, HC, B2, SR>;
   const int smem = (SR && HC) ? F32Smem::kBytesRand : F32Smem::kBytesNoRand;
-  static bool configured = false;  // per instantiation; the attribute is per function and idempotent
-  if (!configured) {
+  static std::atomic<uint64_t> configured{0};  // per call site (template instantiation) and device
+  int dev;
+  if (device_needs_config(configured, &dev)) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, F32Smem::kBytesRand);
     if (e != cudaSuccess) return e;
-    configured = true;
+    device_configured(configured, dev);
   }
   kern<<<(unsigned)((int64_t)a.tiles_r * a.tiles_c), 256, smem, s>>>(a);
   count_launch();
