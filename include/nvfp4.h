@@ -141,8 +141,8 @@ NVFP4_API nvfp4_status nvfp4_quantize(const void* x_bf16, int64_t rows, int64_t 
  *   FP32 by the tensor cores; the product of the two tensor decode scales is applied once at the end.
  *   accumulate != 0 adds the product to the existing contents of an fp32 D (gradient accumulation,
  *   Section 4.1); it is rejected for bf16 outputs.
- *   Both operands must have the same format.  MXFP4 operands (no tensor-level scale, the block scales
- *   are powers of two) need M % 256 == 0 and N % 256 == 0; other shapes return NVFP4_ERR_UNIMPLEMENTED.
+ *   Both operands must have the same format (MXFP4 operands carry no tensor-level scale and power-of-two
+ *   block scales per 32 elements).
  */
 NVFP4_API nvfp4_status nvfp4_gemm(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D,
                                   int32_t d_is_fp32, int64_t ldd, int32_t accumulate,

@@ -110,7 +110,6 @@ nvfp4_status gemm_prepare(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D,
   if (A->sf_layout != NVFP4_SF_SWIZZLED || B->sf_layout != NVFP4_SF_SWIZZLED) return NVFP4_ERR_ARG;
   if (A->format != B->format) return NVFP4_ERR_ARG;
   if (A->format != NVFP4_FORMAT_NVFP4 && A->format != NVFP4_FORMAT_MXFP4) return NVFP4_ERR_ARG;
-  if (A->format == NVFP4_FORMAT_MXFP4 && (M % 256 != 0 || N % 256 != 0)) return NVFP4_ERR_UNIMPLEMENTED;
   if (accumulate && !d_is_fp32) return NVFP4_ERR_ARG;
   if (ldd < N) return NVFP4_ERR_SHAPE;
   const int64_t esz = d_is_fp32 ? 4 : 2;
@@ -135,7 +134,6 @@ int gemm_tile(const GemmArgs& g) {
   // (exposed epilogue), 128 x 128 tiles two (the epilogue overlaps the next tile), so the wide tile pays off
   // once the main loop is long enough to amortise the epilogue.
   int tile_n = g_tile_n.load(std::memory_order_relaxed);
-  if (g.mx) return 512;  // MXFP4 runs on the CTA-pair kernel only
   if (tile_n != 128 && tile_n != 256 && tile_n != 512) {
     if (M % 256 == 0 && N % 256 == 0)
       tile_n = 512;

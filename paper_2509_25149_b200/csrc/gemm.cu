@@ -79,7 +79,9 @@ struct Cfg {
 };
 
 // ------------------------------------------------------------------------------------ kernel ----
-template <int BN>
+// MX = true: MXFP4 operands (UE8M0 scale per 32 elements): half the scale atoms per k-block, one atom serving two
+// K = 64 steps through the scale-id field of the instruction descriptor (see gemm_2cta.cuh).
+template <int BN, bool MX>
 __global__ void __launch_bounds__(kThreads, 1)
     gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const GemmArgs g) {
@@ -102,7 +104,8 @@ __global__ void __launch_bounds__(kThreads, 1)
   const int tiles_m = g.M / BM, tiles_n = g.N / BN;
   const int n_tiles = tiles_m * tiles_n;
   const int k_blocks = g.K / BK;
-  const int64_t sf_atoms_per_row_group = g.K / 64;
+  const int64_t sf_atoms_per_row_group = g.K / (MX ? 128 : 64);
+  constexpr int kAtomsKb = MX ? 2 : 4;  // scale atoms per 256-deep k-block and 128-row group
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::kStages; ++s) {
@@ -142,14 +145,15 @@ __global__ void __launch_bounds__(kThreads, 1)
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x100u + stage))) break;
           const uint32_t st = base + stage * C::kStageBytes;
-          mbar_expect_tx(full_bar(stage), C::kStageBytes);
+          mbar_expect_tx(full_bar(stage), C::kABytes + C::kBBytes + (1 + BN / 128) * kAtomsKb * 512);
           tma_load_2d(st, &map_a, kb * BK_BYTES, m_blk * BM, full_bar(stage));
           tma_load_2d(st + C::kABytes, &map_b, kb * BK_BYTES, n_blk * BN, full_bar(stage));
-          bulk_load(st + C::kABytes + C::kBBytes, sfa + (int64_t)kb * 2048, C::kSfaBytes, full_bar(stage));
+          bulk_load(st + C::kABytes + C::kBBytes, sfa + (int64_t)kb * kAtomsKb * 512, kAtomsKb * 512, full_bar(stage));
 #pragma unroll
           for (int grp = 0; grp < BN / 128; ++grp)
             bulk_load(st + C::kABytes + C::kBBytes + C::kSfaBytes + grp * 2048,
-                      sfb + ((int64_t)grp * sf_atoms_per_row_group + (int64_t)kb * 4) * 512, 2048, full_bar(stage));
+                      sfb + ((int64_t)grp * sf_atoms_per_row_group + (int64_t)kb * kAtomsKb) * 512, kAtomsKb * 512,
+                      full_bar(stage));
           if (++stage == C::kStages) {
             stage = 0;
             phase ^= 1u;
@@ -174,7 +178,7 @@ __global__ void __launch_bounds__(kThreads, 1)
           const uint32_t lo = sf_lo0 + stage * (C::kStageBytes >> 4);
           const uint32_t sf_t = tmem + C::kSfCol + stage * C::kSfBufCols;
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
+          for (int j = 0; j < kAtomsKb; ++j) {
             tc_cp_sf(sf_t + j * 4, make_desc(lo + j * 32, kDescHiSf));
 #pragma unroll
             for (int grp = 0; grp < BN / 128; ++grp)
@@ -196,6 +200,7 @@ __global__ void __launch_bounds__(kThreads, 1)
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
       constexpr uint32_t idesc = instr_desc_nvf4(BM, BN);
+      constexpr uint32_t idesc_mx[2] = {instr_desc_mxf4(BM, BN, 0), instr_desc_mxf4(BM, BN, 2)};
       const uint32_t a_lo0 = ((base >> 4) & 0x3fffu) | (1u << 16);
       const uint32_t b_lo0 = (((base + C::kABytes) >> 4) & 0x3fffu) | (1u << 16);
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -211,8 +216,13 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             // advancing 64 elements of K = 32 bytes inside the 128-byte swizzle span: +2 in the address field
-            tc_mma_nvf4(d_tmem, make_desc(a_lo + 2 * j, kDescHiOperand), make_desc(b_lo + 2 * j, kDescHiOperand), idesc,
-                        sf_t + j * 4, sf_t + C::kSfaCols + j * (BN / 32), (kb > 0 || j > 0) ? 1u : 0u);
+            if (MX)
+              tc_mma_mxf4(d_tmem, make_desc(a_lo + 2 * j, kDescHiOperand), make_desc(b_lo + 2 * j, kDescHiOperand),
+                          idesc_mx[j & 1], sf_t + (j >> 1) * 4, sf_t + C::kSfaCols + (j >> 1) * (BN / 32),
+                          (kb > 0 || j > 0) ? 1u : 0u);
+            else
+              tc_mma_nvf4(d_tmem, make_desc(a_lo + 2 * j, kDescHiOperand), make_desc(b_lo + 2 * j, kDescHiOperand), idesc,
+                          sf_t + j * 4, sf_t + C::kSfaCols + j * (BN / 32), (kb > 0 || j > 0) ? 1u : 0u);
           }
           tc_commit(empty_bar(stage));  // frees the stage once the MMAs above have read it
           if (++stage == C::kStages) {
@@ -306,13 +316,13 @@ bool make_code_map(CUtensorMap* map, const void* codes, int64_t rows, int64_t k_
                      BK_BYTES, (uint32_t)box_rows, true);
 }
 
-template <int BN>
+template <int BN, bool MX>
 cudaError_t launch_t(const GemmArgs& g, const void* a_codes, const void* b_codes, int num_sms, cudaStream_t s) {
   using C = Cfg<BN>;
   CUtensorMap map_a, map_b;
   if (!make_code_map(&map_a, a_codes, g.M, g.K / 2, BM) || !make_code_map(&map_b, b_codes, g.N, g.K / 2, BN))
     return cudaErrorInvalidValue;
-  auto kern = gemm_kernel<BN>;
+  auto kern = gemm_kernel<BN, MX>;
   static std::atomic<uint64_t> configured{0};  // per call site (template instantiation) and device
   int dev;
   if (device_needs_config(configured, &dev)) {
@@ -401,11 +411,11 @@ cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_co
   int num_sms = 0;
   cudaError_t e = sm_count(&num_sms);
   if (e != cudaSuccess) return e;
-  if (g.mx && !(g.M % 256 == 0 && g.N % 256 == 0)) return cudaErrorNotSupported;
-  if ((tile_n == 512 || g.mx) && g.M % 256 == 0 && g.N % 256 == 0)
+  if (tile_n == 512 && g.M % 256 == 0 && g.N % 256 == 0)
     return launch_pair(g, a_codes, b_codes, nullptr, nullptr, nullptr, num_sms, s);
-  if (tile_n == 256 && g.N % 256 == 0) return launch_t<256>(g, a_codes, b_codes, num_sms, s);
-  return launch_t<128>(g, a_codes, b_codes, num_sms, s);
+  if (tile_n == 256 && g.N % 256 == 0)
+    return g.mx ? launch_t<256, true>(g, a_codes, b_codes, num_sms, s) : launch_t<256, false>(g, a_codes, b_codes, num_sms, s);
+  return g.mx ? launch_t<128, true>(g, a_codes, b_codes, num_sms, s) : launch_t<128, false>(g, a_codes, b_codes, num_sms, s);
 }
 
 cudaError_t launch_gemm_two(const GemmArgs& g0, const void* a0, const void* b0, const GemmArgs& g1, const void* a1,

@@ -57,13 +57,35 @@ def test_gemm_against_fp64_product_of_decoded_operands(shape, fp32):
     P.assert_gemm_close(run_gemm(a, b, fp32), Dref, T, not fp32, f"mx gemm {shape}")
 
 
-def test_gemm_rejects_mixed_formats_and_ragged_mx_shapes():
-    a = oracle.quantize_mx(synth.bits(synth.normal_bf16((128, 256), 1.0, 1)))
-    A = upload_mx(a)
-    D = torch.empty((128, 128), dtype=torch.float32, device="cuda")
-    with pytest.raises(B.NVFP4Error) as e:
-        B.nvfp4_gemm(A, A, D)  # M, N = 128: only the CTA-pair kernel handles this format
-    assert e.value.status == 8
+@pytest.mark.parametrize("shape", [(128, 128, 256), (384, 640, 768), (256, 256, 1024)])
+@pytest.mark.parametrize("tile_n", [128, 256])
+@pytest.mark.parametrize("fp32", [False, True])
+def test_gemm_one_cta_kernel(shape, tile_n, fp32):
+    """Shapes with M or N not a multiple of 256 (and the forced tile widths) take the one-CTA kernel."""
+    M, N, K = shape
+    a = oracle.quantize_mx(synth.bits(synth.normal_with_outliers_bf16((M, K), 0.01, 50.0, 35, 36)))
+    b = oracle.quantize_mx(synth.bits(synth.normal_bf16((N, K), 0.02, 37)), block_rows=32)
+    Dref, T = reference(a, b)
+    B.nvfp4_set_gemm_tile_n(tile_n)
+    try:
+        D = run_gemm(a, b, fp32)
+    finally:
+        B.nvfp4_set_gemm_tile_n(0)
+    P.assert_gemm_close(D, Dref, T, not fp32, f"mx one-CTA {shape} tile {tile_n}")
+    if shape == (256, 256, 1024) and fp32:  # exact pairing of scale bytes with blocks in this kernel too
+        rng = np.random.default_rng(6)
+        mk = lambda R: oracle.QuantizedMX(np.full((R, K // 2), 0x22, np.uint8),
+                                          (127 + rng.integers(-3, 4, size=(R, K // 32))).astype(np.uint8), R, K)
+        a, b = mk(M), mk(N)
+        B.nvfp4_set_gemm_tile_n(tile_n)
+        try:
+            D = run_gemm(a, b, True)
+        finally:
+            B.nvfp4_set_gemm_tile_n(0)
+        assert np.array_equal(D.astype(np.float64), reference(a, b)[0])
+
+
+def test_gemm_rejects_mixed_formats():
     n = P.upload(oracle.quantize(synth.bits(synth.normal_bf16((256, 256), 1.0, 2))))
     m = upload_mx(oracle.quantize_mx(synth.bits(synth.normal_bf16((256, 256), 1.0, 3))))
     with pytest.raises(B.NVFP4Error) as e:
