@@ -197,25 +197,18 @@ def run_cuda(args):
     ws_f = torch.empty(B.nvfp4_linear_fwd_workspace_bytes(M, K), dtype=torch.uint8, device="cuda")
     ws_b = torch.empty(B.nvfp4_linear_bwd_workspace_bytes(M, N), dtype=torch.uint8, device="cuda")
 
-    # N > 1: the FP32 all-reduce of dW runs beside the next step's kernels; two dW buffers alternate and a buffer
-    # is rewritten only after its own exchange has finished (every step's exchange is inside the timed region, the
-    # last one is waited for before the closing event)
-    dWs = [dW, torch.empty_like(dW)] if world > 1 else [dW]
-    pending = [None] * len(dWs)
-    counter = [0]
+    # N > 1: the FP32 all-reduce of dW runs beside the next step's kernels (two dW buffers alternate, a buffer is
+    # rewritten only after its own exchange has finished); every step's exchange is inside the timed region, the
+    # last one is waited for before the closing event
+    exchange = dp.OverlappedGradExchange(dW)
 
     def step():
-        i = counter[0] % len(dWs)
-        counter[0] += 1
-        dp.wait_weight_grad(pending[i])
+        buf = exchange.acquire()
         B.nvfp4_linear_fwd(X, W, opts, Y, X_col, W_row, W_col, False, ws_f)
-        B.nvfp4_linear_bwd(dY, X_col, W_col, K, opts, dX, dWs[i], False, ws_b)
-        pending[i] = dp.allreduce_weight_grad(dWs[i], async_op=True)  # None at N = 1
+        B.nvfp4_linear_bwd(dY, X_col, W_col, K, opts, dX, buf, False, ws_b)
+        exchange.release(buf)  # asynchronous all-reduce; a no-op at N = 1
 
-    def drain():
-        for j in range(len(pending)):
-            dp.wait_weight_grad(pending[j])
-            pending[j] = None
+    drain = exchange.drain
 
     def barrier():
         if world > 1:

@@ -60,3 +60,36 @@ def reduce_scatter_weight_grad(dW: torch.Tensor, out: torch.Tensor) -> None:
     else:
         assert out.numel() == dW.numel()
         out.copy_(dW.view_as(out))
+
+
+class OverlappedGradExchange:
+    """Weight-gradient buffers whose exchange runs beside the next step's kernels.
+
+    Each step takes a buffer (`acquire`: waits for the exchange that buffer was last handed to), lets the Wgrad GEMM
+    write it, and hands it back (`release`: starts the asynchronous FP32 all-reduce).  With two buffers the exchange
+    of step i overlaps the forward and backward kernels of step i + 1; `drain` waits for everything in flight.
+    Without a process group (one GPU) there is one buffer and the exchange is a no-op."""
+
+    def __init__(self, like: torch.Tensor, n_buffers: int = 2):
+        multi = dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1
+        n = max(1, n_buffers) if multi else 1
+        self.buffers = [like] + [torch.empty_like(like) for _ in range(n - 1)]
+        self.pending = [None] * n
+        self.steps = 0
+
+    def acquire(self) -> torch.Tensor:
+        i = self.steps % len(self.buffers)
+        wait_weight_grad(self.pending[i])
+        self.pending[i] = None
+        return self.buffers[i]
+
+    def release(self, buf: torch.Tensor) -> None:
+        i = self.steps % len(self.buffers)
+        assert buf is self.buffers[i], "release the buffer of the current step"
+        self.pending[i] = allreduce_weight_grad(buf, async_op=True)
+        self.steps += 1
+
+    def drain(self) -> None:
+        for i, w in enumerate(self.pending):
+            wait_weight_grad(w)
+            self.pending[i] = None

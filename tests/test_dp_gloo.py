@@ -44,6 +44,21 @@ def _worker(rank, world, port, out):
         assert torch.equal(ref, dW), "asynchronous all-reduce differs from the blocking one"
         b0, e0 = dp.weight_grad_shard(48, rank, world)
         assert torch.equal(shard, dW[b0:e0]), "reduce-scatter shard differs from the rows of the all-reduced dW"
+        # the overlapped exchange the bench uses at N > 1: buffers alternate, each step's sum is complete when the
+        # buffer comes round again (and after drain)
+        ex = dp.OverlappedGradExchange(torch.zeros(6))
+        assert len(ex.buffers) == 2
+        seen = []
+        for step in range(5):
+            buf = ex.acquire()
+            if step >= 2:
+                seen.append(buf.clone())  # the exchange started two steps ago has finished
+            buf.fill_(float(step * 10 + rank + 1))
+            ex.release(buf)
+        ex.drain()
+        want = lambda st: float(sum(st * 10 + r + 1 for r in range(world)))
+        assert [float(t[0]) for t in seen] == [want(0), want(1), want(2)]
+        assert float(ex.buffers[1][0]) == want(3) and float(ex.buffers[0][0]) == want(4)
         # replicated weights quantize to identical bytes on every rank (deterministic RNE)
         W = synth.normal_bf16((48, 64), 0.02, 3)
         wq = torch.from_numpy(oracle.quantize(synth.bits(W), block_rows=16).codes.copy())
@@ -85,6 +100,10 @@ def test_token_shard_and_offsets():
     assert dp.allreduce_weight_grad(t, async_op=True) is None
     dp.wait_weight_grad(None)
     assert torch.equal(t, torch.ones(4))
+    ex = dp.OverlappedGradExchange(t)  # one buffer, exchange is a no-op
+    assert len(ex.buffers) == 1 and ex.acquire() is t
+    ex.release(t)
+    ex.drain()
     o = torch.empty(4)
     dp.reduce_scatter_weight_grad(t, o)
     assert torch.equal(o, t) and dp.weight_grad_shard(20480, 1, 8) == (2560, 5120)
