@@ -176,6 +176,8 @@ def run_cuda(args):
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     B.lib()
+    if args.gemm_tile:
+        B.nvfp4_set_gemm_tile_n(args.gemm_tile)
 
     # inputs: rank r owns its own 8192-token shard (different seeds per rank), W is replicated
     p = synth.config3()
@@ -585,6 +587,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--gemm-tile", type=int, default=0, choices=[0, 128, 256, 512, 768],
+                    help="force a GEMM tile configuration (0: the library's choice); for experiments")
     ap.add_argument("--format", default="nvfp4", choices=["nvfp4", "mxfp4"],
                     help="mxfp4: run the step in the paper's comparison format (extra measurement)")
     args = ap.parse_args()

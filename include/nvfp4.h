@@ -136,6 +136,7 @@ NVFP4_API nvfp4_status nvfp4_quantize(const void* x_bf16, int64_t rows, int64_t 
  * nvfp4_gemm -- Eq. 5: D[i][j] = s_dec^A * s_dec^B * sum_blocks S^A[i,b] S^B[j,b] sum_{k in b} a[i,k] b[j,k]
  *   A [M x K], B [N x K]: quantized copies whose columns are the contraction dimension, scales in
  *   the NVFP4_SF_SWIZZLED layout, M % 128 == 0, N % 128 == 0, K % 256 == 0 (K = A->cols = B->cols).
+ *   Shapes with M % 256 == 0 run on CTA pairs (256 x 256 or 256 x 384 tiles), others on one CTA per tile.
  *   D: device, row-major [M x N] with leading dimension ldd (elements, >= N, ldd*elemsize % 16 == 0),
  *   bf16 (round-to-nearest-even) when d_is_fp32 == 0, else fp32.  Partial sums are accumulated in
  *   FP32 by the tensor cores; the product of the two tensor decode scales is applied once at the end.
@@ -230,7 +231,10 @@ NVFP4_API nvfp4_status nvfp4_device_status(void* cuda_stream, uint32_t* detail);
 
 /* Tuning knob: which GEMM tiling to use.  128 / 256 = one CTA per 128 x 128 / 128 x 256 output tile;
  * 512 = a CTA pair per 256 x 256 tile (needs M % 256 == 0 and N % 256 == 0, otherwise 128 is used);
- * 0 = choose by shape.  Returns 0, or -1 for any other value.  Process-wide; results do not depend on it
+ * 768 = a CTA pair per 256 x 384 tile, plus up to two 256-wide tiles per row of tiles (needs M % 256 == 0,
+ * N % 128 == 0 and N >= 256, otherwise as 512);
+ * 0 = choose by shape (for the pair kernels: the tile width whose static schedule is estimated shorter).
+ * Returns 0, or -1 for any other value.  Process-wide; results do not depend on it
  * beyond FP32 summation order. */
 NVFP4_API int32_t nvfp4_set_gemm_tile_n(int32_t tile_n);
 

@@ -134,9 +134,11 @@ int gemm_tile(const GemmArgs& g) {
   // (exposed epilogue), 128 x 128 tiles two (the epilogue overlaps the next tile), so the wide tile pays off
   // once the main loop is long enough to amortise the epilogue.
   int tile_n = g_tile_n.load(std::memory_order_relaxed);
-  if (tile_n != 128 && tile_n != 256 && tile_n != 512) {
+  if (tile_n != 128 && tile_n != 256 && tile_n != 512 && tile_n != 768) {
     if (M % 256 == 0 && N % 256 == 0)
-      tile_n = 512;
+      tile_n = prefer_wide_tiles(g, nullptr) ? 768 : 512;  // CTA pairs: the tile width with the shorter schedule
+    else if (M % 256 == 0 && N % 128 == 0 && N >= 256)
+      tile_n = 768;
     else
       tile_n = (K >= (d_is_fp32 ? 16384 : 8192)) ? 256 : 128;
   }
@@ -260,11 +262,14 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, c
     GemmArgs gd, gw;
     if ((st = gemm_prepare(&g_row, W_col_saved, dX_bf16, 0, K, 0, gd)) != NVFP4_OK) return st;
     if ((st = gemm_prepare(&g_col, X_col_saved, dW_fp32, 1, K, accumulate_dw, gw)) != NVFP4_OK) return st;
-    if (gemm_tile(gd) == 512 && gemm_tile(gw) == 512) {
+    const int td = gemm_tile(gd), tw = gemm_tile(gw);
+    if ((td == 512 || td == 768) && (tw == 512 || tw == 768)) {
+      const bool forced = g_tile_n.load(std::memory_order_relaxed) != 0;
       const bool dgrad_first = gd.K >= gw.K;
-      const cudaError_t e = dgrad_first
-                                ? launch_gemm_two(gd, g_row.codes, W_col_saved->codes, gw, g_col.codes, X_col_saved->codes, s)
-                                : launch_gemm_two(gw, g_col.codes, X_col_saved->codes, gd, g_row.codes, W_col_saved->codes, s);
+      const bool wide = forced ? td == 768 : prefer_wide_tiles(dgrad_first ? gd : gw, dgrad_first ? &gw : &gd);
+      const cudaError_t e =
+          dgrad_first ? launch_gemm_two(gd, g_row.codes, W_col_saved->codes, gw, g_col.codes, X_col_saved->codes, wide, s)
+                      : launch_gemm_two(gw, g_col.codes, X_col_saved->codes, gd, g_row.codes, W_col_saved->codes, wide, s);
       return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
     }
   }
@@ -324,7 +329,7 @@ nvfp4_status nvfp4_device_status(void* cuda_stream, uint32_t* detail) {
 }
 
 int32_t nvfp4_set_gemm_tile_n(int32_t tile_n) {
-  if (tile_n != 0 && tile_n != 128 && tile_n != 256 && tile_n != 512) return -1;
+  if (tile_n != 0 && tile_n != 128 && tile_n != 256 && tile_n != 512 && tile_n != 768) return -1;
   g_tile_n.store(tile_n, std::memory_order_relaxed);
   return 0;
 }

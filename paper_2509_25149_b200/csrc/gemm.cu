@@ -18,9 +18,12 @@
 #include <cuda_bf16.h>
 
 #include "common.cuh"
+#include <vector>
+
 #include "gemm.h"
 #include "tc_ptx.cuh"
 #include "gemm_2cta.cuh"
+#include "gemm_wide.cuh"
 
 namespace nvfp4 {
 
@@ -390,6 +393,108 @@ cudaError_t launch_pair(const GemmArgs& g0, const void* a0, const void* b0, cons
   return cudaGetLastError();
 }
 
+// N = 128 q = 384 a + 256 b with b in {0, 1, 2}: a wide column tiles, b narrow ones (q >= 2)
+bool wide_split(int N, int* n_wide, int* n_narrow) {
+  if (N % 128 != 0 || N < 256) return false;
+  const int q = N / 128;
+  const int b = (q % 3 == 0) ? 0 : (q % 3 == 1) ? 2 : 1;
+  if (q - 2 * b < 0) return false;
+  *n_wide = (q - 2 * b) / 3;
+  *n_narrow = b;
+  return true;
+}
+
+bool wide_eligible(const GemmArgs& g) {
+  int a, b;
+  return g.M % 256 == 0 && g.K % 256 == 0 && wide_split(g.N, &a, &b);
+}
+
+wide::WProblem wide_problem(const GemmArgs& g) {
+  int a = 0, b = 0;
+  wide_split(g.N, &a, &b);
+  return wide::WProblem{g.M, g.N, g.K, g.sfa, g.sfb, g.a_global, g.b_global, g.d_is_fp32, g.accumulate, a, a + b};
+}
+
+bool make_wide_maps(const GemmArgs& g, const void* a_codes, const void* b_codes, CUtensorMap* m) {
+  // m[0] A (128-row boxes), m[1] B (128-row boxes), m[2] B (64-row boxes), m[3] D
+  bool ok = make_code_map(&m[0], a_codes, g.M, g.K / 2, 128) && make_code_map(&m[1], b_codes, g.N, g.K / 2, 128) &&
+            make_code_map(&m[2], b_codes, g.N, g.K / 2, 64);
+  if (g.d_is_fp32)
+    ok = ok && make_map_2d(&m[3], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g.d, (uint64_t)g.N, (uint64_t)g.M,
+                           (uint64_t)g.ldd * 4, 32, 128, true);
+  else
+    ok = ok && make_map_2d(&m[3], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, g.d, (uint64_t)g.N, (uint64_t)g.M,
+                           (uint64_t)g.ldd * 2, 64, 128, true);
+  return ok;
+}
+
+// Estimated makespan (in units of one 256-deep k-block of a 256 x 256 tile) of the static round-robin schedule
+// both pair kernels use, for one or two problems: tile t goes to pair t % pairs in the kernels' tile order.  A tile
+// costs its k-blocks times its width factor plus the accumulator hand-over.
+double pair_makespan(const GemmArgs* const* gs, int n_problems, bool wide_tiles, int pairs) {
+  std::vector<double> load((size_t)pairs, 0.0);
+  constexpr int kGroupM = 8;
+  int64_t t = 0;
+  for (int pi = 0; pi < n_problems; ++pi) {
+    const GemmArgs& g = *gs[pi];
+    int n_wide = 0, n_narrow = g.N / 256;
+    if (wide_tiles) wide_split(g.N, &n_wide, &n_narrow);
+    const int tiles_m = g.M / 256, tiles_n = n_wide + n_narrow;
+    const double kb = g.K / 256.0;
+    for (int m0 = 0; m0 < tiles_m; m0 += kGroupM) {
+      const int gm = tiles_m - m0 < kGroupM ? tiles_m - m0 : kGroupM;
+      for (int n_idx = 0; n_idx < tiles_n; ++n_idx) {
+        const bool w = n_idx < n_wide;
+        const double cost = w ? 1.5 * kb + 3.3 : kb + (wide_tiles ? 2.9 : 2.5);
+        for (int i = 0; i < gm; ++i, ++t) load[(size_t)(t % pairs)] += cost;
+      }
+    }
+  }
+  double worst = 0.0;
+  for (double v : load) worst = v > worst ? v : worst;
+  // the wide tiles move 17 % fewer operand bytes per flop; under the power cap that showed as ~3 % more clock
+  return wide_tiles ? worst * 0.97 : worst;
+}
+
+// g1 == nullptr: one problem
+cudaError_t launch_wide(const GemmArgs& g0, const void* a0, const void* b0, const GemmArgs* g1, const void* a1,
+                        const void* b1, int num_sms, cudaStream_t s) {
+  CUtensorMap m[8];
+  if (!make_wide_maps(g0, a0, b0, &m[0])) return cudaErrorInvalidValue;
+  if (g1) {
+    if (!make_wide_maps(*g1, a1, b1, &m[4])) return cudaErrorInvalidValue;
+  } else {
+    for (int i = 0; i < 4; ++i) m[4 + i] = m[i];
+  }
+  if (g1 && g1->mx != g0.mx) return cudaErrorInvalidValue;
+  static std::atomic<uint64_t> configured{0};  // per device
+  int dev;
+  if (device_needs_config(configured, &dev)) {
+    cudaError_t e = cudaFuncSetAttribute(wide::gemm_wide_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         wide::kWSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(wide::gemm_wide_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             wide::kWSmemBytes);
+    if (e != cudaSuccess) return e;
+    device_configured(configured, dev);
+  }
+  wide::WArgs a{};
+  a.p[0] = wide_problem(g0);
+  a.p[1] = wide_problem(g1 ? *g1 : g0);
+  a.n_tiles0 = (g0.M / 256) * a.p[0].tiles_n;
+  a.n_tiles = a.n_tiles0 + (g1 ? (g1->M / 256) * a.p[1].tiles_n : 0);
+  const int max_pairs = num_sms / 2;
+  const int pairs = a.n_tiles < max_pairs ? a.n_tiles : max_pairs;
+  if (g0.mx)
+    wide::gemm_wide_kernel<true><<<2 * pairs, wide::kWThreads, wide::kWSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5],
+                                                                                        m[6], m[7], a);
+  else
+    wide::gemm_wide_kernel<false><<<2 * pairs, wide::kWThreads, wide::kWSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5],
+                                                                                         m[6], m[7], a);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t sm_count(int* n) {
   static std::atomic<int> cache[64] = {};  // per device ordinal
   int dev = 0;
@@ -411,7 +516,8 @@ cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_co
   int num_sms = 0;
   cudaError_t e = sm_count(&num_sms);
   if (e != cudaSuccess) return e;
-  if (tile_n == 512 && g.M % 256 == 0 && g.N % 256 == 0)
+  if (tile_n == 768 && wide_eligible(g)) return launch_wide(g, a_codes, b_codes, nullptr, nullptr, nullptr, num_sms, s);
+  if ((tile_n == 512 || tile_n == 768) && g.M % 256 == 0 && g.N % 256 == 0)
     return launch_pair(g, a_codes, b_codes, nullptr, nullptr, nullptr, num_sms, s);
   if (tile_n == 256 && g.N % 256 == 0)
     return g.mx ? launch_t<256, true>(g, a_codes, b_codes, num_sms, s) : launch_t<256, false>(g, a_codes, b_codes, num_sms, s);
@@ -419,11 +525,22 @@ cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_co
 }
 
 cudaError_t launch_gemm_two(const GemmArgs& g0, const void* a0, const void* b0, const GemmArgs& g1, const void* a1,
-                            const void* b1, cudaStream_t s) {
+                            const void* b1, bool wide_tiles, cudaStream_t s) {
   int num_sms = 0;
   cudaError_t e = sm_count(&num_sms);
   if (e != cudaSuccess) return e;
+  if (wide_tiles && wide_eligible(g0) && wide_eligible(g1)) return launch_wide(g0, a0, b0, &g1, a1, b1, num_sms, s);
   return launch_pair(g0, a0, b0, &g1, a1, b1, num_sms, s);
+}
+
+bool prefer_wide_tiles(const GemmArgs& g0, const GemmArgs* g1) {
+  if (!wide_eligible(g0) || (g1 && !wide_eligible(*g1))) return false;
+  if (g0.N % 256 != 0 || (g1 && g1->N % 256 != 0)) return true;  // only the wide kernel takes N = 128 (2k + 1)
+  int num_sms = 0;
+  if (sm_count(&num_sms) != cudaSuccess) return false;
+  const GemmArgs* gs[2] = {&g0, g1};
+  const int n = g1 ? 2 : 1, pairs = num_sms / 2;
+  return pair_makespan(gs, n, true, pairs) < pair_makespan(gs, n, false, pairs);
 }
 
 cudaError_t read_device_status(cudaStream_t s, uint32_t* code) {

@@ -17,12 +17,16 @@ struct GemmArgs {
   int mx;                 // operands are MXFP4 (UE8M0 scale per 32 elements) instead of NVFP4
 };
 
-// tile_n: 128 or 256 (256 needs N % 256 == 0, otherwise 128 is used)
+// tile_n: 128 or 256 (one CTA per tile; 256 needs N % 256 == 0, otherwise 128 is used), 512 (CTA pairs, 256 x 256
+// tiles; M, N % 256 == 0) or 768 (CTA pairs, 256 x 384 tiles; M % 256 == 0, N % 128 == 0, N >= 256)
 cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_codes, int tile_n, cudaStream_t s);
 // Two independent GEMMs in one launch of the CTA-pair kernel (all of M, N multiples of 256, K of 256): the tiles of
 // g0 are worked through first, then those of g1, on one persistent grid.
+// wide_tiles: 256 x 384 tiles (gemm_wide.cuh) when both shapes allow, else 256 x 256.
 cudaError_t launch_gemm_two(const GemmArgs& g0, const void* a0, const void* b0, const GemmArgs& g1, const void* a1,
-                            const void* b1, cudaStream_t s);
+                            const void* b1, bool wide_tiles, cudaStream_t s);
+// Scheduling estimate: do 256 x 384 tiles beat 256 x 256 tiles for this problem (or pair of problems in one launch)?
+bool prefer_wide_tiles(const GemmArgs& g0, const GemmArgs* g1);
 cudaError_t read_device_status(cudaStream_t s, uint32_t* code);
 
 }  // namespace nvfp4

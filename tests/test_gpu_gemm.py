@@ -31,7 +31,7 @@ def run_gemm(a, b, fp32, tile_n, accumulate=False, D0=None):
         B.nvfp4_set_gemm_tile_n(0)
 
 
-@pytest.mark.parametrize("tile_n", [128, 256, 512])
+@pytest.mark.parametrize("tile_n", [128, 256, 512, 768])
 def test_exact_all_ones(tile_n):
     # every code 1.0 (nibble 2), every block scale 1.0 (0x38), tensor scales 1: each output = K exactly
     M, N, K = 256, 256, 512
@@ -41,7 +41,7 @@ def test_exact_all_ones(tile_n):
     assert np.array_equal(D, np.full((M, N), float(K), np.float32))
 
 
-@pytest.mark.parametrize("tile_n", [128, 256, 512])
+@pytest.mark.parametrize("tile_n", [128, 256, 512, 768])
 def test_exact_small_integers_and_power_of_two_scales(tile_n):
     # codes in {0, +-1, +-2}, power-of-two scales: every partial sum is exact in FP32 in any order
     rng = np.random.default_rng(1)
@@ -62,7 +62,7 @@ def test_exact_small_integers_and_power_of_two_scales(tile_n):
 
 @pytest.mark.parametrize("shape", [(128, 128, 256), (256, 384, 512), (384, 640, 768), (128, 256, 2048),
                                    (256, 256, 256), (512, 768, 1024), (256, 512, 3072)])
-@pytest.mark.parametrize("tile_n", [128, 256, 512])
+@pytest.mark.parametrize("tile_n", [128, 256, 512, 768])
 @pytest.mark.parametrize("fp32", [False, True])
 def test_against_fp64_product_of_decoded_operands(shape, tile_n, fp32):
     M, N, K = shape
@@ -116,3 +116,33 @@ def test_gemm_is_deterministic(tile_n):
     a, b = operands(256, 256, 1024, 5)
     D1, D2 = run_gemm(a, b, True, tile_n), run_gemm(a, b, True, tile_n)
     assert np.array_equal(D1, D2)
+
+
+@pytest.mark.parametrize("shape", [(256, 384, 256), (256, 640, 512), (512, 768, 1024), (256, 1152, 768), (512, 512, 512),
+                                   (768, 1408, 256), (256, 256, 2048)])
+@pytest.mark.parametrize("fp32", [False, True])
+def test_wide_tiles_against_fp64_product(shape, fp32):
+    """256 x 384 tiles: N = 384 a + 256 b with every b in {0, 1, 2}, one and several k-blocks, both outputs."""
+    M, N, K = shape
+    a, b = operands(M, N, K, 41)
+    Dref, T = P.gemm_reference(a, b)
+    P.assert_gemm_close(run_gemm(a, b, fp32, 768), Dref, T, not fp32, f"wide {shape}")
+
+
+def test_wide_tiles_exact_pairing_and_accumulate():
+    rng = np.random.default_rng(9)
+    M, N, K = 512, 1408, 1024  # three wide tiles + one narrow... 1408 = 11 x 128 = 384 * 1 + 256 * 4? no: q = 11 -> b = 1, a = 3
+    nib = np.array([0, 2, 4, 10, 12], dtype=np.uint8)  # 0, 1, 2, -1, -2
+
+    def make(R):
+        c = nib[rng.integers(0, 5, size=(R, K))]
+        codes = (c[:, 0::2] | (c[:, 1::2] << 4)).astype(np.uint8)
+        scales = (rng.integers(5, 10, size=(R, K // 16)).astype(np.uint8) << 3)  # 2^-2 .. 2^2
+        return oracle.Quantized(codes, scales, np.array([1.0, 0.5], np.float32), R, K)
+
+    a, b = make(M), make(N)
+    Dref, _ = P.gemm_reference(a, b)
+    assert np.array_equal(run_gemm(a, b, True, 768).astype(np.float64), Dref)  # every partial sum exact
+    D0 = torch.randn((M, N), device="cuda")
+    D = run_gemm(a, b, True, 768, accumulate=True, D0=D0)
+    assert np.allclose(D - D0.cpu().numpy(), Dref, rtol=0, atol=1e-3 * np.abs(D0.cpu().numpy()).max() + 1e-3)
