@@ -409,6 +409,8 @@ def run_case(args):
 
     kind, r, c, k = CASES[args.case]
     torch.cuda.set_device(0)
+    if args.gemm_tile:
+        B.nvfp4_set_gemm_tile_n(args.gemm_tile)
     g = torch.Generator(device="cuda").manual_seed(1)
     mask = synth.DEFAULT_RHT_SIGN_MASK
     if kind == "step":
