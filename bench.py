@@ -27,9 +27,10 @@ METRIC = "NVFP4 GEMM TFLOP/s vs FP4 peak; quantize+RHT+SR GB/s vs HBM peak"
 M, N, K = 8192, 20480, 5120
 WORKLOAD = "cfg3_ffn_up_fwd_bwd_M8192_K5120_N20480"
 # DRAM bytes (read + write) from a one-pass ncu capture of this workload at full size, cold caches
-# (profiles/dram_traffic_cfg3_step.md): mean of Fprop / Dgrad / Wgrad per launch, and the six quantizer kernels summed.
-GEMM_DRAM_BYTES_PER_LAUNCH = (560.2e6 + 541.5e6 + 655.6e6) / 3
-QUANT_DRAM_BYTES_PER_STEP = 1511.3e6
+# (profiles/dram_traffic_cfg3_step.md): the step's two GEMM launches divided by its three GEMMs, and the six quantizer
+# kernels summed.
+GEMM_DRAM_BYTES_PER_LAUNCH = (548.0e6 + 1136.3e6) / 3  # Fprop launch + merged Dgrad/Wgrad launch, per GEMM
+QUANT_DRAM_BYTES_PER_STEP = 1514.3e6
 SLAB = (4096, 2048, 5120)     # tokens, out-features, in-features of the CPU-baseline sample (one run)
 SLAB_REF = (512, 1024, 5120)  # per-step sample of the `--impl reference` arm (many steps)
 
