@@ -1,11 +1,12 @@
 // Block-scaled FP4 GEMM on CTA pairs with 256 x 384 output tiles.
 //
-// With all 148 SMs busy the main loop of the 256 x 256 pair kernel (gemm_2cta.cuh) is bound by the delivery of
-// operand bytes from L2, not by the tensor pipe: what shortens it is fewer bytes per flop, i.e. a larger tile.
-// Tensor memory decides how large: 512 columns hold a 384-column FP32 accumulator plus two 64-column slots for the
-// scale factors.  A 256 x 384 tile moves (256 + 384) / (256 * 384) operand rows per output, 17 % less than 256 x 256,
-// and has a third fewer accumulator hand-overs per output.  N is cut into 384-wide tiles plus zero, one or two
-// 256-wide ones (N = 128 q = 384 a + 256 b); both widths run through the same code.
+// The largest tile a CTA pair can hold: tensor memory has 512 columns, enough for a 384-column FP32 accumulator plus
+// two 64-column slots for the scale factors.  A 256 x 384 tile moves (256 + 384) / (256 * 384) operand rows per
+// output, 17 % less than the 256 x 256 tile of gemm_2cta.cuh, and has a third fewer accumulator hand-overs per
+// output.  With all 148 SMs on the tensor pipe the part is power-capped, so less data movement per flop shows up as
+// a little more clock rather than as a shorter k-block; the price is a coarser schedule, which is why the host
+// picks the tile width per problem from an estimate of the schedule.  N is cut into 384-wide tiles plus zero, one
+// or two 256-wide ones (N = 128 q = 384 a + 256 b); both widths run through the same code.
 //
 // Per K = 64 step the 384 columns take two instructions (N = 256 and N = 128; the B tile of a CTA is its 128 rows
 // of the first 256 and its 64 rows of the last 128).  Roles as in the pair kernel; differences:
@@ -225,6 +226,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
     int stage = 0;
     uint32_t phase = 0, it = 0;  // it: k-blocks processed so far (selects the slot)
     const uint32_t sff_leader = map_to_cta(sff_bar(0), 0);
+    uint32_t r[64];  // the slot's 64 columns; entries of a narrow tile's third group keep stale (unused) values
+#pragma unroll
+    for (int i = 0; i < 64; ++i) r[i] = 0u;
     for (int tile = pair_id; tile < n_tiles; tile += n_pairs) {
       bool ok = true;
       int prob, m_blk, n0, width;
@@ -241,9 +245,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
         if (!ok) break;
         tc_fence_after();
         const uint32_t sf_s = base + stage * kWStageBytes + kWABytes + kWBBytes + lane * 16;
-        uint32_t r[64];
-#pragma unroll
-        for (int i = 0; i < 64; ++i) r[i] = 0u;
 #pragma unroll
         for (int j = 0; j < kAtomsKb; ++j) {
           const uint4 a = lds128(sf_s + j * 512);
