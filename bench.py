@@ -248,6 +248,34 @@ def run_cuda(args):
     ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps)
     B.nvfp4_device_status()
 
+    # ---- the same step with the quantized weight reused (micro-batches between optimizer steps): extra figure ----
+    def step_cached():
+        buf = exchange.acquire()
+        B.nvfp4_linear_fwd(X, None, opts, Y, X_col, W_row, W_col, True, ws_f)
+        B.nvfp4_linear_bwd(dY, X_col, W_col, K, opts, dX, buf, False, ws_b)
+        exchange.release(buf)
+
+    # blocks of 20 steps alternate between the two variants so that both see the same clocks (the step is
+    # power-capped: a block timed right after another one inherits its clock state)
+    def timed_block(fn, n=20):
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        b0.record()
+        for _ in range(n):
+            fn()
+        drain()
+        b1.record()
+        torch.cuda.synchronize()
+        return b0.elapsed_time(b1) / n
+
+    barrier()
+    alt = {"full": [], "cached": []}
+    for _ in range(8):
+        alt["full"].append(timed_block(step))
+        alt["cached"].append(timed_block(step_cached))
+    barrier()
+    ms_alt_full = max_over_ranks(sum(alt["full"]) / len(alt["full"]))
+    ms_step_cached = max_over_ranks(sum(alt["cached"]) / len(alt["cached"]))
+
     # ---- per-kernel pass: the same sequence as separate C-ABI calls with events around each ----
     x_row = alloc(M, K)
     g_row, g_col = alloc(M, N), alloc(N, M)
@@ -359,6 +387,9 @@ def run_cuda(args):
                        "parallelism": f"dp{world}", "l2": "inputs (629 MB bf16 per step) exceed the 126 MB L2",
                        "step": "quantize W (2D), quantize X, Fprop, quantize dY (SR), Dgrad, Wgrad"
                                + (", FP32 all-reduce of dW" if world > 1 else "")},
+            # extra: the step with the quantized weight reused (no quantize W), and the full step again, timed in
+            # alternating blocks of 20 steps
+            "ms_per_step_w_cached": ms_step_cached, "ms_per_step_alternating": ms_alt_full,
             "gemm_tflops": gemm_tflops, "quant_gbs": q_gbs,
             "kernel_ms": {k: round(v, 4) for k, v in kern_ms.items()},
             "roofline": {"bound": "tensor", "kernel": "gemm_kernel (mean of Fprop, Dgrad, Wgrad)",
