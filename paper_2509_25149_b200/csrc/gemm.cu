@@ -18,6 +18,8 @@
 #include <cuda_bf16.h>
 
 #include "common.cuh"
+#include <algorithm>
+#include <mutex>
 #include <vector>
 
 #include "gemm.h"
@@ -538,9 +540,28 @@ bool prefer_wide_tiles(const GemmArgs& g0, const GemmArgs* g1) {
   if (g0.N % 256 != 0 || (g1 && g1->N % 256 != 0)) return true;  // only the wide kernel takes N = 128 (2k + 1)
   int num_sms = 0;
   if (sm_count(&num_sms) != cudaSuccess) return false;
+  // the estimate walks every tile of both schedules: remember the answers for the shapes seen (a training loop
+  // repeats a handful of them)
+  struct Entry { int key[7]; bool wide; };
+  static std::mutex mu;
+  static std::vector<Entry> seen;
+  const int key[7] = {g0.M, g0.N, g0.K, g1 ? g1->M : 0, g1 ? g1->N : 0, g1 ? g1->K : 0, num_sms};
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    for (const Entry& e : seen)
+      if (std::equal(key, key + 7, e.key)) return e.wide;
+  }
   const GemmArgs* gs[2] = {&g0, g1};
   const int n = g1 ? 2 : 1, pairs = num_sms / 2;
-  return pair_makespan(gs, n, true, pairs) < pair_makespan(gs, n, false, pairs);
+  const bool wide = pair_makespan(gs, n, true, pairs) < pair_makespan(gs, n, false, pairs);
+  std::lock_guard<std::mutex> lock(mu);
+  if (seen.size() < 256) {
+    Entry e{};
+    std::copy(key, key + 7, e.key);
+    e.wide = wide;
+    seen.push_back(e);
+  }
+  return wide;
 }
 
 cudaError_t read_device_status(cudaStream_t s, uint32_t* code) {
