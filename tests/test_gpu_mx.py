@@ -226,3 +226,72 @@ def test_linear_layer_in_mxfp4_matches_the_oracle_pipeline():
     with pytest.raises(B.NVFP4Error) as e:
         B.nvfp4_linear_fwd(X.cuda(), W.cuda(), opts, Y, B.alloc_tensor(K, M), W_row, W_col, False, ws_f)
     assert e.value.status == 4
+
+
+def test_full_size_layer_in_mxfp4_sampled():
+    """The bench's cfg 3 layer (M 8192, K 5120, N 20480) in MXFP4: stored operands on sampled slabs, the three
+    products on sampled rows x columns against operand rows the oracle remakes from the sources."""
+    p = synth.config3()
+    M, N, K = p.M, p.N, p.K
+    mx = dict(format=B.FORMAT_MXFP4)
+    X, W, dY = p.X.cuda(), p.W.cuda(), p.dY.cuda()
+    X_col, W_row, W_col = B.alloc_tensor(K, M, **mx), B.alloc_tensor(N, K, **mx), B.alloc_tensor(K, N, **mx)
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((N, K), dtype=torch.float32, device="cuda")
+    ws_f = torch.empty(B.nvfp4_linear_fwd_workspace_bytes(M, K), dtype=torch.uint8, device="cuda")
+    ws_b = torch.empty(B.nvfp4_linear_bwd_workspace_bytes(M, N), dtype=torch.uint8, device="cuda")
+    opts = B.quant_opts(rht_sign_mask=MASK32, seed=p.sr_seed, sr_offset=p.sr_offset)
+    B.nvfp4_linear_fwd(X, W, opts, Y, X_col, W_row, W_col, False, ws_f)
+    B.nvfp4_linear_bwd(dY, X_col, W_col, K, opts, dX, dW, False, ws_b)
+    B.nvfp4_device_status()
+    for t in (Y, dX, dW):
+        assert torch.isfinite(t.float()).all()
+
+    xb, wb, gb = synth.bits(p.X), synth.bits(p.W), synth.bits(p.dY)
+    sr = dict(rounding=oracle.SR, seed=p.sr_seed, sr_offset=p.sr_offset)
+
+    def rows_of(src_bits, rows, *, colwise, block_rows=1, rht=False, **kw):
+        """Rows of a copy, remade by the oracle from 32-row (or 32-column) slabs of the source."""
+        n_src_cols = src_bits.shape[1]
+        codes, scales = [], []
+        for r in rows:
+            g0 = (int(r) // 32) * 32
+            if colwise:
+                q = oracle.quantize_mx(src_bits[:, g0:g0 + 32], colwise=True, block_rows=block_rows, rht=rht,
+                                       sign_mask=MASK32, sr_cols=n_src_cols, sr_col0=g0, **kw)
+            else:
+                q = oracle.quantize_mx(src_bits[g0:g0 + 32], block_rows=block_rows, sr_cols=n_src_cols, sr_row0=g0, **kw)
+            codes.append(q.codes[int(r) - g0])
+            scales.append(q.scales[int(r) - g0])
+        n_cols = src_bits.shape[0] if colwise else n_src_cols
+        return oracle.QuantizedMX(np.stack(codes), np.stack(scales), len(rows), n_cols)
+
+    # stored weight copies: sampled rows, bit-exact
+    rng = np.random.default_rng(11)
+    wr, wc = P.download_mx(W_row), P.download_mx(W_col)
+    rows = np.sort(rng.choice(N, 8, replace=False))
+    ref = rows_of(wb, rows, colwise=False, block_rows=32)
+    assert np.array_equal(wr[0][rows], ref.codes) and np.array_equal(wr[1][rows], ref.scales)
+    cols = np.sort(rng.choice(K, 8, replace=False))
+    ref = rows_of(wb, cols, colwise=True, block_rows=32)
+    assert np.array_equal(wc[0][cols], ref.codes) and np.array_equal(wc[1][cols], ref.scales)
+
+    def check(D, a, b, rows, cols, bf16, loose, what):
+        Dref, T = oracle.gemm_tn(oracle.dequantize_mx(a), oracle.dequantize_mx(b))
+        got = D[torch.from_numpy(rows).cuda()][:, torch.from_numpy(cols).cuda()].float().cpu().numpy()
+        if loose:  # transformed operands: the few codes the protocol may excuse move single products
+            err = np.abs(got - Dref)
+            assert np.count_nonzero(err > 1e-3 * T + 1e-30) <= 1e-3 * err.size and np.all(err <= 2e-2 * T + 1e-30), what
+        else:
+            P.assert_gemm_close(got, Dref, T, bf16, what)
+
+    r12 = np.sort(rng.choice(M, 12, replace=False))
+    c256 = np.sort(rng.choice(N, 256, replace=False))
+    check(Y, rows_of(xb, r12, colwise=False), rows_of(wb, c256, colwise=False, block_rows=32), r12, c256, True, False, "Fprop")
+    k256 = np.sort(rng.choice(K, 256, replace=False))
+    check(dX, rows_of(gb, r12, colwise=False, **sr), rows_of(wb, k256, colwise=True, block_rows=32), r12, k256, True, False,
+          "Dgrad")
+    n12 = np.sort(rng.choice(N, 12, replace=False))
+    check(dW, rows_of(gb, n12, colwise=True, rht=True, **sr), rows_of(xb, k256, colwise=True, rht=True), n12, k256, False,
+          True, "Wgrad")
