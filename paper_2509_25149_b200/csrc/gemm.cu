@@ -431,7 +431,8 @@ bool make_wide_maps(const GemmArgs& g, const void* a_codes, const void* b_codes,
 }
 
 // Estimated makespan (in units of one 256-deep k-block of a 256 x 256 tile) of the static round-robin schedule
-// both pair kernels use, for one or two problems: tile t goes to pair t % pairs in the kernels' tile order.  A tile
+// the pair kernels use, for one or two problems: round r hands tiles r * pairs .. to the pairs in order, odd rounds
+// in reverse order.  A tile
 // costs its k-blocks times its width factor plus the accumulator hand-over.
 double pair_makespan(const GemmArgs* const* gs, int n_problems, bool wide_tiles, int pairs) {
   std::vector<double> load((size_t)pairs, 0.0);
@@ -448,7 +449,10 @@ double pair_makespan(const GemmArgs* const* gs, int n_problems, bool wide_tiles,
       for (int n_idx = 0; n_idx < tiles_n; ++n_idx) {
         const bool w = n_idx < n_wide;
         const double cost = w ? 1.5 * kb + 3.3 : kb + (wide_tiles ? 2.9 : 2.5);
-        for (int i = 0; i < gm; ++i, ++t) load[(size_t)(t % pairs)] += cost;
+        for (int i = 0; i < gm; ++i, ++t) {
+          const int64_t rnd = t / pairs, p = t % pairs;
+          load[(size_t)((rnd & 1) ? pairs - 1 - p : p)] += cost;  // odd rounds run through the pairs in reverse
+        }
       }
     }
   }

@@ -267,6 +267,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     n_blk = in_grp / gm;
   };
   auto k_blocks_of = [&](int tile) { return g.p[tile >= g.n_tiles0 ? 1 : 0].K / 256; };
+  // Tiles go to the pairs in rounds, odd rounds in reverse pair order (a snake): the pairs that got the extra tiles
+  // of one round get none in the next, and neighbouring rounds of a pair touch neighbouring operand blocks.
+  auto next_tile = [&](int rnd) { return rnd * n_pairs + ((rnd & 1) ? n_pairs - 1 - pair_id : pair_id); };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -300,7 +303,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = pair_id; tile < n_tiles && ok; tile += n_pairs) {
+      for (int rnd = 0, tile = pair_id; tile < n_tiles && ok; tile = next_tile(++rnd)) {
         int prob, m_blk, n_blk;
         tile_coords(tile, prob, m_blk, n_blk);
         const Problem& pr = g.p[prob];
@@ -345,7 +348,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     int stage = 0;
     uint32_t phase = 0;
     const uint32_t sff_leader = map_to_cta(sff_bar(0), 0);
-    for (int tile = pair_id; tile < n_tiles; tile += n_pairs) {
+    for (int rnd = 0, tile = pair_id; tile < n_tiles; tile = next_tile(++rnd)) {
       bool ok = true;
       const int k_blocks = k_blocks_of(tile);
       for (int kb = 0; kb < k_blocks; ++kb) {
@@ -400,7 +403,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       constexpr uint32_t idesc_mx[2] = {instr_desc_mxf4(256, 256, 0), instr_desc_mxf4(256, 256, 2)};
       const uint32_t a_lo0 = ((base >> 4) & 0x3fffu) | (1u << 16);
       const uint32_t b_lo0 = (((base + kABytes) >> 4) & 0x3fffu) | (1u << 16);
-      for (int tile = pair_id; tile < n_tiles && ok; tile += n_pairs) {
+      for (int rnd = 0, tile = pair_id; tile < n_tiles && ok; tile = next_tile(++rnd)) {
         if (!(ok = mbar_wait_cluster(acce_bar, acc_phase ^ 1u, abort_flag, 0x300u))) break;
         tc_fence_after();
         const int k_blocks = k_blocks_of(tile);
@@ -447,7 +450,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + half * 128;
     const uint32_t stage_buf = staging + half * 16384;
     int buf = 0;
-    for (int tile = pair_id; tile < n_tiles; tile += n_pairs) {
+    for (int rnd = 0, tile = pair_id; tile < n_tiles; tile = next_tile(++rnd)) {
       int prob, m_blk, n_blk;
       tile_coords(tile, prob, m_blk, n_blk);
       const CUtensorMap* map_d = prob ? &map_d1 : &map_d0;

@@ -145,6 +145,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
     n0 = n_idx < n_wide ? n_idx * 384 : n_wide * 384 + (n_idx - n_wide) * 256;
   };
   auto k_blocks_of = [&](int tile) { return g.p[tile >= g.n_tiles0 ? 1 : 0].K / 256; };
+  // Tiles go to the pairs in rounds, odd rounds in reverse pair order (a snake): the pairs that got the larger or
+  // the extra tiles of one round get the smaller ones, or none, in the next.
+  auto next_tile = [&](int rnd) { return rnd * n_pairs + ((rnd & 1) ? n_pairs - 1 - pair_id : pair_id); };
   constexpr int kAtomsKb = MX ? 2 : 4;  // scale atoms per 256-deep k-block and 128-row group
 
   if (threadIdx.x == 0) {
@@ -179,7 +182,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = pair_id; tile < n_tiles && ok; tile += n_pairs) {
+      for (int rnd = 0, tile = pair_id; tile < n_tiles && ok; tile = next_tile(++rnd)) {
         int prob, m_blk, n0, width;
         tile_coords(tile, prob, m_blk, n0, width);
         const WProblem& pr = g.p[prob];
@@ -229,7 +232,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
     uint32_t r[64];  // the slot's 64 columns; entries of a narrow tile's third group keep stale (unused) values
 #pragma unroll
     for (int i = 0; i < 64; ++i) r[i] = 0u;
-    for (int tile = pair_id; tile < n_tiles; tile += n_pairs) {
+    for (int rnd = 0, tile = pair_id; tile < n_tiles; tile = next_tile(++rnd)) {
       bool ok = true;
       int prob, m_blk, n0, width;
       tile_coords(tile, prob, m_blk, n0, width);
@@ -285,7 +288,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
       constexpr uint32_t id128_mx[2] = {instr_desc_mxf4(256, 128, 0), instr_desc_mxf4(256, 128, 2)};
       const uint32_t a_lo0 = ((base >> 4) & 0x3fffu) | (1u << 16);
       const uint32_t b_lo0 = (((base + kWABytes) >> 4) & 0x3fffu) | (1u << 16);
-      for (int tile = pair_id; tile < n_tiles && ok; tile += n_pairs) {
+      for (int rnd = 0, tile = pair_id; tile < n_tiles && ok; tile = next_tile(++rnd)) {
         int prob, m_blk, n0, width;
         tile_coords(tile, prob, m_blk, n0, width);
         const bool is_wide = width == 384;
@@ -342,7 +345,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
     const uint32_t acce_leader = map_to_cta(acce_bar, 0);
     const int row_in_tile = quad * 32 + lane;
     const uint32_t stage_buf = staging + half * 16384;
-    for (int tile = pair_id; tile < n_tiles; tile += n_pairs) {
+    for (int rnd = 0, tile = pair_id; tile < n_tiles; tile = next_tile(++rnd)) {
       int prob, m_blk, n0, width;
       tile_coords(tile, prob, m_blk, n0, width);
       const CUtensorMap* map_d = prob ? &map_d1 : &map_d0;
