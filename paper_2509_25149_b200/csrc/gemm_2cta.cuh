@@ -267,8 +267,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     n_blk = in_grp / gm;
   };
   auto k_blocks_of = [&](int tile) { return g.p[tile >= g.n_tiles0 ? 1 : 0].K / 256; };
-  // Tiles go to the pairs in rounds, odd rounds in reverse pair order (a snake): the pairs that got the extra tiles
-  // of one round get none in the next, and neighbouring rounds of a pair touch neighbouring operand blocks.
+  // Tiles go to the pairs in rounds, odd rounds in reverse pair order (a snake): with two problems of different
+  // depth in one launch, the pairs that drew the deeper or the extra tiles of one round draw the shallower ones, or
+  // none, in the next.  A balance measure only: on one problem it times the same as the plain round-robin.
   auto next_tile = [&](int rnd) { return rnd * n_pairs + ((rnd & 1) ? n_pairs - 1 - pair_id : pair_id); };
 
   if (threadIdx.x == 0) {

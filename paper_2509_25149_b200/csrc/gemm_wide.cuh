@@ -146,7 +146,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
   };
   auto k_blocks_of = [&](int tile) { return g.p[tile >= g.n_tiles0 ? 1 : 0].K / 256; };
   // Tiles go to the pairs in rounds, odd rounds in reverse pair order (a snake): the pairs that got the larger or
-  // the extra tiles of one round get the smaller ones, or none, in the next.
+  // the extra tiles of one round get the smaller ones, or none, in the next.  A balance measure only: with equal
+  // tiles it times the same as the plain round-robin.
   auto next_tile = [&](int rnd) { return rnd * n_pairs + ((rnd & 1) ? n_pairs - 1 - pair_id : pair_id); };
   constexpr int kAtomsKb = MX ? 2 : 4;  // scale atoms per 256-deep k-block and 128-row group
 
