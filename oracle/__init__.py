@@ -69,6 +69,10 @@ def lib():
                 "orc_quantize_f32": (c.c_int, [f32p, c.c_int64, c.c_int64, c.c_int64, c.c_int, c.c_int,
                                                c.c_int, c.c_uint16, c.c_int, c.c_uint64, c.c_uint64,
                                                c.c_float, c.c_int64, c.c_int64, c.c_int64, u8p, u8p, f32p, f32p]),
+                "orc_rht_d": (c.c_int, [f32p, c.c_int, u32p, f32p]),
+                "orc_quantize_rht": (c.c_int, [u16p, c.c_int64, c.c_int64, c.c_int64, c.c_int, c.c_int, u32p,
+                                               c.c_int, c.c_uint64, c.c_uint64, c.c_float, c.c_int64, c.c_int64,
+                                               c.c_int64, u8p, u8p, f32p, f32p]),
                 "orc_dequantize": (None, [u8p, u8p, f32p, c.c_int64, c.c_int64, f64p]),
                 "orc_dequantize_local": (None, [u8p, u8p, c.c_int64, c.c_int64, f64p]),
                 "orc_gemm_tn": (None, [f64p, f64p, c.c_int64, c.c_int64, c.c_int64, f64p, f64p]),
@@ -144,6 +148,21 @@ def rht16(x, sign_mask: int):
     return y
 
 
+def _sign_words(sign_mask: int):
+    return np.array([(sign_mask >> (32 * i)) & 0xFFFFFFFF for i in range(4)], dtype=np.uint32)
+
+
+def rht_d(x, d: int, sign_mask: int):
+    """Transform of size d (a power of two up to 128) of one chunk; bit j of sign_mask negates input j."""
+    xin = np.ascontiguousarray(x, dtype=np.float32)
+    assert xin.shape == (d,)
+    y = np.zeros(d, dtype=np.float32)
+    w = _sign_words(sign_mask)
+    if lib().orc_rht_d(_p(xin, ctypes.c_float), d, _p(w, ctypes.c_uint32), _p(y, ctypes.c_float)) != 0:
+        raise ValueError("transform size must be a power of two in [2, 128]")
+    return y
+
+
 def global_scale(amax: float):
     e, d = ctypes.c_float(), ctypes.c_float()
     lib().orc_global_scale(np.float32(amax), ctypes.byref(e), ctypes.byref(d))
@@ -201,12 +220,15 @@ class Quantized:
 
 
 def quantize(x_bf16_bits, *, colwise=False, block_rows=1, rht=False, sign_mask=0, rounding=RNE,
-             seed=0, sr_offset=0, amax_override=None, return_y=False, sr_row0=0, sr_cols=0, sr_col0=0) -> Quantized:
+             seed=0, sr_offset=0, amax_override=None, return_y=False, sr_row0=0, sr_cols=0, sr_col0=0,
+             rht_dim=16) -> Quantized:
     """Quantize one copy of a bf16 tensor given as a 2-D uint16 array of bit patterns (or of a binary32 tensor given
     as a float32 array).
 
     sr_row0 / sr_col0 / sr_cols: the array is the block starting at (sr_row0, sr_col0) of a larger source with
-    sr_cols columns (only the index of the stochastic-rounding draws depends on it)."""
+    sr_cols columns (only the index of the stochastic-rounding draws depends on it).
+    rht_dim: size of the transform when rht is set (16 = the recipe; 2, 4, 8, 128 = the sizes of Appendix E.4.2,
+    bf16 sources with 1x16 blocks only); sign_mask then carries rht_dim bits."""
     x = np.asarray(x_bf16_bits)
     f32 = x.dtype == np.float32  # a binary32 source instead of bf16 bit patterns
     assert (x.dtype == np.uint16 or f32) and x.ndim == 2
@@ -219,11 +241,20 @@ def quantize(x_bf16_bits, *, colwise=False, block_rows=1, rht=False, sign_mask=0
     scales = np.zeros((R, C // 16), dtype=np.uint8)
     glob = np.zeros(2, dtype=np.float32)
     y = np.zeros((R, C), dtype=np.float32) if return_y else None
-    fn, src = (lib().orc_quantize_f32, _p(x, ctypes.c_float)) if f32 else (lib().orc_quantize, _p(x, ctypes.c_uint16))
-    rc = fn(src, sr, sc, ld, int(colwise), block_rows, int(rht), sign_mask, rounding, seed, sr_offset,
-            np.float32(-1.0 if amax_override is None else amax_override), sr_row0, sr_cols, sr_col0,
-            _p(codes, ctypes.c_uint8), _p(scales, ctypes.c_uint8), _p(glob, ctypes.c_float),
+    amax_arg = np.float32(-1.0 if amax_override is None else amax_override)
+    outs = (_p(codes, ctypes.c_uint8), _p(scales, ctypes.c_uint8), _p(glob, ctypes.c_float),
             _p(y, ctypes.c_float) if return_y else None)
+    if rht and rht_dim != 16:
+        if f32 or block_rows != 1:
+            raise ValueError("other transform sizes: bf16 source and 1x16 blocks only")
+        w = _sign_words(sign_mask)
+        rc = lib().orc_quantize_rht(_p(x, ctypes.c_uint16), sr, sc, ld, int(colwise), rht_dim, _p(w, ctypes.c_uint32),
+                                    rounding, seed, sr_offset, amax_arg, sr_row0, sr_cols, sr_col0, *outs)
+    else:
+        fn, src = ((lib().orc_quantize_f32, _p(x, ctypes.c_float)) if f32
+                   else (lib().orc_quantize, _p(x, ctypes.c_uint16)))
+        rc = fn(src, sr, sc, ld, int(colwise), block_rows, int(rht), sign_mask & 0xFFFF, rounding, seed, sr_offset,
+                amax_arg, sr_row0, sr_cols, sr_col0, *outs)
     if rc != 0:
         raise ValueError(f"orc_quantize rejected the shape (rc={rc})")
     return Quantized(codes, scales, glob, R, C, y)
@@ -268,6 +299,35 @@ def gemm_blockscaled(a: Quantized, b: Quantized):
                                _p(bc, ctypes.c_uint8), _p(bsf, ctypes.c_uint8), _p(bg, ctypes.c_float),
                                a.rows, b.rows, a.cols, _p(D, ctypes.c_double))
     return D
+
+
+# ------------------------------------------- layers kept in BF16 (Section 4.1) ----
+def _bf16_bits_to_f64(bits):
+    b = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def linear_bf16_fwd(x_bits, w_bits):
+    """A linear layer left in BF16 (Section 4.1 keeps the most sensitive layers in higher precision; Appendix D
+    switches all of them late in training): Y = X W^T of the bf16 values, exact products summed in binary64.
+    Returns (Y, T) with T = |X| |W|^T, the scale of the accumulation-error tolerance."""
+    return gemm_tn(_bf16_bits_to_f64(x_bits), _bf16_bits_to_f64(w_bits))
+
+
+def linear_bf16_bwd(dy_bits, x_bits, w_bits):
+    """dX = dY W and dW = dY^T X (Section 4.1's Dgrad and Wgrad) of the bf16 values, in binary64.
+    Returns ((dX, T_dX), (dW, T_dW))."""
+    dy, x, w = _bf16_bits_to_f64(dy_bits), _bf16_bits_to_f64(x_bits), _bf16_bits_to_f64(w_bits)
+    return gemm_tn(dy, np.ascontiguousarray(w.T)), gemm_tn(np.ascontiguousarray(dy.T), np.ascontiguousarray(x.T))
+
+
+# ------------------------------- quantization-error metric (Appendix E.2) ----
+def quant_error(x, x_hat):
+    """Squared error of a decoded tensor against its source and the source's squared norm, in binary64:
+    (sum (x - x_hat)^2, sum x^2); their ratio is the relative quantization error of the tensor."""
+    x = np.asarray(x, dtype=np.float64)
+    e = x - np.asarray(x_hat, dtype=np.float64)
+    return float(np.sum(e * e)), float(np.sum(x * x))
 
 
 # ----------------------------------------------------------------- MXFP4 ----

@@ -187,6 +187,26 @@ ORC_EXPORT void orc_rht16(const float x[16], uint16_t sign_mask, float y[16]) {
   }
 }
 
+/* Other transform sizes (Appendix E.4.2 compares d = 2, 4, 16 and 128): the
+ * Sylvester matrix of order d = 2^m has the same entry rule (parity of the bits
+ * j and k share), the normalisation is 1/sqrt(d), and the sign vector has d
+ * entries: bit (j & 31) of sign_words[j >> 5].  y_k = (1/sqrt d) sum_j s_j x_j
+ * h(j,k), accumulated and normalised in binary64, rounded once to binary32.
+ * Returns -1 unless d is a power of two in [2, 128]. */
+ORC_EXPORT int orc_rht_d(const float* x, int d, const uint32_t* sign_words, float* y) {
+  if (d < 2 || d > 128 || (d & (d - 1))) return -1;
+  const double norm = sqrt((double)d);
+  for (int k = 0; k < d; ++k) {
+    double acc = 0.0;
+    for (int j = 0; j < d; ++j) {
+      double s = ((sign_words[j >> 5] >> (j & 31)) & 1u) ? -1.0 : 1.0;
+      acc += s * (double)x[j] * (double)orc_hadamard16_entry(j, k);
+    }
+    y[k] = (float)(acc / norm);
+  }
+  return 0;
+}
+
 /* ------------------------------------------------------------------------- */
 /* Two-level scaling (Appendix B.1, B.2)                                      */
 /* ------------------------------------------------------------------------- */
@@ -259,12 +279,14 @@ ORC_EXPORT int64_t orc_sf_swizzled_offset(int64_t r, int64_t kb, int64_t n_kb) {
  */
 static int quantize_source(const uint16_t* x_bf16, const float* x_f32, int64_t src_rows, int64_t src_cols,
                            int64_t ld, int colwise, int block_rows, int rht, uint16_t sign_mask,
+                           int rht_dim, const uint32_t* sign_words,
                            int rounding, uint64_t seed, uint64_t sr_offset,
                            float amax_override, int64_t sr_row0, int64_t sr_cols, int64_t sr_col0,
                            uint8_t* codes, uint8_t* scales, float* global, float* y_out) {
   const int64_t R = colwise ? src_cols : src_rows;
   const int64_t C = colwise ? src_rows : src_cols;
   if ((block_rows != 1 && block_rows != 16) || C % 16 || R % block_rows) return -1;
+  if (rht && rht_dim != 16 && (rht_dim < 2 || rht_dim > 128 || (rht_dim & (rht_dim - 1)) || C % rht_dim)) return -1;
   float* y = (float*)malloc(sizeof(float) * (size_t)(R * C));
   if (!y) return -2;
 
@@ -277,13 +299,21 @@ static int quantize_source(const uint16_t* x_bf16, const float* x_f32, int64_t s
     }
 
   /* Appendix C: rotate every aligned chunk of 16 along the contraction dim */
-  if (rht) {
+  if (rht && rht_dim == 16) {
 #pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < R; ++r)
       for (int64_t c0 = 0; c0 < C; c0 += 16) {
         float t[16];
         orc_rht16(&y[r * C + c0], sign_mask, t);
         memcpy(&y[r * C + c0], t, sizeof t);
+      }
+  } else if (rht) { /* Appendix E.4.2: every aligned chunk of rht_dim elements instead */
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < R; ++r)
+      for (int64_t c0 = 0; c0 < C; c0 += rht_dim) {
+        float t[128];
+        orc_rht_d(&y[r * C + c0], rht_dim, sign_words, t);
+        memcpy(&y[r * C + c0], t, sizeof(float) * (size_t)rht_dim);
       }
   }
 
@@ -346,8 +376,21 @@ ORC_EXPORT int orc_quantize(const uint16_t* x_bf16, int64_t src_rows, int64_t sr
                             int rounding, uint64_t seed, uint64_t sr_offset,
                             float amax_override, int64_t sr_row0, int64_t sr_cols, int64_t sr_col0,
                             uint8_t* codes, uint8_t* scales, float* global, float* y_out) {
-  return quantize_source(x_bf16, NULL, src_rows, src_cols, ld, colwise, block_rows, rht, sign_mask, rounding, seed,
-                         sr_offset, amax_override, sr_row0, sr_cols, sr_col0, codes, scales, global, y_out);
+  return quantize_source(x_bf16, NULL, src_rows, src_cols, ld, colwise, block_rows, rht, sign_mask, 16, NULL,
+                         rounding, seed, sr_offset, amax_override, sr_row0, sr_cols, sr_col0, codes, scales, global, y_out);
+}
+
+/* The same procedure with a transform of another size (Appendix E.4.2): every aligned chunk of rht_dim elements
+ * along the contraction dimension is rotated (several per 16-block for rht_dim < 16, one per eight blocks for 128);
+ * blocks, scales and rounding are unchanged.  sign_words: rht_dim sign bits. */
+ORC_EXPORT int orc_quantize_rht(const uint16_t* x_bf16, int64_t src_rows, int64_t src_cols, int64_t ld,
+                                int colwise, int rht_dim, const uint32_t* sign_words,
+                                int rounding, uint64_t seed, uint64_t sr_offset,
+                                float amax_override, int64_t sr_row0, int64_t sr_cols, int64_t sr_col0,
+                                uint8_t* codes, uint8_t* scales, float* global, float* y_out) {
+  return quantize_source(x_bf16, NULL, src_rows, src_cols, ld, colwise, 1, 1, (uint16_t)sign_words[0], rht_dim,
+                         sign_words, rounding, seed, sr_offset, amax_override, sr_row0, sr_cols, sr_col0, codes,
+                         scales, global, y_out);
 }
 
 /* The same procedure from a binary32 source (Appendix B: "from higher precision (FP32 or BF16)"): only step one,
@@ -357,8 +400,8 @@ ORC_EXPORT int orc_quantize_f32(const float* x_f32, int64_t src_rows, int64_t sr
                                 int rounding, uint64_t seed, uint64_t sr_offset,
                                 float amax_override, int64_t sr_row0, int64_t sr_cols, int64_t sr_col0,
                                 uint8_t* codes, uint8_t* scales, float* global, float* y_out) {
-  return quantize_source(NULL, x_f32, src_rows, src_cols, ld, colwise, block_rows, rht, sign_mask, rounding, seed,
-                         sr_offset, amax_override, sr_row0, sr_cols, sr_col0, codes, scales, global, y_out);
+  return quantize_source(NULL, x_f32, src_rows, src_cols, ld, colwise, block_rows, rht, sign_mask, 16, NULL,
+                         rounding, seed, sr_offset, amax_override, sr_row0, sr_cols, sr_col0, codes, scales, global, y_out);
 }
 
 /* Decode: x^ = (+-magnitude) * fp32(block scale) * s_dec, in binary64 (exact:
