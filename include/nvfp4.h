@@ -150,6 +150,35 @@ NVFP4_API nvfp4_status nvfp4_gemm(const nvfp4_tensor* A, const nvfp4_tensor* B, 
                                   void* cuda_stream);
 
 /*
+ * nvfp4_gemm_bf16 -- the GEMM of a linear layer that is kept in BF16 (Section 4.1: a small share of the layers,
+ * the last ones above all, stay in higher precision; Appendix D: all of them late in training).
+ *   D[M x N] = op(A) op(B)^T, products of bf16 values accumulated in FP32 by the tensor cores.
+ *   A: device bf16.  a_layout NVFP4_K_MAJOR : stored [M][K], leading dimension lda >= K (contraction contiguous);
+ *                    a_layout NVFP4_MN_MAJOR: stored [K][M], lda >= M (the operand is read transposed).
+ *   B: device bf16.  b_layout NVFP4_K_MAJOR : stored [N][K], ldb >= K;  NVFP4_MN_MAJOR: stored [K][N], ldb >= N.
+ *   D: device, row-major [M x N], ldd >= N, bf16 (round-to-nearest-even) or fp32 (d_is_fp32 != 0);
+ *      accumulate != 0 adds into an fp32 D.
+ *   M, N multiples of 256, K of 64; pointers 16-byte aligned, lda, ldb multiples of 8, ldd * elemsize of 16.
+ *   Nothing is enqueued on error.
+ */
+enum { NVFP4_K_MAJOR = 0, NVFP4_MN_MAJOR = 1 };
+NVFP4_API nvfp4_status nvfp4_gemm_bf16(const void* A, int32_t a_layout, int64_t lda, const void* B, int32_t b_layout,
+                                       int64_t ldb, int64_t M, int64_t N, int64_t K, void* D, int32_t d_is_fp32,
+                                       int64_t ldd, int32_t accumulate, void* cuda_stream);
+
+/*
+ * The same layer as nvfp4_linear_fwd / _bwd without quantization (Section 4.1, Appendix D), on the same row-major
+ * operands X [M x K], W [N x K], dY [M x N], all contiguous bf16; no transposed copies are made:
+ *   fwd: Y  = X W^T (bf16);   bwd: dX = dY W (bf16), dW = dY^T X (fp32, accumulate_dw != 0 adds into it);
+ *   dX or dW may be NULL to skip that GEMM.  M, N, K multiples of 256.
+ */
+NVFP4_API nvfp4_status nvfp4_linear_bf16_fwd(const void* X, const void* W, int64_t M, int64_t N, int64_t K,
+                                             void* Y_bf16, void* cuda_stream);
+NVFP4_API nvfp4_status nvfp4_linear_bf16_bwd(const void* dY, const void* X, const void* W, int64_t M, int64_t N,
+                                             int64_t K, void* dX_bf16, float* dW_fp32, int32_t accumulate_dw,
+                                             void* cuda_stream);
+
+/*
  * Linear layer, Section 4.1 (three GEMMs, each quantizing its inputs):
  *   X [M x K] bf16 (tokens x in-features), W [N x K] bf16, dY [M x N] bf16, all contiguous.
  *   M, N, K multiples of 256.

@@ -71,6 +71,11 @@ def lib() -> ctypes.CDLL:
         L.nvfp4_linear_fwd_noalloc_max_bytes.restype, L.nvfp4_linear_fwd_noalloc_max_bytes.argtypes = c.c_size_t, []
         L.nvfp4_linear_bwd.restype = i32
         L.nvfp4_linear_bwd.argtypes = [vp, TP, TP, i64, i64, i64, OP, vp, vp, i32, vp, c.c_size_t, vp]
+        L.nvfp4_gemm_bf16.restype = i32
+        L.nvfp4_gemm_bf16.argtypes = [vp, i32, i64, vp, i32, i64, i64, i64, i64, vp, i32, i64, i32, vp]
+        L.nvfp4_linear_bf16_fwd.restype, L.nvfp4_linear_bf16_fwd.argtypes = i32, [vp, vp, i64, i64, i64, vp, vp]
+        L.nvfp4_linear_bf16_bwd.restype = i32
+        L.nvfp4_linear_bf16_bwd.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, i32, vp]
         L.nvfp4_dequantize.restype, L.nvfp4_dequantize.argtypes = i32, [TP, vp, vp]
         L.nvfp4_rht16.restype, L.nvfp4_rht16.argtypes = i32, [vp, i64, i64, i64, i32, u32, vp, vp]
         L.nvfp4_device_status.restype, L.nvfp4_device_status.argtypes = i32, [vp, c.POINTER(u32)]
@@ -199,6 +204,48 @@ def nvfp4_linear_bwd(dY: torch.Tensor, X_col_saved: Optional[NVFP4Tensor], W_col
                                   dW.data_ptr() if dW is not None else None, int(accumulate_dw),
                                   workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
            "nvfp4_linear_bwd")
+
+
+K_MAJOR, MN_MAJOR = 0, 1
+
+
+def nvfp4_gemm_bf16(A: torch.Tensor, B: torch.Tensor, D: torch.Tensor, a_layout: int = K_MAJOR,
+                    b_layout: int = K_MAJOR, accumulate: bool = False) -> None:
+    """D[M x N] = op(A) op(B)^T in BF16.  K_MAJOR: the operand is [M or N][K]; MN_MAJOR: it is [K][M or N]."""
+    for t in (A, B):
+        assert t.is_cuda and t.dim() == 2 and t.stride(1) == 1 and t.dtype == torch.bfloat16
+    assert D.is_cuda and D.dim() == 2 and D.stride(1) == 1 and D.dtype in (torch.bfloat16, torch.float32)
+    M, N = D.shape
+    K = A.shape[0] if a_layout == MN_MAJOR else A.shape[1]
+    assert tuple(A.shape) == ((K, M) if a_layout == MN_MAJOR else (M, K))
+    assert tuple(B.shape) == ((K, N) if b_layout == MN_MAJOR else (N, K))
+    _check(lib().nvfp4_gemm_bf16(A.data_ptr(), a_layout, A.stride(0), B.data_ptr(), b_layout, B.stride(0), M, N, K,
+                                 D.data_ptr(), int(D.dtype == torch.float32), D.stride(0), int(accumulate), _stream()),
+           "nvfp4_gemm_bf16")
+
+
+def nvfp4_linear_bf16_fwd(X: torch.Tensor, W: torch.Tensor, Y: torch.Tensor) -> None:
+    M, K = X.shape
+    N = W.shape[0]
+    assert X.is_contiguous() and W.is_contiguous() and Y.is_contiguous() and tuple(W.shape) == (N, K)
+    assert X.dtype == W.dtype == Y.dtype == torch.bfloat16 and tuple(Y.shape) == (M, N)
+    _check(lib().nvfp4_linear_bf16_fwd(X.data_ptr(), W.data_ptr(), M, N, K, Y.data_ptr(), _stream()),
+           "nvfp4_linear_bf16_fwd")
+
+
+def nvfp4_linear_bf16_bwd(dY: torch.Tensor, X: Optional[torch.Tensor], W: Optional[torch.Tensor], K: int,
+                          dX: Optional[torch.Tensor], dW: Optional[torch.Tensor], accumulate_dw: bool = False) -> None:
+    M, N = dY.shape
+    assert dY.is_contiguous() and dY.dtype == torch.bfloat16
+    assert dX is None or (W is not None and W.is_contiguous() and tuple(W.shape) == (N, K) and dX.is_contiguous()
+                          and dX.dtype == torch.bfloat16 and tuple(dX.shape) == (M, K))
+    assert dW is None or (X is not None and X.is_contiguous() and tuple(X.shape) == (M, K) and dW.is_contiguous()
+                          and dW.dtype == torch.float32 and tuple(dW.shape) == (N, K))
+    _check(lib().nvfp4_linear_bf16_bwd(dY.data_ptr(), X.data_ptr() if X is not None else None,
+                                       W.data_ptr() if W is not None else None, M, N, K,
+                                       dX.data_ptr() if dX is not None else None,
+                                       dW.data_ptr() if dW is not None else None, int(accumulate_dw), _stream()),
+           "nvfp4_linear_bf16_bwd")
 
 
 def nvfp4_dequantize(t: NVFP4Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:

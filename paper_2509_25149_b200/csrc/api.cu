@@ -302,6 +302,50 @@ nvfp4_status nvfp4_linear_fwd_noalloc(const void* X, const void* W, int64_t M, i
                           scratch_of_device[dev], NVFP4_NOALLOC_SCRATCH_BYTES, cuda_stream);
 }
 
+nvfp4_status nvfp4_gemm_bf16(const void* A, int32_t a_layout, int64_t lda, const void* B, int32_t b_layout, int64_t ldb,
+                             int64_t M, int64_t N, int64_t K, void* D, int32_t d_is_fp32, int64_t ldd,
+                             int32_t accumulate, void* cuda_stream) {
+  if (!A || !B || !D) return NVFP4_ERR_NULL;
+  if ((a_layout != NVFP4_K_MAJOR && a_layout != NVFP4_MN_MAJOR) || (b_layout != NVFP4_K_MAJOR && b_layout != NVFP4_MN_MAJOR))
+    return NVFP4_ERR_ARG;
+  if (M <= 0 || N <= 0 || K <= 0 || M % 256 != 0 || N % 256 != 0 || K % 64 != 0) return NVFP4_ERR_SHAPE;
+  if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff || (M / 256) * (N / 256) > 0x7fffffff) return NVFP4_ERR_SHAPE;
+  if (lda < (a_layout == NVFP4_MN_MAJOR ? M : K) || ldb < (b_layout == NVFP4_MN_MAJOR ? N : K) || ldd < N)
+    return NVFP4_ERR_SHAPE;
+  if (accumulate && !d_is_fp32) return NVFP4_ERR_ARG;
+  const int64_t esz = d_is_fp32 ? 4 : 2;
+  if (lda % 8 != 0 || ldb % 8 != 0 || (ldd * esz) % 16 != 0 || !aligned(A, 16) || !aligned(B, 16) || !aligned(D, 16))
+    return NVFP4_ERR_ALIGN;
+  DenseGemmArgs g{};
+  g.a = A; g.b = B; g.d = D;
+  g.lda = lda; g.ldb = ldb; g.ldd = ldd;
+  g.M = (int)M; g.N = (int)N; g.K = (int)K;
+  g.a_mn = a_layout == NVFP4_MN_MAJOR; g.b_mn = b_layout == NVFP4_MN_MAJOR;
+  g.d_is_fp32 = d_is_fp32 != 0; g.accumulate = accumulate != 0;
+  return launch_gemm_bf16(g, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_linear_bf16_fwd(const void* X, const void* W, int64_t M, int64_t N, int64_t K, void* Y_bf16,
+                                   void* cuda_stream) {
+  return nvfp4_gemm_bf16(X, NVFP4_K_MAJOR, K, W, NVFP4_K_MAJOR, K, M, N, K, Y_bf16, 0, N, 0, cuda_stream);
+}
+
+nvfp4_status nvfp4_linear_bf16_bwd(const void* dY, const void* X, const void* W, int64_t M, int64_t N, int64_t K,
+                                   void* dX_bf16, float* dW_fp32, int32_t accumulate_dw, void* cuda_stream) {
+  if (!dY) return NVFP4_ERR_NULL;
+  if (!dX_bf16 && !dW_fp32) return NVFP4_ERR_NULL;
+  nvfp4_status st;
+  // Dgrad: dX[M x K] = dY[M x N] W[N x K]; the contraction runs over W's rows
+  if (dX_bf16 && (st = nvfp4_gemm_bf16(dY, NVFP4_K_MAJOR, N, W, NVFP4_MN_MAJOR, K, M, K, N, dX_bf16, 0, K, 0,
+                                       cuda_stream)) != NVFP4_OK)
+    return st;
+  // Wgrad: dW[N x K] = dY^T X; the contraction runs over the tokens, the rows of both operands
+  if (dW_fp32 && (st = nvfp4_gemm_bf16(dY, NVFP4_MN_MAJOR, N, X, NVFP4_MN_MAJOR, K, N, K, M, dW_fp32, 1, K,
+                                       accumulate_dw, cuda_stream)) != NVFP4_OK)
+    return st;
+  return NVFP4_OK;
+}
+
 nvfp4_status nvfp4_dequantize(const nvfp4_tensor* t, float* out, void* cuda_stream) {
   if (!t || !out || !t->codes || !t->scales || !t->global) return NVFP4_ERR_NULL;
   nvfp4_status st = check_copy(t, t->rows, t->cols);

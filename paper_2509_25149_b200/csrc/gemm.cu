@@ -26,6 +26,7 @@
 #include "tc_ptx.cuh"
 #include "gemm_2cta.cuh"
 #include "gemm_wide.cuh"
+#include "gemm_bf16.cuh"
 
 namespace nvfp4 {
 
@@ -566,6 +567,38 @@ bool prefer_wide_tiles(const GemmArgs& g0, const GemmArgs* g1) {
     seen.push_back(e);
   }
   return wide;
+}
+
+cudaError_t launch_gemm_bf16(const DenseGemmArgs& g, cudaStream_t s) {
+  int num_sms = 0;
+  cudaError_t e = sm_count(&num_sms);
+  if (e != cudaSuccess) return e;
+  CUtensorMap map_a, map_b, map_d;
+  const CUtensorMapDataType bf = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  bool ok = g.a_mn ? make_map_2d(&map_a, bf, 2, g.a, (uint64_t)g.M, (uint64_t)g.K, (uint64_t)g.lda * 2, 64, 64, true)
+                   : make_map_2d(&map_a, bf, 2, g.a, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.lda * 2, 64, 128, true);
+  ok = ok && (g.b_mn ? make_map_2d(&map_b, bf, 2, g.b, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.ldb * 2, 64, 64, true)
+                     : make_map_2d(&map_b, bf, 2, g.b, (uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.ldb * 2, 64, 128, true));
+  if (g.d_is_fp32)
+    ok = ok && make_map_2d(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g.d, (uint64_t)g.N, (uint64_t)g.M,
+                           (uint64_t)g.ldd * 4, 32, 128, true);
+  else
+    ok = ok && make_map_2d(&map_d, bf, 2, g.d, (uint64_t)g.N, (uint64_t)g.M, (uint64_t)g.ldd * 2, 64, 128, true);
+  if (!ok) return cudaErrorInvalidValue;
+  static std::atomic<uint64_t> configured{0};  // per device
+  int dev;
+  if (device_needs_config(configured, &dev)) {
+    e = cudaFuncSetAttribute(dense::gemm_bf16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             dense::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    device_configured(configured, dev);
+  }
+  dense::Args a{g.M, g.N, g.K, g.a_mn, g.b_mn, g.d_is_fp32, g.accumulate};
+  const int n_tiles = (g.M / 256) * (g.N / 256), max_pairs = num_sms / 2;
+  const int pairs = n_tiles < max_pairs ? n_tiles : max_pairs;
+  dense::gemm_bf16_pair_kernel<<<2 * pairs, dense::kThreads, dense::kSmemBytes, s>>>(map_a, map_b, map_d, a);
+  count_launch();
+  return cudaGetLastError();
 }
 
 cudaError_t read_device_status(cudaStream_t s, uint32_t* code) {

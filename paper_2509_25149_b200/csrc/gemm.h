@@ -29,4 +29,18 @@ cudaError_t launch_gemm_two(const GemmArgs& g0, const void* a0, const void* b0, 
 bool prefer_wide_tiles(const GemmArgs& g0, const GemmArgs* g1);
 cudaError_t read_device_status(cudaStream_t s, uint32_t* code);
 
+// BF16 GEMM D[M x N] = A B^T on CTA pairs (gemm_bf16.cuh) for layers kept in higher precision.
+// a_mn / b_mn = 0: the operand is stored [M or N][K] (contraction contiguous); 1: stored [K][M or N].
+// M, N multiples of 256, K of 64; leading dimensions in elements.
+struct DenseGemmArgs {
+  const void* a;
+  const void* b;
+  void* d;
+  int64_t lda, ldb, ldd;
+  int M, N, K;
+  int a_mn, b_mn;
+  int d_is_fp32, accumulate;
+};
+cudaError_t launch_gemm_bf16(const DenseGemmArgs& g, cudaStream_t s);
+
 }  // namespace nvfp4
