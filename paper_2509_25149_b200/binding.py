@@ -25,6 +25,7 @@ EXPORTED = (
     "nvfp4_linear_fwd", "nvfp4_linear_bwd", "nvfp4_dequantize", "nvfp4_rht16", "nvfp4_device_status",
     "nvfp4_set_gemm_tile_n", "nvfp4_status_string", "nvfp4_launch_count",
     "nvfp4_linear_fwd_noalloc", "nvfp4_linear_fwd_noalloc_max_bytes",
+    "nvfp4_gemm_bf16", "nvfp4_linear_bf16_fwd", "nvfp4_linear_bf16_bwd",
 )
 
 
