@@ -179,6 +179,26 @@ NVFP4_API nvfp4_status nvfp4_linear_bf16_bwd(const void* dY, const void* X, cons
                                              void* cuda_stream);
 
 /*
+ * Quantization-error metrics (Appendix E.2: the layers whose FP4 weight gradients carry the largest quantization
+ * error are the ones worth keeping in higher precision; such a metric can drive that choice).
+ *
+ * nvfp4_quant_error: out2 = { sum (x - x^)^2, sum x^2 } over the tensor, x^ the decoded row-wise copy q of the bf16
+ *   source x [rows x cols] (leading dimension ld; same alignment rules as nvfp4_quantize).  q is NVFP4 or MXFP4,
+ *   scales linear or swizzled, and must be a copy WITHOUT the Hadamard transform (a transformed copy lives in the
+ *   rotated space).  The ratio of the two sums is the relative squared quantization error.
+ * nvfp4_sq_error: out2 = { sum (ref - test)^2, sum ref^2 } of two dense row-major [rows x cols] tensors, each bf16 or
+ *   fp32 (e.g. dW from nvfp4_linear_bwd against dW from nvfp4_linear_bf16_bwd).  cols % 8 == 0, leading dimensions
+ *   multiples of 8, pointers 16-byte (bf16) / 32-byte (fp32) aligned.
+ * out2: DEVICE double[2], written in stream order (zeroed, then accumulated in FP64; the order of the additions, and
+ *   with it the last bits, vary from run to run).
+ */
+NVFP4_API nvfp4_status nvfp4_quant_error(const void* x_bf16, int64_t rows, int64_t cols, int64_t ld,
+                                         const nvfp4_tensor* q, double* out2, void* cuda_stream);
+NVFP4_API nvfp4_status nvfp4_sq_error(const void* ref, int32_t ref_is_fp32, int64_t ld_ref, const void* test,
+                                      int32_t test_is_fp32, int64_t ld_test, int64_t rows, int64_t cols,
+                                      double* out2, void* cuda_stream);
+
+/*
  * Linear layer, Section 4.1 (three GEMMs, each quantizing its inputs):
  *   X [M x K] bf16 (tokens x in-features), W [N x K] bf16, dY [M x N] bf16, all contiguous.
  *   M, N, K multiples of 256.

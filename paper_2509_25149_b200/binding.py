@@ -25,7 +25,7 @@ EXPORTED = (
     "nvfp4_linear_fwd", "nvfp4_linear_bwd", "nvfp4_dequantize", "nvfp4_rht16", "nvfp4_device_status",
     "nvfp4_set_gemm_tile_n", "nvfp4_status_string", "nvfp4_launch_count",
     "nvfp4_linear_fwd_noalloc", "nvfp4_linear_fwd_noalloc_max_bytes",
-    "nvfp4_gemm_bf16", "nvfp4_linear_bf16_fwd", "nvfp4_linear_bf16_bwd",
+    "nvfp4_gemm_bf16", "nvfp4_linear_bf16_fwd", "nvfp4_linear_bf16_bwd", "nvfp4_quant_error", "nvfp4_sq_error",
 )
 
 
@@ -77,6 +77,9 @@ def lib() -> ctypes.CDLL:
         L.nvfp4_linear_bf16_fwd.restype, L.nvfp4_linear_bf16_fwd.argtypes = i32, [vp, vp, i64, i64, i64, vp, vp]
         L.nvfp4_linear_bf16_bwd.restype = i32
         L.nvfp4_linear_bf16_bwd.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, i32, vp]
+        L.nvfp4_quant_error.restype, L.nvfp4_quant_error.argtypes = i32, [vp, i64, i64, i64, TP, vp, vp]
+        L.nvfp4_sq_error.restype = i32
+        L.nvfp4_sq_error.argtypes = [vp, i32, i64, vp, i32, i64, i64, i64, vp, vp]
         L.nvfp4_dequantize.restype, L.nvfp4_dequantize.argtypes = i32, [TP, vp, vp]
         L.nvfp4_rht16.restype, L.nvfp4_rht16.argtypes = i32, [vp, i64, i64, i64, i32, u32, vp, vp]
         L.nvfp4_device_status.restype, L.nvfp4_device_status.argtypes = i32, [vp, c.POINTER(u32)]
@@ -247,6 +250,27 @@ def nvfp4_linear_bf16_bwd(dY: torch.Tensor, X: Optional[torch.Tensor], W: Option
                                        dX.data_ptr() if dX is not None else None,
                                        dW.data_ptr() if dW is not None else None, int(accumulate_dw), _stream()),
            "nvfp4_linear_bf16_bwd")
+
+
+def nvfp4_quant_error(x: torch.Tensor, q: NVFP4Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Device tensor {sum (x - decode(q))^2, sum x^2} (float64) for the row-wise copy q of x."""
+    assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1 and x.dtype == torch.bfloat16
+    out = torch.empty(2, dtype=torch.float64, device=x.device) if out is None else out
+    _check(lib().nvfp4_quant_error(x.data_ptr(), x.shape[0], x.shape[1], x.stride(0), _ref(q), out.data_ptr(),
+                                   _stream()), "nvfp4_quant_error")
+    return out
+
+
+def nvfp4_sq_error(ref: torch.Tensor, test: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Device tensor {sum (ref - test)^2, sum ref^2} (float64) of two 2-D tensors, each bf16 or fp32."""
+    for t in (ref, test):
+        assert t.is_cuda and t.dim() == 2 and t.stride(1) == 1 and t.dtype in (torch.bfloat16, torch.float32)
+    assert ref.shape == test.shape
+    out = torch.empty(2, dtype=torch.float64, device=ref.device) if out is None else out
+    _check(lib().nvfp4_sq_error(ref.data_ptr(), int(ref.dtype == torch.float32), ref.stride(0), test.data_ptr(),
+                                int(test.dtype == torch.float32), test.stride(0), ref.shape[0], ref.shape[1],
+                                out.data_ptr(), _stream()), "nvfp4_sq_error")
+    return out
 
 
 def nvfp4_dequantize(t: NVFP4Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:

@@ -346,6 +346,33 @@ nvfp4_status nvfp4_linear_bf16_bwd(const void* dY, const void* X, const void* W,
   return NVFP4_OK;
 }
 
+nvfp4_status nvfp4_quant_error(const void* x_bf16, int64_t rows, int64_t cols, int64_t ld, const nvfp4_tensor* q,
+                               double* out2, void* cuda_stream) {
+  if (!x_bf16 || !q || !out2) return NVFP4_ERR_NULL;
+  if (rows <= 0 || cols <= 0 || ld < cols) return NVFP4_ERR_SHAPE;
+  nvfp4_status st = check_copy(q, rows, cols);
+  if (st != NVFP4_OK) return st;
+  if (cols % (q->format == NVFP4_FORMAT_MXFP4 ? 32 : 16) != 0) return NVFP4_ERR_SHAPE;
+  if (!aligned(x_bf16, 32) || ld % 16 != 0 || !aligned(out2, 8)) return NVFP4_ERR_ALIGN;
+  return launch_quant_error(x_bf16, rows, cols, ld, *q, out2, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? NVFP4_OK
+             : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_sq_error(const void* ref, int32_t ref_is_fp32, int64_t ld_ref, const void* test,
+                            int32_t test_is_fp32, int64_t ld_test, int64_t rows, int64_t cols, double* out2,
+                            void* cuda_stream) {
+  if (!ref || !test || !out2) return NVFP4_ERR_NULL;
+  if (rows <= 0 || cols <= 0 || cols % 8 != 0 || ld_ref < cols || ld_test < cols) return NVFP4_ERR_SHAPE;
+  if (!aligned(ref, ref_is_fp32 ? 32 : 16) || !aligned(test, test_is_fp32 ? 32 : 16) || ld_ref % 8 != 0 ||
+      ld_test % 8 != 0 || !aligned(out2, 8))
+    return NVFP4_ERR_ALIGN;
+  return launch_sq_error(ref, ref_is_fp32 != 0, ld_ref, test, test_is_fp32 != 0, ld_test, rows, cols, out2,
+                         static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? NVFP4_OK
+             : NVFP4_ERR_CUDA;
+}
+
 nvfp4_status nvfp4_dequantize(const nvfp4_tensor* t, float* out, void* cuda_stream) {
   if (!t || !out || !t->codes || !t->scales || !t->global) return NVFP4_ERR_NULL;
   nvfp4_status st = check_copy(t, t->rows, t->cols);

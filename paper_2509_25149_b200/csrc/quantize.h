@@ -37,4 +37,10 @@ cudaError_t launch_dequantize(const nvfp4_tensor& t, float* out, cudaStream_t s)
 cudaError_t launch_rht16(const void* x, int64_t rows, int64_t cols, int64_t ld, int colwise, uint32_t mask,
                          float* out, cudaStream_t s);
 
+// metrics.cu: out = {sum (x - decode(q))^2, sum x^2} of a row-wise copy; {sum (ref - test)^2, sum ref^2} of two tensors
+cudaError_t launch_quant_error(const void* x, int64_t rows, int64_t cols, int64_t ld, const nvfp4_tensor& q,
+                               double* out, cudaStream_t s);
+cudaError_t launch_sq_error(const void* ref, bool ref_fp32, int64_t ld_ref, const void* test, bool test_fp32,
+                            int64_t ld_test, int64_t rows, int64_t cols, double* out, cudaStream_t s);
+
 }  // namespace nvfp4

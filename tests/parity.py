@@ -37,6 +37,13 @@ def upload(q: oracle.Quantized, device="cuda") -> B.NVFP4Tensor:
                          torch.from_numpy(np.ascontiguousarray(q.glob)).to(device), q.rows, q.cols, B.SF_SWIZZLED)
 
 
+def upload_linear(q: oracle.Quantized, device="cuda") -> B.NVFP4Tensor:
+    """Oracle copy -> device tensors with the scales in the plain [rows][blocks] layout."""
+    return B.NVFP4Tensor(torch.from_numpy(np.ascontiguousarray(q.codes)).to(device),
+                         torch.from_numpy(np.ascontiguousarray(q.scales)).to(device),
+                         torch.from_numpy(np.ascontiguousarray(q.glob)).to(device), q.rows, q.cols, B.SF_LINEAR)
+
+
 def gpu_quantize(x: torch.Tensor, *, rowwise=True, colwise=False, sf_layout=B.SF_SWIZZLED, **opt):
     """x: CPU bf16 tensor.  Returns (row copy or None, col copy or None) as device NVFP4Tensors."""
     xd = x.cuda()
