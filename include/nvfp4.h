@@ -108,6 +108,13 @@ typedef struct nvfp4_quant_opts {
   uint64_t seed;          /* Philox4x32-10 key                                                        */
   uint64_t sr_offset;     /* Philox counter words 2..3; words 0..1 = (row-major source index) >> 4,   */
                           /* and the element uses byte (index & 15) of the 16 output bytes            */
+  int32_t rht_dim;        /* size d of the transform: 0 = the format's own (16; 32 for MXFP4); 2, 4,  */
+                          /* 8 or 128 = the other sizes of Appendix E.4.2 (NVFP4 outputs, bf16 source,*/
+                          /* 1x16 blocks): every aligned d-chunk along the copy's contraction         */
+                          /* dimension is multiplied by S * H_d / sqrt(d); d = 128 needs that         */
+                          /* dimension to be a multiple of 128.  Sign bit of chunk position j is bit  */
+                          /* j of rht_sign_mask (j < 32), else bit (j & 31) of                        */
+  uint32_t rht_sign_mask_ext[3]; /* rht_sign_mask_ext[(j >> 5) - 1]                                   */
 } nvfp4_quant_opts;
 
 /*

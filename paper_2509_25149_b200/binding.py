@@ -38,7 +38,8 @@ class CTensor(ctypes.Structure):
 class CQuantOpts(ctypes.Structure):
     _fields_ = [("block_rows", ctypes.c_int32), ("rounding", ctypes.c_int32), ("rht_rowwise", ctypes.c_int32),
                 ("rht_colwise", ctypes.c_int32), ("rht_sign_mask", ctypes.c_uint32), ("flags", ctypes.c_int32),
-                ("seed", ctypes.c_uint64), ("sr_offset", ctypes.c_uint64)]
+                ("seed", ctypes.c_uint64), ("sr_offset", ctypes.c_uint64), ("rht_dim", ctypes.c_int32),
+                ("rht_sign_mask_ext", ctypes.c_uint32 * 3)]
 
 
 class NVFP4Error(RuntimeError):
@@ -131,8 +132,11 @@ def alloc_tensor(rows: int, cols: int, sf_layout: int = SF_SWIZZLED, device="cud
 
 
 def quant_opts(block_rows=1, rounding=ROUND_NEAREST_EVEN, rht_rowwise=False, rht_colwise=False, rht_sign_mask=0,
-               flags=0, seed=0, sr_offset=0) -> CQuantOpts:
-    return CQuantOpts(block_rows, rounding, int(rht_rowwise), int(rht_colwise), rht_sign_mask, flags, seed, sr_offset)
+               flags=0, seed=0, sr_offset=0, rht_dim=0) -> CQuantOpts:
+    """rht_sign_mask: up to 128 sign bits (bit j negates input j of a chunk); rht_dim: 0 = the format's own size."""
+    ext = (ctypes.c_uint32 * 3)(*[(rht_sign_mask >> (32 * i)) & 0xFFFFFFFF for i in (1, 2, 3)])
+    return CQuantOpts(block_rows, rounding, int(rht_rowwise), int(rht_colwise), rht_sign_mask & 0xFFFFFFFF, flags, seed,
+                      sr_offset, rht_dim, ext)
 
 
 def _ref(t: Optional[NVFP4Tensor]):

@@ -1,5 +1,6 @@
 // C-ABI entry points: argument validation and the stream-ordered composition of the kernels.
 #include <atomic>
+#include <cmath>
 
 #include "common.cuh"
 #include "gemm.h"
@@ -54,6 +55,14 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
   if (o->flags & ~(NVFP4_SR_INDEPENDENT_COPIES | NVFP4_AMAX_PROVIDED | NVFP4_INPUT_FP32)) return NVFP4_ERR_ARG;
   const bool f32 = (o->flags & NVFP4_INPUT_FP32) != 0;
   if (f32 && (mx || o->rht_rowwise || o->rht_colwise)) return NVFP4_ERR_UNIMPLEMENTED;
+  // transform size: 0 = the format's own (16, or 32 for MXFP4); 2, 4, 8, 128 are the sizes of Appendix E.4.2
+  const int32_t rd = o->rht_dim;
+  const bool any_rht = o->rht_rowwise || o->rht_colwise;
+  const bool other_dim = any_rht && rd != 0 && rd != (mx ? 32 : 16);
+  if (rd != 0 && rd != 2 && rd != 4 && rd != 8 && rd != 16 && rd != 32 && rd != 128) return NVFP4_ERR_ARG;
+  if (other_dim && (mx || rd == 32 || rd == 16)) return NVFP4_ERR_UNIMPLEMENTED;
+  if (other_dim && rd == 128 && ((o->rht_rowwise && rowwise && cols % 128 != 0) || (o->rht_colwise && colwise && rows % 128 != 0)))
+    return NVFP4_ERR_SHAPE;
   if (rows > (int64_t)1 << 30 || cols > (int64_t)1 << 30 || ((rows + 127) / 128) * ((cols + 127) / 128) > 0x7fffffff)
     return NVFP4_ERR_SHAPE;
   nvfp4_status st;
@@ -89,6 +98,22 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
   if (f32) {
     if (!(o->flags & NVFP4_AMAX_PROVIDED) && launch_amax_f32(a, hr, hc, s) != cudaSuccess) return NVFP4_ERR_CUDA;
     return launch_quantize_f32(a, hr, hc, b2, sr, s) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+  }
+  if (other_dim) {
+    RhtArgs ra{};
+    ra.q = a;
+    ra.d = rd;
+    ra.has_row = hr; ra.has_col = hc;
+    ra.rht_row = hr && o->rht_rowwise; ra.rht_col = hc && o->rht_colwise;
+    ra.sign_words[0] = o->rht_sign_mask;
+    for (int i = 0; i < 3; ++i) ra.sign_words[1 + i] = o->rht_sign_mask_ext[i];
+    if (rd < 16) {
+      const uint32_t low = o->rht_sign_mask & ((1u << rd) - 1u);
+      for (int p = 0; p < 16; p += rd) ra.mask16 |= low << p;
+    }
+    ra.norm = (float)(1.0 / sqrt((double)rd));
+    return launch_quantize_rht(ra, (o->flags & NVFP4_AMAX_PROVIDED) != 0, sr, s) == cudaSuccess ? NVFP4_OK
+                                                                                                  : NVFP4_ERR_CUDA;
   }
   if (!(o->flags & NVFP4_AMAX_PROVIDED)) {
     if (launch_amax(a, hr, hc, o->rht_rowwise != 0, o->rht_colwise != 0, s) != cudaSuccess) return NVFP4_ERR_CUDA;

@@ -23,6 +23,17 @@ struct QuantArgs {
   int tiles_r, tiles_c;  // 128 x 128 tiles of the source
 };
 
+// Another transform size (quantize_rht.cu): d = 2, 4, 8 or 128 on the copies flagged rht_row / rht_col
+struct RhtArgs {
+  QuantArgs q;
+  int d;
+  int has_row, has_col, rht_row, rht_col;
+  uint32_t mask16;         // d <= 16: the d sign bits repeated over sixteen positions
+  uint32_t sign_words[4];  // d = 128: sign bit of position p is bit (p & 31) of word p >> 5
+  float norm;              // fl(1 / sqrt(d))
+};
+cudaError_t launch_quantize_rht(const RhtArgs& ra, bool amax_provided, bool sr, cudaStream_t s);
+
 cudaError_t launch_amax(const QuantArgs& a, bool has_row, bool has_col, bool rht_row, bool rht_col,
                         cudaStream_t s);
 cudaError_t launch_quantize(const QuantArgs& a, bool has_row, bool has_col, bool block2d, bool rht_row,

@@ -66,25 +66,45 @@ def assert_exact(gpu: B.NVFP4Tensor, ref: oracle.Quantized, what=""):
                           f"{codes[tuple(bad[0])]:#x} vs {ref.codes[tuple(bad[0])]:#x}"
 
 
-def assert_rht_close(x_bits: np.ndarray, gpu: B.NVFP4Tensor, y_gpu: np.ndarray, *, colwise, sign_mask, rounding,
-                     seed=0, sr_offset=0, what=""):
+def canon_zero(nibbles: np.ndarray) -> np.ndarray:
+    """E2M1 has two zeros (codes 0 and 8).  Which one a transformed element gets depends on the order in which
+    signed zeros are added, which no passage fixes; they decode to the same value, so compare them as equal."""
+    out = nibbles.copy()
+    out[out == 8] = 0
+    return out
+
+
+def assert_exact_up_to_zero_sign(gpu: B.NVFP4Tensor, ref: oracle.Quantized, what=""):
+    """Bit-exact scales and tensor words; codes equal except that -0 and +0 are the same code."""
+    codes, scales, glob = download(gpu)
+    assert glob.view(np.uint32).tolist() == ref.glob.view(np.uint32).tolist(), f"{what}: global {glob} vs {ref.glob}"
+    assert np.array_equal(scales, ref.scales), f"{what}: scale bytes"
+    bad = np.argwhere(canon_zero(unpack(codes)) != canon_zero(unpack(ref.codes)))
+    assert bad.size == 0, f"{what}: {len(bad)} codes differ, first at {bad[0]}"
+
+
+def assert_rht_close(x_bits: np.ndarray, gpu: B.NVFP4Tensor, y_gpu, *, colwise, sign_mask, rounding,
+                     seed=0, sr_offset=0, what="", rht_dim=16):
     """Tolerance protocol for transformed copies (the transform is computed in a different order on the GPU):
     values within 1e-5 of the scale of their dot product; amax within 1e-5; then, with the oracle re-run on the
     GPU's amax, scale bytes equal except where the pre-rounding scale is within 1e-5 of an E4M3 midpoint, and
     codes equal except where the pre-rounding value is within 1e-5 of a rounding threshold (an excused code must
-    still be an adjacent grid point).  Excused items must stay below 1e-3 of all elements."""
+    still be an adjacent grid point).  Excused items must stay below 1e-3 of all elements.
+    y_gpu may be None (no device-side dump of the transformed values for that transform size): step (1) is skipped."""
     codes, scales, glob = download(gpu)
+    d = rht_dim
     ref0 = oracle.quantize(x_bits, colwise=colwise, rht=True, sign_mask=sign_mask, rounding=rounding, seed=seed,
-                           sr_offset=sr_offset, return_y=True)
+                           sr_offset=sr_offset, return_y=True, rht_dim=d)
     # (1) transformed values
-    xs = synth.from_bits(x_bits).to(torch.float64).numpy()
-    src = xs.T if colwise else xs
-    l1 = np.abs(src).reshape(src.shape[0], -1, 16).sum(axis=2).repeat(16, axis=1) / 4
-    assert np.all(np.abs(y_gpu.astype(np.float64) - ref0.y) <= 1e-5 * l1 + 1e-30), f"{what}: transformed values"
+    if y_gpu is not None:
+        xs = synth.from_bits(x_bits).to(torch.float64).numpy()
+        src = xs.T if colwise else xs
+        l1 = np.abs(src).reshape(src.shape[0], -1, d).sum(axis=2).repeat(d, axis=1) / np.sqrt(d)
+        assert np.all(np.abs(y_gpu.astype(np.float64) - ref0.y) <= 1e-5 * l1 + 1e-30), f"{what}: transformed values"
     # (2) amax
     assert abs(float(glob[0]) - float(ref0.amax)) <= 1e-5 * float(ref0.amax), f"{what}: amax"
     ref = oracle.quantize(x_bits, colwise=colwise, rht=True, sign_mask=sign_mask, rounding=rounding, seed=seed,
-                          sr_offset=sr_offset, amax_override=float(glob[0]), return_y=True)
+                          sr_offset=sr_offset, amax_override=float(glob[0]), return_y=True, rht_dim=d)
     assert glob.view(np.uint32).tolist() == ref.glob.view(np.uint32).tolist(), f"{what}: s_dec from the same amax"
     s_enc, s_dec = oracle.global_scale(float(glob[0]))
     # (3) scale bytes
@@ -98,7 +118,7 @@ def assert_rht_close(x_bits: np.ndarray, gpu: B.NVFP4Tensor, y_gpu: np.ndarray, 
     assert not np.any(sdiff & ~near), f"{what}: {np.count_nonzero(sdiff & ~near)} unexcused scale bytes"
     assert np.all(np.abs(scales.astype(int) - ref.scales.astype(int))[sdiff] == 1), f"{what}: excused scale not adjacent"
     # (4) codes in blocks whose scale agrees
-    got, want = unpack(codes), unpack(ref.codes)
+    got, want = canon_zero(unpack(codes)), canon_zero(unpack(ref.codes))
     cdiff = (got != want) & ~np.repeat(sdiff, 16, axis=1)
     excused = 0
     for r, c in np.argwhere(cdiff):
@@ -199,7 +219,7 @@ def assert_mx_rht_close(x_bits: np.ndarray, gpu: B.NVFP4Tensor, *, colwise, sign
     sdiff = scales != ref.scales
     assert not np.any(sdiff & ~near), f"{what}: {np.count_nonzero(sdiff & ~near)} unexcused scale bytes"
     assert np.all(np.abs(scales.astype(int) - ref.scales.astype(int))[sdiff] == 1), f"{what}: excused scale not adjacent"
-    got, want = unpack(codes), unpack(ref.codes)
+    got, want = canon_zero(unpack(codes)), canon_zero(unpack(ref.codes))
     cdiff = (got != want) & ~np.repeat(sdiff, 32, axis=1)
     excused = 0
     for r, c in np.argwhere(cdiff):

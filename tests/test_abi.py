@@ -25,7 +25,7 @@ def test_every_declared_symbol_is_exported():
 
 
 def test_struct_layouts_match_the_header():
-    assert ctypes.sizeof(B.CTensor) == 48 and ctypes.sizeof(B.CQuantOpts) == 40
+    assert ctypes.sizeof(B.CTensor) == 48 and ctypes.sizeof(B.CQuantOpts) == 56
     assert B.CTensor.rows.offset == 24 and B.CQuantOpts.seed.offset == 24
 
 
