@@ -429,6 +429,12 @@ CASES = {
     "gemm_fprop_mx": ("gemm_mx", 4096, 5120, 5120), # MXFP4 operands, bf16 output
     "quant_w_f32": ("qw_f32", 20480, 5120, 0),      # 16x16 blocks, both copies, from a binary32 source (419 MB)
     "step": ("step", 8192, 20480, 5120),           # the whole cfg 3 fwd + bwd step, full size: ONE-PASS captures only
+    "gemm_bf16_fprop": ("bf16", 4096, 5120, 5120),  # BF16 layer (Section 4.1): Y = X W^T, both operands K-major
+    "gemm_bf16_wgrad": ("bf16_wgrad", 5120, 5120, 4096),  # dW = dY^T X, both operands read transposed, fp32 output
+    "step_bf16": ("step_bf16", 8192, 20480, 5120),  # the cfg 3 layer kept in BF16, fwd + bwd, full size
+    "quant_dy_rht4": ("qdy_rht4", 4096, 20480, 0),    # Appendix E.4.2: 4 x 4 transform
+    "quant_dy_rht128": ("qdy_rht128", 4096, 20480, 0),  # Appendix E.4.2: 128 x 128 transform
+    "quant_error": ("qerr", 4096, 20480, 0),        # Appendix E.2: decode-and-compare reduction (2.5625 B / element)
 }
 
 
@@ -461,6 +467,44 @@ def run_case(args):
             B.nvfp4_linear_fwd(X, W, o, Y, X_col, W_row, W_col, False, ws_f)
             B.nvfp4_linear_bwd(dY, X_col, W_col, k, o, dX, dW, False, ws_b)
         work, unit = 3 * 2.0 * r * c * k / 1e12, "TFLOP/s"
+    elif kind == "step_bf16":
+        X = torch.randn((r, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        W = (torch.randn((c, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
+        dY = (torch.randn((r, c), generator=g, device="cuda", dtype=torch.float32) * 1e-4).to(torch.bfloat16)
+        Y = torch.empty((r, c), dtype=torch.bfloat16, device="cuda")
+        dX = torch.empty((r, k), dtype=torch.bfloat16, device="cuda")
+        dW = torch.empty((c, k), dtype=torch.float32, device="cuda")
+
+        def fn():
+            B.nvfp4_linear_bf16_fwd(X, W, Y)
+            B.nvfp4_linear_bf16_bwd(dY, X, W, k, dX, dW)
+        work, unit = 3 * 2.0 * r * c * k / 1e12, "TFLOP/s"
+    elif kind in ("bf16", "bf16_wgrad"):
+        if kind == "bf16":
+            a = torch.randn((r, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+            b = (torch.randn((c, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
+            D = torch.empty((r, c), dtype=torch.bfloat16, device="cuda")
+            fn = lambda: B.nvfp4_gemm_bf16(a, b, D)
+        else:  # operands stored [tokens][features]: the contraction runs down their rows
+            a = torch.randn((k, r), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+            b = torch.randn((k, c), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+            D = torch.empty((r, c), dtype=torch.float32, device="cuda")
+            fn = lambda: B.nvfp4_gemm_bf16(a, b, D, B.MN_MAJOR, B.MN_MAJOR)
+        work, unit = 2.0 * r * c * k / 1e12, "TFLOP/s"
+    elif kind == "qerr":
+        x = torch.randn((r, c), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        q = B.alloc_tensor(r, c)
+        B.nvfp4_quantize(x, B.quant_opts(), q, None)
+        out = torch.empty(2, dtype=torch.float64, device="cuda")
+        fn = lambda: B.nvfp4_quant_error(x, q, out)
+        work, unit = r * c * 2.5625 / 1e9, "GB/s"
+    elif kind in ("qdy_rht4", "qdy_rht128"):
+        x = (torch.randn((r, c), generator=g, device="cuda", dtype=torch.float32) * 1e-4).to(torch.bfloat16)
+        row, col = B.alloc_tensor(r, c), B.alloc_tensor(c, r)
+        o = B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True, rht_dim=4 if kind == "qdy_rht4" else 128,
+                         rht_sign_mask=0x5A5A73E51234ABCD0F0F3C3C999973E5)
+        fn = lambda: B.nvfp4_quantize(x, o, row, col)
+        work, unit = r * c * 5.125 / 1e9, "GB/s"
     elif kind == "gemm_mx":
         a_src = torch.randn((r, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
         b_src = (torch.randn((c, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)

@@ -24,15 +24,15 @@ namespace nvfp4 {
 namespace {
 
 struct RhtSmem {
-  static constexpr int kTile = 0;                     // 128 rows x 256 B of bf16
-  static constexpr int kColCodes = 32768;             // 128 columns x 64 B
+  static constexpr int kColCodes = 0;                 // 128 columns x 64 B
   static constexpr int kSfRow = kColCodes + 8192;     // 1 KB
   static constexpr int kSfCol = kSfRow + 1024;        // 1 KB
   static constexpr int kGlobalScales = kSfCol + 1024; // 4 floats
   static constexpr int kRed = kGlobalScales + 64;     // 2 x 8 floats (amax pass)
   static constexpr int kRand = kRed + 64;             // 128 rows x 128 B
-  static constexpr int kU = kRand + 16384;            // 128 x 128 floats (d = 128, transposed copy only)
-  static constexpr int kBytesSmall = kU;
+  static constexpr int kTile = kRand + 16384;         // d <= 16: 128 rows x 256 B of bf16
+  static constexpr int kU = kTile;                    // d = 128 (transposed copy): 128 x 128 floats instead
+  static constexpr int kBytesSmall = kTile + 32768;
   static constexpr int kBytesBig = kU + 65536;
 };
 
@@ -58,7 +58,7 @@ __device__ __forceinline__ uint32_t chunk_signs(const RhtArgs& ra, int c16) {
 }
 
 template <int MODE, bool SR>
-__global__ void __launch_bounds__(256) quantize_rht_kernel(const RhtArgs ra) {
+__global__ void __launch_bounds__(256, 3) quantize_rht_kernel(const RhtArgs ra) {
   const QuantArgs& a = ra.q;
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -96,10 +96,19 @@ __global__ void __launch_bounds__(256) quantize_rht_kernel(const RhtArgs ra) {
 #pragma unroll
       for (int k = 0; k < 8; ++k) raw[i][k] = 0u;
     }
-    if (has_col) {
+    if (has_col && d_col == 128) {  // FP32 tile: the cross-group stages run in place on it
+      float* dst = reinterpret_cast<float*>(smem + RhtSmem::kU) + r * 128 + cb * 16;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        *reinterpret_cast<float4*>(dst + 4 * k) = make_float4(bf16_lo(raw[i][2 * k]), bf16_hi(raw[i][2 * k]),
+                                                              bf16_lo(raw[i][2 * k + 1]), bf16_hi(raw[i][2 * k + 1]));
+    } else if (has_col) {  // halves written in lane-dependent order so that a quarter warp covers all 32 banks
       uint8_t* dst = smem + RhtSmem::kTile + r * 256 + cb * 32;
-      *reinterpret_cast<uint4*>(dst) = make_uint4(raw[i][0], raw[i][1], raw[i][2], raw[i][3]);
-      *reinterpret_cast<uint4*>(dst + 16) = make_uint4(raw[i][4], raw[i][5], raw[i][6], raw[i][7]);
+      const int first = ((lane >> 2) & 1) * 16;
+      *reinterpret_cast<uint4*>(dst + first) =
+          first ? make_uint4(raw[i][4], raw[i][5], raw[i][6], raw[i][7]) : make_uint4(raw[i][0], raw[i][1], raw[i][2], raw[i][3]);
+      *reinterpret_cast<uint4*>(dst + (16 - first)) =
+          first ? make_uint4(raw[i][0], raw[i][1], raw[i][2], raw[i][3]) : make_uint4(raw[i][4], raw[i][5], raw[i][6], raw[i][7]);
     }
   }
   __syncthreads();
@@ -170,9 +179,9 @@ __global__ void __launch_bounds__(256) quantize_rht_kernel(const RhtArgs ra) {
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
           const int p = 16 * g + j;  // position in the 128-chunk = row inside the tile
-          uint32_t word = *reinterpret_cast<const uint32_t*>(smem + RhtSmem::kTile + p * 256 + cp * 4);
-          if ((ra.sign_words[p >> 5] >> (p & 31)) & 1u) word ^= 0x80008000u;
-          v[g] = make_float2(bf16_lo(word), bf16_hi(word));
+          const float2 x = *reinterpret_cast<const float2*>(U + p * 128 + 2 * cp);
+          const bool neg = (ra.sign_words[p >> 5] >> (p & 31)) & 1u;
+          v[g] = neg ? make_float2(-x.x, -x.y) : x;
         }
 #pragma unroll
         for (int h = 1; h < 8; h <<= 1)
@@ -237,7 +246,8 @@ __global__ void __launch_bounds__(256) quantize_rht_kernel(const RhtArgs ra) {
 #pragma unroll
         for (int odd = 0; odd < 2; ++odd) {
           const int c = 2 * cp + odd;
-          *reinterpret_cast<uint2*>(smem + RhtSmem::kColCodes + c * 64 + q * 8) = odd ? codes1 : codes0;
+          // unit q of column c sits at slot (q ^ (c >> 1)) & 7: neighbouring lanes hit different banks
+          *reinterpret_cast<uint2*>(smem + RhtSmem::kColCodes + c * 64 + (((q ^ (c >> 1)) & 7) << 3)) = odd ? codes1 : codes0;
           const uint32_t byte = odd ? byte1 : byte0;
           const int pos = a.c_swz ? ((q >> 2) * 512 + (c & 31) * 16 + (c >> 5) * 4 + (q & 3)) : (c * 8 + q);
           smem[RhtSmem::kSfCol + pos] = (uint8_t)byte;
@@ -276,7 +286,7 @@ __global__ void __launch_bounds__(256) quantize_rht_kernel(const RhtArgs ra) {
       const int c = unit >> 3, qq = unit & 7;  // column, 16-row group
       if (col0 + c >= a.cols || row0 + 16 * qq >= a.rows) continue;
       *reinterpret_cast<uint2*>(a.c_codes + (col0 + c) * pitch + (row0 >> 1) + qq * 8) =
-          *reinterpret_cast<const uint2*>(smem + RhtSmem::kColCodes + c * 64 + qq * 8);
+          *reinterpret_cast<const uint2*>(smem + RhtSmem::kColCodes + c * 64 + (((qq ^ (c >> 1)) & 7) << 3));
     }
   }
 #pragma unroll
