@@ -27,7 +27,7 @@ def rotated_amax(x: torch.Tensor, mask: int) -> float:
 
 
 def check_copy_slabs(x: torch.Tensor, gpu: B.NVFP4Tensor, *, colwise, block_rows=1, rht=False, mask=0, rounding=0,
-                     seed=0, sr_offset=0, what=""):
+                     seed=0, sr_offset=0, what="", rht_dim=16):
     codes, scales, glob = P.download(gpu)
     R = x.shape[0]
     n_bad = n_tot = 0
@@ -35,7 +35,7 @@ def check_copy_slabs(x: torch.Tensor, gpu: B.NVFP4Tensor, *, colwise, block_rows
         slab = synth.bits(x[r0:r0 + 128])
         ref = oracle.quantize(slab, colwise=colwise, block_rows=block_rows, rht=rht, sign_mask=mask, rounding=rounding,
                               seed=seed, sr_offset=sr_offset, amax_override=float(glob[0]), sr_row0=r0,
-                              sr_cols=x.shape[1])
+                              sr_cols=x.shape[1], rht_dim=rht_dim)
         assert glob.view(np.uint32)[1] == ref.glob.view(np.uint32)[1], f"{what}: s_dec"
         if colwise:
             got_c, got_s = codes[:, r0 // 2:(r0 + 128) // 2], scales[:, r0 // 16:(r0 + 128) // 16]
@@ -48,7 +48,7 @@ def check_copy_slabs(x: torch.Tensor, gpu: B.NVFP4Tensor, *, colwise, block_rows
             # rotated copies: equal except next to a rounding threshold (butterfly vs float64 summation order)
             sd = got_s != ref.scales
             assert np.all(np.abs(got_s.astype(int) - ref.scales.astype(int))[sd] <= 1), f"{what}: scale not adjacent"
-            g, w = P.unpack(got_c), P.unpack(ref.codes)
+            g, w = P.canon_zero(P.unpack(got_c)), P.canon_zero(P.unpack(ref.codes))
             cd = (g != w) & ~np.repeat(sd, 16, axis=1)
             assert np.all(np.abs((g & 7).astype(int) - (w & 7).astype(int))[cd] <= 1), f"{what}: code not adjacent"
             n_bad += int(cd.sum()) + 16 * int(sd.sum())
@@ -233,3 +233,59 @@ def test_config5_qkv_projection_shapes():
                        True, "cfg5 qkv Dgrad", 6)
     check_gemm_samples(dW, Operand(g_col, p.dY, colwise=True, rht=True, mask=mask, **sr),
                        Operand(X_col, p.X, colwise=True, rht=True, mask=mask), False, "cfg5 qkv Wgrad", 7)
+
+
+def test_config3_full_size_variants_bf16_layer_transform_sizes_error_metric():
+    """The recipe's variants at the benchmark's size: the layer kept in BF16 (Section 4.1) on sampled rows x columns,
+    dY quantized with the 4 x 4 and 128 x 128 transforms (Appendix E.4.2) on sampled slabs, and the error metric
+    (Appendix E.2) of the full dY copy against sums the oracle forms from sampled slabs scaled to the tensor."""
+    p = synth.config3()
+    M, N, K = p.M, p.N, p.K
+    X, W, dY = p.X.cuda(), p.W.cuda(), p.dY.cuda()
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    dW = torch.zeros((N, K), dtype=torch.float32, device="cuda")
+    B.nvfp4_linear_bf16_fwd(X, W, Y)
+    B.nvfp4_linear_bf16_bwd(dY, X, W, K, dX, dW)
+    B.nvfp4_device_status()
+    rng = np.random.default_rng(5)
+    f64 = lambda t: t.float().numpy().astype(np.float64)
+
+    def sample(D, A, Bm, bf16, what):  # D = A Bm^T with A [rows x k], Bm [cols x k] given as CPU bf16 tensors
+        rows = np.sort(rng.choice(A.shape[0], 12, replace=False))
+        cols = np.sort(rng.choice(Bm.shape[0], 384, replace=False))
+        Dref, T = oracle.gemm_tn(f64(A[rows]), f64(Bm[cols]))
+        got = D[torch.from_numpy(rows).cuda()][:, torch.from_numpy(cols).cuda()].float().cpu().numpy()
+        tol = 1e-4 * T + (2.0 ** -8 * np.abs(Dref) if bf16 else 0.0) + 1e-30
+        assert np.all(np.abs(got - Dref) <= tol), what
+
+    sample(Y, p.X, p.W, True, "BF16 Fprop")
+    sample(dX, p.dY, p.W.t().contiguous(), True, "BF16 Dgrad")
+    sample(dW, p.dY.t().contiguous(), p.X.t().contiguous(), False, "BF16 Wgrad")
+
+    # transform sizes on dY (stochastic rounding, plain row copy + rotated transposed copy)
+    big_mask = 0x5A5A_73E5_1234_ABCD_0F0F_3C3C_9999_73E5
+    g_row, g_col = B.alloc_tensor(M, N), B.alloc_tensor(N, M)
+    for d in (4, 128):
+        m = big_mask & ((1 << d) - 1)
+        B.nvfp4_quantize(dY, B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True, rht_sign_mask=m, rht_dim=d,
+                                          seed=p.sr_seed, sr_offset=p.sr_offset), g_row, g_col)
+        check_copy_slabs(p.dY, g_row, colwise=False, rounding=oracle.SR, seed=p.sr_seed, sr_offset=p.sr_offset,
+                         what=f"dY row beside d={d}")
+        check_copy_slabs(p.dY, g_col, colwise=True, rht=True, mask=m, rounding=oracle.SR, seed=p.sr_seed,
+                         sr_offset=p.sr_offset, what=f"dY col d={d}", rht_dim=d)
+
+    # error metric of the row-wise copy: the oracle's sums over three 128-row slabs against the kernel's over the
+    # same slabs (views of the full-size tensors), and the full-tensor value for plausibility
+    for r0 in (0, M // 2, M - 128):
+        ref = oracle.quantize(synth.bits(p.dY[r0:r0 + 128]), rounding=oracle.SR, seed=p.sr_seed, sr_offset=p.sr_offset,
+                              amax_override=float(g_row.glob[0]), sr_row0=r0, sr_cols=N)
+        e_ref, n_ref = oracle.quant_error(f64(p.dY[r0:r0 + 128]), oracle.dequantize(ref))
+        # scale atoms of a 128-row slab are contiguous: rows r0 .. r0 + 127 form the atom row r0 / 128
+        slab = B.NVFP4Tensor(g_row.codes[r0:r0 + 128], g_row.scales.view(-1)[(r0 // 128) * (N // 64) * 512:].contiguous(),
+                             g_row.glob, 128, N, B.SF_SWIZZLED)
+        out = B.nvfp4_quant_error(dY[r0:r0 + 128], slab).cpu().numpy()
+        assert abs(out[0] - e_ref) <= 1e-5 * e_ref and abs(out[1] - n_ref) <= 1e-5 * n_ref, (r0, out, e_ref, n_ref)
+    full = B.nvfp4_quant_error(dY, g_row).cpu().numpy()
+    assert abs(full[1] - float((p.dY.double() ** 2).sum())) <= 1e-6 * full[1]
+    assert 2e-3 < full[0] / full[1] < 5e-2
