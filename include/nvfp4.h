@@ -165,7 +165,8 @@ NVFP4_API nvfp4_status nvfp4_gemm(const nvfp4_tensor* A, const nvfp4_tensor* B, 
  *   B: device bf16.  b_layout NVFP4_K_MAJOR : stored [N][K], ldb >= K;  NVFP4_MN_MAJOR: stored [K][N], ldb >= N.
  *   D: device, row-major [M x N], ldd >= N, bf16 (round-to-nearest-even) or fp32 (d_is_fp32 != 0);
  *      accumulate != 0 adds into an fp32 D.
- *   M, N multiples of 256, K of 64; pointers 16-byte aligned, lda, ldb multiples of 8, ldd * elemsize of 16.
+ *   M, N, K multiples of 8 (the kernel works on 256 x 256 x 64 tiles; ragged edges are zero-filled on load and
+ *   clipped on store by the tensor maps); pointers 16-byte aligned, lda, ldb multiples of 8, ldd * elemsize of 16.
  *   Nothing is enqueued on error.
  */
 enum { NVFP4_K_MAJOR = 0, NVFP4_MN_MAJOR = 1 };
@@ -177,7 +178,7 @@ NVFP4_API nvfp4_status nvfp4_gemm_bf16(const void* A, int32_t a_layout, int64_t 
  * The same layer as nvfp4_linear_fwd / _bwd without quantization (Section 4.1, Appendix D), on the same row-major
  * operands X [M x K], W [N x K], dY [M x N], all contiguous bf16; no transposed copies are made:
  *   fwd: Y  = X W^T (bf16);   bwd: dX = dY W (bf16), dW = dY^T X (fp32, accumulate_dw != 0 adds into it);
- *   dX or dW may be NULL to skip that GEMM.  M, N, K multiples of 256.
+ *   dX or dW may be NULL to skip that GEMM.  M, N, K multiples of 8.
  */
 NVFP4_API nvfp4_status nvfp4_linear_bf16_fwd(const void* X, const void* W, int64_t M, int64_t N, int64_t K,
                                              void* Y_bf16, void* cuda_stream);

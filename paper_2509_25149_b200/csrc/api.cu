@@ -333,8 +333,9 @@ nvfp4_status nvfp4_gemm_bf16(const void* A, int32_t a_layout, int64_t lda, const
   if (!A || !B || !D) return NVFP4_ERR_NULL;
   if ((a_layout != NVFP4_K_MAJOR && a_layout != NVFP4_MN_MAJOR) || (b_layout != NVFP4_K_MAJOR && b_layout != NVFP4_MN_MAJOR))
     return NVFP4_ERR_ARG;
-  if (M <= 0 || N <= 0 || K <= 0 || M % 256 != 0 || N % 256 != 0 || K % 64 != 0) return NVFP4_ERR_SHAPE;
-  if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff || (M / 256) * (N / 256) > 0x7fffffff) return NVFP4_ERR_SHAPE;
+  if (M <= 0 || N <= 0 || K <= 0 || M % 8 != 0 || N % 8 != 0 || K % 8 != 0) return NVFP4_ERR_SHAPE;
+  if (M > 0x7fffff00 || N > 0x7fffff00 || K > 0x7fffff00 || ((M + 255) / 256) * ((N + 255) / 256) > 0x7fffffff)
+    return NVFP4_ERR_SHAPE;
   if (lda < (a_layout == NVFP4_MN_MAJOR ? M : K) || ldb < (b_layout == NVFP4_MN_MAJOR ? N : K) || ldd < N)
     return NVFP4_ERR_SHAPE;
   if (accumulate && !d_is_fp32) return NVFP4_ERR_ARG;

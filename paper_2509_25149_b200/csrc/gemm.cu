@@ -594,7 +594,7 @@ cudaError_t launch_gemm_bf16(const DenseGemmArgs& g, cudaStream_t s) {
     device_configured(configured, dev);
   }
   dense::Args a{g.M, g.N, g.K, g.a_mn, g.b_mn, g.d_is_fp32, g.accumulate};
-  const int n_tiles = (g.M / 256) * (g.N / 256), max_pairs = num_sms / 2;
+  const int n_tiles = ((g.M + 255) / 256) * ((g.N + 255) / 256), max_pairs = num_sms / 2;
   const int pairs = n_tiles < max_pairs ? n_tiles : max_pairs;
   dense::gemm_bf16_pair_kernel<<<2 * pairs, dense::kThreads, dense::kSmemBytes, s>>>(map_a, map_b, map_d, a);
   count_launch();

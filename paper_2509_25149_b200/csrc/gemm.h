@@ -31,7 +31,7 @@ cudaError_t read_device_status(cudaStream_t s, uint32_t* code);
 
 // BF16 GEMM D[M x N] = A B^T on CTA pairs (gemm_bf16.cuh) for layers kept in higher precision.
 // a_mn / b_mn = 0: the operand is stored [M or N][K] (contraction contiguous); 1: stored [K][M or N].
-// M, N multiples of 256, K of 64; leading dimensions in elements.
+// M, N, K multiples of 8 (tiles of 256 x 256 x 64 with zero-filled / clipped edges); leading dimensions in elements.
 struct DenseGemmArgs {
   const void* a;
   const void* b;

@@ -76,8 +76,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
   const uint32_t rank = cluster_ctarank();  // 0 = leader
   const bool leader = rank == 0;
   const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int tiles_m = g.M / 256, tiles_n = g.N / 256, n_tiles = tiles_m * tiles_n;
-  const int k_blocks = g.K / 64;
+  // ragged edges: loads beyond the operands read zeros, stores beyond D are clipped (both by the tensor maps)
+  const int tiles_m = (g.M + 255) / 256, tiles_n = (g.N + 255) / 256, n_tiles = tiles_m * tiles_n;
+  const int k_blocks = (g.K + 63) / 64;
   // groups of eight row-blocks sweep all column-blocks before the next group starts (L2 reuse of A and B)
   constexpr int kGroupM = 8;
   auto tile_coords = [&](int tile, int& m_blk, int& n_blk) {

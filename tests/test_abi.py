@@ -77,7 +77,7 @@ def test_argument_validation_happens_before_any_launch():
     g16 = lambda M, N, K, lda=None, ldb=None, ldd=None, al=0, bl=0, fp32=0, acc=0, A=fake: L.nvfp4_gemm_bf16(
         A, al, lda or K, fake, bl, ldb or K, M, N, K, fake, fp32, ldd or N, acc, None)
     assert g16(256, 256, 64, A=None) == 1
-    assert g16(128, 256, 64) == 2 and g16(256, 384, 64) == 2 and g16(256, 256, 32) == 2      # tile multiples
+    assert g16(124, 256, 64) == 2 and g16(256, 380, 64) == 2 and g16(256, 256, 36) == 2      # multiples of 8
     assert g16(256, 256, 64, lda=32) == 2 and g16(256, 256, 64, ldd=128) == 2                 # leading dimensions
     assert g16(256, 256, 64, al=1, lda=64) == 2                                                # [K][M] needs lda >= M
     assert g16(256, 256, 64, al=2) == 4 and g16(256, 256, 64, acc=1) == 4                      # layout id; bf16 accumulate

@@ -96,7 +96,27 @@ def test_accumulate_and_leading_dimensions():
     with pytest.raises(B.NVFP4Error):
         B.nvfp4_gemm_bf16(x.cuda(), w.cuda(), torch.empty((M, N), dtype=torch.bfloat16, device="cuda"), accumulate=True)
     with pytest.raises(B.NVFP4Error):
-        B.nvfp4_gemm_bf16(x.cuda()[:128], w.cuda(), torch.empty((128, N), dtype=torch.bfloat16, device="cuda"))
+        B.nvfp4_gemm_bf16(x.cuda()[:124], w.cuda(), torch.empty((124, N), dtype=torch.bfloat16, device="cuda"))
+
+
+@pytest.mark.parametrize("shape", [(8, 8, 8), (264, 136, 72), (1000, 520, 200), (136, 2056, 4104)])
+def test_ragged_shapes_every_layout(shape):
+    """M, N, K that are not multiples of the 256 x 256 x 64 tile: edges are zero-filled on load, clipped on store."""
+    M, N, K = shape
+    x = synth.normal_bf16((M, K), 1.0, 41)
+    w = synth.normal_bf16((N, K), 0.1, 42)
+    Dref, T = oracle.gemm_tn(f64(x), f64(w))
+    for a_layout, b_layout in LAYOUTS:
+        a = x.t().contiguous() if a_layout == B.MN_MAJOR else x
+        b = w.t().contiguous() if b_layout == B.MN_MAJOR else w
+        for fp32 in (False, True):
+            # the output sits inside a larger buffer whose other elements must survive
+            buf = torch.full((M + 8, N + 8), 7.0, dtype=torch.float32 if fp32 else torch.bfloat16, device="cuda")
+            B.nvfp4_gemm_bf16(a.cuda(), b.cuda(), buf[:M, :N], a_layout, b_layout)
+            B.nvfp4_device_status()
+            out = buf.float().cpu().numpy()
+            assert_close(out[:M, :N], Dref, T, not fp32, f"{shape} {a_layout}{b_layout} fp32={fp32}")
+            assert np.all(out[M:, :] == 7.0) and np.all(out[:, N:] == 7.0), "stores beyond M x N"
 
 
 def test_linear_layer_fwd_bwd():
