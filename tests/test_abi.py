@@ -83,3 +83,39 @@ def test_argument_validation_happens_before_any_launch():
     assert g16(256, 256, 64, al=2) == 4 and g16(256, 256, 64, acc=1) == 4                      # layout id; bf16 accumulate
     assert g16(256, 256, 64, lda=68) == 3                                                      # lda % 8
     assert L.nvfp4_linear_bf16_bwd(fake, fake, fake, 256, 256, 256, None, None, 0, None) == 1
+
+
+def test_header_is_plain_c_and_cxx():
+    import subprocess
+    hdr = os.path.join(ROOT, "include", "nvfp4.h")
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c", hdr], check=True)
+    subprocess.run(["g++", "-std=c++17", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", hdr], check=True)
+
+
+def test_plain_c_client_compiles_and_links():
+    """The C client under tests/c uses nothing but the header, the shared library and the CUDA runtime."""
+    import subprocess, tempfile
+    B.lib()
+    libdir = os.path.join(ROOT, "paper_2509_25149_b200")
+    with tempfile.TemporaryDirectory() as tmp:
+        exe = os.path.join(tmp, "abi_roundtrip")
+        subprocess.run(["gcc", "-std=c99", "-O1", "-Wall", "-Werror", os.path.join(ROOT, "tests", "c", "abi_roundtrip.c"),
+                        "-I", os.path.join(ROOT, "include"), "-I", "/usr/local/cuda/include", "-L", libdir,
+                        "-lnvfp4_b200", "-L", "/usr/local/cuda/lib64", "-lcudart", f"-Wl,-rpath,{libdir}", "-o", exe],
+                       check=True)
+        assert os.path.exists(exe)
+
+
+@pytest.mark.gpu
+def test_plain_c_client_runs():
+    import subprocess, tempfile
+    B.lib()
+    libdir = os.path.join(ROOT, "paper_2509_25149_b200")
+    with tempfile.TemporaryDirectory() as tmp:
+        exe = os.path.join(tmp, "abi_roundtrip")
+        subprocess.run(["gcc", "-std=c99", "-O1", os.path.join(ROOT, "tests", "c", "abi_roundtrip.c"),
+                        "-I", os.path.join(ROOT, "include"), "-I", "/usr/local/cuda/include", "-L", libdir,
+                        "-lnvfp4_b200", "-L", "/usr/local/cuda/lib64", "-lcudart", f"-Wl,-rpath,{libdir}", "-o", exe],
+                       check=True)
+        r = subprocess.run([exe], capture_output=True, text=True, timeout=120)
+        assert r.returncode == 0 and r.stdout.startswith("ok"), (r.returncode, r.stdout, r.stderr)
