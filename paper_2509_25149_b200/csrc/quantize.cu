@@ -142,12 +142,14 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t v) {
   return r;
 }
 
+// d, norm: size of the transform (2, 4, 8 or 16: H_16 is replaced by the block-diagonal matrix of 16 / d copies of
+// H_d) and its normalisation 1 / sqrt(d), applied to the maximum.
 template <bool PLAIN>
 __global__ void __launch_bounds__(256) amax_rot_col_kernel(const uint16_t* __restrict__ x, int64_t rows,
                                                            int64_t cols, int64_t ld, uint32_t sign_mask,
                                                            int tiles_c, float* __restrict__ out_plain0,
                                                            float* __restrict__ out_plain1,
-                                                           float* __restrict__ out_rot_col) {
+                                                           float* __restrict__ out_rot_col, int d, float norm) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
   const int64_t tr = blockIdx.x / tiles_c, tc = blockIdx.x % tiles_c;
@@ -166,9 +168,11 @@ __global__ void __launch_bounds__(256) amax_rot_col_kernel(const uint16_t* __res
     }
   }
 
-  // A fragments: entry (k, j) = +-1 as bf16, negative iff popc(k & j) is odd XOR sign bit j
+  // A fragments: entry (k, j) = +-1 as bf16 inside the d x d diagonal blocks (0 outside), negative iff
+  // popc(k & j) is odd XOR sign bit j
   auto entry = [&](int k, int j) -> uint32_t {
-    return ((__popc(k & j) ^ (sign_mask >> j)) & 1u) ? 0xBF80u : 0x3F80u;
+    if ((k ^ j) >= d) return 0u;
+    return ((__popc(k & j & (d - 1)) ^ (sign_mask >> j)) & 1u) ? 0xBF80u : 0x3F80u;
   };
   const uint32_t a0 = entry(g, 2 * t) | (entry(g, 2 * t + 1) << 16);
   const uint32_t a1 = entry(g + 8, 2 * t) | (entry(g + 8, 2 * t + 1) << 16);
@@ -196,7 +200,7 @@ __global__ void __launch_bounds__(256) amax_rot_col_kernel(const uint16_t* __res
       m_col = fmaxf(fmaxf(m_col, fmaxf(fabsf(d0), fabsf(d1))), fmaxf(fabsf(d2), fabsf(d3)));
     }
   }
-  m_col *= 0.25f;
+  m_col *= norm;
   float m_plain = PLAIN ? fmaxf(bf16_lo(acc), bf16_hi(acc)) : 0.f;
 
   __shared__ float red[2][8];
@@ -588,10 +592,10 @@ cudaError_t launch_amax(const QuantArgs& a, bool has_row, bool has_col, bool rht
     const unsigned tiles = (unsigned)(((a.rows + 127) / 128) * tiles_c);
     if (plain)
       amax_rot_col_kernel<true><<<tiles, 256, 0, s>>>(a.x, a.rows, a.cols, a.ld, a.sign_mask, tiles_c, plain0, plain1,
-                                                      rot_col);
+                                                      rot_col, 16, 0.25f);
     else
       amax_rot_col_kernel<false><<<tiles, 256, 0, s>>>(a.x, a.rows, a.cols, a.ld, a.sign_mask, tiles_c, plain0,
-                                                       plain1, rot_col);
+                                                       plain1, rot_col, 16, 0.25f);
     count_launch();
     return cudaGetLastError();
   }
@@ -605,6 +609,25 @@ cudaError_t launch_amax(const QuantArgs& a, bool has_row, bool has_col, bool rht
   NVFP4_AMAX(false, true, false)
 #undef NVFP4_AMAX
   return cudaErrorInvalidValue;
+}
+
+// Pass 1 of the transposed copy with a d x d transform (d = 2, 4, 8), and the plain amax of the row-wise copy
+// beside it: the tensor-core kernel above with a block-diagonal matrix.  sign_mask: the d sign bits repeated to 16.
+cudaError_t launch_amax_rot_col_small(const QuantArgs& a, bool has_row, uint32_t mask16, int d, float norm,
+                                      cudaStream_t s) {
+  cudaError_t e;
+  if (has_row && (e = cudaMemsetAsync(a.r_global, 0, sizeof(float), s)) != cudaSuccess) return e;
+  if ((e = cudaMemsetAsync(a.c_global, 0, sizeof(float), s)) != cudaSuccess) return e;
+  const int tiles_c = (int)((a.cols + 255) / 256);
+  const unsigned tiles = (unsigned)(((a.rows + 127) / 128) * tiles_c);
+  if (has_row)
+    amax_rot_col_kernel<true><<<tiles, 256, 0, s>>>(a.x, a.rows, a.cols, a.ld, mask16, tiles_c, a.r_global, nullptr,
+                                                    a.c_global, d, norm);
+  else
+    amax_rot_col_kernel<false><<<tiles, 256, 0, s>>>(a.x, a.rows, a.cols, a.ld, mask16, tiles_c, nullptr, nullptr,
+                                                     a.c_global, d, norm);
+  count_launch();
+  return cudaGetLastError();
 }
 
 template <bool HR, bool HC, bool B2, bool RR, bool RC, bool SR>

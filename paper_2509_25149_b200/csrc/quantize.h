@@ -33,6 +33,8 @@ struct RhtArgs {
   float norm;              // fl(1 / sqrt(d))
 };
 cudaError_t launch_quantize_rht(const RhtArgs& ra, bool amax_provided, bool sr, cudaStream_t s);
+cudaError_t launch_amax_rot_col_small(const QuantArgs& a, bool has_row, uint32_t mask16, int d, float norm,
+                                      cudaStream_t s);
 
 cudaError_t launch_amax(const QuantArgs& a, bool has_row, bool has_col, bool rht_row, bool rht_col,
                         cudaStream_t s);

@@ -336,7 +336,10 @@ cudaError_t launch_mode(const RhtArgs& ra, cudaStream_t s) {
 
 cudaError_t launch_quantize_rht(const RhtArgs& ra, bool amax_provided, bool sr, cudaStream_t s) {
   cudaError_t e;
-  if (!amax_provided) {
+  if (!amax_provided && ra.d <= 16 && ra.has_col && ra.rht_col && !ra.rht_row) {
+    // the recipe's case (plain row-wise copy, transformed transposed copy): pass 1 on the tensor cores, HBM-bound
+    if ((e = launch_amax_rot_col_small(ra.q, ra.has_row != 0, ra.mask16, ra.d, ra.norm, s)) != cudaSuccess) return e;
+  } else if (!amax_provided) {
     if (ra.has_row && (e = cudaMemsetAsync(ra.q.r_global, 0, sizeof(float), s)) != cudaSuccess) return e;
     if (ra.has_col && (e = cudaMemsetAsync(ra.q.c_global, 0, sizeof(float), s)) != cudaSuccess) return e;
     if ((e = launch_mode<0, false>(ra, s)) != cudaSuccess) return e;
