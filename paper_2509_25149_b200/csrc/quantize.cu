@@ -302,7 +302,10 @@ __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const Qu
     }
   }
 
-  if (HAS_COL) {
+  // 16x16 blocks with both copies requested: the transposed copy holds the very codes of the row-wise one
+  // (Section 4.3), so it is made by transposing nibbles; the raw tile is not needed a second time
+  constexpr bool kNibbleTranspose = BLOCK2D && HAS_ROW && HAS_COL;
+  if (HAS_COL && !kNibbleTranspose) {
     // stage the raw tile; halves are written in lane-dependent order so that a quarter warp covers
     // all 32 banks
     const int first = (lane >> 2) & 1;
@@ -384,6 +387,8 @@ __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const Qu
       uint2 codes = convert16<SR>(f, enc, Nu14FromWords{rnd});
       if (ok[i])
         *reinterpret_cast<uint2*>(a.r_codes + (row0 + r) * (a.cols >> 1) + ((col0 + cb * 16) >> 1)) = codes;
+      if (kNibbleTranspose)  // row r, bytes [8 cb, 8 cb + 8): byte k = columns (2k, 2k + 1) of the chunk
+        *reinterpret_cast<uint2*>(smem + QuantSmem::kTile + r * 64 + cb * 8) = ok[i] ? codes : make_uint2(0u, 0u);
       const int pos = a.r_swz ? ((cb >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (cb & 3)) : (r * 8 + cb);
       smem[QuantSmem::kSfRow + pos] = (uint8_t)byte;
     }
@@ -396,6 +401,41 @@ __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const Qu
 #pragma unroll 1
     for (int it = 0; it < 2; ++it) {
       const int cp = lane + 32 * it;  // column pair: tile columns 2cp, 2cp+1
+      if (kNibbleTranspose) {
+        // byte [row][cp] of the staged row-wise codes = (column 2cp in the low nibble, 2cp + 1 in the high one)
+        uint32_t w[4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          uint32_t b[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) b[j] = smem[QuantSmem::kTile + (q * 16 + 4 * m + j) * 64 + cp];
+          w[m] = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
+        }
+        auto gather = [](uint32_t x) {  // four nibbles, one per byte -> 16 bits
+          const uint32_t t = (x | (x >> 4)) & 0x00FF00FFu;
+          return (t | (t >> 8)) & 0xFFFFu;
+        };
+        uint32_t lo[4], hi[4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          lo[m] = gather(w[m] & 0x0F0F0F0Fu);
+          hi[m] = gather((w[m] >> 4) & 0x0F0F0F0Fu);
+        }
+        const uint2 codes0 = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
+        const uint2 codes1 = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+        const uint32_t byte = smem[QuantSmem::kBlkByte + q * 8 + (cp >> 3)];
+        const int sel = (lane >> 3) & 1;
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+          const int odd = s ^ sel;
+          const int c = 2 * cp + odd;
+          *reinterpret_cast<uint2*>(smem + QuantSmem::kColCodes + c * 64 + (((q ^ (c >> 1)) & 7) << 3)) =
+              odd ? codes1 : codes0;
+          const int pos = a.c_swz ? ((q >> 2) * 512 + (c & 31) * 16 + (c >> 5) * 4 + (q & 3)) : (c * 8 + q);
+          smem[QuantSmem::kSfCol + pos] = (uint8_t)byte;
+        }
+        continue;
+      }
       float f0[16], f1[16];
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
