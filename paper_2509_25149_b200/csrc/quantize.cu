@@ -381,7 +381,16 @@ __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const Qu
         byte = blk_byte;
         enc = blk_enc;
       } else {
-        block_scales(RHT_ROW ? 0.25f * amax16(f) : amax16(f), r_senc, r_sdec, byte, enc);
+        float bmax;
+        if (RHT_ROW) {
+          bmax = 0.25f * amax16(f);
+        } else {  // untransformed: the maximum of the bf16 pairs themselves, two elements per instruction
+          uint32_t acc = 0;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) acc = absmax_bf16x2(acc, raw[i][k]);
+          bmax = fmaxf(bf16_lo(acc), bf16_hi(acc));
+        }
+        block_scales(bmax, r_senc, r_sdec, byte, enc);
         if (RHT_ROW) enc *= 0.25f;
       }
       uint2 codes = convert16<SR>(f, enc, Nu14FromWords{rnd});
