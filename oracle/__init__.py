@@ -301,6 +301,41 @@ def gemm_blockscaled(a: Quantized, b: Quantized):
     return D
 
 
+# ------------------------- global scale at row granularity (Appendix B.1, last sentence) ----
+class QuantizedRows:
+    """A row-wise copy whose FP32 scale is taken per row: glob[r] = {amax of row r, s_dec of row r}."""
+
+    def __init__(self, codes, scales, glob, rows, cols):
+        self.codes, self.scales, self.glob = codes, scales, glob
+        self.rows, self.cols = rows, cols
+
+
+def quantize_rowscale(x_bf16_bits, *, rounding=RNE, seed=0, sr_offset=0, sr_row0=0, sr_cols=0, sr_col0=0) -> QuantizedRows:
+    """Appendix B.1 closes with the remark that the global scale could span a row instead of the tensor, which
+    removes the pass that computes the tensor amax.  Written out: every row is quantized as a tensor of its own
+    (Eq. 1 from the row's amax, then Eq. 2-4 unchanged); the stochastic-rounding draws stay keyed by the element's
+    position in the whole source."""
+    x = np.asarray(x_bf16_bits)
+    assert x.dtype == np.uint16 and x.ndim == 2
+    R, C = x.shape
+    codes = np.zeros((R, C // 2), dtype=np.uint8)
+    scales = np.zeros((R, C // 16), dtype=np.uint8)
+    glob = np.zeros((R, 2), dtype=np.float32)
+    for r in range(R):
+        q = quantize(x[r:r + 1], rounding=rounding, seed=seed, sr_offset=sr_offset, sr_row0=sr_row0 + r,
+                     sr_cols=sr_cols if sr_cols else C, sr_col0=sr_col0)
+        codes[r], scales[r], glob[r] = q.codes[0], q.scales[0], q.glob
+    return QuantizedRows(codes, scales, glob, R, C)
+
+
+def dequantize_rowscale(q: QuantizedRows):
+    """x^ = code * block scale * the row's decode scale, in binary64."""
+    out = np.zeros((q.rows, q.cols), dtype=np.float64)
+    for r in range(q.rows):
+        out[r] = dequantize(Quantized(q.codes[r:r + 1], q.scales[r:r + 1], q.glob[r], 1, q.cols))[0]
+    return out
+
+
 # ------------------------------------------- layers kept in BF16 (Section 4.1) ----
 def _bf16_bits_to_f64(bits):
     b = np.ascontiguousarray(bits, dtype=np.uint16)

@@ -152,3 +152,41 @@ def test_quant_error_by_hand_and_on_the_grid():
     e_rne, n = oracle.quant_error(xf, oracle.dequantize(oracle.quantize(synth.bits(x))))
     e_sr, _ = oracle.quant_error(xf, oracle.dequantize(oracle.quantize(synth.bits(x), rounding=oracle.SR, seed=1)))
     assert 2e-3 < e_rne / n < 3e-2 and e_rne < e_sr < 4 * e_rne
+
+
+# ------------------------------------------- row-granular global scale ----
+def test_rowscale_reduces_to_the_tensor_scale_and_decouples_rows():
+    """Appendix B.1's closing remark: a global scale per row.  Pins: rows sharing one amax give the tensor-scaled
+    result bit for bit; a row's bytes do not depend on the other rows; an outlier row no longer costs the small
+    rows their resolution; on-grid rows decode exactly; SR draws are those of the whole-tensor positions."""
+    x = synth.normal_bf16((32, 256), 1.0, 91)
+    xb = synth.bits(x).copy()
+    # (a) give every row the same maximum: per-row scaling must equal per-tensor scaling
+    top = np.uint16(0x4120)  # 10.0 in bf16, above every N(0,1) sample
+    xb[:, 7] = top
+    a = oracle.quantize_rowscale(xb)
+    b = oracle.quantize(xb)
+    assert np.array_equal(a.codes, b.codes) and np.array_equal(a.scales, b.scales)
+    assert np.all(a.glob == b.glob[None, :])
+    # (b) rows are independent: changing row 3 leaves all other rows' bytes alone
+    xb2 = xb.copy()
+    xb2[3, 100] = np.uint16(0x447A)  # 1000.0
+    c = oracle.quantize_rowscale(xb2)
+    keep = np.arange(32) != 3
+    assert np.array_equal(c.codes[keep], a.codes[keep]) and np.array_equal(c.glob[keep], a.glob[keep])
+    assert c.glob[3, 0] == 1000.0
+    # (c) with a per-tensor scale the same outlier flushes small blocks of OTHER rows to zero, with row scales not
+    small = synth.normal_bf16((8, 64), 1e-4, 92)
+    sb = synth.bits(small).copy()
+    sb[0, 0] = np.uint16(0x4F00)  # 2^31 in row 0
+    xs = synth.from_bits(sb).to(torch.float64).numpy()
+    e_tensor = np.abs(oracle.dequantize(oracle.quantize(sb)) - xs)[1:].max()
+    e_rows = np.abs(oracle.dequantize_rowscale(oracle.quantize_rowscale(sb)) - xs)[1:].max()
+    assert e_rows < 0.2 * np.abs(xs[1:]).max() and e_tensor == np.abs(xs[1:]).max(), (e_rows, e_tensor)  # flushed to zero
+    # (d) stochastic rounding: row r of the row-scaled copy is the 1-row tensor quantized with the draws of the
+    # positions (r, c) of the whole source
+    q = oracle.quantize_rowscale(xb, rounding=oracle.SR, seed=5, sr_offset=2)
+    one = oracle.quantize(xb[9:10], rounding=oracle.SR, seed=5, sr_offset=2, sr_row0=9, sr_cols=256)
+    assert np.array_equal(q.codes[9], one.codes[0])
+    v = oracle.dequantize_rowscale(q)
+    assert np.all(np.abs(v - synth.from_bits(xb).to(torch.float64).numpy()) <= 2.0 * 10.0 / 6 * 1.07)
