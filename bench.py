@@ -455,6 +455,8 @@ CASES = {
     "step_bf16": ("step_bf16", 8192, 20480, 5120),  # the cfg 3 layer kept in BF16, fwd + bwd, full size
     "quant_dy_rht4": ("qdy_rht4", 4096, 20480, 0),    # Appendix E.4.2: 4 x 4 transform
     "quant_dy_rht128": ("qdy_rht128", 4096, 20480, 0),  # Appendix E.4.2: 128 x 128 transform
+    "quant_x_rowscale": ("q_rows", 16384, 5120, 0),  # App. B.1 closing remark: one pass, global scale per row, RNE
+    "quant_dy_rowscale": ("q_rows_sr", 4096, 20480, 0),  # the same with stochastic rounding on gradient-shaped rows
     "quant_error": ("qerr", 4096, 20480, 0),        # Appendix E.2: decode-and-compare reduction (2.5625 B / element)
 }
 
@@ -512,6 +514,12 @@ def run_case(args):
             D = torch.empty((r, c), dtype=torch.float32, device="cuda")
             fn = lambda: B.nvfp4_gemm_bf16(a, b, D, B.MN_MAJOR, B.MN_MAJOR)
         work, unit = 2.0 * r * c * k / 1e12, "TFLOP/s"
+    elif kind in ("q_rows", "q_rows_sr"):
+        x = torch.randn((r, c), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        row = B.alloc_tensor(r, c, format=B.FORMAT_NVFP4_ROWSCALE)
+        o = B.quant_opts(rounding=B.ROUND_STOCHASTIC if kind == "q_rows_sr" else B.ROUND_NEAREST_EVEN, seed=1)
+        fn = lambda: B.nvfp4_quantize(x, o, row, None)
+        work, unit = r * c * 2.5625 / 1e9, "GB/s"
     elif kind == "qerr":
         x = torch.randn((r, c), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
         q = B.alloc_tensor(r, c)

@@ -52,8 +52,13 @@ enum { NVFP4_SF_LINEAR = 0, NVFP4_SF_SWIZZLED = 1 };
    format the paper compares against (Section 2, Section 5, Appendix B.4): E2M1 elements with one UE8M0
    power-of-two scale per 32 elements, the decode scale amax_b / 6 rounded UP to a power of two, no
    tensor-level scale (global = {0, 1}), transform size 32 on the weight-gradient operands, 32x32 blocks
-   for weights. */
-enum { NVFP4_FORMAT_NVFP4 = 0, NVFP4_FORMAT_MXFP4 = 1 };
+   for weights.
+   NVFP4_ROWSCALE is NVFP4 with the FP32 "global" scale taken per ROW of the copy instead of per tensor (the
+   closing remark of Appendix B.1: a global scale spanning a row avoids the extra pass through device memory
+   that the tensor amax costs): global holds rows pairs {amax of the row, s_dec of the row}, Eq. 1 per row,
+   Eq. 2-4 unchanged.  Row-wise copies only; nvfp4_quantize makes them in ONE pass and nvfp4_gemm applies the
+   vectors in its epilogue (D[i][j] = s_dec^A[i] * s_dec^B[j] * sum ...). */
+enum { NVFP4_FORMAT_NVFP4 = 0, NVFP4_FORMAT_MXFP4 = 1, NVFP4_FORMAT_NVFP4_ROWSCALE = 2 };
 enum {
   /* the column-wise copy draws its stochastic-rounding bits from a second stream (bit 63 of
      sr_offset set) instead of sharing the draw of the same source element with the row-wise copy */
@@ -87,7 +92,8 @@ typedef struct nvfp4_tensor {
   int32_t sf_layout;
   int32_t format;   /* NVFP4_FORMAT_NVFP4 (0) or NVFP4_FORMAT_MXFP4; MXFP4: scales hold rows * cols/32 UE8M0
                        bytes (byte b = 2^(b-127)), same two layouts with 32-element blocks (swizzled needs
-                       cols % 128 == 0), global is written as {0, 1} and not used */
+                       cols % 128 == 0), global is written as {0, 1} and not used;
+                       NVFP4_FORMAT_NVFP4_ROWSCALE: global is float[2 * rows] */
 } nvfp4_tensor;
 
 /*
@@ -129,6 +135,8 @@ typedef struct nvfp4_quant_opts {
  *             colwise->rows == cols, colwise->cols == rows.
  *   At least one copy must be requested.  With block_rows == 16 both copies hold the same
  *   quantized values (transposed) and no Hadamard transform is allowed.
+ *   rowwise->format == NVFP4_FORMAT_NVFP4_ROWSCALE: one pass, colwise must be NULL, block_rows 1, no transform,
+ *   bf16 source; rowwise->global receives 2 * rows floats.
  * Two passes over x: a tensor-amax reduction (in the rotated space for a transformed copy),
  * then transform + scale + round + pack.  Stochastic rounding rounds up iff
  * u + 0.5 < 256 * frac, u = the 8-bit Philox draw of the source position, frac = the position of
@@ -150,7 +158,8 @@ NVFP4_API nvfp4_status nvfp4_quantize(const void* x_bf16, int64_t rows, int64_t 
  *   accumulate != 0 adds the product to the existing contents of an fp32 D (gradient accumulation,
  *   Section 4.1); it is rejected for bf16 outputs.
  *   Both operands must have the same format (MXFP4 operands carry no tensor-level scale and power-of-two
- *   block scales per 32 elements).
+ *   block scales per 32 elements); an NVFP4_ROWSCALE operand combines with an NVFP4 or another NVFP4_ROWSCALE
+ *   operand and needs M % 256 == 0 and N % 256 == 0 (the scale vectors are applied by the CTA-pair kernel).
  */
 NVFP4_API nvfp4_status nvfp4_gemm(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D,
                                   int32_t d_is_fp32, int64_t ldd, int32_t accumulate,

@@ -18,7 +18,7 @@ OK = 0
 ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
 SF_LINEAR, SF_SWIZZLED = 0, 1
 SR_INDEPENDENT_COPIES, AMAX_PROVIDED, INPUT_FP32 = 1, 2, 4
-FORMAT_NVFP4, FORMAT_MXFP4 = 0, 1
+FORMAT_NVFP4, FORMAT_MXFP4, FORMAT_NVFP4_ROWSCALE = 0, 1, 2
 
 EXPORTED = (
     "nvfp4_quantize", "nvfp4_gemm", "nvfp4_linear_fwd_workspace_bytes", "nvfp4_linear_bwd_workspace_bytes",
@@ -123,7 +123,7 @@ class NVFP4Tensor:
 def alloc_tensor(rows: int, cols: int, sf_layout: int = SF_SWIZZLED, device="cuda",
                  format: int = FORMAT_NVFP4) -> NVFP4Tensor:
     block = 32 if format == FORMAT_MXFP4 else 16
-    glob = torch.zeros((2,), dtype=torch.float32, device=device)
+    glob = torch.zeros((2 * rows if format == FORMAT_NVFP4_ROWSCALE else 2,), dtype=torch.float32, device=device)
     if format == FORMAT_MXFP4:
         glob[1] = 1.0
     return NVFP4Tensor(torch.empty((rows, cols // 2), dtype=torch.uint8, device=device),

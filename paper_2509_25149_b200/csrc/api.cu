@@ -27,7 +27,8 @@ nvfp4_status check_copy(const nvfp4_tensor* t, int64_t rows, int64_t cols) {
   if (!t->codes || !t->scales || !t->global) return NVFP4_ERR_NULL;
   if (t->rows != rows || t->cols != cols) return NVFP4_ERR_SHAPE;
   if (t->sf_layout != NVFP4_SF_LINEAR && t->sf_layout != NVFP4_SF_SWIZZLED) return NVFP4_ERR_ARG;
-  if (t->format != NVFP4_FORMAT_NVFP4 && t->format != NVFP4_FORMAT_MXFP4) return NVFP4_ERR_ARG;
+  if (t->format != NVFP4_FORMAT_NVFP4 && t->format != NVFP4_FORMAT_MXFP4 && t->format != NVFP4_FORMAT_NVFP4_ROWSCALE)
+    return NVFP4_ERR_ARG;
   const int64_t atom_cols = t->format == NVFP4_FORMAT_MXFP4 ? 128 : 64;  // four blocks of 32 / 16 elements
   if (t->sf_layout == NVFP4_SF_SWIZZLED && (rows % 128 != 0 || cols % atom_cols != 0)) return NVFP4_ERR_SHAPE;
   if (!aligned(t->codes, 16) || !aligned(t->scales, 16) || !aligned(t->global, 8)) return NVFP4_ERR_ALIGN;
@@ -42,6 +43,29 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
   if (ld < cols) return NVFP4_ERR_SHAPE;
   if (ld % 16 != 0 || !aligned(x, 32)) return NVFP4_ERR_ALIGN;
   const int32_t fmt = rowwise ? rowwise->format : colwise->format;
+  if (fmt == NVFP4_FORMAT_NVFP4_ROWSCALE) {
+    // one pass, row-wise copy only (a scale per row of the transposed copy would be a statistic over all source rows)
+    if (colwise) return NVFP4_ERR_ARG;
+    if (o->block_rows != 1 || o->rht_rowwise || o->rht_colwise) return NVFP4_ERR_ARG;
+    if (o->rounding != NVFP4_ROUND_NEAREST_EVEN && o->rounding != NVFP4_ROUND_STOCHASTIC) return NVFP4_ERR_ARG;
+    if (o->flags & ~NVFP4_SR_INDEPENDENT_COPIES) return NVFP4_ERR_ARG;
+    if (rows > (int64_t)1 << 30 || cols > (int64_t)1 << 30) return NVFP4_ERR_SHAPE;
+    nvfp4_status st0 = check_copy(rowwise, rows, cols);
+    if (st0 != NVFP4_OK) return st0;
+    QuantArgs a{};
+    a.x = static_cast<const uint16_t*>(x);
+    a.rows = rows; a.cols = cols; a.ld = ld;
+    a.r_codes = rowwise->codes; a.r_scales = rowwise->scales; a.r_global = rowwise->global;
+    a.r_swz = rowwise->sf_layout == NVFP4_SF_SWIZZLED;
+    a.seed_lo = (uint32_t)o->seed; a.seed_hi = (uint32_t)(o->seed >> 32);
+    for (uint32_t r = 0; r < 10; ++r) {  // Philox key schedule
+      a.rk[2 * r] = a.seed_lo + r * 0x9E3779B9u;
+      a.rk[2 * r + 1] = a.seed_hi + r * 0xBB67AE85u;
+    }
+    a.off_lo = (uint32_t)o->sr_offset; a.off_hi = (uint32_t)(o->sr_offset >> 32);
+    return launch_quantize_rowscale(a, o->rounding == NVFP4_ROUND_STOCHASTIC, s) == cudaSuccess ? NVFP4_OK
+                                                                                                  : NVFP4_ERR_CUDA;
+  }
   if (fmt != NVFP4_FORMAT_NVFP4 && fmt != NVFP4_FORMAT_MXFP4) return NVFP4_ERR_ARG;
   if (rowwise && colwise && rowwise->format != colwise->format) return NVFP4_ERR_ARG;
   const bool mx = fmt == NVFP4_FORMAT_MXFP4;
@@ -133,8 +157,11 @@ nvfp4_status gemm_prepare(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D,
   if (M <= 0 || N <= 0 || K <= 0 || M % 128 != 0 || N % 128 != 0 || K % 256 != 0) return NVFP4_ERR_SHAPE;
   if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff || (M / 128) * (N / 128) > 0x7fffffff) return NVFP4_ERR_SHAPE;
   if (A->sf_layout != NVFP4_SF_SWIZZLED || B->sf_layout != NVFP4_SF_SWIZZLED) return NVFP4_ERR_ARG;
-  if (A->format != B->format) return NVFP4_ERR_ARG;
-  if (A->format != NVFP4_FORMAT_NVFP4 && A->format != NVFP4_FORMAT_MXFP4) return NVFP4_ERR_ARG;
+  const bool a_rs = A->format == NVFP4_FORMAT_NVFP4_ROWSCALE, b_rs = B->format == NVFP4_FORMAT_NVFP4_ROWSCALE;
+  // a row-scaled NVFP4 operand mixes with a tensor-scaled one; MXFP4 only with MXFP4
+  if ((a_rs ? NVFP4_FORMAT_NVFP4 : A->format) != (b_rs ? NVFP4_FORMAT_NVFP4 : B->format)) return NVFP4_ERR_ARG;
+  if (!a_rs && A->format != NVFP4_FORMAT_NVFP4 && A->format != NVFP4_FORMAT_MXFP4) return NVFP4_ERR_ARG;
+  if ((a_rs || b_rs) && (M % 256 != 0 || N % 256 != 0)) return NVFP4_ERR_SHAPE;
   if (accumulate && !d_is_fp32) return NVFP4_ERR_ARG;
   if (ldd < N) return NVFP4_ERR_SHAPE;
   const int64_t esz = d_is_fp32 ? 4 : 2;
@@ -148,6 +175,8 @@ nvfp4_status gemm_prepare(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D,
   g.M = (int)M; g.N = (int)N; g.K = (int)K;
   g.d_is_fp32 = d_is_fp32 != 0; g.accumulate = accumulate != 0;
   g.mx = A->format == NVFP4_FORMAT_MXFP4;
+  g.a_rows = a_rs ? A->global : nullptr;
+  g.b_rows = b_rs ? B->global : nullptr;
   return NVFP4_OK;
 }
 
@@ -231,6 +260,7 @@ nvfp4_status nvfp4_linear_fwd(const void* X, const void* W, int64_t M, int64_t N
   if (W_row->sf_layout != NVFP4_SF_SWIZZLED) return NVFP4_ERR_ARG;
   // the format of the layer is the format of its weight copy (MXFP4: 32-element blocks, transform size 32)
   const int32_t fmt = W_row->format;
+  if (fmt != NVFP4_FORMAT_NVFP4 && fmt != NVFP4_FORMAT_MXFP4) return NVFP4_ERR_ARG;  // per-tensor scales only
   if ((W_col_saved && W_col_saved->format != fmt) || (X_col_saved && X_col_saved->format != fmt)) return NVFP4_ERR_ARG;
 
   if (!w_is_cached) {
@@ -267,6 +297,7 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, c
   if (X_col_saved && (st = check_copy(X_col_saved, K, M)) != NVFP4_OK) return st;
 
   const int32_t fmt = W_col_saved ? W_col_saved->format : X_col_saved->format;
+  if (fmt != NVFP4_FORMAT_NVFP4 && fmt != NVFP4_FORMAT_MXFP4) return NVFP4_ERR_ARG;  // per-tensor scales only
   if (W_col_saved && X_col_saved && W_col_saved->format != X_col_saved->format) return NVFP4_ERR_ARG;
   uint8_t* p = static_cast<uint8_t*>(workspace);
   nvfp4_tensor g_row = carve(p, M, N, fmt);

@@ -356,7 +356,7 @@ bool make_pair_maps(const GemmArgs& g, const void* a_codes, const void* b_codes,
 }
 
 pair::Problem pair_problem(const GemmArgs& g) {
-  return pair::Problem{g.M, g.N, g.K, g.sfa, g.sfb, g.a_global, g.b_global, g.d_is_fp32, g.accumulate};
+  return pair::Problem{g.M, g.N, g.K, g.sfa, g.sfb, g.a_global, g.b_global, g.d_is_fp32, g.accumulate, g.a_rows, g.b_rows};
 }
 
 // g1 == nullptr: one problem
@@ -388,10 +388,22 @@ cudaError_t launch_pair(const GemmArgs& g0, const void* a0, const void* b0, cons
   a.n_tiles = a.n_tiles0 + (g1 ? (g1->M / 256) * (g1->N / 256) : 0);
   const int max_pairs = num_sms / 2;
   const int pairs = a.n_tiles < max_pairs ? a.n_tiles : max_pairs;
-  if (g0.mx)
+  const bool rows = a.p[0].a_rows || a.p[0].b_rows || a.p[1].a_rows || a.p[1].b_rows;
+  if (rows) {
+    if (g0.mx) return cudaErrorInvalidValue;
+    static std::atomic<uint64_t> configured_rows{0};
+    if (device_needs_config(configured_rows, &dev)) {
+      cudaError_t e = cudaFuncSetAttribute(pair::gemm_pair_kernel<false, true>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, pair::kSmemBytes);
+      if (e != cudaSuccess) return e;
+      device_configured(configured_rows, dev);
+    }
+    pair::gemm_pair_kernel<false, true><<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5], a);
+  } else if (g0.mx) {
     pair::gemm_pair_kernel<true><<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5], a);
-  else
+  } else {
     pair::gemm_pair_kernel<false><<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5], a);
+  }
   count_launch();
   return cudaGetLastError();
 }
@@ -523,6 +535,10 @@ cudaError_t launch_gemm(const GemmArgs& g, const void* a_codes, const void* b_co
   int num_sms = 0;
   cudaError_t e = sm_count(&num_sms);
   if (e != cudaSuccess) return e;
+  if (g.a_rows || g.b_rows) {  // scale vectors are applied by the 256 x 256 pair kernel's epilogue only
+    if (g.M % 256 != 0 || g.N % 256 != 0) return cudaErrorInvalidValue;
+    return launch_pair(g, a_codes, b_codes, nullptr, nullptr, nullptr, num_sms, s);
+  }
   if (tile_n == 768 && wide_eligible(g)) return launch_wide(g, a_codes, b_codes, nullptr, nullptr, nullptr, num_sms, s);
   if ((tile_n == 512 || tile_n == 768) && g.M % 256 == 0 && g.N % 256 == 0)
     return launch_pair(g, a_codes, b_codes, nullptr, nullptr, nullptr, num_sms, s);

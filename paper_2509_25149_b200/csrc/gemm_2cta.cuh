@@ -28,7 +28,8 @@ constexpr int kSfaBytes = 4 * 512;   // own 128 rows, four K64 steps
 constexpr int kSfbBytes = 8 * 512;   // all 256 rows of B (both CTAs need them), four K64 steps
 constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 38 KB
 constexpr int kStagingBytes = 2 * 16384;  // one 128 x 128-byte store buffer per epilogue group
-constexpr int kSmemBytes = kStages * kStageBytes + kStagingBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+constexpr int kBetaBytes = 2 * 128 * 4;   // column scales of the tile, one half per epilogue group (row-scaled B)
+constexpr int kSmemBytes = kStages * kStageBytes + kStagingBytes + 1024 /*alignment*/ + 256 /*barriers*/ + kBetaBytes;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSfCol = 256;          // after the 256 accumulator columns: one 48-column slot per stage
 constexpr int kSfSlotCols = 48;      // SFA 4 x 4, SFB 4 x 8
@@ -42,6 +43,10 @@ struct Problem {
   const float* a_global;
   const float* b_global;
   int d_is_fp32, accumulate;
+  // Global scale per row instead of per tensor (Appendix B.1, closing remark): {amax, s_dec} pairs, one per row of
+  // the operand; NULL = the operand carries the usual per-tensor words in a_global / b_global
+  const float* a_rows;
+  const float* b_rows;
 };
 // One launch works through the tiles of up to two independent GEMMs (problem 0 first): Dgrad and Wgrad of a
 // linear layer share no output, so their tiles can fill the same persistent grid and the partial last round of
@@ -180,10 +185,11 @@ __device__ __forceinline__ void tc2_mma_mxf4(uint32_t d_tmem, uint64_t adesc, ui
 // Epilogue helper: 128 accumulator columns of one row per thread (registers) -> alpha, conversion -> 128-byte
 // swizzled rows of a staging buffer -> TMA store (or reduce-add) of 128 x 128-byte boxes.  Two staging buffers
 // alternate; a buffer is rewritten only after the store issued two boxes earlier has finished reading it.
-template <bool FP32>
+// BETA: the 128 columns additionally carry their own factors (float[128] in shared memory at `beta`).
+template <bool FP32, bool BETA = false>
 __device__ __forceinline__ void store_half(const uint32_t (&r)[128], float alpha, int et, int bar_id, int row_in_tile,
                                            uint32_t stage_buf, int& buf, const CUtensorMap* map_d, int x0, int row0,
-                                           int accumulate) {
+                                           int accumulate, const float* beta = nullptr) {
   constexpr int kChunks = FP32 ? 4 : 2;
   constexpr int kChunkCols = FP32 ? 32 : 64;
 #pragma unroll
@@ -196,12 +202,21 @@ __device__ __forceinline__ void store_half(const uint32_t (&r)[128], float alpha
       uint32_t p[4];
       if (FP32) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) p[e] = __float_as_uint(__uint_as_float(r[c * 32 + 4 * j + e]) * alpha);
+        for (int e = 0; e < 4; ++e) {
+          float v = __uint_as_float(r[c * 32 + 4 * j + e]) * alpha;
+          if (BETA) v *= beta[c * 32 + 4 * j + e];
+          p[e] = __float_as_uint(v);
+        }
       } else {
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[c * 64 + 8 * j + 2 * e]) * alpha,
-                                                   __uint_as_float(r[c * 64 + 8 * j + 2 * e + 1]) * alpha);
+          float v0 = __uint_as_float(r[c * 64 + 8 * j + 2 * e]) * alpha;
+          float v1 = __uint_as_float(r[c * 64 + 8 * j + 2 * e + 1]) * alpha;
+          if (BETA) {
+            v0 *= beta[c * 64 + 8 * j + 2 * e];
+            v1 *= beta[c * 64 + 8 * j + 2 * e + 1];
+          }
+          __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
           p[e] = *reinterpret_cast<uint32_t*>(&h);
         }
       }
@@ -225,7 +240,10 @@ __device__ __forceinline__ void store_half(const uint32_t (&r)[128], float alpha
 // MX = false: NVFP4 (E4M3 scale per 16 elements: one 512-byte atom per 128 rows and K = 64).
 // MX = true : MXFP4 (UE8M0 scale per 32 elements: one atom per 128 rows and K = 128, so half the atoms, the same
 //             slots in shared and tensor memory half used, and the byte pair picked by the instruction descriptor).
-template <bool MX>
+// ROWS = true: at least one operand carries its global scale per row (a_rows / b_rows); the epilogue then applies a
+// factor per output row and / or per output column.  A separate instantiation so that the common kernel keeps its
+// register budget.
+template <bool MX, bool ROWS = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_b0,
                      const __grid_constant__ CUtensorMap map_d0, const __grid_constant__ CUtensorMap map_a1,
@@ -444,8 +462,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     const int et = (threadIdx.x - 96) & 127;  // 0..127 inside the group
     const int bar_id = 1 + half;
     uint32_t acc_phase = 0;
-    const float alpha0 = __fmul_rn(g.p[0].a_global[1], g.p[0].b_global[1]);
-    const float alpha1 = __fmul_rn(g.p[1].a_global[1], g.p[1].b_global[1]);
+    // per-tensor decode scales; an operand with per-row scales contributes 1 here and its vector below
+    const float alpha0 = __fmul_rn((ROWS && g.p[0].a_rows) ? 1.f : g.p[0].a_global[1], (ROWS && g.p[0].b_rows) ? 1.f : g.p[0].b_global[1]);
+    const float alpha1 = __fmul_rn((ROWS && g.p[1].a_rows) ? 1.f : g.p[1].a_global[1], (ROWS && g.p[1].b_rows) ? 1.f : g.p[1].b_global[1]);
+    float* beta = reinterpret_cast<float*>(base_ptr + kStages * kStageBytes + kStagingBytes + 256) + half * 128;
     const uint32_t acce_leader = map_to_cta(acce_bar, 0);
     const int row_in_tile = quad * 32 + lane;
     const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + half * 128;
@@ -455,8 +475,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       int prob, m_blk, n_blk;
       tile_coords(tile, prob, m_blk, n_blk);
       const CUtensorMap* map_d = prob ? &map_d1 : &map_d0;
-      const float alpha = prob ? alpha1 : alpha0;
+      float alpha = prob ? alpha1 : alpha0;
       const int d_is_fp32 = g.p[prob].d_is_fp32, accumulate = g.p[prob].accumulate;
+      const float* a_rows = ROWS ? g.p[prob].a_rows : nullptr;
+      const float* b_rows = ROWS ? g.p[prob].b_rows : nullptr;
+      if (a_rows) alpha *= a_rows[2 * (int64_t)(m_blk * 256 + (int)rank * 128 + quad * 32 + lane) + 1];
+      // the group's 128 column factors; the first barrier inside store_half orders this write before their use, its
+      // last one orders their use before the next tile's write
+      if (b_rows) beta[et] = b_rows[2 * (int64_t)(n_blk * 256 + half * 128 + et) + 1];
       mbar_wait_cluster(accf_bar, acc_phase, abort_flag, 0x400u);
       // agree on giving up: a warp that timed out still joins this barrier, then everyone reads the flag
       asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
@@ -472,12 +498,20 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(acce_leader);
-      if (d_is_fp32)
+      if (ROWS && b_rows) {
+        if (d_is_fp32)
+          store_half<true, true>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, map_d, n_blk * 256 + half * 128,
+                                 row0, accumulate, beta);
+        else
+          store_half<false, true>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, map_d, n_blk * 256 + half * 128,
+                                  row0, accumulate, beta);
+      } else if (d_is_fp32) {
         store_half<true>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, map_d, n_blk * 256 + half * 128, row0,
                          accumulate);
-      else
+      } else {
         store_half<false>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, map_d, n_blk * 256 + half * 128, row0,
                           accumulate);
+      }
       acc_phase ^= 1u;
     }
     if (et == 0) bulk_wait_all<0>();  // all stores have left shared memory and are visible

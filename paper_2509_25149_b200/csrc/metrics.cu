@@ -67,11 +67,11 @@ __global__ void __launch_bounds__(256) quant_error_kernel(const uint16_t* __rest
                                                           int64_t ld, const uint8_t* __restrict__ codes,
                                                           const uint8_t* __restrict__ scales,
                                                           const float* __restrict__ global, int swz,
-                                                          double* __restrict__ out) {
+                                                          int per_row, double* __restrict__ out) {
   const int64_t n_cb = cols >> 4;                 // 16-element chunks per row
   const int64_t n_sb = MX ? (cols >> 5) : n_cb;   // scale blocks per row
   const int64_t n_chunks = rows * n_cb;
-  const float s_dec = MX ? 1.f : global[1];
+  const float s_dec_t = MX ? 1.f : global[1];
   double err = 0.0, ref = 0.0;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n_chunks; i += (int64_t)gridDim.x * blockDim.x) {
     int64_t r, cb;
@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(256) quant_error_kernel(const uint16_t* __rest
       asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)byte));
       sf = __half2float(__ushort_as_half((unsigned short)(h2 & 0xffffu)));
     }
-    const float scale = __fmul_rn(sf, s_dec);
+    const float scale = __fmul_rn(sf, per_row ? global[2 * r + 1] : s_dec_t);  // per_row: {amax, s_dec} per row
     float e = 0.f, n = 0.f;
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
@@ -167,10 +167,10 @@ cudaError_t launch_quant_error(const void* x, int64_t rows, int64_t cols, int64_
   const int swz = q.sf_layout == NVFP4_SF_SWIZZLED;
   if (q.format == NVFP4_FORMAT_MXFP4)
     quant_error_kernel<true><<<grid, 256, 0, s>>>(static_cast<const uint16_t*>(x), rows, cols, ld, q.codes, q.scales,
-                                                  q.global, swz, out);
+                                                  q.global, swz, 0, out);
   else
     quant_error_kernel<false><<<grid, 256, 0, s>>>(static_cast<const uint16_t*>(x), rows, cols, ld, q.codes, q.scales,
-                                                   q.global, swz, out);
+                                                   q.global, swz, q.format == NVFP4_FORMAT_NVFP4_ROWSCALE, out);
   count_launch();
   return cudaGetLastError();
 }

@@ -564,9 +564,9 @@ __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const Qu
 // ---------------------------------------------------------------------------------------------
 __global__ void dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ scales,
                                   const float* __restrict__ global, int64_t rows, int64_t cols, int swz,
-                                  int mx, float* __restrict__ out) {
+                                  int mx, int per_row, float* __restrict__ out) {
   const int64_t n = rows * cols;
-  const float s_dec = global[1];
+  const float s_dec_t = global[1];
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / cols, c = i % cols;
     const uint32_t byte = codes[r * (cols >> 1) + (c >> 1)];
@@ -585,7 +585,7 @@ __global__ void dequantize_kernel(const uint8_t* __restrict__ codes, const uint8
       asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(sb));
       sf = __half2float(__ushort_as_half((unsigned short)(h2 & 0xffffu)));
     }
-    out[i] = __fmul_rn(__fmul_rn(m, sf), s_dec);
+    out[i] = __fmul_rn(__fmul_rn(m, sf), per_row ? global[2 * r + 1] : s_dec_t);
   }
 }
 
@@ -725,7 +725,8 @@ cudaError_t launch_quantize(const QuantArgs& a, bool has_row, bool has_col, bool
 
 cudaError_t launch_dequantize(const nvfp4_tensor& t, float* out, cudaStream_t s) {
   dequantize_kernel<<<1184, 256, 0, s>>>(t.codes, t.scales, t.global, t.rows, t.cols,
-                                         t.sf_layout == NVFP4_SF_SWIZZLED, t.format == NVFP4_FORMAT_MXFP4, out);
+                                         t.sf_layout == NVFP4_SF_SWIZZLED, t.format == NVFP4_FORMAT_MXFP4,
+                                         t.format == NVFP4_FORMAT_NVFP4_ROWSCALE, out);
   count_launch();
   return cudaGetLastError();
 }

@@ -50,6 +50,8 @@ cudaError_t launch_dequantize(const nvfp4_tensor& t, float* out, cudaStream_t s)
 cudaError_t launch_rht16(const void* x, int64_t rows, int64_t cols, int64_t ld, int colwise, uint32_t mask,
                          float* out, cudaStream_t s);
 
+// quantize_rowscale.cu: row-wise copy with {amax, s_dec} per row in a.r_global[2 * rows], one pass
+cudaError_t launch_quantize_rowscale(const QuantArgs& a, bool sr, cudaStream_t s);
 // metrics.cu: out = {sum (x - decode(q))^2, sum x^2} of a row-wise copy; {sum (ref - test)^2, sum ref^2} of two tensors
 cudaError_t launch_quant_error(const void* x, int64_t rows, int64_t cols, int64_t ld, const nvfp4_tensor& q,
                                double* out, cudaStream_t s);
