@@ -17,7 +17,7 @@ from . import build as _build
 OK = 0
 ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
 SF_LINEAR, SF_SWIZZLED = 0, 1
-SR_INDEPENDENT_COPIES, AMAX_PROVIDED, INPUT_FP32 = 1, 2, 4
+SR_INDEPENDENT_COPIES, AMAX_PROVIDED, INPUT_FP32, LINEAR_ROW_SCALES = 1, 2, 4, 8
 FORMAT_NVFP4, FORMAT_MXFP4, FORMAT_NVFP4_ROWSCALE = 0, 1, 2
 
 EXPORTED = (
@@ -148,7 +148,7 @@ def nvfp4_quantize(x: torch.Tensor, opts: CQuantOpts, rowwise: Optional[NVFP4Ten
     assert x.is_cuda and x.dtype in (torch.bfloat16, torch.float32) and x.dim() == 2 and x.stride(1) == 1
     if x.dtype == torch.float32 and not (opts.flags & INPUT_FP32):  # a binary32 source is announced by a flag
         opts = CQuantOpts(opts.block_rows, opts.rounding, opts.rht_rowwise, opts.rht_colwise, opts.rht_sign_mask,
-                          opts.flags | INPUT_FP32, opts.seed, opts.sr_offset)
+                          opts.flags | INPUT_FP32, opts.seed, opts.sr_offset, opts.rht_dim, opts.rht_sign_mask_ext)
     assert (x.dtype == torch.float32) == bool(opts.flags & INPUT_FP32)
     _check(lib().nvfp4_quantize(x.data_ptr(), x.shape[0], x.shape[1], x.stride(0), ctypes.byref(opts), _ref(rowwise),
                                 _ref(colwise), _stream()), "nvfp4_quantize")

@@ -212,6 +212,11 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline size_t copy_bytes(int64_t rows, int64_t cols) {
   return align_up((size_t)(rows * cols / 2), 256) + align_up((size_t)(rows * cols / 16), 256) + 256;
 }
+// the same with room for {amax, s_dec} per row (forward-only calls with row scales)
+inline size_t copy_bytes_rows(int64_t rows, int64_t cols) {
+  return align_up((size_t)(rows * cols / 2), 256) + align_up((size_t)(rows * cols / 16), 256) +
+         align_up((size_t)rows * 8, 256);
+}
 // carve one swizzled-scale copy [rows x cols] out of a workspace
 nvfp4_tensor carve(uint8_t*& p, int64_t rows, int64_t cols, int32_t format = NVFP4_FORMAT_NVFP4) {
   nvfp4_tensor t{};
@@ -240,7 +245,7 @@ nvfp4_status nvfp4_gemm(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D, i
   return gemm_impl(A, B, D, d_is_fp32, ldd, accumulate, static_cast<cudaStream_t>(cuda_stream));
 }
 
-size_t nvfp4_linear_fwd_workspace_bytes(int64_t M, int64_t K) { return copy_bytes(M, K); }
+size_t nvfp4_linear_fwd_workspace_bytes(int64_t M, int64_t K) { return copy_bytes_rows(M, K); }
 size_t nvfp4_linear_bwd_workspace_bytes(int64_t M, int64_t N) { return 2 * copy_bytes(M, N); }
 
 nvfp4_status nvfp4_linear_fwd(const void* X, const void* W, int64_t M, int64_t N, int64_t K,
@@ -270,6 +275,24 @@ nvfp4_status nvfp4_linear_fwd(const void* X, const void* W, int64_t M, int64_t N
     if ((st = quantize_impl(W, N, K, K, &wo, W_row, W_col_saved, s)) != NVFP4_OK) return st;
   }
   uint8_t* p = static_cast<uint8_t*>(workspace);
+  if (opts->flags & NVFP4_LINEAR_ROW_SCALES) {
+    // forward-only call: X gets a global scale per row in one pass (Appendix B.1, closing remark) and Fprop applies
+    // the vector in its epilogue.  No transposed copy can be made this way, so none may be requested.
+    if (X_col_saved || fmt != NVFP4_FORMAT_NVFP4) return NVFP4_ERR_ARG;
+    nvfp4_tensor x_rows{};
+    x_rows.codes = p;
+    p += align_up((size_t)(M * K / 2), 256);
+    x_rows.scales = p;
+    p += align_up((size_t)(M * K / 16), 256);
+    x_rows.global = reinterpret_cast<float*>(p);
+    x_rows.rows = M; x_rows.cols = K; x_rows.sf_layout = NVFP4_SF_SWIZZLED;
+    x_rows.format = NVFP4_FORMAT_NVFP4_ROWSCALE;
+    nvfp4_quant_opts ro{};
+    ro.block_rows = 1;
+    ro.rounding = NVFP4_ROUND_NEAREST_EVEN;
+    if ((st = quantize_impl(X, M, K, K, &ro, &x_rows, nullptr, s)) != NVFP4_OK) return st;
+    return gemm_impl(&x_rows, W_row, Y_bf16, 0, N, 0, s);
+  }
   nvfp4_tensor x_row = carve(p, M, K, fmt);
   nvfp4_quant_opts xo{};
   xo.block_rows = 1;

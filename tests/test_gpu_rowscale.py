@@ -115,3 +115,24 @@ def test_row_scales_keep_small_rows_alive_next_to_an_outlier_row_and_metric_agre
     err_rows = np.abs(dec - xf)[small].max()
     err_tensor = np.abs(B.nvfp4_dequantize(t_tensor).cpu().numpy() - xf)[small].max()
     assert err_rows < 0.2 * np.abs(xf[small]).max() and err_tensor == np.abs(xf[small]).max()
+
+
+def test_forward_only_layer_with_row_scaled_activations():
+    """nvfp4_linear_fwd with NVFP4_LINEAR_ROW_SCALES: X quantized in one pass with a scale per token, W with 16x16
+    blocks and its tensor scale, Fprop applying the token vector in its epilogue."""
+    M, N, K = 512, 768, 1024
+    x = synth.normal_with_outliers_bf16((M, K), 0.01, 40.0, 51, 52)
+    x[::5] *= 100.0
+    w = synth.normal_bf16((N, K), 0.02, 53)
+    W_row = B.alloc_tensor(N, K)
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(B.nvfp4_linear_fwd_workspace_bytes(M, K), dtype=torch.uint8, device="cuda")
+    o = B.quant_opts(flags=B.LINEAR_ROW_SCALES)
+    B.nvfp4_linear_fwd(x.cuda(), w.cuda(), o, Y, None, W_row, None, False, ws)
+    B.nvfp4_device_status()
+    qa = oracle.quantize_rowscale(synth.bits(x))
+    qb = oracle.quantize(synth.bits(w), block_rows=16)
+    Dref, T = oracle.gemm_tn(oracle.dequantize_rowscale(qa), oracle.dequantize(qb))
+    P.assert_gemm_close(Y.float().cpu().numpy(), Dref, T, True, "forward-only layer")
+    with pytest.raises(B.NVFP4Error):  # a saved transposed copy cannot be made with row scales
+        B.nvfp4_linear_fwd(x.cuda(), w.cuda(), o, Y, B.alloc_tensor(K, M), W_row, None, False, ws)
