@@ -226,7 +226,8 @@ NVFP4_API nvfp4_status nvfp4_sq_error(const void* ref, int32_t ref_is_fp32, int6
  * nvfp4_linear_fwd: Y = X W^T (bf16).  Quantizes X row-wise (1x16, RNE) for Fprop and, when
  *   X_col_saved is given, column-wise with the Hadamard transform for the later Wgrad; quantizes W
  *   with 16x16 blocks into W_row (Fprop) and W_col_saved (Dgrad) unless w_is_cached != 0, in which
- *   case W_row must already hold the quantized weight.  opts supplies rht_sign_mask, and the flag
+ *   case W_row must already hold the quantized weight.  opts supplies rht_sign_mask (and rht_dim, when another
+ *   transform size than the format's own is wanted: the same value must then be given to nvfp4_linear_bwd), and the flag
  *   NVFP4_LINEAR_ROW_SCALES for forward-only calls (then X_col_saved must be NULL).
  *   workspace: device scratch of nvfp4_linear_fwd_workspace_bytes(M, K) for the row-wise copy of X.
  * nvfp4_linear_bwd: dX = dY W (bf16), dW = dY^T X (fp32).  Quantizes dY with stochastic rounding

@@ -299,6 +299,8 @@ nvfp4_status nvfp4_linear_fwd(const void* X, const void* W, int64_t M, int64_t N
   xo.rounding = NVFP4_ROUND_NEAREST_EVEN;
   xo.rht_colwise = 1;
   xo.rht_sign_mask = opts->rht_sign_mask;
+  xo.rht_dim = opts->rht_dim;  // 0 = the format's own size; Appendix E.4.2's other sizes pass through
+  for (int i = 0; i < 3; ++i) xo.rht_sign_mask_ext[i] = opts->rht_sign_mask_ext[i];
   if ((st = quantize_impl(X, M, K, K, &xo, &x_row, X_col_saved, s)) != NVFP4_OK) return st;
   return gemm_impl(&x_row, W_row, Y_bf16, 0, N, 0, s);
 }
@@ -330,6 +332,8 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, c
   go.rounding = NVFP4_ROUND_STOCHASTIC;
   go.rht_colwise = 1;
   go.rht_sign_mask = opts->rht_sign_mask;
+  go.rht_dim = opts->rht_dim;
+  for (int i = 0; i < 3; ++i) go.rht_sign_mask_ext[i] = opts->rht_sign_mask_ext[i];
   go.seed = opts->seed;
   go.sr_offset = opts->sr_offset;
   go.flags = opts->flags & NVFP4_SR_INDEPENDENT_COPIES;

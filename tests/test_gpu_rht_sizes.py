@@ -99,3 +99,35 @@ def test_larger_transform_lowers_the_rotated_amax_and_the_gemm_still_cancels():
         rel = np.linalg.norm(dW.cpu().numpy() - ref) / np.linalg.norm(ref)
         assert rel < 0.25, (d, rel)  # FP4 noise only: a transform that did not cancel would give rel ~ 1
     assert amax[128] < amax[4]
+
+
+@pytest.mark.parametrize("d", [4, 128])
+def test_linear_layer_with_another_transform_size(d):
+    """nvfp4_linear_fwd / _bwd pass rht_dim through to both Wgrad operands: dW must match the product of the
+    oracle's operands made with the same size (and would be far off if only one side used it)."""
+    M, N, K = 256, 256, 256
+    x = synth.normal_with_outliers_bf16((M, K), 0.01, 20.0, 71, 72)
+    w = synth.normal_bf16((N, K), 0.02, 73)
+    dy = synth.normal_bf16((M, N), 0.01, 74)
+    m = mask_for(d)
+    o = B.quant_opts(rht_sign_mask=m, rht_dim=d, seed=5, sr_offset=1)
+    X_col, W_row, W_col = B.alloc_tensor(K, M), B.alloc_tensor(N, K), B.alloc_tensor(K, N)
+    Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    dX = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((N, K), dtype=torch.float32, device="cuda")
+    ws_f = torch.empty(B.nvfp4_linear_fwd_workspace_bytes(M, K), dtype=torch.uint8, device="cuda")
+    ws_b = torch.empty(B.nvfp4_linear_bwd_workspace_bytes(M, N), dtype=torch.uint8, device="cuda")
+    B.nvfp4_linear_fwd(x.cuda(), w.cuda(), o, Y, X_col, W_row, W_col, False, ws_f)
+    B.nvfp4_linear_bwd(dy.cuda(), X_col, W_col, K, o, dX, dW, False, ws_b)
+    B.nvfp4_device_status()
+    P.assert_rht_close(synth.bits(x), X_col, None, colwise=True, sign_mask=m, rounding=oracle.RNE, what="X col", rht_dim=d)
+    gx = oracle.quantize(synth.bits(x), colwise=True, rht=True, sign_mask=m, rht_dim=d, amax_override=float(X_col.glob.cpu()[0]))
+    # the layer's dY copy lives in its workspace: remake it with the same options to learn its amax (protocol)
+    g_col = B.alloc_tensor(N, M)
+    B.nvfp4_quantize(dy.cuda(), B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True, rht_sign_mask=m, rht_dim=d,
+                                             seed=5, sr_offset=1), None, g_col)
+    gg = oracle.quantize(synth.bits(dy), colwise=True, rht=True, sign_mask=m, rht_dim=d, rounding=oracle.SR, seed=5,
+                         sr_offset=1, amax_override=float(g_col.glob.cpu()[0]))
+    Dref, T = oracle.gemm_tn(oracle.dequantize(gg), oracle.dequantize(gx))
+    err = np.abs(dW.cpu().numpy() - Dref)
+    assert np.count_nonzero(err > 1e-3 * T + 1e-30) <= 1e-3 * err.size and np.all(err <= 2e-2 * T + 1e-30)
