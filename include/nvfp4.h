@@ -54,8 +54,7 @@ enum { NVFP4_SF_LINEAR = 0, NVFP4_SF_SWIZZLED = 1 };
    tensor-level scale (global = {0, 1}), transform size 32 on the weight-gradient operands, 32x32 blocks
    for weights.
    NVFP4_ROWSCALE is NVFP4 with the FP32 "global" scale taken per ROW of the copy instead of per tensor (the
-   closing remark of Appendix B.1: a global scale spanning a row avoids the extra pass through device memory
-   that the tensor amax costs): global holds rows pairs {amax of the row, s_dec of the row}, Eq. 1 per row,
+   closing remark of Appendix B.1: with one global scale per row no separate amax sweep over the whole tensor is needed): global holds rows pairs {amax of the row, s_dec of the row}, Eq. 1 per row,
    Eq. 2-4 unchanged.  Row-wise copies only; nvfp4_quantize makes them in ONE pass and nvfp4_gemm applies the
    vectors in its epilogue (D[i][j] = s_dec^A[i] * s_dec^B[j] * sum ...). */
 enum { NVFP4_FORMAT_NVFP4 = 0, NVFP4_FORMAT_MXFP4 = 1, NVFP4_FORMAT_NVFP4_ROWSCALE = 2 };
@@ -65,7 +64,7 @@ enum {
   NVFP4_SR_INDEPENDENT_COPIES = 1,
   /* global[0] of each requested copy already holds the tensor amax: skip the reduction pass */
   NVFP4_AMAX_PROVIDED = 2,
-  /* the source is binary32 instead of bf16 (Appendix B: "from higher precision (FP32 or BF16)"), e.g. weights
+  /* the source is binary32 instead of bf16 (Appendix B names FP32 as well as BF16 as the precision converted from), e.g. weights
      quantized from their FP32 master copy.  NVFP4 outputs without the Hadamard transform only; ld counts floats */
   NVFP4_INPUT_FP32 = 4,
   /* nvfp4_linear_fwd only, forward-only calls (X_col_saved == NULL): quantize X with a global scale per row in
@@ -74,8 +73,8 @@ enum {
 };
 
 /*
- * One quantized copy of a tensor (Appendix B.3: "the quantized values, the local and global
- * decode scales are stored in memory").  The copy is a row-major [rows x cols] matrix whose
+ * One quantized copy of a tensor (Appendix B.3: what is kept in memory is the codes, the block decode scales and
+ * the tensor decode scale).  The copy is a row-major [rows x cols] matrix whose
  * columns are the dot-product (contraction) dimension of the GEMM that will read it.
  *   codes : rows * cols/2 bytes; element (r, c) is the E2M1 nibble of byte [r][c/2], even c in
  *           the low nibble.  E2M1 = sign, 2 exponent bits, 1 mantissa bit (Section 2).

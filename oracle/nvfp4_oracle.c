@@ -393,7 +393,7 @@ ORC_EXPORT int orc_quantize_rht(const uint16_t* x_bf16, int64_t src_rows, int64_
                          scales, global, y_out);
 }
 
-/* The same procedure from a binary32 source (Appendix B: "from higher precision (FP32 or BF16)"): only step one,
+/* The same procedure from a binary32 source (Appendix B names FP32 as well as BF16 as the precision converted from): only step one,
  * reading the element, differs. */
 ORC_EXPORT int orc_quantize_f32(const float* x_f32, int64_t src_rows, int64_t src_cols, int64_t ld,
                                 int colwise, int block_rows, int rht, uint16_t sign_mask,

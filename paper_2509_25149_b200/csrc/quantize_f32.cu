@@ -1,4 +1,4 @@
-// NVFP4 quantizer for a binary32 source (Appendix B: "converting a tensor from higher precision (FP32 or BF16)"),
+// NVFP4 quantizer for a binary32 source (Appendix B names FP32 as well as BF16 as the precision converted from),
 // e.g. weights quantized straight from their FP32 master copy.  Same two passes and the same arithmetic as the bf16
 // kernels of quantize.cu, only the element read differs: the tile is staged as FP32 (64 KB), a chunk is two 32-byte
 // loads.  No Hadamard transform (the recipe transforms activations and gradients, which are bf16).

@@ -397,7 +397,7 @@ def test_column_slab_with_given_amax_equals_the_rows_of_the_transposed_copy():
 
 
 def test_binary32_source_follows_the_same_procedure():
-    """Appendix B converts "from higher precision (FP32 or BF16)": a binary32 source differs only in how the
+    """Appendix B names FP32 as well as BF16 as the precision converted from: a binary32 source differs only in how the
     element is read."""
     x = _random_bits((32, 64), 31, scale=1.0)
     xf = synth.from_bits(x).float().numpy()
