@@ -71,3 +71,34 @@ def test_gemm_with_a_thousand_row_blocks():
         a = oracle.quantize(synth.bits(a_src[g0:g0 + 16].cpu()), amax_override=amax_a)
         Dref, T = P.gemm_reference(a, b, rows=[int(r) - g0])
         P.assert_gemm_close(D[int(r)].float().cpu().numpy()[None, :], Dref, T, True, f"row {r}")
+
+
+def test_bf16_gemm_with_more_than_2_pow_31_outputs_and_row_scaled_copy_past_the_boundary():
+    """Variants at the edge of the size range: a BF16 GEMM whose output has 2.7e9 elements (exact integer data,
+    sampled rows compared in full) and the one-pass row-scaled quantizer on a tensor with more than 2^31 elements
+    (the draw counter and the code offsets of the last rows must not wrap)."""
+    M, N, K = 65536, 40960, 64
+    g = torch.Generator(device="cuda").manual_seed(7)
+    a = torch.randint(-2, 3, (M, K), generator=g, device="cuda").to(torch.bfloat16)
+    b = torch.randint(-2, 3, (N, K), generator=g, device="cuda").to(torch.bfloat16)
+    D = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    assert D.numel() > 2 ** 31
+    B.nvfp4_gemm_bf16(a, b, D)
+    B.nvfp4_device_status()
+    rows = torch.tensor([0, 255, 256, 32767, 52428, 52429, 65535], device="cuda")  # 52429 * 40960 > 2^31
+    ref = oracle.gemm_tn(a[rows].float().cpu().numpy(), b.float().cpu().numpy(), want_T=False)
+    assert np.array_equal(D[rows].float().cpu().numpy().astype(np.float64), ref)  # |sum| <= 256: exact in bf16
+    del D
+
+    R, C = 139264, 16384  # 2.28e9 elements, rows held by four warps
+    x = _big_tensor(R, C, 9, 1.0)
+    t = B.alloc_tensor(R, C, format=B.FORMAT_NVFP4_ROWSCALE)
+    B.nvfp4_quantize(x, B.quant_opts(rounding=B.ROUND_STOCHASTIC, seed=4, sr_offset=(1 << 33) + 5), t, None)
+    torch.cuda.synchronize()
+    for r0 in (0, 131072, R - 128):  # 131072 * 16384 = 2^31
+        ref = oracle.quantize_rowscale(synth.bits(x[r0:r0 + 128].cpu()), rounding=oracle.SR, seed=4,
+                                       sr_offset=(1 << 33) + 5, sr_row0=r0, sr_cols=C)
+        assert np.array_equal(t.codes[r0:r0 + 128].cpu().numpy(), ref.codes), f"codes of rows {r0}.."
+        assert np.array_equal(t.glob.view(R, 2)[r0:r0 + 128].cpu().numpy().view(np.uint32), ref.glob.view(np.uint32))
+        sc = t.scales.view(-1)[(r0 // 128) * (C // 64) * 512:((r0 // 128) + 1) * (C // 64) * 512].cpu().numpy()
+        assert np.array_equal(oracle.sf_unswizzle(sc, 128, C // 16), ref.scales), f"scales of rows {r0}.."
