@@ -313,8 +313,11 @@ __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const Qu
     for (int i = 0; i < 4; ++i) {
       const int r = warp * 16 + i * 4 + (lane >> 3);
       uint8_t* dst = smem + QuantSmem::kTile + r * QuantSmem::kTilePitch + cb * 32;
-      uint4 h0 = make_uint4(raw[i][0], raw[i][1], raw[i][2], raw[i][3]);
-      uint4 h1 = make_uint4(raw[i][4], raw[i][5], raw[i][6], raw[i][7]);
+      // the transform of the transposed copy negates whole source rows (input j of a chunk = row j of a 16-row
+      // group): the staged tile carries those signs already, one mask per row instead of one per word later
+      const uint32_t sg = (RHT_COL && ((a.sign_mask >> (r & 15)) & 1u)) ? 0x80008000u : 0u;
+      uint4 h0 = make_uint4(raw[i][0] ^ sg, raw[i][1] ^ sg, raw[i][2] ^ sg, raw[i][3] ^ sg);
+      uint4 h1 = make_uint4(raw[i][4] ^ sg, raw[i][5] ^ sg, raw[i][6] ^ sg, raw[i][7] ^ sg);
       if (first) {
         *reinterpret_cast<uint4*>(dst + 16) = h1;
         *reinterpret_cast<uint4*>(dst) = h0;
@@ -448,9 +451,8 @@ __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const Qu
       float f0[16], f1[16];
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        uint32_t word = *reinterpret_cast<const uint32_t*>(smem + QuantSmem::kTile + (q * 16 + j) * QuantSmem::kTilePitch + cp * 4);
-        if (RHT_COL) word ^= sign_pair(a.sign_mask, j, j);
-        f0[j] = bf16_lo(word);
+        const uint32_t word = *reinterpret_cast<const uint32_t*>(smem + QuantSmem::kTile + (q * 16 + j) * QuantSmem::kTilePitch + cp * 4);
+        f0[j] = bf16_lo(word);  // signs of the transform were applied when the tile was staged
         f1[j] = bf16_hi(word);
       }
       if (RHT_COL) {  // values are 4 * y from here on; the 1/4 is folded into amax and encode scale (exact)
