@@ -29,8 +29,8 @@ WORKLOAD = "cfg3_ffn_up_fwd_bwd_M8192_K5120_N20480"
 # DRAM bytes (read + write) from a one-pass ncu capture of this workload at full size, cold caches
 # (profiles/dram_traffic_cfg3_step.md): the step's two GEMM launches divided by its three GEMMs, and the six quantizer
 # kernels summed.
-GEMM_DRAM_BYTES_PER_LAUNCH = (548.0e6 + 1136.3e6) / 3  # Fprop launch + merged Dgrad/Wgrad launch, per GEMM
-QUANT_DRAM_BYTES_PER_STEP = 1514.3e6
+GEMM_DRAM_BYTES_PER_LAUNCH = (547.2e6 + 1092.6e6) / 3  # Fprop launch + merged Dgrad/Wgrad launch, per GEMM
+QUANT_DRAM_BYTES_PER_STEP = 1509.3e6
 SLAB = (4096, 2048, 5120)     # tokens, out-features, in-features of the CPU-baseline sample (one run)
 SLAB_REF = (512, 1024, 5120)  # per-step sample of the `--impl reference` arm (many steps)
 
