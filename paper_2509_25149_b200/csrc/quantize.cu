@@ -405,7 +405,9 @@ __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const Qu
       smem[QuantSmem::kSfRow + pos] = (uint8_t)byte;
     }
   }
-  __syncthreads();
+  // Phase 2 of a warp reads only what the same warp staged in phase 1 (its own 16 rows of the tile, their random
+  // bytes, its 16x16 scales), so the warps need not wait for each other here
+  __syncwarp();
 
   // ------------------------------------------------------------------ phase 2 ----
   if (HAS_COL) {

@@ -167,6 +167,9 @@ __global__ void __launch_bounds__(256, 3) quantize_rht_kernel(const RhtArgs ra) 
   }
 
   // ------------------------------------------------------------------ phase 2: transposed copy ----
+  // A warp reads back only what the same warp stored above (the random bytes of its own 16 rows; the tile was
+  // staged before the barrier), so a warp-level barrier orders it; d = 128 adds a CTA barrier after its first pass.
+  __syncwarp();
   if (has_col) {
     float* U = reinterpret_cast<float*>(smem + RhtSmem::kU);
     if (d_col == 128) {
