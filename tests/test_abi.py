@@ -74,6 +74,14 @@ def test_argument_validation_happens_before_any_launch():
                               fake, 1 << 30, None) == 2
     assert L.nvfp4_linear_bwd(fake, None, None, 256, 256, 256, ctypes.byref(o), None, None, 0, fake, 1 << 30,
                               None) == 1
+    # a row-scaled operand (format 2) pairs with NVFP4 only, and only on 256 x 256 tiles
+    ar = B.CTensor(fake, fake, fake, 256, 256, B.SF_SWIZZLED, 2)
+    bm = B.CTensor(fake, fake, fake, 256, 256, B.SF_SWIZZLED, 1)
+    bn = B.CTensor(fake, fake, fake, 128, 256, B.SF_SWIZZLED, 0)
+    assert L.nvfp4_gemm(ctypes.byref(ar), ctypes.byref(bm), fake, 0, 256, 0, None) == 4
+    assert L.nvfp4_gemm(ctypes.byref(ar), ctypes.byref(bn), fake, 0, 128, 0, None) == 2
+    rs = B.CTensor(fake, fake, fake, 64, 128, B.SF_LINEAR, 2)
+    assert q(fake, 64, 128, 128, ctypes.byref(o), ctypes.byref(rs), ctypes.byref(rs), None) == 4   # no transposed copy
     g16 = lambda M, N, K, lda=None, ldb=None, ldd=None, al=0, bl=0, fp32=0, acc=0, A=fake: L.nvfp4_gemm_bf16(
         A, al, lda or K, fake, bl, ldb or K, M, N, K, fake, fp32, ldd or N, acc, None)
     assert g16(256, 256, 64, A=None) == 1
