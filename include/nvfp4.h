@@ -286,8 +286,13 @@ NVFP4_API nvfp4_status nvfp4_linear_fwd_noalloc(const void* X, const void* W, in
  * nvfp4_dequantize: out[r][c] = code * fp32(block scale) * s_dec as fp32 (the decode of Section 2).
  * nvfp4_rht16: the transformed values y = x*(S*H_16) of the row-wise (colwise == 0, out [rows x cols])
  *   or column-wise (colwise != 0, out [cols x rows]) copy, fp32, as the quantizer sees them.
+ * nvfp4_e2m1_sr: codes[i] = the E2M1 code (4 bits in a byte) of the already scaled value v[i] under the
+ *   stochastic-rounding rule of Section 4.4 with the 8-bit draw u[i], computed by the device routine the
+ *   quantizer kernels use; v, u, codes are device arrays of n elements.
  */
 NVFP4_API nvfp4_status nvfp4_dequantize(const nvfp4_tensor* t, float* out, void* cuda_stream);
+NVFP4_API nvfp4_status nvfp4_e2m1_sr(const float* v, const uint8_t* u, int64_t n, uint8_t* codes,
+                                     void* cuda_stream);
 NVFP4_API nvfp4_status nvfp4_rht16(const void* x_bf16, int64_t rows, int64_t cols, int64_t ld,
                                    int32_t colwise, uint32_t sign_mask, float* out,
                                    void* cuda_stream);

@@ -55,6 +55,7 @@ def lib():
                 "orc_e4m3_encode_rne": (c.c_uint8, [c.c_float]),
                 "orc_e2m1_encode_rne": (c.c_uint8, [c.c_float]),
                 "orc_e2m1_encode_sr": (c.c_uint8, [c.c_float, c.c_uint8]),
+                "orc_e2m1_encode_sr_many": (None, [f32p, u8p, c.c_int64, u8p]),
                 "orc_philox4x32_10": (None, [u32p, u32p, u32p]),
                 "orc_sr_draw": (c.c_uint8, [c.c_uint64, c.c_uint64, c.c_uint64]),
                 "orc_hadamard16_entry": (c.c_int, [c.c_int, c.c_int]),
@@ -122,6 +123,16 @@ def e2m1_encode_rne(v: float) -> int:
 
 def e2m1_encode_sr(v: float, u: int) -> int:
     return int(lib().orc_e2m1_encode_sr(np.float32(v), u))
+
+
+def e2m1_encode_sr_many(v, u):
+    """orc_e2m1_encode_sr applied element by element to float32 values `v` and uint8 draws `u`."""
+    v = np.ascontiguousarray(v, dtype=np.float32).ravel()
+    u = np.ascontiguousarray(u, dtype=np.uint8).ravel()
+    assert v.size == u.size
+    out = np.empty(v.size, dtype=np.uint8)
+    lib().orc_e2m1_encode_sr_many(_p(v, ctypes.c_float), _p(u, ctypes.c_uint8), v.size, _p(out, ctypes.c_uint8))
+    return out
 
 
 def philox4x32_10(ctr, key):

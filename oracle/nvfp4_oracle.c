@@ -118,6 +118,11 @@ ORC_EXPORT uint8_t orc_e2m1_encode_sr(float v, uint8_t u) {
   return (uint8_t)(sign | (lo + up));
 }
 
+/* The same, element by element over arrays (a loop around the scalar routine, for sweeps in tests). */
+ORC_EXPORT void orc_e2m1_encode_sr_many(const float* v, const uint8_t* u, int64_t n, uint8_t* out) {
+  for (int64_t i = 0; i < n; ++i) out[i] = orc_e2m1_encode_sr(v[i], u[i]);
+}
+
 /* ------------------------------------------------------------------------- */
 /* Philox4x32-10 counter-based generator (Salmon et al., SC'11).              */
 /* The paper leaves the random source open; the draw is keyed by              */

@@ -22,7 +22,7 @@ FORMAT_NVFP4, FORMAT_MXFP4, FORMAT_NVFP4_ROWSCALE = 0, 1, 2
 
 EXPORTED = (
     "nvfp4_quantize", "nvfp4_gemm", "nvfp4_linear_fwd_workspace_bytes", "nvfp4_linear_bwd_workspace_bytes",
-    "nvfp4_linear_fwd", "nvfp4_linear_bwd", "nvfp4_dequantize", "nvfp4_rht16", "nvfp4_device_status",
+    "nvfp4_linear_fwd", "nvfp4_linear_bwd", "nvfp4_dequantize", "nvfp4_rht16", "nvfp4_e2m1_sr", "nvfp4_device_status",
     "nvfp4_set_gemm_tile_n", "nvfp4_status_string", "nvfp4_launch_count",
     "nvfp4_linear_fwd_noalloc", "nvfp4_linear_fwd_noalloc_max_bytes",
     "nvfp4_gemm_bf16", "nvfp4_linear_bf16_fwd", "nvfp4_linear_bf16_bwd", "nvfp4_quant_error", "nvfp4_sq_error",
@@ -83,6 +83,7 @@ def lib() -> ctypes.CDLL:
         L.nvfp4_sq_error.argtypes = [vp, i32, i64, vp, i32, i64, i64, i64, vp, vp]
         L.nvfp4_dequantize.restype, L.nvfp4_dequantize.argtypes = i32, [TP, vp, vp]
         L.nvfp4_rht16.restype, L.nvfp4_rht16.argtypes = i32, [vp, i64, i64, i64, i32, u32, vp, vp]
+        L.nvfp4_e2m1_sr.restype, L.nvfp4_e2m1_sr.argtypes = i32, [vp, vp, i64, vp, vp]
         L.nvfp4_device_status.restype, L.nvfp4_device_status.argtypes = i32, [vp, c.POINTER(u32)]
         L.nvfp4_set_gemm_tile_n.restype, L.nvfp4_set_gemm_tile_n.argtypes = i32, [i32]
         L.nvfp4_status_string.restype, L.nvfp4_status_string.argtypes = c.c_char_p, [i32]
@@ -289,6 +290,15 @@ def nvfp4_rht16(x: torch.Tensor, colwise: bool, sign_mask: int) -> torch.Tensor:
     out = torch.empty((R, C), dtype=torch.float32, device=x.device)
     _check(lib().nvfp4_rht16(x.data_ptr(), x.shape[0], x.shape[1], x.stride(0), int(colwise), sign_mask,
                              out.data_ptr(), _stream()), "nvfp4_rht16")
+    return out
+
+
+def nvfp4_e2m1_sr(v: torch.Tensor, u: torch.Tensor) -> torch.Tensor:
+    """E2M1 codes of the scaled fp32 values `v` under stochastic rounding with the uint8 draws `u` (test aid)."""
+    assert v.dtype == torch.float32 and u.dtype == torch.uint8 and v.numel() == u.numel()
+    v, u = v.contiguous(), u.contiguous()
+    out = torch.empty(v.numel(), dtype=torch.uint8, device=v.device)
+    _check(lib().nvfp4_e2m1_sr(v.data_ptr(), u.data_ptr(), v.numel(), out.data_ptr(), _stream()), "nvfp4_e2m1_sr")
     return out
 
 

@@ -476,6 +476,13 @@ nvfp4_status nvfp4_rht16(const void* x_bf16, int64_t rows, int64_t cols, int64_t
              : NVFP4_ERR_CUDA;
 }
 
+nvfp4_status nvfp4_e2m1_sr(const float* v, const uint8_t* u, int64_t n, uint8_t* codes, void* cuda_stream) {
+  if (!v || !u || !codes) return NVFP4_ERR_NULL;
+  if (n <= 0) return NVFP4_ERR_SHAPE;
+  return launch_e2m1_sr(v, u, n, codes, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? NVFP4_OK
+                                                                                                 : NVFP4_ERR_CUDA;
+}
+
 nvfp4_status nvfp4_device_status(void* cuda_stream, uint32_t* detail) {
   uint32_t code = 0;
   if (read_device_status(static_cast<cudaStream_t>(cuda_stream), &code) != cudaSuccess) return NVFP4_ERR_CUDA;

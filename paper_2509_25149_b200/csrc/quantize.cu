@@ -365,7 +365,9 @@ __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const Qu
         uint4 qc = q;
         if (a.off_hi_col != a.off_hi)
           qc = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), a.off_lo, a.off_hi_col, a.rk);
-        *reinterpret_cast<uint4*>(smem + QuantSmem::kRand + r * 128 + ((cb ^ ((r >> 2) & 7)) << 4)) = qc;
+        // staged complemented: the conversion wants 255 - draw
+        *reinterpret_cast<uint4*>(smem + QuantSmem::kRand + r * 128 + ((cb ^ ((r >> 2) & 7)) << 4)) =
+            make_uint4(~qc.x, ~qc.y, ~qc.z, ~qc.w);
       }
     }
     if (HAS_ROW) {
@@ -481,18 +483,20 @@ __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const Qu
           enc1 *= 0.25f;
         }
       }
-      uint32_t two[16];
-#pragma unroll
-      for (int j = 0; j < 16; ++j) two[j] = 0u;
+      uint2 codes0, codes1;
       if (SR) {
-        // low / high byte of two[j] = draw of source element (row 16q + j, column 2cp / 2cp + 1)
+        // low / high byte of ntwo[j] = 255 - draw of source element (row 16q + j, column 2cp / 2cp + 1)
+        uint32_t ntwo[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j)
-          two[j] = *reinterpret_cast<const uint16_t*>(smem + QuantSmem::kRand + (q * 16 + j) * 128 +
-                                                     (((cp >> 3) ^ ((4 * q + (j >> 2)) & 7)) << 4) + (cp & 7) * 2);
+          ntwo[j] = *reinterpret_cast<const uint16_t*>(smem + QuantSmem::kRand + (q * 16 + j) * 128 +
+                                                      (((cp >> 3) ^ ((4 * q + (j >> 2)) & 7)) << 4) + (cp & 7) * 2);
+        convert16x2_sr(f0, f1, enc0, enc1, ntwo, codes0, codes1);
+      } else {
+        const uint32_t none[4] = {0u, 0u, 0u, 0u};
+        codes0 = convert16<false>(f0, enc0, Nu14FromWords{none});
+        codes1 = convert16<false>(f1, enc1, Nu14FromWords{none});
       }
-      uint2 codes0 = convert16<SR>(f0, enc0, Nu14FromPairs<0>{two});
-      uint2 codes1 = convert16<SR>(f1, enc1, Nu14FromPairs<1>{two});
       // staging: column c holds eight 8-byte units, unit q stored at (q ^ (c >> 1)) & 7; the column a
       // lane writes first alternates with bit 3 of the lane so that a half warp covers all banks
       const int sel = (lane >> 3) & 1;
@@ -612,6 +616,19 @@ __global__ void rht16_kernel(const uint16_t* __restrict__ x, int64_t rows, int64
     fwht16(f);
 #pragma unroll
     for (int j = 0; j < 16; ++j) out[r * C + kb * 16 + j] = f[j] * 0.25f;
+  }
+}
+
+// codes[i] = stochastic rounding of v[i] with the draw u[i], through the very conversion the quantizer uses
+__global__ void e2m1_sr_kernel(const float* __restrict__ v, const uint8_t* __restrict__ u, int64_t n,
+                               uint8_t* __restrict__ codes) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    // the element sits in the low slot on even i and in the high slot on odd i, the other slot holds a decoy
+    const float w = __fmul_rz(v[i], kSrTowardsZero), decoy = __fmul_rz(-v[i] * 0.75f, kSrTowardsZero);
+    const uint32_t nu = 255u - u[i], nd = (uint32_t)(i * 37) & 255u;
+    const uint32_t d = (i & 1) ? e2m1x2_sr(decoy, w, (nu << 24) | (nd << 16) | 0x8080u)
+                               : e2m1x2_sr(w, decoy, (nd << 24) | (nu << 16) | 0x8080u);
+    codes[i] = (uint8_t)((i & 1) ? (d >> 8) & 15u : d & 15u);
   }
 }
 
@@ -738,6 +755,12 @@ cudaError_t launch_dequantize(const nvfp4_tensor& t, float* out, cudaStream_t s)
 cudaError_t launch_rht16(const void* x, int64_t rows, int64_t cols, int64_t ld, int colwise, uint32_t mask,
                          float* out, cudaStream_t s) {
   rht16_kernel<<<1184, 256, 0, s>>>(static_cast<const uint16_t*>(x), rows, cols, ld, colwise, mask, out);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_e2m1_sr(const float* v, const uint8_t* u, int64_t n, uint8_t* codes, cudaStream_t s) {
+  e2m1_sr_kernel<<<1184, 256, 0, s>>>(v, u, n, codes);
   count_launch();
   return cudaGetLastError();
 }

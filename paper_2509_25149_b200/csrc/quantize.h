@@ -47,6 +47,7 @@ cudaError_t launch_quantize_mx(const QuantArgs& a, bool has_row, bool has_col, b
 cudaError_t launch_amax_f32(const QuantArgs& a, bool has_row, bool has_col, cudaStream_t s);
 cudaError_t launch_quantize_f32(const QuantArgs& a, bool has_row, bool has_col, bool block2d, bool sr, cudaStream_t s);
 cudaError_t launch_dequantize(const nvfp4_tensor& t, float* out, cudaStream_t s);
+cudaError_t launch_e2m1_sr(const float* v, const uint8_t* u, int64_t n, uint8_t* codes, cudaStream_t s);
 cudaError_t launch_rht16(const void* x, int64_t rows, int64_t cols, int64_t ld, int colwise, uint32_t mask,
                          float* out, cudaStream_t s);
 

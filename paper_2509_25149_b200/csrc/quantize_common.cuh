@@ -44,26 +44,40 @@ __device__ __forceinline__ uint32_t sign_pair(uint32_t mask, int j0, int j1) {
   return (((mask >> j0) & 1u) << 15) | (((mask >> j1) & 1u) << 31);
 }
 
-// 16 scaled values -> 16 E2M1 nibbles (element 0 in the lowest nibble of .x).  For stochastic rounding `nu14(i)`
-// returns the complemented 8-bit draw of element i placed in bits [21, 29).
-template <bool SR, class Nu14>
-__device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, Nu14 nu14) {
-  uint2 out;
-  float v[16];
+// Eq. 4 for sixteen values: v = fl(y * s_enc,b), two lanes per instruction; for stochastic rounding the result is
+// then moved one binary32 towards zero, which is what e2m1x2_sr() expects.
+template <bool SR>
+__device__ __forceinline__ void scale16(const float (&f)[16], float s_enc_b, float (&v)[16]) {
 #pragma unroll
-  for (int i = 0; i < 16; i += 2) {  // Eq. 4: v = fl(y * s_enc,b), two lanes per instruction
-    const float2 p = mul2(make_float2(f[i], f[i + 1]), make_float2(s_enc_b, s_enc_b));
+  for (int i = 0; i < 16; i += 2) {
+    float2 p = mul2(make_float2(f[i], f[i + 1]), make_float2(s_enc_b, s_enc_b));
+    if (SR) p = mul2_rz(p, make_float2(kSrTowardsZero, kSrTowardsZero));
     v[i] = p.x;
     v[i + 1] = p.y;
   }
+}
+
+// 16 scaled values -> 16 E2M1 nibbles (element 0 in the lowest nibble of .x).  For stochastic rounding
+// `draws.rbits(i, j)` returns the random word of e2m1x2_sr() for elements i (low) and j (high).
+template <bool SR, class Draws>
+__device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, Draws draws) {
+  uint2 out;
+  float v[16];
+  scale16<SR>(f, s_enc_b, v);
   if (!SR) {
     const float(&lo)[8] = *reinterpret_cast<const float(*)[8]>(&v[0]);
     const float(&hi)[8] = *reinterpret_cast<const float(*)[8]>(&v[8]);
     out.x = e2m1x8_rne(lo);
     out.y = e2m1x8_rne(hi);
   } else {
-    out.x = e2m1x8_sr(&v[0], nu14, 0);
-    out.y = e2m1x8_sr(&v[8], nu14, 8);
+    uint32_t even[4], odd[4];  // nibbles 0 and 2 of each: elements (4k, 4k + 2) and (4k + 1, 4k + 3)
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      even[k] = e2m1x2_sr(v[4 * k], v[4 * k + 2], draws.rbits(4 * k, 4 * k + 2));
+      odd[k] = e2m1x2_sr(v[4 * k + 1], v[4 * k + 3], draws.rbits(4 * k + 1, 4 * k + 3));
+    }
+    out.x = (even[0] | (even[1] << 16)) | ((odd[0] | (odd[1] << 16)) << 4);
+    out.y = (even[2] | (even[3] << 16)) | ((odd[2] | (odd[3] << 16)) << 4);
   }
   return out;
 }
@@ -71,20 +85,39 @@ __device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, 
 // draws packed four to a word, byte i = element i (the row-wise copy: straight from the Philox output)
 struct Nu14FromWords {
   const uint32_t (&rnd)[4];
-  __device__ __forceinline__ uint32_t operator()(int i) const {
-    const uint32_t nr = ~rnd[i >> 2];
-    const int b = i & 3;
-    return (b == 0 ? (nr << 21) : b == 1 ? (nr << 13) : b == 2 ? (nr << 5) : (nr >> 3)) & 0x1FE00000u;
+  __device__ __forceinline__ uint32_t rbits(int i, int j) const {  // i, j in the same word, i even <=> j even
+    return __byte_perm(~rnd[i >> 2], 0x80808080u, (i & 1) ? 0x3144u : 0x2044u);
   }
 };
 // draws of two adjacent columns, 16 bits per row (the transposed copy: read back from shared memory)
 template <int COL>
 struct Nu14FromPairs {
   const uint32_t (&two)[16];
-  __device__ __forceinline__ uint32_t operator()(int i) const {
-    return (COL == 0 ? (~two[i] << 21) : (~two[i] << 13)) & 0x1FE00000u;
+  __device__ __forceinline__ uint32_t rbits(int i, int j) const {
+    const uint32_t picked = __byte_perm(two[i], two[j], COL == 0 ? 0x4000u : 0x5100u);  // bytes 2, 3 = draws of i, j
+    return (~picked & 0xFFFF0000u) | 0x8080u;
   }
 };
+
+// Two columns of sixteen rows at once (the transposed copy of the main kernel): element j of both columns goes into
+// one conversion.  ntwo[j]: low byte = 255 - draw of (row j, first column), next byte = the same for the second one.
+__device__ __forceinline__ void convert16x2_sr(const float (&f0)[16], const float (&f1)[16], float enc0, float enc1,
+                                               const uint32_t (&ntwo)[16], uint2& out0, uint2& out1) {
+  float v0[16], v1[16];
+  scale16<true>(f0, enc0, v0);
+  scale16<true>(f1, enc1, v1);
+  uint32_t e[8];  // byte 0 = first column, rows (2m, 2m + 1); byte 1 = second column
+#pragma unroll
+  for (int m = 0; m < 8; ++m) {
+    const uint32_t a = e2m1x2_sr(v0[2 * m], v1[2 * m], __byte_perm(ntwo[2 * m], 0x80808080u, 0x1044u));
+    const uint32_t b = e2m1x2_sr(v0[2 * m + 1], v1[2 * m + 1], __byte_perm(ntwo[2 * m + 1], 0x80808080u, 0x1044u));
+    e[m] = a | (b << 4);
+  }
+  const uint32_t p0 = __byte_perm(e[0], e[1], 0x5140u), p1 = __byte_perm(e[2], e[3], 0x5140u);
+  const uint32_t p2 = __byte_perm(e[4], e[5], 0x5140u), p3 = __byte_perm(e[6], e[7], 0x5140u);
+  out0 = make_uint2(__byte_perm(p0, p1, 0x5410u), __byte_perm(p2, p3, 0x5410u));
+  out1 = make_uint2(__byte_perm(p0, p1, 0x7632u), __byte_perm(p2, p3, 0x7632u));
+}
 
 __device__ __forceinline__ float amax16(const float (&f)[16]) {
   float m = 0.f;
