@@ -13,7 +13,7 @@ CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libnvfp4_b200.so")
 SOURCES = ("quantize.cu", "quantize_mx.cu", "quantize_f32.cu", "quantize_rht.cu", "quantize_rowscale.cu", "metrics.cu", "gemm.cu", "api.cu")
-HEADERS = ("common.cuh", "quantize.h", "quantize_common.cuh", "gemm.h", "tc_ptx.cuh", "gemm_2cta.cuh", "gemm_wide.cuh", "gemm_bf16.cuh")
+HEADERS = ("common.cuh", "quantize.h", "quantize_common.cuh", "gemm.h", "tc_ptx.cuh", "async_ptx.cuh", "gemm_2cta.cuh", "gemm_wide.cuh", "gemm_bf16.cuh")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-O3", "-lineinfo",
               "-Xcompiler", "-fPIC,-fvisibility=hidden", f"-I{os.path.join(ROOT, 'include')}", f"-I{CSRC}"]
 

@@ -114,6 +114,7 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
   a.off_hi_col = (o->flags & NVFP4_SR_INDEPENDENT_COPIES) ? (a.off_hi | 0x80000000u) : a.off_hi;
   a.tiles_r = (int)((rows + 127) / 128);
   a.tiles_c = (int)((cols + 127) / 128);
+  if (device_status_word(&a.status) != cudaSuccess) return NVFP4_ERR_CUDA;
 
   const bool hr = rowwise != nullptr, hc = colwise != nullptr;
   const bool b2 = o->block_rows == blk, sr = o->rounding == NVFP4_ROUND_STOCHASTIC;

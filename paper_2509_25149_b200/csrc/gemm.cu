@@ -617,6 +617,21 @@ cudaError_t launch_gemm_bf16(const DenseGemmArgs& g, cudaStream_t s) {
   return cudaGetLastError();
 }
 
+cudaError_t device_status_word(unsigned int** word) {
+  static std::atomic<unsigned int*> cache[64] = {};  // per device ordinal
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  unsigned int* p = (dev >= 0 && dev < 64) ? cache[dev].load(std::memory_order_acquire) : nullptr;
+  if (!p) {
+    e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_device_status);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) cache[dev].store(p, std::memory_order_release);
+  }
+  *word = p;
+  return cudaSuccess;
+}
+
 cudaError_t read_device_status(cudaStream_t s, uint32_t* code) {
   cudaError_t e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return e;

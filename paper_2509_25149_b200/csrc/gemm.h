@@ -30,6 +30,8 @@ cudaError_t launch_gemm_two(const GemmArgs& g0, const void* a0, const void* b0, 
 // Scheduling estimate: do 256 x 384 tiles beat 256 x 256 tiles for this problem (or pair of problems in one launch)?
 bool prefer_wide_tiles(const GemmArgs& g0, const GemmArgs* g1);
 cudaError_t read_device_status(cudaStream_t s, uint32_t* code);
+// device address of the status word on the current device (for kernels of other translation units)
+cudaError_t device_status_word(unsigned int** word);
 
 // BF16 GEMM D[M x N] = A B^T on CTA pairs (gemm_bf16.cuh) for layers kept in higher precision.
 // a_mn / b_mn = 0: the operand is stored [M or N][K] (contraction contiguous); 1: stored [K][M or N].

@@ -6,6 +6,9 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
+#include "async_ptx.cuh"
 #include "common.cuh"
 #include "quantize.h"
 #include "quantize_common.cuh"
@@ -225,50 +228,122 @@ __global__ void __launch_bounds__(256) amax_rot_col_kernel(const uint16_t* __res
 }
 
 // ---------------------------------------------------------------------------------------------
-// Pass 2: one CTA per 128 x 128 tile of the source.
-//   phase 1  each thread owns four 1x16 chunks (32-byte loads), produces the row-wise copy from
-//            registers and stages the raw tile (and the random bytes) in shared memory;
-//   phase 2  each thread owns 16 rows x 2 columns of the staged tile and produces the transposed copy
-//            into a swizzled staging buffer;
+// Pass 2: persistent CTAs (two per SM), each working through 128 x 128 tiles of the source.  The tiles arrive by
+// TMA (cp.async.bulk.tensor, this GPU's memory, no multicast) in a ring of two 32 KB buffers: the load of tile
+// k + 2 is issued as soon as tile k has been consumed, so a tile is in flight during the whole of the previous one;
+// out-of-range parts of a ragged tile are zero-filled by the copy.
+//   set-up   once per CTA: Eq. 1, and the table  E4M3 byte -> encode scale  of each copy (the text after Eq. 3:
+//            s_enc,b = 1 / (fp32(S_b) * s_dec) has only 127 possible values per tensor), so a block costs one
+//            conversion and one shared-memory read instead of an IEEE reciprocal;
+//   phase 1  each thread owns four 1x16 chunks of the tile and produces the row-wise copy (and, for stochastic
+//            rounding, stages the random bytes of its chunks in shared memory);
+//   phase 2  each thread owns 16 rows x 2 columns of the tile and produces the transposed copy into a swizzled
+//            staging buffer;
 //   phase 3  staged codes and scale bytes leave with 16-byte stores.
-// Tiles are visited in reverse order so that the end of the tensor, which pass 1 touched last, is read
-// first while it may still sit in L2.
+// A warp's phase 2 reads only what the same warp staged in phase 1, and the buffers phase 3 reads are double
+// buffered, so a tile needs one CTA barrier.  Tiles are visited in reverse order so that the end of the tensor,
+// which pass 1 touched last, is read first while it may still sit in L2.
 // ---------------------------------------------------------------------------------------------
-template <int PITCH>
-struct QuantSmemT {
-  static constexpr int kTile = 0;                    // 128 rows of bf16, kTilePitch bytes apart
-  static constexpr int kTilePitch = PITCH;           // 256, or 256 + 16 for the tensor-core transform: eight
-                                                     // consecutive rows then start in eight different 16-byte bank
-                                                     // groups (conflict-free 8x8 matrix loads)
-  static constexpr int kColCodes = 128 * kTilePitch; // 128 columns x 64 B
-  static constexpr int kSfRow = kColCodes + 8192;    // 1 KB
-  static constexpr int kSfCol = kSfRow + 1024;       // 1 KB
-  static constexpr int kBlkEnc = kSfCol + 1024;      // 64 floats (16x16 mode)
-  static constexpr int kBlkByte = kBlkEnc + 256;     // 64 bytes
-  static constexpr int kGlobalScales = kBlkByte + 64;  // s_enc, s_dec of the row-wise and the column-wise copy
-  static constexpr int kRand = kGlobalScales + 64;   // 128 rows x 128 B (stochastic rounding only); the 16-byte
-                                                     // chunk cb of row r sits at slot cb ^ ((r >> 2) & 7)
-  static constexpr int kBytesNoRand = kRand;
-  static constexpr int kBytesRand = kRand + 16384;
+struct QuantSmem {
+  static constexpr int kTile = 0;                     // 2 x (128 rows x 256 B of bf16), filled by TMA
+  static constexpr int kColCodes = 65536;             // 2 x (128 columns x 64 B)
+  static constexpr int kSfRow = kColCodes + 2 * 8192; // 2 x 1 KB
+  static constexpr int kSfCol = kSfRow + 2 * 1024;    // 2 x 1 KB
+  static constexpr int kBlkEnc = kSfCol + 2 * 1024;   // 64 floats (16x16 mode)
+  static constexpr int kBlkByte = kBlkEnc + 256;      // 64 bytes
+  static constexpr int kGlobalScales = kBlkByte + 64; // s_enc, s_dec of the row-wise and the column-wise copy
+  static constexpr int kEncRow = kGlobalScales + 64;  // 128 floats: encode scale by E4M3 byte, row-wise copy
+  static constexpr int kEncCol = kEncRow + 512;       // the same for the transposed copy
+  static constexpr int kBars = kEncCol + 512;         // two "tile landed" barriers, then the abort word
+  static constexpr int kRand = kBars + 32;            // 128 rows x 128 B of complemented draws (stochastic rounding),
+                                                      // or 128 rows x 64 B of row-wise codes (16x16 blocks, both copies)
+  static constexpr int kTileBytes = 32768;
+  static constexpr int bytes(bool rand, bool row_codes) { return kRand + (rand ? 16384 : row_codes ? 8192 : 0); }
 };
-// the transposed copy with the transform uses the padded pitch
-template <bool HAS_COL, bool BLOCK2D, bool RHT_COL>
-using QuantSmemFor = QuantSmemT<256>;
+
+// Bounded wait for a tile (2 s): on expiry the abort word of the CTA and the device status word are set.
+constexpr uint32_t kQuantWaitCode = 0x51000001u;
+__device__ __forceinline__ bool quant_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                           unsigned int* status) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (true) {
+    if (mbar_try(bar, parity)) return true;
+    if ((++spins & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = kQuantWaitCode;
+        if (status) atomicCAS(status, 0u, kQuantWaitCode);
+        return false;
+      }
+    }
+  }
+}
+
+// max(m, |a|, |b|)
+__device__ __forceinline__ float amax3(float m, float a, float b) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(m), "f"(fabsf(a)), "f"(fabsf(b)));
+  return r;
+}
+__device__ __forceinline__ float amax16_3(const float (&f)[16]) {
+  float m = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; i += 2) m = amax3(m, f[i], f[i + 1]);
+  return m;
+}
+
+// Eq. 2-3: the stored E4M3 byte of a block, S_b = e4m3(fl(fl(amax_b / 6) * s_enc))
+__device__ __forceinline__ uint32_t block_scale_byte(float amax_b, float s_enc) {
+  const float t = __fmul_rn(div6_rn(amax_b), s_enc);
+  uint16_t packed;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %1;" : "=h"(packed) : "f"(t));
+  return packed & 0xffu;
+}
+// the text after Eq. 3: encode scale of a block from its stored byte, fl(1 / fl(fp32(S_b) * s_dec)), 0 for S_b = 0
+__device__ __forceinline__ float encode_scale_of_byte(uint32_t byte, float s_dec) {
+  uint32_t h2;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)byte));
+  const float sf = __half2float(__ushort_as_half((unsigned short)(h2 & 0xffffu)));
+  const float d = __fmul_rn(sf, s_dec);
+  return (byte == 0u) ? 0.0f : fminf(__frcp_rn(d), kFltMax);
+}
 
 template <bool HAS_ROW, bool HAS_COL, bool BLOCK2D, bool RHT_ROW, bool RHT_COL, bool SR>
-__global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const QuantArgs a) {
-  using QuantSmem = QuantSmemFor<HAS_COL, BLOCK2D, RHT_COL>;
+__global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant__ CUtensorMap src_map,
+                                                          const QuantArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = (int)(gridDim.x - 1 - blockIdx.x);
-  const int64_t row0 = (int64_t)(tile / a.tiles_c) * 128;
-  const int64_t col0 = (int64_t)(tile % a.tiles_c) * 128;
-  const int64_t n_cb = a.cols >> 4;  // 16-blocks per source row
-  const int64_t n_rb = a.rows >> 4;  // 16-blocks per source column
+  const int n_cb = (int)(a.cols >> 4);  // 16-blocks per source row
+  const int n_rb = (int)(a.rows >> 4);  // 16-blocks per source column
+  // 16x16 blocks with both copies requested: the transposed copy holds the very codes of the row-wise one
+  // (Section 4.3), so it is made by transposing nibbles; the raw tile is not needed a second time
+  constexpr bool kNibbleTranspose = BLOCK2D && HAS_ROW && HAS_COL;
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + QuantSmem::kBars + 16);
+  const uint32_t bar0 = smem_u32(smem + QuantSmem::kBars), tile0 = smem_u32(smem + QuantSmem::kTile);
 
-  // Eq. 1 once per CTA (two IEEE divisions per copy), broadcast through shared memory
+  const int total = a.tiles_r * a.tiles_c, stride = (int)gridDim.x;
+  const int first = total - 1 - (int)blockIdx.x;         // this CTA's tiles: first, first - stride, ...
+  const int n_mine = first >= 0 ? first / stride + 1 : 0;
+  auto issue_load = [&](int k) {  // tile k of this CTA into buffer k & 1 (one thread)
+    const int t = first - k * stride, tr = t / a.tiles_c, tc = t - tr * a.tiles_c;
+    const uint32_t bar = bar0 + 8 * (k & 1);
+    mbar_expect_tx(bar, QuantSmem::kTileBytes);
+    tma_load_2d(tile0 + (k & 1) * QuantSmem::kTileBytes, &src_map, tc * 128, tr * 128, bar);
+  };
+
+  // ------------------------------------------------------------------ set-up ----
   float* g_sc = reinterpret_cast<float*>(smem + QuantSmem::kGlobalScales);
   if (threadIdx.x == 0) {
+    mbar_init(bar0, 1);
+    mbar_init(bar0 + 8, 1);
+    *abort_flag = 0u;
+    fence_mbarrier_init();
+    fence_proxy_async_smem();
+    if (n_mine > 0) issue_load(0);
+    if (n_mine > 1) issue_load(1);
+    // Eq. 1 (two IEEE divisions per copy)
     float re = 1.f, rd = 1.f, ce = 1.f, cd = 1.f;
     if (HAS_ROW || BLOCK2D) global_scales(HAS_ROW ? a.r_global[0] : a.c_global[0], re, rd);
     if (HAS_COL) {
@@ -285,283 +360,297 @@ __global__ void __launch_bounds__(256, BLOCK2D ? 4 : 3) quantize_kernel(const Qu
       if (HAS_COL) a.c_global[1] = cd;
     }
   }
-
-  // ------------------------------------------------------------------ phase 1 ----
-  const int cb = lane & 7;  // chunk column inside the tile
-  uint32_t raw[4][8];
-  bool ok[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = warp * 16 + i * 4 + (lane >> 3);
-    ok[i] = (row0 + r < a.rows) && (col0 + cb * 16 < a.cols);
-    if (ok[i]) {
-      ldg256_stream(a.x + (row0 + r) * a.ld + col0 + cb * 16, raw[i]);
-    } else {
-#pragma unroll
-      for (int k = 0; k < 8; ++k) raw[i][k] = 0u;
-    }
-  }
-
-  // 16x16 blocks with both copies requested: the transposed copy holds the very codes of the row-wise one
-  // (Section 4.3), so it is made by transposing nibbles; the raw tile is not needed a second time
-  constexpr bool kNibbleTranspose = BLOCK2D && HAS_ROW && HAS_COL;
-  if (HAS_COL && !kNibbleTranspose) {
-    // stage the raw tile; halves are written in lane-dependent order so that a quarter warp covers
-    // all 32 banks
-    const int first = (lane >> 2) & 1;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int r = warp * 16 + i * 4 + (lane >> 3);
-      uint8_t* dst = smem + QuantSmem::kTile + r * QuantSmem::kTilePitch + cb * 32;
-      // the transform of the transposed copy negates whole source rows (input j of a chunk = row j of a 16-row
-      // group): the staged tile carries those signs already, one mask per row instead of one per word later
-      const uint32_t sg = (RHT_COL && ((a.sign_mask >> (r & 15)) & 1u)) ? 0x80008000u : 0u;
-      uint4 h0 = make_uint4(raw[i][0] ^ sg, raw[i][1] ^ sg, raw[i][2] ^ sg, raw[i][3] ^ sg);
-      uint4 h1 = make_uint4(raw[i][4] ^ sg, raw[i][5] ^ sg, raw[i][6] ^ sg, raw[i][7] ^ sg);
-      if (first) {
-        *reinterpret_cast<uint4*>(dst + 16) = h1;
-        *reinterpret_cast<uint4*>(dst) = h0;
-      } else {
-        *reinterpret_cast<uint4*>(dst) = h0;
-        *reinterpret_cast<uint4*>(dst + 16) = h1;
-      }
-    }
-  }
-
-  __syncthreads();  // the loads above are in flight; the global scales are in shared memory now
+  __syncthreads();
   const float r_senc = g_sc[0], r_sdec = g_sc[1], c_senc = g_sc[2], c_sdec = g_sc[3];
-
-  float blk_amax = 0.f;  // 16x16 mode: running amax of the lane's chunk column over the warp's 16 rows
-  if (BLOCK2D) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      uint32_t acc = 0;
-#pragma unroll
-      for (int k = 0; k < 8; ++k) acc = absmax_bf16x2(acc, raw[i][k]);
-      blk_amax = fmaxf(blk_amax, fmaxf(bf16_lo(acc), bf16_hi(acc)));
+  const float* enc_row = reinterpret_cast<const float*>(smem + QuantSmem::kEncRow);
+  const float* enc_col = reinterpret_cast<const float*>(smem + QuantSmem::kEncCol);
+  if (!BLOCK2D) {
+    // with the transform the kernel works on 4 * y: the 1/4 is folded into the block amax and the encode scale (exact)
+    if (threadIdx.x < 128) {
+      if (HAS_ROW)
+        reinterpret_cast<float*>(smem + QuantSmem::kEncRow)[threadIdx.x] =
+            encode_scale_of_byte(threadIdx.x, r_sdec) * (RHT_ROW ? 0.25f : 1.0f);
+    } else {
+      if (HAS_COL)
+        reinterpret_cast<float*>(smem + QuantSmem::kEncCol)[threadIdx.x - 128] =
+            encode_scale_of_byte(threadIdx.x - 128, c_sdec) * (RHT_COL ? 0.25f : 1.0f);
     }
-    blk_amax = fmaxf(blk_amax, __shfl_xor_sync(0xffffffffu, blk_amax, 8));
-    blk_amax = fmaxf(blk_amax, __shfl_xor_sync(0xffffffffu, blk_amax, 16));
-  }
-  uint32_t blk_byte = 0;
-  float blk_enc = 0.f;
-  if (BLOCK2D) {
-    block_scales(blk_amax, r_senc, r_sdec, blk_byte, blk_enc);
-    if (lane < 8) {
-      reinterpret_cast<float*>(smem + QuantSmem::kBlkEnc)[warp * 8 + cb] = blk_enc;
-      smem[QuantSmem::kBlkByte + warp * 8 + cb] = (uint8_t)blk_byte;
-    }
+    __syncthreads();
   }
 
+  // per-thread constants of phase 1: chunk column cb, row rl + 4 i for chunk i
+  const int cb = lane & 7, rl = warp * 16 + (lane >> 3);
+  const uint32_t tile_ld = rl * 256 + cb * 32;     // chunk i of the thread inside a tile buffer: + 1024 i
+  const uint32_t rand_st = QuantSmem::kRand + rl * 128 + cb * 16;  // + 512 i
+  // sign of source row j of a 16-row group (the transform of the transposed copy negates whole source rows: input j
+  // of a chunk = row j of the group) for both halves of a bf16 pair: bits 15 and 31 of sign2 << (15 - j)
+  const uint32_t sign2 = (a.sign_mask & 0xffffu) * 0x10001u;
+  const int sf_row_pos = a.r_swz ? ((cb >> 2) * 512 + (rl & 31) * 16 + (rl >> 5) * 4 + (cb & 3)) : (rl * 8 + cb);
+  const int sf_row_step = a.r_swz ? 64 : 32;
+  const int64_t r_pitch = a.cols >> 1;  // bytes per row of the row-wise codes
+
+  int k = 0;
+  for (; k < n_mine; ++k) {
+    const int buf = k & 1;
+    const int tile = first - k * stride;
+    const int tr = tile / a.tiles_c, tc = tile - tr * a.tiles_c;
+    const int64_t row0 = (int64_t)tr * 128, col0 = (int64_t)tc * 128;
+    const bool full_tile = (row0 + 128 <= a.rows) && (col0 + 128 <= a.cols);
+    uint8_t* const col_codes = smem + QuantSmem::kColCodes + buf * 8192;
+    uint8_t* const sf_row = smem + QuantSmem::kSfRow + buf * 1024;
+    uint8_t* const sf_col = smem + QuantSmem::kSfCol + buf * 1024;
+    const uint8_t* const tile_buf = smem + QuantSmem::kTile + buf * QuantSmem::kTileBytes;
+    quant_wait(bar0 + 8 * buf, (uint32_t)(k >> 1) & 1u, abort_flag, a.status);  // the tile has landed
+
+    auto phases_1_2 = [&](auto full_c) {
+      constexpr bool FULL = decltype(full_c)::value;
+      // ---------------------------------------------------------------- phase 1 ----
+      const int rows_left = FULL ? 128 : (int)(a.rows - row0) - rl;         // chunk i exists iff 4 i < rows_left
+      const bool col_ok = FULL || (col0 + cb * 16 < a.cols);
+      uint32_t raw[4][8];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = warp * 16 + i * 4 + (lane >> 3);
-    uint32_t rnd[4] = {0u, 0u, 0u, 0u};
-    if (SR) {
-      const uint64_t g = (uint64_t)(row0 + r) * (uint64_t)n_cb + (uint64_t)((col0 >> 4) + cb);
-      uint4 q = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), a.off_lo, a.off_hi, a.rk);
-      rnd[0] = q.x; rnd[1] = q.y; rnd[2] = q.z; rnd[3] = q.w;
-      if (HAS_COL) {
-        uint4 qc = q;
-        if (a.off_hi_col != a.off_hi)
-          qc = philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), a.off_lo, a.off_hi_col, a.rk);
-        // staged complemented: the conversion wants 255 - draw
-        *reinterpret_cast<uint4*>(smem + QuantSmem::kRand + r * 128 + ((cb ^ ((r >> 2) & 7)) << 4)) =
-            make_uint4(~qc.x, ~qc.y, ~qc.z, ~qc.w);
+      for (int i = 0; i < 4; ++i) {
+        const uint4 h0 = *reinterpret_cast<const uint4*>(tile_buf + tile_ld + i * 1024);
+        const uint4 h1 = *reinterpret_cast<const uint4*>(tile_buf + tile_ld + i * 1024 + 16);
+        raw[i][0] = h0.x; raw[i][1] = h0.y; raw[i][2] = h0.z; raw[i][3] = h0.w;
+        raw[i][4] = h1.x; raw[i][5] = h1.y; raw[i][6] = h1.z; raw[i][7] = h1.w;
       }
-    }
-    if (HAS_ROW) {
-      float f[16];
+
+      uint32_t blk_byte = 0;
+      float blk_enc = 0.f;
+      if (BLOCK2D) {  // amax of the lane's chunk column over the warp's 16 rows: one scale per 16 x 16 block
+        float blk_amax = 0.f;
 #pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        uint32_t word = raw[i][k];
-        if (RHT_ROW) word ^= sign_pair(a.sign_mask, 2 * k, 2 * k + 1);
-        f[2 * k] = bf16_lo(word);
-        f[2 * k + 1] = bf16_hi(word);
-      }
-      if (RHT_ROW) fwht16(f);  // values are 4 * y: the 1/4 is folded into the amax and the encode scale (exact)
-      uint32_t byte;
-      float enc;
-      if (BLOCK2D) {
-        byte = blk_byte;
-        enc = blk_enc;
-      } else {
-        float bmax;
-        if (RHT_ROW) {
-          bmax = 0.25f * amax16(f);
-        } else {  // untransformed: the maximum of the bf16 pairs themselves, two elements per instruction
+        for (int i = 0; i < 4; ++i) {
           uint32_t acc = 0;
 #pragma unroll
           for (int k = 0; k < 8; ++k) acc = absmax_bf16x2(acc, raw[i][k]);
-          bmax = fmaxf(bf16_lo(acc), bf16_hi(acc));
+          blk_amax = fmaxf(blk_amax, fmaxf(bf16_lo(acc), bf16_hi(acc)));
         }
-        block_scales(bmax, r_senc, r_sdec, byte, enc);
-        if (RHT_ROW) enc *= 0.25f;
+        blk_amax = fmaxf(blk_amax, __shfl_xor_sync(0xffffffffu, blk_amax, 8));
+        blk_amax = fmaxf(blk_amax, __shfl_xor_sync(0xffffffffu, blk_amax, 16));
+        block_scales(blk_amax, r_senc, r_sdec, blk_byte, blk_enc);
+        if (lane < 8) {
+          reinterpret_cast<float*>(smem + QuantSmem::kBlkEnc)[warp * 8 + cb] = blk_enc;
+          smem[QuantSmem::kBlkByte + warp * 8 + cb] = (uint8_t)blk_byte;
+        }
       }
-      uint2 codes = convert16<SR>(f, enc, Nu14FromWords{rnd});
-      if (ok[i])
-        *reinterpret_cast<uint2*>(a.r_codes + (row0 + r) * (a.cols >> 1) + ((col0 + cb * 16) >> 1)) = codes;
-      if (kNibbleTranspose)  // row r, bytes [8 cb, 8 cb + 8): byte k = columns (2k, 2k + 1) of the chunk
-        *reinterpret_cast<uint2*>(smem + QuantSmem::kTile + r * 64 + cb * 8) = ok[i] ? codes : make_uint2(0u, 0u);
-      const int pos = a.r_swz ? ((cb >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (cb & 3)) : (r * 8 + cb);
-      smem[QuantSmem::kSfRow + pos] = (uint8_t)byte;
-    }
-  }
-  // Phase 2 of a warp reads only what the same warp staged in phase 1 (its own 16 rows of the tile, their random
-  // bytes, its 16x16 scales), so the warps need not wait for each other here
-  __syncwarp();
 
-  // ------------------------------------------------------------------ phase 2 ----
-  if (HAS_COL) {
-    const int q = warp;  // 16-row group inside the tile
+      uint64_t g = 0;  // Philox counter of chunk 0: the chunk's index in the source, 16-blocks numbered row by row
+      if (SR) g = (uint64_t)(row0 + rl) * (uint64_t)n_cb + (uint64_t)((col0 >> 4) + cb);
+      uint8_t* r_out = HAS_ROW ? a.r_codes + (row0 + rl) * r_pitch + ((col0 + cb * 16) >> 1) : nullptr;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        uint32_t rnd[4] = {0u, 0u, 0u, 0u};
+        if (SR) {
+          const uint64_t gi = g + (uint64_t)(4 * i) * (uint64_t)n_cb;
+          uint4 q = philox4x32_10((uint32_t)gi, (uint32_t)(gi >> 32), a.off_lo, a.off_hi, a.rk);
+          rnd[0] = q.x; rnd[1] = q.y; rnd[2] = q.z; rnd[3] = q.w;
+          if (HAS_COL && !kNibbleTranspose) {
+            uint4 qc = q;
+            if (a.off_hi_col != a.off_hi)
+              qc = philox4x32_10((uint32_t)gi, (uint32_t)(gi >> 32), a.off_lo, a.off_hi_col, a.rk);
+            // staged complemented: the conversion wants 255 - draw
+            *reinterpret_cast<uint4*>(smem + rand_st + i * 512) = make_uint4(~qc.x, ~qc.y, ~qc.z, ~qc.w);
+          }
+        }
+        if (HAS_ROW) {
+          float f[16];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            uint32_t word = raw[i][k];
+            if (RHT_ROW) word ^= sign_pair(a.sign_mask, 2 * k, 2 * k + 1);
+            f[2 * k] = bf16_lo(word);
+            f[2 * k + 1] = bf16_hi(word);
+          }
+          if (RHT_ROW) fwht16(f);  // values are 4 * y from here on
+          uint32_t byte;
+          float enc;
+          if (BLOCK2D) {
+            byte = blk_byte;
+            enc = blk_enc;
+          } else {
+            const float m = amax16_3(f);
+            byte = block_scale_byte(RHT_ROW ? 0.25f * m : m, r_senc);
+            enc = enc_row[byte];
+          }
+          const uint2 codes = convert16<SR>(f, enc, Nu14FromWords{rnd});
+          if (FULL || (col_ok && 4 * i < rows_left)) *reinterpret_cast<uint2*>(r_out + (int64_t)(4 * i) * r_pitch) = codes;
+          if (kNibbleTranspose)  // row r, bytes [8 cb, 8 cb + 8): byte k = columns (2k, 2k + 1) of the chunk
+            *reinterpret_cast<uint2*>(smem + QuantSmem::kRand + (rl + 4 * i) * 64 + cb * 8) =
+                (FULL || (col_ok && 4 * i < rows_left)) ? codes : make_uint2(0u, 0u);
+          sf_row[sf_row_pos + i * sf_row_step] = (uint8_t)byte;
+        }
+      }
+      // Phase 2 of a warp reads only what the same warp staged in phase 1 (its own 16 rows of the tile, their random
+      // bytes, its 16x16 scales), so the warps need not wait for each other here
+      __syncwarp();
+
+      // ---------------------------------------------------------------- phase 2 ----
+      if (HAS_COL) {
+        const int q = warp;  // 16-row group inside the tile
 #pragma unroll 1
-    for (int it = 0; it < 2; ++it) {
-      const int cp = lane + 32 * it;  // column pair: tile columns 2cp, 2cp+1
-      if (kNibbleTranspose) {
-        // byte [row][cp] of the staged row-wise codes = (column 2cp in the low nibble, 2cp + 1 in the high one)
-        uint32_t w[4];
+        for (int it = 0; it < 2; ++it) {
+          const int cp = lane + 32 * it;  // column pair: tile columns 2cp, 2cp+1
+          const int sel = (lane >> 3) & 1;
+          if (kNibbleTranspose) {
+            // byte [row][cp] of the staged row-wise codes = (column 2cp in the low nibble, 2cp + 1 in the high one)
+            uint32_t w[4];
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-          uint32_t b[4];
+            for (int m = 0; m < 4; ++m) {
+              uint32_t b[4];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) b[j] = smem[QuantSmem::kTile + (q * 16 + 4 * m + j) * 64 + cp];
-          w[m] = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
+              for (int j = 0; j < 4; ++j) b[j] = smem[QuantSmem::kRand + (q * 16 + 4 * m + j) * 64 + cp];
+              w[m] = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
+            }
+            auto gather = [](uint32_t x) {  // four nibbles, one per byte -> 16 bits
+              const uint32_t t = (x | (x >> 4)) & 0x00FF00FFu;
+              return (t | (t >> 8)) & 0xFFFFu;
+            };
+            uint32_t lo[4], hi[4];
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+              lo[m] = gather(w[m] & 0x0F0F0F0Fu);
+              hi[m] = gather((w[m] >> 4) & 0x0F0F0F0Fu);
+            }
+            const uint2 codes0 = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
+            const uint2 codes1 = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+            const uint32_t byte = smem[QuantSmem::kBlkByte + q * 8 + (cp >> 3)];
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+              const int odd = s ^ sel;
+              const int c = 2 * cp + odd;
+              *reinterpret_cast<uint2*>(col_codes + c * 64 + (((q ^ (c >> 1)) & 7) << 3)) = odd ? codes1 : codes0;
+              const int pos = a.c_swz ? ((q >> 2) * 512 + (c & 31) * 16 + (c >> 5) * 4 + (q & 3)) : (c * 8 + q);
+              sf_col[pos] = (uint8_t)byte;
+            }
+            continue;
+          }
+          float f0[16], f1[16];
+          const uint8_t* tp = tile_buf + q * 16 * 256 + cp * 4;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            uint32_t word = *reinterpret_cast<const uint32_t*>(tp + j * 256);
+            if (RHT_COL) word ^= (sign2 << (15 - j)) & 0x80008000u;
+            f0[j] = bf16_lo(word);
+            f1[j] = bf16_hi(word);
+          }
+          if (RHT_COL) {  // values are 4 * y from here on
+            float2 v[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = make_float2(f0[j], f1[j]);
+            fwht16_pairs(v);  // both columns in one pass of packed adds
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              f0[j] = v[j].x;
+              f1[j] = v[j].y;
+            }
+          }
+          uint32_t byte0, byte1;
+          float enc0, enc1;
+          if (BLOCK2D) {
+            enc0 = enc1 = reinterpret_cast<const float*>(smem + QuantSmem::kBlkEnc)[q * 8 + (cp >> 3)];
+            byte0 = byte1 = smem[QuantSmem::kBlkByte + q * 8 + (cp >> 3)];
+          } else {
+            const float m0 = amax16_3(f0), m1 = amax16_3(f1);
+            byte0 = block_scale_byte(RHT_COL ? 0.25f * m0 : m0, c_senc);
+            byte1 = block_scale_byte(RHT_COL ? 0.25f * m1 : m1, c_senc);
+            enc0 = enc_col[byte0];
+            enc1 = enc_col[byte1];
+          }
+          uint2 codes0, codes1;
+          if (SR) {
+            // low / high byte of ntwo[j] = 255 - draw of source element (row 16q + j, column 2cp / 2cp + 1)
+            uint32_t ntwo[16];
+            const uint8_t* rp = smem + QuantSmem::kRand + q * 16 * 128 + cp * 2;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) ntwo[j] = *reinterpret_cast<const uint16_t*>(rp + j * 128);
+            convert16x2_sr(f0, f1, enc0, enc1, ntwo, codes0, codes1);
+          } else {
+            const uint32_t none[4] = {0u, 0u, 0u, 0u};
+            codes0 = convert16<false>(f0, enc0, Nu14FromWords{none});
+            codes1 = convert16<false>(f1, enc1, Nu14FromWords{none});
+          }
+          // staging: column c holds eight 8-byte units, unit q stored at (q ^ (c >> 1)) & 7; the column a
+          // lane writes first alternates with bit 3 of the lane so that a half warp covers all banks
+#pragma unroll
+          for (int s = 0; s < 2; ++s) {
+            const int odd = s ^ sel;
+            const int c = 2 * cp + odd;
+            *reinterpret_cast<uint2*>(col_codes + c * 64 + (((q ^ (c >> 1)) & 7) << 3)) = odd ? codes1 : codes0;
+            const uint32_t byte = odd ? byte1 : byte0;
+            const int pos = a.c_swz ? ((q >> 2) * 512 + (c & 31) * 16 + (c >> 5) * 4 + (q & 3)) : (c * 8 + q);
+            sf_col[pos] = (uint8_t)byte;
+          }
         }
-        auto gather = [](uint32_t x) {  // four nibbles, one per byte -> 16 bits
-          const uint32_t t = (x | (x >> 4)) & 0x00FF00FFu;
-          return (t | (t >> 8)) & 0xFFFFu;
-        };
-        uint32_t lo[4], hi[4];
-#pragma unroll
-        for (int m = 0; m < 4; ++m) {
-          lo[m] = gather(w[m] & 0x0F0F0F0Fu);
-          hi[m] = gather((w[m] >> 4) & 0x0F0F0F0Fu);
-        }
-        const uint2 codes0 = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
-        const uint2 codes1 = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
-        const uint32_t byte = smem[QuantSmem::kBlkByte + q * 8 + (cp >> 3)];
-        const int sel = (lane >> 3) & 1;
-#pragma unroll
-        for (int s = 0; s < 2; ++s) {
-          const int odd = s ^ sel;
-          const int c = 2 * cp + odd;
-          *reinterpret_cast<uint2*>(smem + QuantSmem::kColCodes + c * 64 + (((q ^ (c >> 1)) & 7) << 3)) =
-              odd ? codes1 : codes0;
-          const int pos = a.c_swz ? ((q >> 2) * 512 + (c & 31) * 16 + (c >> 5) * 4 + (q & 3)) : (c * 8 + q);
-          smem[QuantSmem::kSfCol + pos] = (uint8_t)byte;
-        }
-        continue;
       }
-      float f0[16], f1[16];
-#pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const uint32_t word = *reinterpret_cast<const uint32_t*>(smem + QuantSmem::kTile + (q * 16 + j) * QuantSmem::kTilePitch + cp * 4);
-        f0[j] = bf16_lo(word);  // signs of the transform were applied when the tile was staged
-        f1[j] = bf16_hi(word);
-      }
-      if (RHT_COL) {  // values are 4 * y from here on; the 1/4 is folded into amax and encode scale (exact)
-        float2 v[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) v[j] = make_float2(f0[j], f1[j]);
-        fwht16_pairs(v);  // both columns in one pass of packed adds
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          f0[j] = v[j].x;
-          f1[j] = v[j].y;
-        }
-      }
-      uint32_t byte0, byte1;
-      float enc0, enc1;
-      if (BLOCK2D) {
-        enc0 = enc1 = reinterpret_cast<const float*>(smem + QuantSmem::kBlkEnc)[q * 8 + (cp >> 3)];
-        byte0 = byte1 = smem[QuantSmem::kBlkByte + q * 8 + (cp >> 3)];
-      } else {
-        block_scales(RHT_COL ? 0.25f * amax16(f0) : amax16(f0), c_senc, c_sdec, byte0, enc0);
-        block_scales(RHT_COL ? 0.25f * amax16(f1) : amax16(f1), c_senc, c_sdec, byte1, enc1);
-        if (RHT_COL) {
-          enc0 *= 0.25f;
-          enc1 *= 0.25f;
-        }
-      }
-      uint2 codes0, codes1;
-      if (SR) {
-        // low / high byte of ntwo[j] = 255 - draw of source element (row 16q + j, column 2cp / 2cp + 1)
-        uint32_t ntwo[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j)
-          ntwo[j] = *reinterpret_cast<const uint16_t*>(smem + QuantSmem::kRand + (q * 16 + j) * 128 +
-                                                      (((cp >> 3) ^ ((4 * q + (j >> 2)) & 7)) << 4) + (cp & 7) * 2);
-        convert16x2_sr(f0, f1, enc0, enc1, ntwo, codes0, codes1);
-      } else {
-        const uint32_t none[4] = {0u, 0u, 0u, 0u};
-        codes0 = convert16<false>(f0, enc0, Nu14FromWords{none});
-        codes1 = convert16<false>(f1, enc1, Nu14FromWords{none});
-      }
-      // staging: column c holds eight 8-byte units, unit q stored at (q ^ (c >> 1)) & 7; the column a
-      // lane writes first alternates with bit 3 of the lane so that a half warp covers all banks
-      const int sel = (lane >> 3) & 1;
-#pragma unroll
-      for (int s = 0; s < 2; ++s) {
-        const int odd = s ^ sel;
-        const int c = 2 * cp + odd;
-        uint2 val = odd ? codes1 : codes0;
-        *reinterpret_cast<uint2*>(smem + QuantSmem::kColCodes + c * 64 + (((q ^ (c >> 1)) & 7) << 3)) = val;
-        const uint32_t byte = odd ? byte1 : byte0;
-        const int pos = a.c_swz ? ((q >> 2) * 512 + (c & 31) * 16 + (c >> 5) * 4 + (q & 3)) : (c * 8 + q);
-        smem[QuantSmem::kSfCol + pos] = (uint8_t)byte;
-      }
-    }
-  }
-  __syncthreads();
+    };
+    if (full_tile)
+      phases_1_2(std::true_type{});
+    else
+      phases_1_2(std::false_type{});
+    __syncthreads();
+    if (*abort_flag) break;  // a wait expired (the word is read after the barrier: the same for every thread)
+    if (threadIdx.x == 0 && k + 2 < n_mine) issue_load(k + 2);  // every warp is done with this buffer
 
-  // ------------------------------------------------------------------ phase 3 ----
-  if (HAS_COL) {
-    const int64_t pitch = a.rows >> 1;  // bytes per row of the transposed copy
-    const bool vec16 = (a.rows & 31) == 0;
+    // ------------------------------------------------------------------ phase 3 ----
+    if (HAS_COL) {
+      const int64_t pitch = a.rows >> 1;  // bytes per row of the transposed copy
+      const bool vec16 = (a.rows & 31) == 0;
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      const int unit = threadIdx.x + 256 * k;
-      const int c = unit >> 2, m = unit & 3;  // column, pair of 16-row groups (2m, 2m+1)
-      if (col0 + c >= a.cols) continue;
-      const int x = (c >> 1) & 7;
-      const int base = ((2 * m) ^ x) & 6;
-      uint4 v = *reinterpret_cast<const uint4*>(smem + QuantSmem::kColCodes + c * 64 + base * 8);
-      if (x & 1) v = make_uint4(v.z, v.w, v.x, v.y);
-      uint8_t* dst = a.c_codes + (col0 + c) * pitch + (row0 >> 1) + m * 16;
-      const int64_t rr = row0 + 32 * m;
-      if (rr + 16 < a.rows && vec16) {
-        *reinterpret_cast<uint4*>(dst) = v;
+      for (int k = 0; k < 2; ++k) {
+        const int unit = threadIdx.x + 256 * k;
+        const int c = unit >> 2, m = unit & 3;  // column, pair of 16-row groups (2m, 2m+1)
+        if (col0 + c >= a.cols) continue;
+        const int x = (c >> 1) & 7;
+        const int base = ((2 * m) ^ x) & 6;
+        uint4 v = *reinterpret_cast<const uint4*>(col_codes + c * 64 + base * 8);
+        if (x & 1) v = make_uint4(v.z, v.w, v.x, v.y);
+        uint8_t* dst = a.c_codes + (col0 + c) * pitch + (row0 >> 1) + m * 16;
+        const int64_t rr = row0 + 32 * m;
+        if (rr + 16 < a.rows && vec16) {
+          *reinterpret_cast<uint4*>(dst) = v;
+        } else {
+          if (rr < a.rows) *reinterpret_cast<uint2*>(dst) = make_uint2(v.x, v.y);
+          if (rr + 16 < a.rows) *reinterpret_cast<uint2*>(dst + 8) = make_uint2(v.z, v.w);
+        }
+      }
+    }
+    // scale bytes
+#pragma unroll
+    for (int which = 0; which < 2; ++which) {
+      if (which == 0 && !HAS_ROW) continue;
+      if (which == 1 && !HAS_COL) continue;
+      const uint8_t* src = which == 0 ? sf_row : sf_col;
+      uint8_t* dst = which == 0 ? a.r_scales : a.c_scales;
+      const int swz = which == 0 ? a.r_swz : a.c_swz;
+      // the copy's row / block coordinates of this tile
+      const int64_t R0 = which == 0 ? row0 : col0, K0 = which == 0 ? (col0 >> 4) : (row0 >> 4);
+      const int64_t Rn = which == 0 ? a.rows : a.cols, n_kb = which == 0 ? n_cb : n_rb;
+      if (swz) {
+        if (threadIdx.x < 64) {
+          const int atom = threadIdx.x >> 5;
+          if (K0 + atom * 4 < n_kb) {
+            const int64_t off = ((R0 >> 7) * (n_kb >> 2) + (K0 >> 2) + atom) * 512 + (threadIdx.x & 31) * 16;
+            *reinterpret_cast<uint4*>(dst + off) = *reinterpret_cast<const uint4*>(src + threadIdx.x * 16);
+          }
+        }
       } else {
-        if (rr < a.rows) *reinterpret_cast<uint2*>(dst) = make_uint2(v.x, v.y);
-        if (rr + 16 < a.rows) *reinterpret_cast<uint2*>(dst + 8) = make_uint2(v.z, v.w);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int idx = threadIdx.x * 4 + k;
+          const int r = idx >> 3, kb = idx & 7;
+          if (R0 + r < Rn && K0 + kb < n_kb) dst[(R0 + r) * n_kb + K0 + kb] = src[idx];
+        }
       }
     }
   }
-  // scale bytes
-#pragma unroll
-  for (int which = 0; which < 2; ++which) {
-    if (which == 0 && !HAS_ROW) continue;
-    if (which == 1 && !HAS_COL) continue;
-    const uint8_t* src = smem + (which == 0 ? QuantSmem::kSfRow : QuantSmem::kSfCol);
-    uint8_t* dst = which == 0 ? a.r_scales : a.c_scales;
-    const int swz = which == 0 ? a.r_swz : a.c_swz;
-    // the copy's row / block coordinates of this tile
-    const int64_t R0 = which == 0 ? row0 : col0, K0 = which == 0 ? (col0 >> 4) : (row0 >> 4);
-    const int64_t Rn = which == 0 ? a.rows : a.cols, n_kb = which == 0 ? n_cb : n_rb;
-    if (swz) {
-      if (threadIdx.x < 64) {
-        const int atom = threadIdx.x >> 5;
-        if (K0 + atom * 4 < n_kb) {
-          const int64_t off = ((R0 >> 7) * (n_kb >> 2) + (K0 >> 2) + atom) * 512 + (threadIdx.x & 31) * 16;
-          *reinterpret_cast<uint4*>(dst + off) = *reinterpret_cast<const uint4*>(src + threadIdx.x * 16);
-        }
-      }
-    } else {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int idx = threadIdx.x * 4 + k;
-        const int r = idx >> 3, kb = idx & 7;
-        if (R0 + r < Rn && K0 + kb < n_kb) dst[(R0 + r) * n_kb + K0 + kb] = src[idx];
+  if (k < n_mine && threadIdx.x == 0) {
+    // left early: tiles k and k + 1 may still be in flight; give each one more bounded wait so that no copy lands
+    // in shared memory after the CTA has gone
+    for (int j = k; j < k + 2 && j < n_mine; ++j) {
+      const unsigned long long t0 = globaltimer_ns();
+      while (!mbar_try(bar0 + 8 * (j & 1), (uint32_t)(j >> 1) & 1u) && globaltimer_ns() - t0 < kWaitLimitNs) {
       }
     }
   }
@@ -703,17 +792,31 @@ cudaError_t launch_amax_rot_col_small(const QuantArgs& a, bool has_row, uint32_t
 template <bool HR, bool HC, bool B2, bool RR, bool RC, bool SR>
 static cudaError_t launch_quant_t(const QuantArgs& a, cudaStream_t s) {
   auto kern = quantize_kernel<HR, HC, B2, RR, RC, SR>;
-  using QuantSmem = QuantSmemFor<HC, B2, RC>;
-  const int smem = (SR && HC) ? QuantSmem::kBytesRand : QuantSmem::kBytesNoRand;
-  static std::atomic<uint64_t> configured{0};  // per call site (template instantiation) and device
+  constexpr bool kRowCodes = B2 && HR && HC;
+  constexpr int smem = QuantSmem::bytes(SR && HC && !kRowCodes, kRowCodes);
+  // the source as a 2-D tensor map: boxes of 128 x 128 bf16 (256-byte rows, no swizzle), zero fill outside
+  CUtensorMap map;
+  if (!make_map_2d(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.x, (uint64_t)a.cols, (uint64_t)a.rows,
+                   (uint64_t)a.ld * 2, 128, 128, false))
+    return cudaErrorInvalidValue;
+  // per call site (template instantiation) and device: the dynamic shared-memory limit, and how many CTAs the device
+  // keeps resident (the persistent grid)
+  static std::atomic<uint64_t> configured{0};
+  static std::atomic<int> resident[64] = {};
   int dev;
   if (device_needs_config(configured, &dev)) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, QuantSmem::kBytesRand);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
+    int sms = 0, per_sm = 0;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev < 0 ? 0 : dev)) != cudaSuccess) return e;
+    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 256, smem)) != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) resident[dev].store(sms * (per_sm > 0 ? per_sm : 1), std::memory_order_relaxed);
     device_configured(configured, dev);
   }
+  const int slots = (dev >= 0 && dev < 64) ? resident[dev].load(std::memory_order_relaxed) : 0;
   const int64_t tiles = (int64_t)a.tiles_r * a.tiles_c;
-  kern<<<(unsigned)tiles, 256, smem, s>>>(a);
+  const int64_t grid = (slots > 0 && tiles > slots) ? slots : tiles;
+  kern<<<(unsigned)grid, 256, smem, s>>>(map, a);
   count_launch();
   return cudaGetLastError();
 }

@@ -21,6 +21,7 @@ struct QuantArgs {
   uint32_t seed_lo, seed_hi, off_lo, off_hi, off_hi_col;
   uint32_t rk[20];       // Philox round keys (seed_lo + r * W0, seed_hi + r * W1), r = 0..9, filled by the host
   int tiles_r, tiles_c;  // 128 x 128 tiles of the source
+  unsigned int* status;  // device status word: a bounded wait that expired leaves its code here (may be NULL)
 };
 
 // Another transform size (quantize_rht.cu): d = 2, 4, 8 or 128 on the copies flagged rht_row / rht_col
