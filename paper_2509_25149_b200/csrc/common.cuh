@@ -108,10 +108,23 @@ __device__ __forceinline__ uint32_t e2m1x8_rne(const float v[8]) {
 //     stays zero, values just above 6 saturate as before.
 constexpr float kSrTowardsZero = 0.99999994f;  // 1 - 2^-24 = 0x3F7FFFFF
 
-// codes of w_lo in nibble 0 and of w_hi in nibble 2; rbits = (nu_hi << 24) | (nu_lo << 16) | 0x8080, nu = 255 - u
+// One conversion: code of w_lo in nibble 0 and of w_hi in nibble 2 of a 16-bit result;
+// rbits = (nu_hi << 24) | (nu_lo << 16) | 0x8080, nu = 255 - u.
 __device__ __forceinline__ uint32_t e2m1x2_sr(float w_lo, float w_hi, uint32_t rbits) {
   uint16_t d;
   asm("cvt.rs.satfinite.e2m1x4.f32 %0, {%1, %2, %1, %3}, %4;" : "=h"(d) : "f"(0.0f), "f"(w_hi), "f"(w_lo), "r"(rbits));
+  return d;
+}
+// Two conversions packed into one word: (a_lo, a_hi) in the low half, (b_lo, b_hi) in the high half
+__device__ __forceinline__ uint32_t e2m1x2_sr_pair(float a_lo, float a_hi, uint32_t ra, float b_lo, float b_hi,
+                                                   uint32_t rb) {
+  uint32_t d;
+  asm("{\n\t.reg .b16 t0, t1;\n\t"
+      "cvt.rs.satfinite.e2m1x4.f32 t0, {%1, %2, %1, %3}, %4;\n\t"
+      "cvt.rs.satfinite.e2m1x4.f32 t1, {%1, %5, %1, %6}, %7;\n\t"
+      "mov.b32 %0, {t0, t1};\n\t}"
+      : "=r"(d)
+      : "f"(0.0f), "f"(a_hi), "f"(a_lo), "r"(ra), "f"(b_hi), "f"(b_lo), "r"(rb));
   return d;
 }
 

@@ -389,11 +389,21 @@ __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant_
   const int sf_row_step = a.r_swz ? 64 : 32;
   const int64_t r_pitch = a.cols >> 1;  // bytes per row of the row-wise codes
 
+  // hoisted constants of phase 2: where a thread stages its two columns' codes and scale bytes (iteration it, column
+  // parity odd); the 16-byte unit of column pair cp and 16-row group q sits at cp * 128 + ((q ^ cp) & 7) * 16
+  const int col_codes_st = lane * 128 + (((warp ^ lane) & 7) << 4);  // + 4096 it
+  const int sf_col_pos = a.c_swz ? ((warp >> 2) * 512 + (lane & 15) * 32 + (lane >> 4) * 4 + (warp & 3)) : (lane * 16 + warp);
+  const int sf_col_odd = a.c_swz ? 16 : 8, sf_col_it = a.c_swz ? 8 : 512;
+
+  const int step_r = stride / a.tiles_c, step_c = stride - step_r * a.tiles_c;  // tile coordinates move by these
+  int tr = first >= 0 ? first / a.tiles_c : 0, tc = first >= 0 ? first - tr * a.tiles_c : 0;
   int k = 0;
-  for (; k < n_mine; ++k) {
+  for (; k < n_mine; ++k, tr -= step_r, tc -= step_c) {
+    if (tc < 0) {
+      tc += a.tiles_c;
+      --tr;
+    }
     const int buf = k & 1;
-    const int tile = first - k * stride;
-    const int tr = tile / a.tiles_c, tc = tile - tr * a.tiles_c;
     const int64_t row0 = (int64_t)tr * 128, col0 = (int64_t)tc * 128;
     const bool full_tile = (row0 + 128 <= a.rows) && (col0 + 128 <= a.cols);
     uint8_t* const col_codes = smem + QuantSmem::kColCodes + buf * 8192;
@@ -492,7 +502,6 @@ __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant_
 #pragma unroll 1
         for (int it = 0; it < 2; ++it) {
           const int cp = lane + 32 * it;  // column pair: tile columns 2cp, 2cp+1
-          const int sel = (lane >> 3) & 1;
           if (kNibbleTranspose) {
             // byte [row][cp] of the staged row-wise codes = (column 2cp in the low nibble, 2cp + 1 in the high one)
             uint32_t w[4];
@@ -516,14 +525,10 @@ __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant_
             const uint2 codes0 = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
             const uint2 codes1 = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
             const uint32_t byte = smem[QuantSmem::kBlkByte + q * 8 + (cp >> 3)];
-#pragma unroll
-            for (int s = 0; s < 2; ++s) {
-              const int odd = s ^ sel;
-              const int c = 2 * cp + odd;
-              *reinterpret_cast<uint2*>(col_codes + c * 64 + (((q ^ (c >> 1)) & 7) << 3)) = odd ? codes1 : codes0;
-              const int pos = a.c_swz ? ((q >> 2) * 512 + (c & 31) * 16 + (c >> 5) * 4 + (q & 3)) : (c * 8 + q);
-              sf_col[pos] = (uint8_t)byte;
-            }
+            *reinterpret_cast<uint4*>(col_codes + col_codes_st + it * 4096) =
+                make_uint4(codes0.x, codes0.y, codes1.x, codes1.y);
+            sf_col[sf_col_pos + it * sf_col_it] = (uint8_t)byte;
+            sf_col[sf_col_pos + it * sf_col_it + sf_col_odd] = (uint8_t)byte;
             continue;
           }
           float f0[16], f1[16];
@@ -571,17 +576,12 @@ __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant_
             codes0 = convert16<false>(f0, enc0, Nu14FromWords{none});
             codes1 = convert16<false>(f1, enc1, Nu14FromWords{none});
           }
-          // staging: column c holds eight 8-byte units, unit q stored at (q ^ (c >> 1)) & 7; the column a
-          // lane writes first alternates with bit 3 of the lane so that a half warp covers all banks
-#pragma unroll
-          for (int s = 0; s < 2; ++s) {
-            const int odd = s ^ sel;
-            const int c = 2 * cp + odd;
-            *reinterpret_cast<uint2*>(col_codes + c * 64 + (((q ^ (c >> 1)) & 7) << 3)) = odd ? codes1 : codes0;
-            const uint32_t byte = odd ? byte1 : byte0;
-            const int pos = a.c_swz ? ((q >> 2) * 512 + (c & 31) * 16 + (c >> 5) * 4 + (q & 3)) : (c * 8 + q);
-            sf_col[pos] = (uint8_t)byte;
-          }
+          // staging: both columns' eight bytes in one 16-byte unit (conflict-free: eight consecutive column pairs hit
+          // eight different units of a 128-byte line)
+          *reinterpret_cast<uint4*>(col_codes + col_codes_st + it * 4096) =
+              make_uint4(codes0.x, codes0.y, codes1.x, codes1.y);
+          sf_col[sf_col_pos + it * sf_col_it] = (uint8_t)byte0;
+          sf_col[sf_col_pos + it * sf_col_it + sf_col_odd] = (uint8_t)byte1;
         }
       }
     };
@@ -595,19 +595,20 @@ __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant_
 
     // ------------------------------------------------------------------ phase 3 ----
     if (HAS_COL) {
+      // a thread takes column pair cp and the 16-row groups (2m, 2m + 1): 16 bytes = 32 rows of each of its two columns
       const int64_t pitch = a.rows >> 1;  // bytes per row of the transposed copy
       const bool vec16 = (a.rows & 31) == 0;
+      const int cp = threadIdx.x >> 2, m = threadIdx.x & 3;
+      const uint8_t* unit = col_codes + cp * 128 + ((((2 * m) ^ cp) & 7) << 4);
+      const uint4 g0 = *reinterpret_cast<const uint4*>(unit);  // group 2m: (first column, second column) x 8 bytes
+      const uint4 g1 = *reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>((uintptr_t)unit ^ 16));
+      const int64_t rr = row0 + 32 * m;
 #pragma unroll
-      for (int k = 0; k < 2; ++k) {
-        const int unit = threadIdx.x + 256 * k;
-        const int c = unit >> 2, m = unit & 3;  // column, pair of 16-row groups (2m, 2m+1)
+      for (int odd = 0; odd < 2; ++odd) {
+        const int c = 2 * cp + odd;
         if (col0 + c >= a.cols) continue;
-        const int x = (c >> 1) & 7;
-        const int base = ((2 * m) ^ x) & 6;
-        uint4 v = *reinterpret_cast<const uint4*>(col_codes + c * 64 + base * 8);
-        if (x & 1) v = make_uint4(v.z, v.w, v.x, v.y);
+        const uint4 v = odd ? make_uint4(g0.z, g0.w, g1.z, g1.w) : make_uint4(g0.x, g0.y, g1.x, g1.y);
         uint8_t* dst = a.c_codes + (col0 + c) * pitch + (row0 >> 1) + m * 16;
-        const int64_t rr = row0 + 32 * m;
         if (rr + 16 < a.rows && vec16) {
           *reinterpret_cast<uint4*>(dst) = v;
         } else {

@@ -70,14 +70,13 @@ __device__ __forceinline__ uint2 convert16(const float (&f)[16], float s_enc_b, 
     out.x = e2m1x8_rne(lo);
     out.y = e2m1x8_rne(hi);
   } else {
-    uint32_t even[4], odd[4];  // nibbles 0 and 2 of each: elements (4k, 4k + 2) and (4k + 1, 4k + 3)
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      even[k] = e2m1x2_sr(v[4 * k], v[4 * k + 2], draws.rbits(4 * k, 4 * k + 2));
-      odd[k] = e2m1x2_sr(v[4 * k + 1], v[4 * k + 3], draws.rbits(4 * k + 1, 4 * k + 3));
-    }
-    out.x = (even[0] | (even[1] << 16)) | ((odd[0] | (odd[1] << 16)) << 4);
-    out.y = (even[2] | (even[3] << 16)) | ((odd[2] | (odd[3] << 16)) << 4);
+    // nibbles 0 and 2 of each 16-bit half: elements (4k, 4k + 2) in `even`, (4k + 1, 4k + 3) in `odd`, k = 0, 1 | 2, 3
+    const uint32_t even01 = e2m1x2_sr_pair(v[0], v[2], draws.rbits(0, 2), v[4], v[6], draws.rbits(4, 6));
+    const uint32_t odd01 = e2m1x2_sr_pair(v[1], v[3], draws.rbits(1, 3), v[5], v[7], draws.rbits(5, 7));
+    const uint32_t even23 = e2m1x2_sr_pair(v[8], v[10], draws.rbits(8, 10), v[12], v[14], draws.rbits(12, 14));
+    const uint32_t odd23 = e2m1x2_sr_pair(v[9], v[11], draws.rbits(9, 11), v[13], v[15], draws.rbits(13, 15));
+    out.x = even01 + odd01 * 16u;  // disjoint nibbles: the sum is the union
+    out.y = even23 + odd23 * 16u;
   }
   return out;
 }
@@ -106,17 +105,19 @@ __device__ __forceinline__ void convert16x2_sr(const float (&f0)[16], const floa
   float v0[16], v1[16];
   scale16<true>(f0, enc0, v0);
   scale16<true>(f1, enc1, v1);
-  uint32_t e[8];  // byte 0 = first column, rows (2m, 2m + 1); byte 1 = second column
+  // rows (r, r + 1) of both columns: byte 0 = first column, byte 1 = second column; rows (r + 2, r + 3) in bytes 2, 3
+  uint32_t e[4];
 #pragma unroll
-  for (int m = 0; m < 8; ++m) {
-    const uint32_t a = e2m1x2_sr(v0[2 * m], v1[2 * m], __byte_perm(ntwo[2 * m], 0x80808080u, 0x1044u));
-    const uint32_t b = e2m1x2_sr(v0[2 * m + 1], v1[2 * m + 1], __byte_perm(ntwo[2 * m + 1], 0x80808080u, 0x1044u));
-    e[m] = a | (b << 4);
+  for (int m = 0; m < 4; ++m) {
+    const int r = 4 * m;
+    const uint32_t a = e2m1x2_sr_pair(v0[r], v1[r], __byte_perm(ntwo[r], 0x80808080u, 0x1044u), v0[r + 2], v1[r + 2],
+                                      __byte_perm(ntwo[r + 2], 0x80808080u, 0x1044u));
+    const uint32_t b = e2m1x2_sr_pair(v0[r + 1], v1[r + 1], __byte_perm(ntwo[r + 1], 0x80808080u, 0x1044u), v0[r + 3],
+                                      v1[r + 3], __byte_perm(ntwo[r + 3], 0x80808080u, 0x1044u));
+    e[m] = a + b * 16u;  // disjoint nibbles
   }
-  const uint32_t p0 = __byte_perm(e[0], e[1], 0x5140u), p1 = __byte_perm(e[2], e[3], 0x5140u);
-  const uint32_t p2 = __byte_perm(e[4], e[5], 0x5140u), p3 = __byte_perm(e[6], e[7], 0x5140u);
-  out0 = make_uint2(__byte_perm(p0, p1, 0x5410u), __byte_perm(p2, p3, 0x5410u));
-  out1 = make_uint2(__byte_perm(p0, p1, 0x7632u), __byte_perm(p2, p3, 0x7632u));
+  out0 = make_uint2(__byte_perm(e[0], e[1], 0x6420u), __byte_perm(e[2], e[3], 0x6420u));
+  out1 = make_uint2(__byte_perm(e[0], e[1], 0x7531u), __byte_perm(e[2], e[3], 0x7531u));
 }
 
 __device__ __forceinline__ float amax16(const float (&f)[16]) {
