@@ -499,7 +499,7 @@ __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant_
       // ---------------------------------------------------------------- phase 2 ----
       if (HAS_COL) {
         const int q = warp;  // 16-row group inside the tile
-#pragma unroll 1
+#pragma unroll
         for (int it = 0; it < 2; ++it) {
           const int cp = lane + 32 * it;  // column pair: tile columns 2cp, 2cp+1
           if (kNibbleTranspose) {
