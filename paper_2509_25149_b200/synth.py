@@ -129,3 +129,53 @@ def config5_layer(layer: int, M: int = 16384) -> LinearProblem:
     return LinearProblem(f"cfg5_{name}_{M}x{N}x{K}", M, N, K, X,
                          normal_bf16((N, K), 0.02, s + W_ID),
                          normal_bf16((M, N), 1e-4, s + DY_ID), sr_offset=layer)
+
+
+# ---------------------------------------------------------------------------------------------
+# The same distributions drawn ON THE DEVICE, in row chunks (for the largest configs, where drawing on the host
+# would dominate a test): torch CUDA generator seeded like the host recipe.  The values differ from the host
+# recipe's (another generator); tests that use these read back the slabs they hand to the oracle.
+# ---------------------------------------------------------------------------------------------
+def _device_tensor(shape, seed: int, make, device="cuda", chunk_rows: int = 4096) -> torch.Tensor:
+    out = torch.empty(shape, dtype=torch.bfloat16, device=device)
+    g = torch.Generator(device=device).manual_seed(seed)
+    for r0 in range(0, shape[0], chunk_rows):
+        r1 = min(shape[0], r0 + chunk_rows)
+        out[r0:r1] = make((r1 - r0, shape[1]), g).to(torch.bfloat16)
+    return out
+
+
+def normal_bf16_device(shape, std: float, seed: int, device="cuda") -> torch.Tensor:
+    return _device_tensor(shape, seed, lambda sh, g: torch.randn(sh, generator=g, device=device) * std, device)
+
+
+def normal_with_outliers_bf16_device(shape, frac: float, factor: float, seed: int, device="cuda") -> torch.Tensor:
+    def make(sh, g):
+        x = torch.randn(sh, generator=g, device=device)
+        return torch.where(torch.rand(sh, generator=g, device=device) < frac, x * factor, x)
+    return _device_tensor(shape, seed, make, device)
+
+
+def squared_relu_bf16_device(shape, seed: int, device="cuda") -> torch.Tensor:
+    return _device_tensor(shape, seed, lambda sh, g: torch.clamp_min(torch.randn(sh, generator=g, device=device), 0).square_(),
+                          device)
+
+
+def config4_device(M: int = 8192, device="cuda") -> LinearProblem:
+    """cfg 4 (FFN down-projection, squared-ReLU input) with the tensors drawn on the device."""
+    s, N, K = 4000, 5120, 20480
+    return LinearProblem(f"cfg4_ffn_down_{M}x{N}x{K}", M, N, K, squared_relu_bf16_device((M, K), s + X_ID, device),
+                         normal_bf16_device((N, K), 0.01, s + W_ID, device),
+                         normal_bf16_device((M, N), 1e-4, s + DY_ID, device))
+
+
+def config5_layer_device(layer: int, M: int = 16384, device="cuda") -> LinearProblem:
+    """One of the four linears of a transformer block at 16384 tokens, drawn on the device."""
+    name, N, K = CONFIG5_LAYERS[layer]
+    s = 5000 + 10 * layer
+    if name == "ffn_down":
+        X = squared_relu_bf16_device((M, K), s + X_ID, device)
+    else:
+        X = normal_with_outliers_bf16_device((M, K), 0.001, 100.0, s + X_ID, device)
+    return LinearProblem(f"cfg5_{name}_{M}x{N}x{K}", M, N, K, X, normal_bf16_device((N, K), 0.02, s + W_ID, device),
+                         normal_bf16_device((M, N), 1e-4, s + DY_ID, device), sr_offset=layer)

@@ -106,8 +106,23 @@ def assert_rht_close(x_bits: np.ndarray, gpu: B.NVFP4Tensor, y_gpu, *, colwise, 
     ref = oracle.quantize(x_bits, colwise=colwise, rht=True, sign_mask=sign_mask, rounding=rounding, seed=seed,
                           sr_offset=sr_offset, amax_override=float(glob[0]), return_y=True, rht_dim=d)
     assert glob.view(np.uint32).tolist() == ref.glob.view(np.uint32).tolist(), f"{what}: s_dec from the same amax"
-    s_enc, s_dec = oracle.global_scale(float(glob[0]))
-    # (3) scale bytes
+    counts = compare_rotated(codes, scales, ref, float(glob[0]), rounding,
+                             lambda r, c: oracle.sr_draw(seed, sr_offset, (c if colwise else r) * x_bits.shape[1] +
+                                                         (r if colwise else c)), what)
+    total = ref.rows * ref.cols
+    assert counts["excused_codes"] + 16 * counts["excused_scales"] <= max(1e-3 * total, 16), f"{what}: too many excused items"
+    counts["elements"] = total
+    return counts
+
+
+def compare_rotated(codes, scales, ref, amax, rounding, draw, what=""):
+    """Steps (3) and (4) of the protocol for transformed copies, on a whole copy or on a slab of one.
+    codes / scales: the GPU's bytes (scales in the linear layout); ref: the oracle's copy of the same elements made
+    with the GPU's tensor amax and `return_y=True`; draw(r, c): the 8-bit draw of element (r, c) of the copy.
+    Scale bytes must be equal except where the pre-rounding scale is within 1e-5 of an E4M3 midpoint (then adjacent);
+    codes, in blocks whose scale agrees, equal except where the pre-rounding value is within 1e-5 of a rounding
+    threshold (then an adjacent grid point).  Returns the number of excused codes and scale bytes."""
+    s_enc, s_dec = oracle.global_scale(amax)
     R, C = ref.rows, ref.cols
     amax_b = np.abs(ref.y).reshape(R, C // 16, 16).max(axis=2)
     t_b = ((amax_b.astype(np.float32) / np.float32(6)) * np.float32(s_enc)).astype(np.float64)
@@ -117,7 +132,7 @@ def assert_rht_close(x_bits: np.ndarray, gpu: B.NVFP4Tensor, y_gpu, *, colwise, 
     sdiff = scales != ref.scales
     assert not np.any(sdiff & ~near), f"{what}: {np.count_nonzero(sdiff & ~near)} unexcused scale bytes"
     assert np.all(np.abs(scales.astype(int) - ref.scales.astype(int))[sdiff] == 1), f"{what}: excused scale not adjacent"
-    # (4) codes in blocks whose scale agrees
+    # codes in blocks whose scale agrees
     got, want = canon_zero(unpack(codes)), canon_zero(unpack(ref.codes))
     cdiff = (got != want) & ~np.repeat(sdiff, 16, axis=1)
     excused = 0
@@ -129,8 +144,7 @@ def assert_rht_close(x_bits: np.ndarray, gpu: B.NVFP4Tensor, y_gpu, *, colwise, 
             thr = E2M1_MIDPOINTS
             step = 0.5 if a < 2 else (1.0 if a < 4 else 2.0)
         else:
-            sr_, sc_ = (c, r) if colwise else (r, c)
-            u = oracle.sr_draw(seed, sr_offset, sr_ * x_bits.shape[1] + sc_)
+            u = draw(int(r), int(c))
             lo = E2M1_GRID[E2M1_GRID <= a].max()
             hi = E2M1_GRID[E2M1_GRID > a].min() if a < 6 else 6.0
             step = max(hi - lo, 0.5)
@@ -138,16 +152,25 @@ def assert_rht_close(x_bits: np.ndarray, gpu: B.NVFP4Tensor, y_gpu, *, colwise, 
         assert np.min(np.abs(thr - a)) <= 1e-5 * max(a, step), f"{what}: code at {(r, c)} differs away from a threshold (v={v})"
         assert abs(int(got[r, c] & 7) - int(want[r, c] & 7)) <= 1, f"{what}: excused code not adjacent"
         excused += 1
-    total = R * C
-    n_block_excused = int(np.count_nonzero(sdiff)) * 16
-    assert excused + n_block_excused <= max(1e-3 * total, 16), f"{what}: too many excused items"
     # blocks with an excused scale: decoded values still within one E2M1 step (in the block's own scale) of y
     if np.any(sdiff):
-        deq = oracle.dequantize(oracle.Quantized(codes, scales, glob, R, C))
+        glob = np.array([amax, s_dec], dtype=np.float32)
+        deq = oracle.dequantize(oracle.Quantized(np.ascontiguousarray(codes), np.ascontiguousarray(scales), glob, R, C))
         sb = np.vectorize(oracle.e4m3_decode)(scales).repeat(16, axis=1) * float(s_dec)
         m = np.repeat(sdiff, 16, axis=1)
         assert np.all(np.abs(deq - ref.y)[m] <= 2.0 * sb[m] * (1 + 2.0 ** -3) + 1e-30), f"{what}: excused block decode"
-    return {"excused_codes": excused, "excused_scales": int(np.count_nonzero(sdiff)), "elements": total}
+    return {"excused_codes": excused, "excused_scales": int(np.count_nonzero(sdiff))}
+
+
+def decode_rows(t: B.NVFP4Tensor, rows) -> np.ndarray:
+    """FP64 decode, by the oracle, of sampled rows of a device copy: the very bytes the GEMM reads."""
+    torch.cuda.synchronize()
+    rows = np.asarray(rows, dtype=np.int64)
+    codes = t.codes[torch.from_numpy(rows).to(t.codes.device)].cpu().numpy()
+    sc = t.scales.cpu().numpy()
+    sc = oracle.sf_unswizzle(sc, t.rows, t.cols // 16) if t.sf_layout == B.SF_SWIZZLED else sc.reshape(t.rows, t.cols // 16)
+    q = oracle.Quantized(np.ascontiguousarray(codes), np.ascontiguousarray(sc[rows]), t.glob.cpu().numpy(), len(rows), t.cols)
+    return oracle.dequantize(q)
 
 
 def gemm_reference(a: oracle.Quantized, b: oracle.Quantized, rows=None, cols=None):

@@ -28,14 +28,17 @@ def rotated_amax(x: torch.Tensor, mask: int) -> float:
 
 def check_copy_slabs(x: torch.Tensor, gpu: B.NVFP4Tensor, *, colwise, block_rows=1, rht=False, mask=0, rounding=0,
                      seed=0, sr_offset=0, what="", rht_dim=16):
+    """Three 128-row slabs of the source (first, interior, last) remade by the oracle with the GPU's tensor amax:
+    bit-exact for untransformed copies, the full tolerance protocol (threshold proximity of every differing scale
+    byte and code, adjacency, at most 1e-3 of the elements) for transformed ones."""
     codes, scales, glob = P.download(gpu)
-    R = x.shape[0]
+    R, n_cols = x.shape[0], x.shape[1]
     n_bad = n_tot = 0
-    for r0 in (0, (R // 128) * 5 // 8 * 128 + 0, R - 128):  # first, an interior and the last 128-row slab
-        slab = synth.bits(x[r0:r0 + 128])
+    for r0 in (0, (R // 128) * 5 // 8 * 128 + 0, R - 128):
+        slab = synth.bits(x[r0:r0 + 128].cpu())  # x may live on the device: only the slab comes to the host
         ref = oracle.quantize(slab, colwise=colwise, block_rows=block_rows, rht=rht, sign_mask=mask, rounding=rounding,
                               seed=seed, sr_offset=sr_offset, amax_override=float(glob[0]), sr_row0=r0,
-                              sr_cols=x.shape[1], rht_dim=rht_dim)
+                              sr_cols=n_cols, rht_dim=rht_dim, return_y=rht)
         assert glob.view(np.uint32)[1] == ref.glob.view(np.uint32)[1], f"{what}: s_dec"
         if colwise:
             got_c, got_s = codes[:, r0 // 2:(r0 + 128) // 2], scales[:, r0 // 16:(r0 + 128) // 16]
@@ -45,13 +48,11 @@ def check_copy_slabs(x: torch.Tensor, gpu: B.NVFP4Tensor, *, colwise, block_rows
             assert np.array_equal(got_s, ref.scales), f"{what}: scale bytes of slab {r0}"
             assert np.array_equal(got_c, ref.codes), f"{what}: codes of slab {r0}"
         else:
-            # rotated copies: equal except next to a rounding threshold (butterfly vs float64 summation order)
-            sd = got_s != ref.scales
-            assert np.all(np.abs(got_s.astype(int) - ref.scales.astype(int))[sd] <= 1), f"{what}: scale not adjacent"
-            g, w = P.canon_zero(P.unpack(got_c)), P.canon_zero(P.unpack(ref.codes))
-            cd = (g != w) & ~np.repeat(sd, 16, axis=1)
-            assert np.all(np.abs((g & 7).astype(int) - (w & 7).astype(int))[cd] <= 1), f"{what}: code not adjacent"
-            n_bad += int(cd.sum()) + 16 * int(sd.sum())
+            # element (r, c) of the slab's copy is source element (r0 + c, r) for a transposed copy, (r0 + r, c) else
+            draw = (lambda r, c: oracle.sr_draw(seed, sr_offset, (r0 + c) * n_cols + r)) if colwise else \
+                   (lambda r, c: oracle.sr_draw(seed, sr_offset, (r0 + r) * n_cols + c))
+            cnt = P.compare_rotated(got_c, got_s, ref, float(glob[0]), rounding, draw, f"{what}, slab {r0}")
+            n_bad += cnt["excused_codes"] + 16 * cnt["excused_scales"]
         n_tot += got_c.size * 2
     assert n_bad <= 1e-3 * n_tot, f"{what}: {n_bad} of {n_tot} elements differ"
 
@@ -70,39 +71,36 @@ class Operand:
         """The sampled rows of the copy, quantized by the oracle from the source (groups of 16 rows of the copy;
         the tensor amax is the GPU's, as the comparison protocol prescribes)."""
         amax = float(self.gpu.glob[0])
-        src_bits = synth.bits(self.src)
         n_cols = self.gpu.cols
         codes = np.zeros((len(rows), n_cols // 2), np.uint8)
         scales = np.zeros((len(rows), n_cols // 16), np.uint8)
         glob = None
         for i, r in enumerate(rows):
             g0 = (int(r) // 16) * 16
-            if self.colwise:
-                q = oracle.quantize(src_bits[:, g0:g0 + 16], amax_override=amax, sr_cols=self.src.shape[1], sr_col0=g0,
-                                    **self.kw)
+            if self.colwise:  # only the 16 source columns / rows of the group are brought to the host
+                q = oracle.quantize(synth.bits(self.src[:, g0:g0 + 16].cpu()), amax_override=amax,
+                                    sr_cols=self.src.shape[1], sr_col0=g0, **self.kw)
             else:
-                q = oracle.quantize(src_bits[g0:g0 + 16], amax_override=amax, sr_cols=self.src.shape[1], sr_row0=g0,
-                                    **self.kw)
+                q = oracle.quantize(synth.bits(self.src[g0:g0 + 16].cpu()), amax_override=amax,
+                                    sr_cols=self.src.shape[1], sr_row0=g0, **self.kw)
             codes[i], scales[i], glob = q.codes[int(r) - g0], q.scales[int(r) - g0], q.glob
         return oracle.Quantized(codes, scales, glob, len(rows), n_cols)
 
 
 def check_gemm_samples(D: torch.Tensor, A: Operand, Bt: Operand, bf16: bool, what: str, seed: int):
-    """Sampled rows x columns of a full-size product against the FP64 product of operand rows the ORACLE made from
-    the sources.  Operands with the transform may differ from the GPU's in the few codes the protocol excuses, so
-    for them a handful of outputs may exceed the bound by the size of one moved product."""
+    """Sampled rows x columns of a full-size product against the FP64 product of the decoded operands, held to
+    1e-3 * sum|a||b| (+ the output rounding for bf16) with no exceptions.  Untransformed operand rows are remade by
+    the ORACLE from the sources (their copies are bit-exact); for a transformed operand, whose copy may differ from
+    the oracle's in the codes the protocol excuses, the rows are the device copy's own bytes (checked against the
+    oracle by check_copy_slabs) decoded by the oracle: the GEMM is judged on the operands it was given."""
     rng = np.random.default_rng(seed)
     rows = np.sort(rng.choice(A.gpu.rows, 12, replace=False))
     cols = np.sort(rng.choice(Bt.gpu.rows, 384, replace=False))
-    a, b = A.oracle_rows(rows), Bt.oracle_rows(cols)
-    Dref, T = oracle.gemm_tn(oracle.dequantize(a), oracle.dequantize(b))
+    a = P.decode_rows(A.gpu, rows) if A.kw["rht"] else oracle.dequantize(A.oracle_rows(rows))
+    b = P.decode_rows(Bt.gpu, cols) if Bt.kw["rht"] else oracle.dequantize(Bt.oracle_rows(cols))
+    Dref, T = oracle.gemm_tn(a, b)
     got = D[torch.from_numpy(rows).cuda()][:, torch.from_numpy(cols).cuda()].float().cpu().numpy()
-    if A.kw["rht"] or Bt.kw["rht"]:
-        err = np.abs(got - Dref)
-        assert np.count_nonzero(err > 1e-3 * T + 1e-30) <= 1e-3 * err.size, what
-        assert np.all(err <= 2e-2 * T + 1e-30), what
-    else:
-        P.assert_gemm_close(got, Dref, T, bf16, what)
+    P.assert_gemm_close(got, Dref, T, bf16, what)
 
 
 def test_config3_full_size_forward_and_backward():

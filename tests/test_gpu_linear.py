@@ -45,22 +45,23 @@ def test_config1_forward_and_backward_match_the_oracle():
     w_col = oracle.quantize(wb, block_rows=16, colwise=True)
     Dref, T = P.gemm_reference(g_row, w_col)
     P.assert_gemm_close(dX.float().cpu().numpy(), Dref, T, True, "Dgrad")
-    # Wgrad: dW = dY_col X_col^T with both operands rotated.  X_col is an output, so it is checked by the
-    # protocol; the reference product is built from the oracle's own copies (X_col re-run on the GPU's amax, as
-    # the protocol prescribes; dY_col lives in the workspace), and the few codes the protocol may excuse are
-    # covered by the tolerance check below.
+    # Wgrad: dW = dY_col X_col^T with both operands rotated.  X_col is an output of the forward call; dY_col lives in
+    # the workspace and is reproduced by nvfp4_quantize with the same options (the kernels are deterministic).  Both
+    # copies go through the tolerance protocol against the oracle first; then dW is held to the GEMM bound against
+    # the FP64 product of those very operand bytes, decoded by the oracle, with no excused entries.
     y_col = B.nvfp4_rht16(p.X.cuda(), True, p.rht_sign_mask).cpu().numpy()
     P.assert_rht_close(xb, X_col, y_col, colwise=True, sign_mask=p.rht_sign_mask, rounding=oracle.RNE, what="X col")
-    _, _, glob = P.download(X_col)
-    x_col = oracle.quantize(xb, colwise=True, rht=True, sign_mask=p.rht_sign_mask, amax_override=float(glob[0]))
-    g_col = oracle.quantize(gb, colwise=True, rht=True, sign_mask=p.rht_sign_mask, rounding=oracle.SR,
-                            seed=p.sr_seed, sr_offset=p.sr_offset)
-    Dref, T = P.gemm_reference(g_col, x_col)
+    g_row_gpu, g_col_gpu = B.alloc_tensor(p.M, p.N), B.alloc_tensor(p.N, p.M)
+    B.nvfp4_quantize(p.dY.cuda(), B.quant_opts(rounding=B.ROUND_STOCHASTIC, rht_colwise=True,
+                                               rht_sign_mask=p.rht_sign_mask, seed=p.sr_seed, sr_offset=p.sr_offset),
+                     g_row_gpu, g_col_gpu)
+    P.assert_exact(g_row_gpu, g_row, "dY row")
+    g_y = B.nvfp4_rht16(p.dY.cuda(), True, p.rht_sign_mask).cpu().numpy()
+    P.assert_rht_close(gb, g_col_gpu, g_y, colwise=True, sign_mask=p.rht_sign_mask, rounding=oracle.SR,
+                       seed=p.sr_seed, sr_offset=p.sr_offset, what="dY col")
+    Dref, T = oracle.gemm_tn(P.decode_rows(g_col_gpu, np.arange(p.N)), P.decode_rows(X_col, np.arange(p.K)))
     dWn = dW.cpu().numpy()
-    err = np.abs(dWn - Dref)
-    # an excused code moves one element by one grid step: allow a handful of outputs beyond 1e-3 T
-    assert np.count_nonzero(err > 1e-3 * T) <= 1e-3 * err.size
-    assert np.all(err <= 2e-2 * T)
+    P.assert_gemm_close(dWn, Dref, T, False, "Wgrad")
     # and the whole layer approximates the unquantized gradients
     exact = p.dY.double().numpy().T @ p.X.double().numpy()
     assert np.linalg.norm(dWn - exact) / np.linalg.norm(exact) < 0.25
