@@ -304,6 +304,14 @@ NVFP4_API nvfp4_status nvfp4_rht16(const void* x_bf16, int64_t rows, int64_t col
  */
 NVFP4_API nvfp4_status nvfp4_device_status(void* cuda_stream, uint32_t* detail);
 
+/*
+ * Test aid for that path: enqueues a one-warp kernel that waits, for at most `limit_ns` nanoseconds
+ * (1 .. 100 000 000), on a barrier nobody arrives at.  The wait runs out, the kernel records the code
+ * 0x7E570001 in the status word and returns by itself; the next nvfp4_device_status() reports
+ * NVFP4_ERR_TIMEOUT with that code, and the device stays usable.  NVFP4_ERR_ARG for a limit out of range.
+ */
+NVFP4_API nvfp4_status nvfp4_test_wait_timeout(uint64_t limit_ns, void* cuda_stream);
+
 /* Tuning knob: which GEMM tiling to use.  128 / 256 = one CTA per 128 x 128 / 128 x 256 output tile;
  * 512 = a CTA pair per 256 x 256 tile (needs M % 256 == 0 and N % 256 == 0, otherwise 128 is used);
  * 768 = a CTA pair per 256 x 384 tile, plus up to two 256-wide tiles per row of tiles (needs M % 256 == 0,

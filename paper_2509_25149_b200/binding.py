@@ -22,7 +22,7 @@ FORMAT_NVFP4, FORMAT_MXFP4, FORMAT_NVFP4_ROWSCALE = 0, 1, 2
 
 EXPORTED = (
     "nvfp4_quantize", "nvfp4_gemm", "nvfp4_linear_fwd_workspace_bytes", "nvfp4_linear_bwd_workspace_bytes",
-    "nvfp4_linear_fwd", "nvfp4_linear_bwd", "nvfp4_dequantize", "nvfp4_rht16", "nvfp4_e2m1_sr", "nvfp4_device_status",
+    "nvfp4_linear_fwd", "nvfp4_linear_bwd", "nvfp4_dequantize", "nvfp4_rht16", "nvfp4_e2m1_sr", "nvfp4_test_wait_timeout", "nvfp4_device_status",
     "nvfp4_set_gemm_tile_n", "nvfp4_status_string", "nvfp4_launch_count",
     "nvfp4_linear_fwd_noalloc", "nvfp4_linear_fwd_noalloc_max_bytes",
     "nvfp4_gemm_bf16", "nvfp4_linear_bf16_fwd", "nvfp4_linear_bf16_bwd", "nvfp4_quant_error", "nvfp4_sq_error",
@@ -84,6 +84,7 @@ def lib() -> ctypes.CDLL:
         L.nvfp4_dequantize.restype, L.nvfp4_dequantize.argtypes = i32, [TP, vp, vp]
         L.nvfp4_rht16.restype, L.nvfp4_rht16.argtypes = i32, [vp, i64, i64, i64, i32, u32, vp, vp]
         L.nvfp4_e2m1_sr.restype, L.nvfp4_e2m1_sr.argtypes = i32, [vp, vp, i64, vp, vp]
+        L.nvfp4_test_wait_timeout.restype, L.nvfp4_test_wait_timeout.argtypes = i32, [ctypes.c_uint64, vp]
         L.nvfp4_device_status.restype, L.nvfp4_device_status.argtypes = i32, [vp, c.POINTER(u32)]
         L.nvfp4_set_gemm_tile_n.restype, L.nvfp4_set_gemm_tile_n.argtypes = i32, [i32]
         L.nvfp4_status_string.restype, L.nvfp4_status_string.argtypes = c.c_char_p, [i32]
@@ -300,6 +301,11 @@ def nvfp4_e2m1_sr(v: torch.Tensor, u: torch.Tensor) -> torch.Tensor:
     out = torch.empty(v.numel(), dtype=torch.uint8, device=v.device)
     _check(lib().nvfp4_e2m1_sr(v.data_ptr(), u.data_ptr(), v.numel(), out.data_ptr(), _stream()), "nvfp4_e2m1_sr")
     return out
+
+
+def nvfp4_test_wait_timeout(limit_ns: int) -> None:
+    """Enqueues the test kernel whose bounded wait runs out after `limit_ns` (the status word then holds 0x7E570001)."""
+    _check(lib().nvfp4_test_wait_timeout(limit_ns, _stream()), "nvfp4_test_wait_timeout")
 
 
 def nvfp4_device_status() -> int:

@@ -35,8 +35,11 @@ nvfp4_status check_copy(const nvfp4_tensor* t, int64_t rows, int64_t cols) {
   return NVFP4_OK;
 }
 
+// check_only: every argument check of the call, no launch (the composed calls validate all their steps first, so
+// that a rejected call has enqueued nothing)
 nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld, const nvfp4_quant_opts* o,
-                           const nvfp4_tensor* rowwise, const nvfp4_tensor* colwise, cudaStream_t s) {
+                           const nvfp4_tensor* rowwise, const nvfp4_tensor* colwise, cudaStream_t s,
+                           bool check_only = false) {
   if (!x || !o) return NVFP4_ERR_NULL;
   if (!rowwise && !colwise) return NVFP4_ERR_NULL;
   if (rows <= 0 || cols <= 0 || rows % 16 != 0 || cols % 16 != 0) return NVFP4_ERR_SHAPE;
@@ -52,6 +55,7 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
     if (rows > (int64_t)1 << 30 || cols > (int64_t)1 << 30) return NVFP4_ERR_SHAPE;
     nvfp4_status st0 = check_copy(rowwise, rows, cols);
     if (st0 != NVFP4_OK) return st0;
+    if (check_only) return NVFP4_OK;
     QuantArgs a{};
     a.x = static_cast<const uint16_t*>(x);
     a.rows = rows; a.cols = cols; a.ld = ld;
@@ -92,6 +96,7 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
   nvfp4_status st;
   if (rowwise && (st = check_copy(rowwise, rows, cols)) != NVFP4_OK) return st;
   if (colwise && (st = check_copy(colwise, cols, rows)) != NVFP4_OK) return st;
+  if (check_only) return NVFP4_OK;
 
   QuantArgs a{};
   a.x = static_cast<const uint16_t*>(x);
@@ -269,12 +274,9 @@ nvfp4_status nvfp4_linear_fwd(const void* X, const void* W, int64_t M, int64_t N
   if (fmt != NVFP4_FORMAT_NVFP4 && fmt != NVFP4_FORMAT_MXFP4) return NVFP4_ERR_ARG;  // per-tensor scales only
   if ((W_col_saved && W_col_saved->format != fmt) || (X_col_saved && X_col_saved->format != fmt)) return NVFP4_ERR_ARG;
 
-  if (!w_is_cached) {
-    nvfp4_quant_opts wo{};
-    wo.block_rows = fmt == NVFP4_FORMAT_MXFP4 ? 32 : 16;
-    wo.rounding = NVFP4_ROUND_NEAREST_EVEN;
-    if ((st = quantize_impl(W, N, K, K, &wo, W_row, W_col_saved, s)) != NVFP4_OK) return st;
-  }
+  nvfp4_quant_opts wo{};
+  wo.block_rows = fmt == NVFP4_FORMAT_MXFP4 ? 32 : 16;
+  wo.rounding = NVFP4_ROUND_NEAREST_EVEN;
   uint8_t* p = static_cast<uint8_t*>(workspace);
   if (opts->flags & NVFP4_LINEAR_ROW_SCALES) {
     // forward-only call: X gets a global scale per row in one pass (Appendix B.1, closing remark) and Fprop applies
@@ -291,6 +293,11 @@ nvfp4_status nvfp4_linear_fwd(const void* X, const void* W, int64_t M, int64_t N
     nvfp4_quant_opts ro{};
     ro.block_rows = 1;
     ro.rounding = NVFP4_ROUND_NEAREST_EVEN;
+    GemmArgs gy;  // every step is validated before the first launch
+    if (!w_is_cached && (st = quantize_impl(W, N, K, K, &wo, W_row, W_col_saved, s, true)) != NVFP4_OK) return st;
+    if ((st = quantize_impl(X, M, K, K, &ro, &x_rows, nullptr, s, true)) != NVFP4_OK) return st;
+    if ((st = gemm_prepare(&x_rows, W_row, Y_bf16, 0, N, 0, gy)) != NVFP4_OK) return st;
+    if (!w_is_cached && (st = quantize_impl(W, N, K, K, &wo, W_row, W_col_saved, s)) != NVFP4_OK) return st;
     if ((st = quantize_impl(X, M, K, K, &ro, &x_rows, nullptr, s)) != NVFP4_OK) return st;
     return gemm_impl(&x_rows, W_row, Y_bf16, 0, N, 0, s);
   }
@@ -302,6 +309,11 @@ nvfp4_status nvfp4_linear_fwd(const void* X, const void* W, int64_t M, int64_t N
   xo.rht_sign_mask = opts->rht_sign_mask;
   xo.rht_dim = opts->rht_dim;  // 0 = the format's own size; Appendix E.4.2's other sizes pass through
   for (int i = 0; i < 3; ++i) xo.rht_sign_mask_ext[i] = opts->rht_sign_mask_ext[i];
+  GemmArgs gy;  // every step is validated before the first launch
+  if (!w_is_cached && (st = quantize_impl(W, N, K, K, &wo, W_row, W_col_saved, s, true)) != NVFP4_OK) return st;
+  if ((st = quantize_impl(X, M, K, K, &xo, &x_row, X_col_saved, s, true)) != NVFP4_OK) return st;
+  if ((st = gemm_prepare(&x_row, W_row, Y_bf16, 0, N, 0, gy)) != NVFP4_OK) return st;
+  if (!w_is_cached && (st = quantize_impl(W, N, K, K, &wo, W_row, W_col_saved, s)) != NVFP4_OK) return st;
   if ((st = quantize_impl(X, M, K, K, &xo, &x_row, X_col_saved, s)) != NVFP4_OK) return st;
   return gemm_impl(&x_row, W_row, Y_bf16, 0, N, 0, s);
 }
@@ -338,6 +350,13 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, c
   go.seed = opts->seed;
   go.sr_offset = opts->sr_offset;
   go.flags = opts->flags & NVFP4_SR_INDEPENDENT_COPIES;
+  {  // every step is validated before the first launch
+    GemmArgs gchk;
+    if ((st = quantize_impl(dY, M, N, N, &go, dX_bf16 ? &g_row : nullptr, dW_fp32 ? &g_col : nullptr, s, true)) != NVFP4_OK)
+      return st;
+    if (dX_bf16 && (st = gemm_prepare(&g_row, W_col_saved, dX_bf16, 0, K, 0, gchk)) != NVFP4_OK) return st;
+    if (dW_fp32 && (st = gemm_prepare(&g_col, X_col_saved, dW_fp32, 1, K, accumulate_dw, gchk)) != NVFP4_OK) return st;
+  }
   if ((st = quantize_impl(dY, M, N, N, &go, dX_bf16 ? &g_row : nullptr, dW_fp32 ? &g_col : nullptr, s)) != NVFP4_OK)
     return st;
   if (dX_bf16 && dW_fp32) {
@@ -374,16 +393,16 @@ nvfp4_status nvfp4_linear_fwd_noalloc(const void* X, const void* W, int64_t M, i
   // `g_noalloc_scratch` names a host-side handle in host code, not a device address: ask the runtime for the
   // address once per device (with that device current) and hand that pointer to the kernels.
   constexpr int kMaxDevices = 64;
-  static void* scratch_of_device[kMaxDevices] = {};
+  static std::atomic<void*> scratch_of_device[kMaxDevices] = {};  // two host threads may make the first call at once
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return NVFP4_ERR_CUDA;
-  if (!scratch_of_device[dev]) {
-    void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return NVFP4_ERR_CUDA;
-    scratch_of_device[dev] = ptr;
+  void* scratch = scratch_of_device[dev].load(std::memory_order_acquire);
+  if (!scratch) {
+    if (cudaGetSymbolAddress(&scratch, g_noalloc_scratch) != cudaSuccess || !scratch) return NVFP4_ERR_CUDA;
+    scratch_of_device[dev].store(scratch, std::memory_order_release);  // every thread computes the same address
   }
-  return nvfp4_linear_fwd(X, W, M, N, K, opts, Y_bf16, X_col_saved, W_row, W_col_saved, w_is_cached,
-                          scratch_of_device[dev], NVFP4_NOALLOC_SCRATCH_BYTES, cuda_stream);
+  return nvfp4_linear_fwd(X, W, M, N, K, opts, Y_bf16, X_col_saved, W_row, W_col_saved, w_is_cached, scratch,
+                          NVFP4_NOALLOC_SCRATCH_BYTES, cuda_stream);
 }
 
 nvfp4_status nvfp4_gemm_bf16(const void* A, int32_t a_layout, int64_t lda, const void* B, int32_t b_layout, int64_t ldb,
@@ -489,6 +508,11 @@ nvfp4_status nvfp4_device_status(void* cuda_stream, uint32_t* detail) {
   if (read_device_status(static_cast<cudaStream_t>(cuda_stream), &code) != cudaSuccess) return NVFP4_ERR_CUDA;
   if (detail) *detail = code;
   return code ? NVFP4_ERR_TIMEOUT : NVFP4_OK;
+}
+
+nvfp4_status nvfp4_test_wait_timeout(uint64_t limit_ns, void* cuda_stream) {
+  if (limit_ns == 0 || limit_ns > 100000000ull) return NVFP4_ERR_ARG;  // at most 0.1 s
+  return launch_wait_probe(limit_ns, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
 int32_t nvfp4_set_gemm_tile_n(int32_t tile_n) {

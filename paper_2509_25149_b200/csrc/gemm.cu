@@ -617,6 +617,25 @@ cudaError_t launch_gemm_bf16(const DenseGemmArgs& g, cudaStream_t s) {
   return cudaGetLastError();
 }
 
+// Test aid: one warp waits, with the given limit, on a barrier nobody arrives at.  The wait runs out, the code lands
+// in the status word, the abort word stops the other lanes, and the kernel returns by itself.
+__global__ void wait_probe_kernel(unsigned long long limit_ns) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ uint32_t abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0u;
+  }
+  __syncthreads();
+  mbar_wait_limit(smem_u32(&bar), 0u, &abort_flag, kWaitProbeCode, limit_ns);
+}
+
+cudaError_t launch_wait_probe(unsigned long long limit_ns, cudaStream_t s) {
+  wait_probe_kernel<<<1, 32, 0, s>>>(limit_ns);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t device_status_word(unsigned int** word) {
   static std::atomic<unsigned int*> cache[64] = {};  // per device ordinal
   int dev = 0;

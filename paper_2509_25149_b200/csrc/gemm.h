@@ -30,6 +30,10 @@ cudaError_t launch_gemm_two(const GemmArgs& g0, const void* a0, const void* b0, 
 // Scheduling estimate: do 256 x 384 tiles beat 256 x 256 tiles for this problem (or pair of problems in one launch)?
 bool prefer_wide_tiles(const GemmArgs& g0, const GemmArgs* g1);
 cudaError_t read_device_status(cudaStream_t s, uint32_t* code);
+// test aid: a bounded wait that is made to run out (a barrier nobody arrives at); leaves kWaitProbeCode in the
+// status word and returns by itself
+constexpr uint32_t kWaitProbeCode = 0x7E570001u;
+cudaError_t launch_wait_probe(unsigned long long limit_ns, cudaStream_t s);
 // device address of the status word on the current device (for kernels of other translation units)
 cudaError_t device_status_word(unsigned int** word);
 

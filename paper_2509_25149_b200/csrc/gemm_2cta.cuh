@@ -183,12 +183,12 @@ __device__ __forceinline__ void tc2_mma_mxf4(uint32_t d_tmem, uint64_t adesc, ui
 }
 
 // Epilogue helper: 128 accumulator columns of one row per thread (registers) -> alpha, conversion -> 128-byte
-// swizzled rows of a staging buffer -> TMA store (or reduce-add) of 128 x 128-byte boxes.  Two staging buffers
-// alternate; a buffer is rewritten only after the store issued two boxes earlier has finished reading it.
+// swizzled rows of the group's staging buffer -> TMA store (or reduce-add) of 128 x 128-byte boxes.  A group has
+// ONE 16 KB buffer: a chunk is converted only after the store of the previous chunk has finished reading it.
 // BETA: the 128 columns additionally carry their own factors (float[128] in shared memory at `beta`).
 template <bool FP32, bool BETA = false>
 __device__ __forceinline__ void store_half(const uint32_t (&r)[128], float alpha, int et, int bar_id, int row_in_tile,
-                                           uint32_t stage_buf, int& buf, const CUtensorMap* map_d, int x0, int row0,
+                                           uint32_t stage_buf, const CUtensorMap* map_d, int x0, int row0,
                                            int accumulate, const float* beta = nullptr) {
   constexpr int kChunks = FP32 ? 4 : 2;
   constexpr int kChunkCols = FP32 ? 32 : 64;
@@ -233,7 +233,6 @@ __device__ __forceinline__ void store_half(const uint32_t (&r)[128], float alpha
         tma_store_2d(map_d, x0 + c * kChunkCols, row0, stage_buf);
       bulk_commit();
     }
-    buf ^= 1;
   }
 }
 
@@ -470,7 +469,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     const int row_in_tile = quad * 32 + lane;
     const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + half * 128;
     const uint32_t stage_buf = staging + half * 16384;
-    int buf = 0;
     for (int rnd = 0, tile = pair_id; tile < n_tiles; tile = next_tile(++rnd)) {
       int prob, m_blk, n_blk;
       tile_coords(tile, prob, m_blk, n_blk);
@@ -484,9 +482,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       // last one orders their use before the next tile's write
       if (b_rows) beta[et] = b_rows[2 * (int64_t)(n_blk * 256 + half * 128 + et) + 1];
       mbar_wait_cluster(accf_bar, acc_phase, abort_flag, 0x400u);
-      // agree on giving up: a warp that timed out still joins this barrier, then everyone reads the flag
-      asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-      if (*abort_flag) break;
+      // agree on giving up: a warp that timed out still joins this barrier, and all 128 threads take ONE decision
+      if (group_gave_up(abort_flag, bar_id, 128)) break;
       tc_fence_after();
       const int row0 = m_blk * 256 + (int)rank * 128;
       // read this warp's 32 lanes x 128 columns in one go and hand the accumulator back at once: the MMA issuer
@@ -500,16 +497,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       if (lane == 0) mbar_arrive_cluster(acce_leader);
       if (ROWS && b_rows) {
         if (d_is_fp32)
-          store_half<true, true>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, map_d, n_blk * 256 + half * 128,
+          store_half<true, true>(r, alpha, et, bar_id, row_in_tile, stage_buf, map_d, n_blk * 256 + half * 128,
                                  row0, accumulate, beta);
         else
-          store_half<false, true>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, map_d, n_blk * 256 + half * 128,
+          store_half<false, true>(r, alpha, et, bar_id, row_in_tile, stage_buf, map_d, n_blk * 256 + half * 128,
                                   row0, accumulate, beta);
       } else if (d_is_fp32) {
-        store_half<true>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, map_d, n_blk * 256 + half * 128, row0,
+        store_half<true>(r, alpha, et, bar_id, row_in_tile, stage_buf, map_d, n_blk * 256 + half * 128, row0,
                          accumulate);
       } else {
-        store_half<false>(r, alpha, et, bar_id, row_in_tile, stage_buf, buf, map_d, n_blk * 256 + half * 128, row0,
+        store_half<false>(r, alpha, et, bar_id, row_in_tile, stage_buf, map_d, n_blk * 256 + half * 128, row0,
                           accumulate);
       }
       acc_phase ^= 1u;

@@ -200,15 +200,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
     uint32_t acc_phase = 0;
     const int row_in_tile = quad * 32 + lane;
     const uint32_t stage_buf = staging + half * 16384;
-    int sbuf = 0, it = 0;
+    int it = 0;
     for (int tile = pair_id; tile < n_tiles; tile += n_pairs, ++it) {
       const int buf = it & 1;
       int m_blk, n_blk;
       tile_coords(tile, m_blk, n_blk);
       mbar_wait_cluster(accf_bar(buf), (acc_phase >> buf) & 1u, abort_flag, 0xC00u + buf);
-      // agree on giving up: a warp that timed out still joins this barrier, then everyone reads the flag
-      asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-      if (*abort_flag) break;
+      // agree on giving up: a warp that timed out still joins this barrier, and all 128 threads take ONE decision
+      if (group_gave_up(abort_flag, bar_id, 128)) break;
       tc_fence_after();
       const int row0 = m_blk * 256 + (int)rank * 128;
       const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + buf * 256 + half * 128;
@@ -220,10 +219,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(acce_bar(buf), 0));
       if (g.d_is_fp32)
-        store_half<true>(r, 1.0f, et, bar_id, row_in_tile, stage_buf, sbuf, &map_d, n_blk * 256 + half * 128, row0,
+        store_half<true>(r, 1.0f, et, bar_id, row_in_tile, stage_buf, &map_d, n_blk * 256 + half * 128, row0,
                          g.accumulate);
       else
-        store_half<false>(r, 1.0f, et, bar_id, row_in_tile, stage_buf, sbuf, &map_d, n_blk * 256 + half * 128, row0,
+        store_half<false>(r, 1.0f, et, bar_id, row_in_tile, stage_buf, &map_d, n_blk * 256 + half * 128, row0,
                           g.accumulate);
       acc_phase ^= 1u << buf;
     }

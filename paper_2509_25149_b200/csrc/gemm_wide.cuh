@@ -354,9 +354,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
       const int d_is_fp32 = g.p[prob].d_is_fp32, accumulate = g.p[prob].accumulate;
       const int cols_half = width >> 1, passes = cols_half >> 6;  // 192 / 3 or 128 / 2
       mbar_wait_cluster(accf_bar, acc_phase, abort_flag, 0x400u);
-      // agree on giving up: a warp that timed out still joins this barrier, then everyone reads the flag
-      asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-      if (*abort_flag) break;
+      // agree on giving up: a warp that timed out still joins this barrier, and all 128 threads take ONE decision
+      if (group_gave_up(abort_flag, bar_id, 128)) break;
       tc_fence_after();
       const int row0 = m_blk * 256 + (int)rank * 128;
       const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + half * cols_half;

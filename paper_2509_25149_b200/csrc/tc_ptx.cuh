@@ -13,8 +13,8 @@ namespace nvfp4 {
 __device__ unsigned int g_device_status = 0;
 
 // Bounded wait.  Returns false when the wait expired or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t code) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                uint32_t code, unsigned long long limit_ns) {
   if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
   uint32_t spins = 0;
@@ -22,13 +22,35 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try(bar, parity)) return true;
     if ((++spins & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      if (globaltimer_ns() - t0 > limit_ns) {
         *abort_flag = code;
         atomicCAS(&g_device_status, 0u, code);
         return false;
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t code) {
+  return mbar_wait_limit(bar, parity, abort_flag, code, kWaitLimitNs);
+}
+
+// One decision for a whole group of `count` threads on a named barrier: every thread contributes what it read from
+// the abort word BEFORE the barrier, and all of them get the OR.  (Reading the word after a plain barrier is not an
+// agreement: another role can set it between two threads' reads, and the threads that went on would then wait at a
+// barrier the others never reach.)
+__device__ __forceinline__ bool group_gave_up(volatile uint32_t* abort_flag, int bar_id, int count) {
+  const uint32_t mine = *abort_flag;
+  uint32_t any;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 p, %1, 0;\n\t"
+      "barrier.cta.red.or.pred.aligned q, %2, %3, p;\n\t"
+      "selp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(any)
+      : "r"(mine), "r"(bar_id), "r"(count)
+      : "memory");
+  return any != 0;
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }

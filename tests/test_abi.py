@@ -74,6 +74,22 @@ def test_argument_validation_happens_before_any_launch():
                               fake, 1 << 30, None) == 2
     assert L.nvfp4_linear_bwd(fake, None, None, 256, 256, 256, ctypes.byref(o), None, None, 0, fake, 1 << 30,
                               None) == 1
+    # the composed calls validate EVERY step before the first launch: an error found in a later step (an option the
+    # X quantizer rejects, a misaligned output of the GEMM) must leave the launch counter where it was
+    w_row, w_col = B.CTensor(fake, fake, fake, 256, 256, B.SF_SWIZZLED, 0), B.CTensor(fake, fake, fake, 256, 256, B.SF_SWIZZLED, 0)
+    x_col = B.CTensor(fake, fake, fake, 256, 256, B.SF_SWIZZLED, 0)
+    before = L.nvfp4_launch_count()
+    fwd = lambda opts, y, wr=w_row: L.nvfp4_linear_fwd(fake, fake, 256, 256, 256, ctypes.byref(opts), y, ctypes.byref(x_col),
+                                                       ctypes.byref(wr), ctypes.byref(w_col), 0, fake, 1 << 30, None)
+    assert fwd(o, fake + 2) == 3                                                               # Y not 16-byte aligned
+    mx = [B.CTensor(fake, fake, fake, 256, 256, B.SF_SWIZZLED, 1) for _ in range(3)]
+    assert L.nvfp4_linear_fwd(fake, fake, 256, 256, 256, ctypes.byref(B.quant_opts(rht_dim=8)), fake, ctypes.byref(mx[0]),
+                              ctypes.byref(mx[1]), ctypes.byref(mx[2]), 0, fake, 1 << 30, None) == 8  # MXFP4 + d = 8
+    assert L.nvfp4_linear_bwd(fake, ctypes.byref(x_col), ctypes.byref(w_col), 256, 256, 256, ctypes.byref(o), fake + 2,
+                              fake, 0, fake, 1 << 30, None) == 3                               # dX not aligned
+    assert L.nvfp4_linear_bwd(fake, ctypes.byref(x_col), ctypes.byref(w_col), 256, 256, 256,
+                              ctypes.byref(B.quant_opts(rht_dim=7)), fake, fake, 0, fake, 1 << 30, None) == 4
+    assert L.nvfp4_launch_count() == before
     # a row-scaled operand (format 2) pairs with NVFP4 only, and only on 256 x 256 tiles
     ar = B.CTensor(fake, fake, fake, 256, 256, B.SF_SWIZZLED, 2)
     bm = B.CTensor(fake, fake, fake, 256, 256, B.SF_SWIZZLED, 1)
