@@ -4,7 +4,9 @@ One step = one pass of the whole path over the FFN up-projection of the 12B-clas
 (tokens M = 8192, K = 5120, N = 20480): quantize W (16x16 blocks, both copies), quantize X (row-wise +
 rotated column-wise), Fprop, quantize dY (stochastic rounding, row-wise + rotated column-wise), Dgrad, Wgrad.
 With --gpus N each rank runs the step on its own 8192-token shard (data parallel, weak scaling) and the FP32
-weight gradient is summed across ranks with one NCCL all-reduce.
+weight gradient is summed across ranks with one NCCL all-reduce.  Under torch.distributed.run the ranks come from the
+environment; a plain `python bench.py --gpus N` starts the N ranks itself (re-running this script under
+torch.distributed.run, rendezvous on 127.0.0.1).
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded slab of the same workload.
 """
@@ -26,11 +28,13 @@ if ROOT not in sys.path:
 METRIC = "NVFP4 GEMM TFLOP/s vs FP4 peak; quantize+RHT+SR GB/s vs HBM peak"
 M, N, K = 8192, 20480, 5120
 WORKLOAD = "cfg3_ffn_up_fwd_bwd_M8192_K5120_N20480"
-# DRAM bytes (read + write) from a one-pass ncu capture of this workload at full size, cold caches
-# (profiles/dram_traffic_cfg3_step.md): the step's two GEMM launches divided by its three GEMMs, and the six quantizer
-# kernels summed.
+# DRAM bytes (read + write).  GEMMs: one-pass ncu capture of this workload at full size, cold caches
+# (profiles/dram_traffic_cfg3_step.md): the step's two GEMM launches divided by its three GEMMs.  Quantizer: ncu
+# captures of the three pass-2 kernels on the reduced --case shapes (profiles/quantize_kernel_dy_x_w.md), 2.80 / 2.73 /
+# 2.72 B per element for W / X / dY, scaled to the step's tensors by their element counts (traffic grows in
+# proportion), plus the amax passes at the 2 B per element the earlier full-size capture measured for them.
 GEMM_DRAM_BYTES_PER_LAUNCH = (547.2e6 + 1092.6e6) / 3  # Fprop launch + merged Dgrad/Wgrad launch, per GEMM
-QUANT_DRAM_BYTES_PER_STEP = 1509.3e6
+QUANT_DRAM_BYTES_PER_STEP = (N * K) * (2.80 + 2.0) + (M * K) * (2.73 + 2.0) + (M * N) * (2.72 + 2.0)
 SLAB = (4096, 2048, 5120)     # tokens, out-features, in-features of the CPU-baseline sample (one run)
 SLAB_REF = (512, 1024, 5120)  # per-step sample of the `--impl reference` arm (many steps)
 
@@ -68,7 +72,18 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([t.strip() for t in line.split(",")])
+            self.rows.append([time.time()] + [t.strip() for t in line.split(",")])
+
+    def median_sm_mhz(self, t0: float, t1: float):
+        """Median SM clock of the samples taken between two host times (None if there is none)."""
+        v = []
+        for r in list(self.rows):
+            try:
+                if t0 <= r[0] <= t1:
+                    v.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+        return statistics.median(v) if v else None
 
     def stop(self):
         if self.proc is None:
@@ -82,9 +97,9 @@ class ClockSampler:
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows:
             try:
-                sm.append(float(r[0]))
-                mx = float(r[1])
-                for nme, v in zip(names, r[3:7]):
+                sm.append(float(r[1]))
+                mx = float(r[2])
+                for nme, v in zip(names, r[4:8]):
                     if v.lower().startswith("active"):
                         reasons.add(nme)
             except (ValueError, IndexError):
@@ -168,14 +183,10 @@ def run_cuda(args):
     from paper_2509_25149_b200 import binding as B
     from paper_2509_25149_b200 import dp, synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
-    torch.cuda.set_device(local)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    ranks = dp.Ranks("nccl")
+    world, rank, local = ranks.world, ranks.rank, ranks.local
     B.lib()
     if args.gemm_tile:
         B.nvfp4_set_gemm_tile_n(args.gemm_tile)
@@ -212,18 +223,7 @@ def run_cuda(args):
         exchange.release(buf)  # asynchronous all-reduce; a no-op at N = 1
 
     drain = exchange.drain
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(ms: float) -> float:
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    barrier, max_over_ranks = ranks.barrier, ranks.max_over_ranks
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -233,19 +233,40 @@ def run_cuda(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-        time.sleep(0.3)
-    # ---- timed region: K steps, device-resident inputs --------------------------------------
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches0 = B.nvfp4_launch_count()
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    drain()
-    e1.record()
-    barrier()
-    launches = B.nvfp4_launch_count() - launches0
-    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps)
+    # ---- declared pre-load: the same step for >= args.preload seconds, so that the timed blocks start from the clock
+    # and power state of a loaded part (the step is power-capped: a region timed right after a pause runs ~10 % fast)
+    t_pre = time.perf_counter()
+    preload_steps = 0
+    while True:
+        for _ in range(20):
+            step()
+        drain()
+        torch.cuda.synchronize()
+        preload_steps += 20
+        if max_over_ranks(time.perf_counter() - t_pre) >= args.preload:
+            break
+    preload_s = time.perf_counter() - t_pre
+    # ---- timed region: args.blocks blocks of EXACTLY args.steps steps, device-resident inputs, each bracketed by a
+    # barrier + synchronize on both sides and timed with CUDA events (max over ranks); the median block is reported
+    ev = [torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)]
+    spans, launch_marks = [], []
+
+    def t_start():
+        launch_marks.append(B.nvfp4_launch_count())
+        spans.append([time.time(), None])
+        ev[0].record()
+
+    def t_stop():
+        ev[1].record()
+        torch.cuda.synchronize()
+        spans[-1][1] = time.time()
+        launch_marks[-1] = B.nvfp4_launch_count() - launch_marks[-1]
+        return ev[0].elapsed_time(ev[1])
+
+    block_ms = dp.timed_blocks(ranks, step, drain, args.steps, args.blocks, t_start, t_stop)
+    ms_step = statistics.median(block_ms)
+    launches = launch_marks[block_ms.index(ms_step)] if ms_step in block_ms else launch_marks[0]
+    block_mhz = [sampler.median_sm_mhz(a, b) if rank == 0 else None for a, b in spans]
     B.nvfp4_device_status()
 
     # ---- the same step with the quantized weight reused (micro-batches between optimizer steps): extra figure ----
@@ -291,7 +312,8 @@ def run_cuda(args):
         ("gemm_wgrad", lambda: B.nvfp4_gemm(g_col, X_col, dW)),
     ]
     per = {name: [] for name, _ in calls}
-    for it in range(args.steps + 2):
+    t_kern0 = time.time()
+    for it in range(min(args.steps, 100) + 2):
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)]
         evs[0].record()
         for i, (_, fn) in enumerate(calls):
@@ -302,7 +324,7 @@ def run_cuda(args):
             for i, (name, _) in enumerate(calls):
                 per[name].append(evs[i].elapsed_time(evs[i + 1]))
     B.nvfp4_device_status()
-    clocks = sampler.stop() if rank == 0 else None
+    kern_mhz = sampler.median_sm_mhz(t_kern0, time.time()) if rank == 0 else None
     kern_ms = {k: sum(v) / len(v) for k, v in per.items()}
 
     # the same layer kept in BF16 (Section 4.1 leaves a share of the layers in higher precision): context for the
@@ -382,21 +404,41 @@ def run_cuda(args):
     d2h = sum(t.numel() * t.element_size() for t in (hY, hdX, hdW))
 
     if rank == 0:
+        clocks = sampler.stop()
+        # the clock record of the timed blocks themselves (the key the timing rules ask for), the whole run beside it
+        timed_mhz = [m for m in block_mhz if m is not None]
+        clocks["sm_mhz_whole_run"] = clocks["sm_mhz"]
+        if timed_mhz:
+            clocks["sm_mhz"] = statistics.median(timed_mhz)
         peaks = measured_peaks()
         flops = step_flops()
         gemm_ms = (kern_ms["gemm_fprop"] + kern_ms["gemm_dgrad"] + kern_ms["gemm_wgrad"]) / 3
         gemm_tflops = 2.0 * M * N * K / (gemm_ms * 1e-3) / 1e12
-        fp4_peak = 4.0 * peaks["bf16_tflops_sustained"]  # FP4 : BF16 dense = 4 : 1 (nominal ratio)
+        # FP4 : BF16 dense = 4 : 1 (nominal ratio).  The denominator is the BURST bf16 figure: the GEMMs are timed one
+        # launch at a time between cooler quantizer kernels, not in a seconds-long GEMM-only loop
+        fp4_peak = 4.0 * peaks["bf16_tflops"]
+        per_gemm = {k: 2.0 * M * N * K / (kern_ms[k] * 1e-3) / 1e12 for k in ("gemm_fprop", "gemm_dgrad", "gemm_wgrad")}
+        # tensor-pipe occupancy at the sampled clock: 16384 dense FP4 MAC / clock / SM x 148 SMs (the 9 PFLOP/s of the
+        # datasheet correspond to 1.86 GHz at that rate; a derived figure, NVIDIA does not publish the per-SM rate)
+        mac_clk_sm, n_sm = 16384, 148
+        pipe = (lambda tf: tf * 1e12 / (kern_mhz * 1e6 * n_sm * mac_clk_sm * 2)) if kern_mhz else (lambda tf: None)
         # quantizer: algorithmic bytes = two reads of the bf16 tensor + both copies (codes + scales)
         q_elems = M * K + N * K + M * N
         # (MXFP4 has no tensor-level scale, hence one read, and one scale byte per 32 elements)
-        q_bytes = q_elems * ((2 + 2 * (0.5 + 1.0 / 32)) if mx else (2 + 2 + 2 * (0.5 + 1.0 / 16)))
+        bpe = (2 + 2 * (0.5 + 1.0 / 32)) if mx else (2 + 2 + 2 * (0.5 + 1.0 / 16))  # algorithmic bytes per element
+        q_bytes = q_elems * bpe
         q_ms = kern_ms["quant_W"] + kern_ms["quant_X"] + kern_ms["quant_dY"]
         q_gbs = q_bytes / (q_ms * 1e-3) / 1e9
         cpu, _ = cpu_baseline(1) if not (args.no_cpu_baseline or mx) else (None, 0)
         line = {
             "metric": METRIC, "value": world * flops / (ms_step * 1e-3) / 1e12, "unit": "TFLOP/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
+            # the timed region: args.blocks blocks of `steps` steps after a declared pre-load; ms_per_step is the median
+            # block; cycles_per_step = ms x median SM MHz of that block's samples (a clock-free figure)
+            "timing": {"preload_s": round(preload_s, 3), "preload_steps": preload_steps, "blocks": args.blocks,
+                       "block_ms_per_step": [round(b, 4) for b in block_ms],
+                       "block_sm_mhz": block_mhz,
+                       "mcycles_per_step": [round(b * m / 1e3, 1) if m else None for b, m in zip(block_ms, block_mhz)]},
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1",
             "data": "synthetic",
             "config": {"workload": WORKLOAD + ("_mxfp4" if mx else ""), "tokens_per_gpu": M, "in_features": K,
@@ -413,28 +455,34 @@ def run_cuda(args):
                            "fp4_step_speedup": ms_step_bf16 / ms_full_beside_bf16},
             "gemm_tflops": gemm_tflops, "quant_gbs": q_gbs,
             "kernel_ms": {k: round(v, 4) for k, v in kern_ms.items()},
-            "roofline": {"bound": "tensor", "kernel": "gemm_kernel (mean of Fprop, Dgrad, Wgrad)",
+            "roofline": {"bound": "tensor", "kernel": "gemm_pair_kernel / gemm_wide_kernel (mean of Fprop, Dgrad, Wgrad)",
                          "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
                          "frac": gemm_tflops / fp4_peak, "traffic": None if mx else GEMM_DRAM_BYTES_PER_LAUNCH,
                          "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum, full-size one-pass "
                                            "capture, mean of the three GEMMs (profiles/dram_traffic_cfg3_step.md)",
-                         "peak_source": f"4 x {peaks['source']} sustained bf16 cuBLAS ({peaks['bf16_tflops_sustained']} TFLOP/s)",
-                         "frac_of_burst": gemm_tflops / (4.0 * peaks["bf16_tflops"]),
-                         "frac_of_datasheet_9pf": gemm_tflops / 9000.0},
+                         "peak_source": f"4 x {peaks['source']} burst bf16 cuBLAS ({peaks['bf16_tflops']} TFLOP/s)",
+                         "frac_of_sustained": gemm_tflops / (4.0 * peaks["bf16_tflops_sustained"]),
+                         "frac_of_datasheet_9pf": gemm_tflops / 9000.0,
+                         "per_gemm": {k: {"tflops": round(v, 1), "frac": v / fp4_peak, "frac_of_datasheet_9pf": v / 9000.0,
+                                          "tensor_pipe_frac": pipe(v)} for k, v in per_gemm.items()},
+                         "tensor_pipe_frac": pipe(gemm_tflops), "tensor_pipe_sm_mhz": kern_mhz,
+                         "tensor_pipe_rate": "16384 FP4 MAC / clock / SM x 148 SMs (derived from the 9 PFLOP/s datasheet figure)"},
             "roofline_quant": {"bound": "hbm", "kernel": "amax kernels + quantize_kernel (W, X, dY)",
                                "achieved": q_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                "frac": q_gbs / peaks["hbm_gbs"], "traffic": None if mx else QUANT_DRAM_BYTES_PER_STEP,
                                "algorithmic_bytes": q_bytes,
                                "peak_source": f"{peaks['source']} copy bandwidth",
-                               "frac_of_datasheet_8tbs": q_gbs / 8000.0},
+                               "frac_of_datasheet_8tbs": q_gbs / 8000.0,
+                               "per_tensor": {k: {"gbs": round(e * bpe / (kern_ms[k] * 1e-3) / 1e9, 1),
+                                                  "frac": e * bpe / (kern_ms[k] * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+                                              for k, e in (("quant_W", N * K), ("quant_X", M * K), ("quant_dY", M * N))}},
             "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                     "overlap": "copies of neighbouring steps overlap the kernels (double-buffered)"},
             "gpu_launches": launches, "clocks": clocks, "cpu_baseline": cpu,
         }
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    ranks.close()
 
 
 # ------------------------------------------------- single-kernel cases (profiling) ----
@@ -693,6 +741,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--blocks", type=int, default=5, help="timed blocks of --steps steps; the median block is reported")
+    ap.add_argument("--preload", type=float, default=1.0, help="seconds of the same step run before the timed blocks")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--gemm-tile", type=int, default=0, choices=[0, 128, 256, 512, 768],
                     help="force a GEMM tile configuration (0: the library's choice); for experiments")
@@ -705,6 +755,10 @@ def main():
         run_config(args)
     elif args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain `python bench.py --gpus N`: start the N ranks (one per GPU) ourselves
+        from paper_2509_25149_b200 import dp
+        sys.exit(dp.spawn_ranks(args.gpus, os.path.abspath(__file__), sys.argv[1:]))
     else:
         run_cuda(args)
 

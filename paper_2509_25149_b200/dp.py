@@ -6,6 +6,11 @@ replicas (paper Section 4.1: weight gradients are accumulated in FP32 across dat
 """
 from __future__ import annotations
 
+import os
+import socket
+import subprocess
+import sys
+
 import torch
 import torch.distributed as dist
 
@@ -93,3 +98,73 @@ class OverlappedGradExchange:
         for i, w in enumerate(self.pending):
             wait_weight_grad(w)
             self.pending[i] = None
+
+
+# ---------------------------------------------------------------------------------------------
+# Rank plumbing of a benchmark / training loop: one process per GPU, started by torch.distributed.run (or by
+# `spawn_ranks`, which starts it), the timed region bracketed by a barrier on both sides and timed as the maximum
+# over ranks.  Backend "nccl" for GPUs, "gloo" for the CPU tests of the same loop.
+# ---------------------------------------------------------------------------------------------
+def free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(n: int, script: str, argv: list[str]) -> int:
+    """Re-runs `script argv` as n ranks on this node under torch.distributed.run (rendezvous on 127.0.0.1);
+    the ranks' output goes to this process's stdout / stderr.  Returns the launcher's exit code."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr",
+           "127.0.0.1", "--master-port", str(free_port()), script, *argv]
+    return subprocess.run(cmd).returncode
+
+
+class Ranks:
+    """World size, rank and local rank from the launcher's environment, and the process group built from them."""
+
+    def __init__(self, backend: str, cuda_device: int | None = None):
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        self.cuda = backend == "nccl"
+        self.device = torch.device("cuda", self.local if cuda_device is None else cuda_device) if self.cuda else torch.device("cpu")
+        if self.world > 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            if self.cuda:
+                dist.init_process_group("nccl", device_id=self.device)
+            else:
+                dist.init_process_group(backend)
+
+    def barrier(self) -> None:
+        if self.world > 1:
+            dist.barrier()
+        if self.cuda:
+            torch.cuda.synchronize()
+
+    def max_over_ranks(self, value: float) -> float:
+        if self.world == 1:
+            return value
+        t = torch.tensor([value], dtype=torch.float64, device=self.device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def close(self) -> None:
+        if self.world > 1 and dist.is_initialized():
+            dist.destroy_process_group()
+
+
+def timed_blocks(ranks: Ranks, step, drain, steps: int, blocks: int, start, stop) -> list[float]:
+    """`blocks` timed regions of exactly `steps` calls of step() followed by drain(), each bracketed by a barrier on
+    both sides; start() / stop() are the caller's timer (stop returns the region's milliseconds).  Returns the
+    milliseconds per step of every block, maximum over ranks."""
+    out = []
+    for _ in range(blocks):
+        ranks.barrier()
+        start()
+        for _ in range(steps):
+            step()
+        drain()
+        ms = stop()
+        ranks.barrier()
+        out.append(ranks.max_over_ranks(ms / steps))
+    return out

@@ -3,6 +3,8 @@ FP32 all-reduce of the weight gradient.  The per-rank arithmetic is done by the 
 unchanged by data parallelism."""
 import os
 import socket
+import sys
+import time
 
 import numpy as np
 import torch
@@ -107,3 +109,59 @@ def test_token_shard_and_offsets():
     o = torch.empty(4)
     dp.reduce_scatter_weight_grad(t, o)
     assert torch.equal(o, t) and dp.weight_grad_shard(20480, 1, 8) == (2560, 5120)
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# The rank loop of bench.py (barrier, exactly K steps, drain, barrier; time = max over ranks; overlapped exchange of
+# the weight gradient) driven by a stub step on two gloo ranks
+# ---------------------------------------------------------------------------------------------------------------
+def _loop_worker(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world),
+                      LOCAL_RANK=str(rank))
+    ranks = dp.Ranks("gloo")
+    try:
+        assert (ranks.world, ranks.rank, ranks.local) == (world, rank, rank) and not ranks.cuda
+        ex = dp.OverlappedGradExchange(torch.zeros(4))
+        calls = {"n": 0}
+
+        def step():  # stands for fwd + bwd: "Wgrad" writes the buffer, the exchange sums it across ranks
+            buf = ex.acquire()
+            buf.fill_(float(calls["n"] + 1) * (rank + 1))
+            ex.release(buf)
+            calls["n"] += 1
+            time.sleep(0.002 * (rank + 1))  # rank 1 is the slow one
+
+        t = [0.0]
+        start = lambda: t.__setitem__(0, time.perf_counter())
+        stop = lambda: (time.perf_counter() - t[0]) * 1e3
+        blocks = dp.timed_blocks(ranks, step, ex.drain, steps=5, blocks=3, start=start, stop=stop)
+        assert calls["n"] == 15 and len(blocks) == 3
+        assert all(b >= 0.002 * world * 1e3 * 0.9 for b in blocks), blocks  # the maximum over ranks: the slow rank's time
+        last = ex.buffers[(calls["n"] - 1) % 2]
+        assert float(last[0]) == 15.0 * sum(r + 1 for r in range(world))  # drained: the last sum is complete
+        assert ranks.max_over_ranks(float(rank)) == float(world - 1)
+        torch.save(torch.tensor(blocks), os.path.join(out_dir, f"blocks{rank}.pt"))
+    finally:
+        ranks.close()
+
+
+def test_bench_rank_loop_with_a_stub_step(tmp_path):
+    mp.spawn(_loop_worker, args=(2, _free_port(), str(tmp_path)), nprocs=2, join=True)
+    b0, b1 = torch.load(tmp_path / "blocks0.pt"), torch.load(tmp_path / "blocks1.pt")
+    assert torch.equal(b0, b1)  # every rank reports the same (maximum) time
+
+
+def test_spawn_ranks_starts_one_process_per_rank(tmp_path):
+    """`bench.py --gpus N` without a launcher re-runs itself through dp.spawn_ranks; here a two-line rank script."""
+    script = tmp_path / "rank_script.py"
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    script.write_text(
+        "import os, sys\n"
+        f"sys.path.insert(0, {root!r})\n"
+        "from paper_2509_25149_b200 import dp\n"
+        "r = dp.Ranks('gloo')\n"
+        "r.barrier()\n"
+        "open(os.path.join(sys.argv[1], f'rank{r.rank}of{r.world}'), 'w').write(str(r.max_over_ranks(float(r.rank))))\n"
+        "r.close()\n")
+    assert dp.spawn_ranks(2, str(script), [str(tmp_path)]) == 0
+    assert (tmp_path / "rank0of2").read_text() == "1.0" and (tmp_path / "rank1of2").read_text() == "1.0"
