@@ -506,6 +506,10 @@ CASES = {
     "quant_x_rowscale": ("q_rows", 16384, 5120, 0),  # App. B.1 closing remark: one pass, global scale per row, RNE
     "quant_dy_rowscale": ("q_rows_sr", 4096, 20480, 0),  # the same with stochastic rounding on gradient-shaped rows
     "quant_error": ("qerr", 4096, 20480, 0),        # Appendix E.2: decode-and-compare reduction (2.5625 B / element)
+    # what bounds a 256-deep k-block of the CTA-pair GEMM: SM cycles and nanoseconds per k-block, measured inside the
+    # kernel, for the full loop and with parts switched off, on all 74 SM pairs and on 37 (balanced shape: 6 tiles of
+    # 80 k-blocks per pair)
+    "gemm_cycles": ("gemm_cycles", 256 * 74, 1536, 20480),
 }
 
 
@@ -522,6 +526,8 @@ def run_case(args):
         B.nvfp4_set_gemm_tile_n(args.gemm_tile)
     g = torch.Generator(device="cuda").manual_seed(1)
     mask = synth.DEFAULT_RHT_SIGN_MASK
+    if kind == "gemm_cycles":
+        return run_gemm_cycles(args, r, c, k)
     if kind == "step":
         X = torch.randn((r, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
         W = (torch.randn((c, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
@@ -635,6 +641,60 @@ def run_case(args):
     B.nvfp4_device_status()
     ms = e0.elapsed_time(e1) / args.steps
     print(json.dumps({"case": args.case, "shape": [r, c, k], "ms": ms, "value": work / (ms * 1e-3), "unit": unit}))
+
+
+def run_gemm_cycles(args, m, n, k):
+    """Table of SM cycles / nanoseconds / effective SM clock per 256-deep k-block of the CTA-pair GEMM (256 x 256
+    tiles), read from the kernel's own cycle and nanosecond counters: everything on, MMAs only, loads only, scale path
+    off, each on all SM pairs and on half of them.  The variants alternate inside one process (`--steps` launches per
+    turn, 4 turns) so that all see the same box and power state."""
+    import torch
+
+    from paper_2509_25149_b200 import binding as B
+
+    g = torch.Generator(device="cuda").manual_seed(1)
+    a_src = torch.randn((m, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    b_src = (torch.randn((n, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
+    A, Bq = B.alloc_tensor(m, k), B.alloc_tensor(n, k)
+    B.nvfp4_quantize(a_src, B.quant_opts(), A, None)
+    B.nvfp4_quantize(b_src, B.quant_opts(block_rows=16), Bq, None)
+    del a_src, b_src
+    D = torch.empty((m, n), dtype=torch.bfloat16, device="cuda")
+    B.nvfp4_set_gemm_tile_n(512)
+    n_pairs = torch.cuda.get_device_properties(0).multi_processor_count // 2
+    probe = torch.zeros(8 * n_pairs, dtype=torch.int64, device="cuda")
+    variants = [("all on", 0), ("no MMAs (loads + scale path)", 1), ("no operand loads (MMAs + scale path)", 2),
+                ("no scale path (loads + MMAs)", 4), ("MMAs only", 6)]
+    rows = {}
+    for turn in range(4):
+        for pairs in (n_pairs, n_pairs // 2):
+            for name, mode in variants:
+                B.nvfp4_set_gemm_experiment(mode, pairs, probe)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                for _ in range(3):
+                    B.nvfp4_gemm(A, Bq, D)
+                e0.record()
+                for _ in range(args.steps):
+                    B.nvfp4_gemm(A, Bq, D)
+                e1.record()
+                torch.cuda.synchronize()
+                p = probe.view(-1, 8)[:pairs].cpu().double()  # the last launch's counters
+                cyc, ns, kb, tiles, wait = p[:, 0], p[:, 1], p[:, 2], p[:, 3], p[:, 4]
+                rows.setdefault((name, pairs), []).append(
+                    (float((cyc / kb).median()), float((ns / kb).median()), float((cyc / ns).median()) * 1e3,
+                     e0.elapsed_time(e1) / args.steps, float((wait / tiles).median())))
+    B.nvfp4_set_gemm_experiment(0, 0, None)
+    B.nvfp4_set_gemm_tile_n(0)
+    B.nvfp4_device_status()
+    table = []
+    for (name, pairs), v in rows.items():
+        t = torch.tensor(v).median(dim=0).values.tolist()
+        table.append({"variant": name, "pairs": pairs, "cycles_per_kblock": round(t[0], 1), "ns_per_kblock": round(t[1], 1),
+                      "sm_mhz": round(t[2], 0), "launch_ms": round(t[3], 4),
+                      "handover_wait_cycles_per_tile": round(t[4], 0)})
+    print(json.dumps({"case": "gemm_cycles", "shape": [m, n, k], "k_blocks_per_pair": (m // 256) * (n // 256) * (k // 256) // n_pairs,
+                      "mma_cycles_per_kblock_at_16384_mac_per_clk_sm": 4 * 256 * 256 * 64 / (2 * 16384),
+                      "launches_per_turn": args.steps, "turns": 4, "table": table}))
 
 
 # ------------------------------------------- other 12B-class configs (extra measurements) ----

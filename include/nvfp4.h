@@ -321,6 +321,22 @@ NVFP4_API nvfp4_status nvfp4_test_wait_timeout(uint64_t limit_ns, void* cuda_str
  * beyond FP32 summation order. */
 NVFP4_API int32_t nvfp4_set_gemm_tile_n(int32_t tile_n);
 
+/*
+ * Measurement aid for the main loop of the CTA-pair GEMM with 256 x 256 tiles (what bounds a 256-deep k-block):
+ * affects that kernel's later launches in this process; (0, 0, NULL) restores normal operation.
+ *   mode      bit 0: the issuer skips the MMAs; bit 1: the producer skips the operand loads; bit 2: the scale atoms
+ *             are neither loaded nor copied to tensor memory; bit 3: the epilogue hands the accumulator back
+ *             unread and stores nothing; bit 4: the issuer does not wait for the accumulator to be handed back.
+ *             With any bit set the OUTPUT IS MEANINGLESS (timing
+ *             only); every barrier is still signalled, so the kernel runs to its end.
+ *   max_pairs > 0: at most that many CTA pairs (SM pairs) take part.
+ *   probe     device array of 8 x uint64 per pair; each pair's issuer writes five: SM cycles and nanoseconds of its
+ *             main loop, the k-blocks and the tiles it went through, and the cycles it spent between issuing a
+ *             tile's last MMA and getting the accumulator back from the epilogue.
+ * Returns 0, or -1 for a value out of range.
+ */
+NVFP4_API int32_t nvfp4_set_gemm_experiment(int32_t mode, int32_t max_pairs, void* probe);
+
 NVFP4_API const char* nvfp4_status_string(nvfp4_status s);
 /* Number of kernel launches this process has enqueued through the library so far. */
 NVFP4_API uint64_t nvfp4_launch_count(void);

@@ -23,7 +23,7 @@ FORMAT_NVFP4, FORMAT_MXFP4, FORMAT_NVFP4_ROWSCALE = 0, 1, 2
 EXPORTED = (
     "nvfp4_quantize", "nvfp4_gemm", "nvfp4_linear_fwd_workspace_bytes", "nvfp4_linear_bwd_workspace_bytes",
     "nvfp4_linear_fwd", "nvfp4_linear_bwd", "nvfp4_dequantize", "nvfp4_rht16", "nvfp4_e2m1_sr", "nvfp4_test_wait_timeout", "nvfp4_device_status",
-    "nvfp4_set_gemm_tile_n", "nvfp4_status_string", "nvfp4_launch_count",
+    "nvfp4_set_gemm_tile_n", "nvfp4_set_gemm_experiment", "nvfp4_status_string", "nvfp4_launch_count",
     "nvfp4_linear_fwd_noalloc", "nvfp4_linear_fwd_noalloc_max_bytes",
     "nvfp4_gemm_bf16", "nvfp4_linear_bf16_fwd", "nvfp4_linear_bf16_bwd", "nvfp4_quant_error", "nvfp4_sq_error",
 )
@@ -87,6 +87,7 @@ def lib() -> ctypes.CDLL:
         L.nvfp4_test_wait_timeout.restype, L.nvfp4_test_wait_timeout.argtypes = i32, [ctypes.c_uint64, vp]
         L.nvfp4_device_status.restype, L.nvfp4_device_status.argtypes = i32, [vp, c.POINTER(u32)]
         L.nvfp4_set_gemm_tile_n.restype, L.nvfp4_set_gemm_tile_n.argtypes = i32, [i32]
+        L.nvfp4_set_gemm_experiment.restype, L.nvfp4_set_gemm_experiment.argtypes = i32, [i32, i32, vp]
         L.nvfp4_status_string.restype, L.nvfp4_status_string.argtypes = c.c_char_p, [i32]
         L.nvfp4_launch_count.restype, L.nvfp4_launch_count.argtypes = c.c_uint64, []
         _lib = L
@@ -315,6 +316,13 @@ def nvfp4_device_status() -> int:
     if st != OK:
         raise NVFP4Error(st, f"nvfp4_device_status (code 0x{detail.value:x})")
     return 0
+
+
+def nvfp4_set_gemm_experiment(mode: int = 0, max_pairs: int = 0, probe: Optional[torch.Tensor] = None) -> None:
+    """Measurement aid of the CTA-pair GEMM (see the header); probe: int64 device tensor of 8 words per pair."""
+    assert probe is None or (probe.dtype == torch.int64 and probe.is_contiguous())
+    if lib().nvfp4_set_gemm_experiment(mode, max_pairs, probe.data_ptr() if probe is not None else None) != 0:
+        raise ValueError("nvfp4_set_gemm_experiment: value out of range")
 
 
 def nvfp4_set_gemm_tile_n(tile_n: int) -> None:

@@ -515,6 +515,12 @@ nvfp4_status nvfp4_test_wait_timeout(uint64_t limit_ns, void* cuda_stream) {
   return launch_wait_probe(limit_ns, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
+int32_t nvfp4_set_gemm_experiment(int32_t mode, int32_t max_pairs, void* probe) {
+  if (mode < 0 || mode > 31 || max_pairs < 0) return -1;
+  set_gemm_experiment(mode, max_pairs, static_cast<unsigned long long*>(probe));
+  return 0;
+}
+
 int32_t nvfp4_set_gemm_tile_n(int32_t tile_n) {
   if (tile_n != 0 && tile_n != 128 && tile_n != 256 && tile_n != 512 && tile_n != 768) return -1;
   g_tile_n.store(tile_n, std::memory_order_relaxed);

@@ -355,6 +355,10 @@ bool make_pair_maps(const GemmArgs& g, const void* a_codes, const void* b_codes,
   return ok;
 }
 
+// measurement aids of the CTA-pair kernel (set_gemm_experiment)
+std::atomic<int> g_exp_mode{0}, g_exp_max_pairs{0};
+std::atomic<unsigned long long*> g_exp_probe{nullptr};
+
 pair::Problem pair_problem(const GemmArgs& g) {
   return pair::Problem{g.M, g.N, g.K, g.sfa, g.sfb, g.a_global, g.b_global, g.d_is_fp32, g.accumulate, g.a_rows, g.b_rows};
 }
@@ -386,7 +390,11 @@ cudaError_t launch_pair(const GemmArgs& g0, const void* a0, const void* b0, cons
   a.p[1] = pair_problem(g1 ? *g1 : g0);
   a.n_tiles0 = (g0.M / 256) * (g0.N / 256);
   a.n_tiles = a.n_tiles0 + (g1 ? (g1->M / 256) * (g1->N / 256) : 0);
-  const int max_pairs = num_sms / 2;
+  int max_pairs = num_sms / 2;
+  const int cap = g_exp_max_pairs.load(std::memory_order_relaxed);  // measurement aids, 0 / NULL normally
+  if (cap > 0 && cap < max_pairs) max_pairs = cap;
+  a.exp = g_exp_mode.load(std::memory_order_relaxed);
+  a.probe = g_exp_probe.load(std::memory_order_relaxed);
   const int pairs = a.n_tiles < max_pairs ? a.n_tiles : max_pairs;
   const bool rows = a.p[0].a_rows || a.p[0].b_rows || a.p[1].a_rows || a.p[1].b_rows;
   if (rows) {
@@ -634,6 +642,12 @@ cudaError_t launch_wait_probe(unsigned long long limit_ns, cudaStream_t s) {
   wait_probe_kernel<<<1, 32, 0, s>>>(limit_ns);
   count_launch();
   return cudaGetLastError();
+}
+
+void set_gemm_experiment(int mode, int max_pairs, unsigned long long* probe) {
+  g_exp_mode.store(mode, std::memory_order_relaxed);
+  g_exp_max_pairs.store(max_pairs, std::memory_order_relaxed);
+  g_exp_probe.store(probe, std::memory_order_relaxed);
 }
 
 cudaError_t device_status_word(unsigned int** word) {

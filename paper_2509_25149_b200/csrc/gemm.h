@@ -29,6 +29,12 @@ cudaError_t launch_gemm_two(const GemmArgs& g0, const void* a0, const void* b0, 
                             const void* b1, bool wide_tiles, cudaStream_t s);
 // Scheduling estimate: do 256 x 384 tiles beat 256 x 256 tiles for this problem (or pair of problems in one launch)?
 bool prefer_wide_tiles(const GemmArgs& g0, const GemmArgs* g1);
+// Measurement aids of the CTA-pair kernel with 256 x 256 tiles (0, 0, NULL = normal operation): mode bit 0 = no MMAs,
+// bit 1 = no operand loads, bit 2 = no scale loads / copies, bit 3 = accumulator handed back unread and nothing
+// stored, bit 4 = the issuer does not wait for the accumulator (results meaningless with any bit set); max_pairs caps the
+// persistent grid; probe = device array of eight 64-bit words per pair (SM cycles and nanoseconds of the issuer's main
+// loop, k-blocks, tiles, cycles waiting for the accumulator hand-over; three unused).
+void set_gemm_experiment(int mode, int max_pairs, unsigned long long* probe);
 cudaError_t read_device_status(cudaStream_t s, uint32_t* code);
 // test aid: a bounded wait that is made to run out (a barrier nobody arrives at); leaves kWaitProbeCode in the
 // status word and returns by itself

@@ -55,6 +55,14 @@ struct Args {
   Problem p[2];
   int n_tiles0;  // tiles of problem 0
   int n_tiles;   // tiles of both problems
+  // Measurement aids (0 / NULL in normal operation).  exp: bit 0 = the issuer skips the MMAs, bit 1 = the producer
+  // skips the operand loads, bit 2 = scale atoms are neither loaded nor copied to tensor memory, bit 3 = the epilogue hands the
+  // accumulator back unread and stores nothing, bit 4 = the issuer does not wait for the accumulator (results are
+  // meaningless with any bit set; the barriers are signalled as usual).  probe: per pair eight 64-bit words, five
+  // written by the issuer: SM cycles and nanoseconds of its main loop, k-blocks and tiles it went through, and the
+  // cycles it spent, after issuing a tile's last MMA, waiting for the accumulator to be handed back.
+  int exp;
+  unsigned long long* probe;
 };
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -338,16 +346,24 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 0x100u + stage))) break;
           const uint32_t st = base + stage * kStageBytes;
           const uint32_t bar = map_to_cta(full_bar(stage), 0);  // the leader's barrier counts both CTAs' operands
-          mbar_expect_tx_cluster(bar, kABytes + kBBytes);
-          tma_load_2d_pair(st, map_a, kb * 128, row_a, bar);
-          tma_load_2d_pair(st + kABytes, map_b, kb * 128, row_b, bar);
+          if (g.exp & 2) {
+            mbar_expect_tx_cluster(bar, 0);  // measurement aid: no operand loads
+          } else {
+            mbar_expect_tx_cluster(bar, kABytes + kBBytes);
+            tma_load_2d_pair(st, map_a, kb * 128, row_a, bar);
+            tma_load_2d_pair(st + kABytes, map_b, kb * 128, row_b, bar);
+          }
           // scale atoms: plain bulk copies counted on this CTA's own barrier (its scale warps wait on it)
-          mbar_expect_tx(sfl_bar(stage), 3 * kAtomsKb * 512);
-          bulk_load(st + kABytes + kBBytes, sfa + (int64_t)kb * kAtomsKb * 512, kAtomsKb * 512, sfl_bar(stage));
-          bulk_load(st + kABytes + kBBytes + kSfaBytes, sfb + (int64_t)kb * kAtomsKb * 512, kAtomsKb * 512,
-                    sfl_bar(stage));
-          bulk_load(st + kABytes + kBBytes + kSfaBytes + 2048, sfb + ((int64_t)sf_atoms_k + kb * kAtomsKb) * 512,
-                    kAtomsKb * 512, sfl_bar(stage));
+          if (g.exp & 4) {
+            mbar_expect_tx(sfl_bar(stage), 0);  // measurement aid: no scale loads
+          } else {
+            mbar_expect_tx(sfl_bar(stage), 3 * kAtomsKb * 512);
+            bulk_load(st + kABytes + kBBytes, sfa + (int64_t)kb * kAtomsKb * 512, kAtomsKb * 512, sfl_bar(stage));
+            bulk_load(st + kABytes + kBBytes + kSfaBytes, sfb + (int64_t)kb * kAtomsKb * 512, kAtomsKb * 512,
+                      sfl_bar(stage));
+            bulk_load(st + kABytes + kBBytes + kSfaBytes + 2048, sfb + ((int64_t)sf_atoms_k + kb * kAtomsKb) * 512,
+                      kAtomsKb * 512, sfl_bar(stage));
+          }
           if (++stage == kStages) {
             stage = 0;
             phase ^= 1u;
@@ -373,6 +389,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
         ok = mbar_wait(sfl_bar(stage), phase, abort_flag, 0x500u + stage);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) break;
+        if (g.exp & 4) {  // measurement aid: no scale copies
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(sff_leader + 8u * stage);
+          if (++stage == kStages) {
+            stage = 0;
+            phase ^= 1u;
+          }
+          continue;
+        }
         const uint32_t sf_s = base + stage * kStageBytes + kABytes + kBBytes + lane * 16;
         uint32_t r[48];
         constexpr int kAtomsKb = MX ? 2 : 4;  // atoms per k-block and 128-row group
@@ -421,8 +446,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       constexpr uint32_t idesc_mx[2] = {instr_desc_mxf4(256, 256, 0), instr_desc_mxf4(256, 256, 2)};
       const uint32_t a_lo0 = ((base >> 4) & 0x3fffu) | (1u << 16);
       const uint32_t b_lo0 = (((base + kABytes) >> 4) & 0x3fffu) | (1u << 16);
+      const long long probe_c0 = g.probe ? clock64() : 0;
+      const unsigned long long probe_t0 = g.probe ? globaltimer_ns() : 0;
+      unsigned long long probe_kb = 0, probe_tiles = 0;
+      long long probe_wait = 0, probe_mark = probe_c0;  // cycles spent waiting for the accumulator to be handed back
       for (int rnd = 0, tile = pair_id; tile < n_tiles && ok; tile = next_tile(++rnd)) {
-        if (!(ok = mbar_wait_cluster(acce_bar, acc_phase ^ 1u, abort_flag, 0x300u))) break;
+        if (!(g.exp & 16) && !(ok = mbar_wait_cluster(acce_bar, acc_phase ^ 1u, abort_flag, 0x300u))) break;
+        if (g.probe) probe_wait += clock64() - probe_mark;
         tc_fence_after();
         const int k_blocks = k_blocks_of(tile);
         for (int kb = 0; kb < k_blocks; ++kb) {
@@ -434,6 +464,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
           const uint32_t sf_t = tmem + kSfCol + stage * kSfSlotCols;
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
+            if (g.exp & 1) break;  // measurement aid: no MMAs
             if (MX)  // one atom (4 columns) serves two K = 64 steps: bytes 0-1, then bytes 2-3
               tc2_mma_mxf4(tmem, make_desc(a_lo + 2 * j, kDescHiOperand), make_desc(b_lo + 2 * j, kDescHiOperand),
                            idesc_mx[j & 1], sf_t + (j >> 1) * 4, sf_t + 16 + (j >> 1) * 8, (kb > 0 || j > 0) ? 1u : 0u);
@@ -450,6 +481,20 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
         if (!ok) break;
         tc2_commit_both(accf_bar, 3);  // accumulators of both CTAs complete
         acc_phase ^= 1u;
+        probe_kb += (unsigned long long)k_blocks;
+        ++probe_tiles;
+        if (g.probe) probe_mark = clock64();
+      }
+      if (g.probe) {
+        // the last commit has been issued, not completed: wait for the accumulator hand-over of the last tile so that
+        // the interval covers the work (bounded like every other wait)
+        mbar_wait_cluster(acce_bar, acc_phase ^ 1u, abort_flag, 0x380u);
+        probe_wait += clock64() - probe_mark;
+        g.probe[8 * pair_id] = (unsigned long long)(clock64() - probe_c0);
+        g.probe[8 * pair_id + 1] = globaltimer_ns() - probe_t0;
+        g.probe[8 * pair_id + 2] = probe_kb;
+        g.probe[8 * pair_id + 3] = probe_tiles;
+        g.probe[8 * pair_id + 4] = (unsigned long long)probe_wait;
       }
     }
   } else if (warp >= 3 && warp <= 10) {
@@ -485,6 +530,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       // agree on giving up: a warp that timed out still joins this barrier, and all 128 threads take ONE decision
       if (group_gave_up(abort_flag, bar_id, 128)) break;
       tc_fence_after();
+      if (g.exp & 8) {  // measurement aid: the accumulator is handed back unread, nothing is stored
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(acce_leader);
+        acc_phase ^= 1u;
+        continue;
+      }
       const int row0 = m_blk * 256 + (int)rank * 128;
       // read this warp's 32 lanes x 128 columns in one go and hand the accumulator back at once: the MMA issuer
       // can start the next tile while the values are converted and stored from registers
