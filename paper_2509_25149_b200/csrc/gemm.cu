@@ -469,7 +469,9 @@ double pair_makespan(const GemmArgs* const* gs, int n_problems, bool wide_tiles,
       const int gm = tiles_m - m0 < kGroupM ? tiles_m - m0 : kGroupM;
       for (int n_idx = 0; n_idx < tiles_n; ++n_idx) {
         const bool w = n_idx < n_wide;
-        const double cost = w ? 1.5 * kb + 3.3 : kb + (wide_tiles ? 2.9 : 2.5);
+        // hand-over per tile in k-block units, fitted to 24 layer shapes timed with both tile widths; the wide
+        // tile drains an fp32 output in six passes before it can release the accumulator
+        const double cost = w ? 1.5 * kb + (g.d_is_fp32 ? 5.3 : 3.3) : kb + (wide_tiles ? 2.9 : 2.5);
         for (int i = 0; i < gm; ++i, ++t) {
           const int64_t rnd = t / pairs, p = t % pairs;
           load[(size_t)((rnd & 1) ? pairs - 1 - p : p)] += cost;  // odd rounds run through the pairs in reverse

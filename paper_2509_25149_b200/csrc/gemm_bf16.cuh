@@ -213,7 +213,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
       const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + buf * 256 + half * 128;
       uint32_t r[128];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) tc_ld32(t_row + q * 32, *reinterpret_cast<uint32_t(*)[32]>(&r[q * 32]));
+      for (int q = 0; q < 8; ++q) tc_ld16(t_row + q * 16, *reinterpret_cast<uint32_t(*)[16]>(&r[q * 16]));
       tc_wait_ld();
       tc_fence_before();
       __syncwarp();

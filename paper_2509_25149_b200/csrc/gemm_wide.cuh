@@ -361,8 +361,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
       const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + half * cols_half;
       for (int p = 0; p < passes; ++p) {
         uint32_t r[64];
-        tc_ld32(t_row + p * 64, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
-        tc_ld32(t_row + p * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+#pragma unroll
+        for (int q = 0; q < 4; ++q) tc_ld16(t_row + p * 64 + q * 16, *reinterpret_cast<uint32_t(*)[16]>(&r[q * 16]));
         tc_wait_ld();
         if (p == passes - 1) {  // the accumulator has been read: the MMA issuer may start the next tile
           tc_fence_before();
