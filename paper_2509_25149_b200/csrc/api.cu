@@ -39,7 +39,7 @@ nvfp4_status check_copy(const nvfp4_tensor* t, int64_t rows, int64_t cols) {
 // that a rejected call has enqueued nothing)
 nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld, const nvfp4_quant_opts* o,
                            const nvfp4_tensor* rowwise, const nvfp4_tensor* colwise, cudaStream_t s,
-                           bool check_only = false) {
+                           bool check_only = false, const SideAmax* side = nullptr, bool chained = false) {
   if (!x || !o) return NVFP4_ERR_NULL;
   if (!rowwise && !colwise) return NVFP4_ERR_NULL;
   if (rows <= 0 || cols <= 0 || rows % 16 != 0 || cols % 16 != 0) return NVFP4_ERR_SHAPE;
@@ -145,12 +145,27 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
     return launch_quantize_rht(ra, (o->flags & NVFP4_AMAX_PROVIDED) != 0, sr, s) == cudaSuccess ? NVFP4_OK
                                                                                                   : NVFP4_ERR_CUDA;
   }
+  // pass 2 may become resident while the previous kernel of this call drains (its own pass 1, or the caller's launch)
+  a.chained = chained;
+  if (side && zero_side_amax(*side, s) != cudaSuccess) return NVFP4_ERR_CUDA;  // not between pass 1 and pass 2
   if (!(o->flags & NVFP4_AMAX_PROVIDED)) {
     if (launch_amax(a, hr, hc, o->rht_rowwise != 0, o->rht_colwise != 0, s) != cudaSuccess) return NVFP4_ERR_CUDA;
+    a.chained = 1;
+  }
+  if (side) {  // only the forward pass's activation quantize carries one (see side_amax_fits)
+    if (!hr || b2 || sr || o->rht_rowwise || (hc && !o->rht_colwise)) return NVFP4_ERR_ARG;
+    return launch_quantize_with_amax_of(a, hc, *side, s) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
   }
   if (launch_quantize(a, hr, hc, b2, o->rht_rowwise != 0, o->rht_colwise != 0, sr, s) != cudaSuccess)
     return NVFP4_ERR_CUDA;
   return NVFP4_OK;
+}
+
+// Whether a quantize of the composed calls (options xo) runs `quantize_kernel`, the kernel that can take a second
+// tensor's plain amax on the side and lets the next kernel of the call set itself up early: bf16 source, NVFP4, the
+// 16-point transform or none.
+bool side_amax_fits(int32_t fmt, const nvfp4_quant_opts& xo) {
+  return fmt == NVFP4_FORMAT_NVFP4 && (xo.rht_dim == 0 || xo.rht_dim == 16) && !(xo.flags & NVFP4_INPUT_FP32);
 }
 
 // argument checks of one GEMM and its launch description
@@ -206,10 +221,11 @@ int gemm_tile(const GemmArgs& g) {
 }
 
 nvfp4_status gemm_impl(const nvfp4_tensor* A, const nvfp4_tensor* B, void* D, int32_t d_is_fp32, int64_t ldd,
-                       int32_t accumulate, cudaStream_t s) {
+                       int32_t accumulate, cudaStream_t s, bool chained = false) {
   GemmArgs g;
   nvfp4_status st = gemm_prepare(A, B, D, d_is_fp32, ldd, accumulate, g);
   if (st != NVFP4_OK) return st;
+  g.chained = chained;
   if (launch_gemm(g, A->codes, B->codes, gemm_tile(g), s) != cudaSuccess) return NVFP4_ERR_CUDA;
   return NVFP4_OK;
 }
@@ -313,9 +329,18 @@ nvfp4_status nvfp4_linear_fwd(const void* X, const void* W, int64_t M, int64_t N
   if (!w_is_cached && (st = quantize_impl(W, N, K, K, &wo, W_row, W_col_saved, s, true)) != NVFP4_OK) return st;
   if ((st = quantize_impl(X, M, K, K, &xo, &x_row, X_col_saved, s, true)) != NVFP4_OK) return st;
   if ((st = gemm_prepare(&x_row, W_row, Y_bf16, 0, N, 0, gy)) != NVFP4_OK) return st;
+  if (!w_is_cached && side_amax_fits(fmt, xo)) {
+    // pass 1 of W (memory-bound) rides on pass 2 of X (issue-bound); W's pass 2 then finds its amax in place
+    const SideAmax w_amax{W, N, K, K, W_row->global, W_col_saved ? W_col_saved->global : nullptr};
+    if ((st = quantize_impl(X, M, K, K, &xo, &x_row, X_col_saved, s, false, &w_amax)) != NVFP4_OK) return st;
+    wo.flags |= NVFP4_AMAX_PROVIDED;
+    if ((st = quantize_impl(W, N, K, K, &wo, W_row, W_col_saved, s, false, nullptr, true)) != NVFP4_OK) return st;
+    return gemm_impl(&x_row, W_row, Y_bf16, 0, N, 0, s, true);
+  }
   if (!w_is_cached && (st = quantize_impl(W, N, K, K, &wo, W_row, W_col_saved, s)) != NVFP4_OK) return st;
   if ((st = quantize_impl(X, M, K, K, &xo, &x_row, X_col_saved, s)) != NVFP4_OK) return st;
-  return gemm_impl(&x_row, W_row, Y_bf16, 0, N, 0, s);
+  // behind the bf16 NVFP4 quantizer the GEMM may set itself up while that kernel drains
+  return gemm_impl(&x_row, W_row, Y_bf16, 0, N, 0, s, side_amax_fits(fmt, xo));
 }
 
 nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, const nvfp4_tensor* W_col_saved,
@@ -365,6 +390,7 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, c
     GemmArgs gd, gw;
     if ((st = gemm_prepare(&g_row, W_col_saved, dX_bf16, 0, K, 0, gd)) != NVFP4_OK) return st;
     if ((st = gemm_prepare(&g_col, X_col_saved, dW_fp32, 1, K, accumulate_dw, gw)) != NVFP4_OK) return st;
+    gd.chained = gw.chained = side_amax_fits(fmt, go);  // behind the bf16 NVFP4 quantizer of dY
     const int td = gemm_tile(gd), tw = gemm_tile(gw);
     if ((td == 512 || td == 768) && (tw == 512 || tw == 768)) {
       const bool forced = g_tile_n.load(std::memory_order_relaxed) != 0;
@@ -376,7 +402,8 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, c
       return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
     }
   }
-  if (dX_bf16 && (st = gemm_impl(&g_row, W_col_saved, dX_bf16, 0, K, 0, s)) != NVFP4_OK) return st;
+  if (dX_bf16 && (st = gemm_impl(&g_row, W_col_saved, dX_bf16, 0, K, 0, s, side_amax_fits(fmt, go))) != NVFP4_OK)
+    return st;
   if (dW_fp32 && (st = gemm_impl(&g_col, X_col_saved, dW_fp32, 1, K, accumulate_dw, s)) != NVFP4_OK) return st;
   return NVFP4_OK;
 }

@@ -55,6 +55,32 @@ __device__ __forceinline__ void fence_mbarrier_init() {
 // orders this thread's earlier generic-proxy accesses to shared memory before later asynchronous-proxy ones (TMA)
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// ---- programmatic dependent launch: a kernel launched with `launch_kernel(..., after_own_kernel = true)` may become
+// resident while the previous kernel of the stream drains; it runs its set-up (barriers, tensor memory, descriptor
+// prefetch, loads of data the previous kernel does not write) and then waits here for that kernel to finish with all
+// its writes visible.  A no-op for a kernel that was launched the ordinary way.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// lets the next kernel of the stream, if it was launched that way, become resident as CTAs of this grid retire
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+#ifdef __CUDACC__
+template <typename... Params, typename... Args>
+inline cudaError_t launch_kernel(void (*kern)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                 bool after_own_kernel, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = after_own_kernel ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<Params>(args)...);
+}
+#endif
+
 // ---- host-side tensor-map encoder (driver entry point fetched through the runtime) ----
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,

@@ -430,14 +430,21 @@ cudaError_t launch_pair(const GemmArgs& g0, const void* a0, const void* b0, cons
       if (e != cudaSuccess) return e;
       device_configured(configured_rows, dev);
     }
-    pair::gemm_pair_kernel<false, true><<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5], a);
-  } else if (g0.mx) {
-    pair::gemm_pair_kernel<true><<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5], a);
-  } else {
-    pair::gemm_pair_kernel<false><<<2 * pairs, pair::kThreads, pair::kSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5], a);
   }
+  const bool chained = g0.chained != 0;
+  const dim3 grid(2 * pairs), block(pair::kThreads);
+  cudaError_t le;
+  if (rows)
+    le = launch_kernel(pair::gemm_pair_kernel<false, true>, grid, block, pair::kSmemBytes, s, chained, m[0], m[1], m[2],
+                       m[3], m[4], m[5], a);
+  else if (g0.mx)
+    le = launch_kernel(pair::gemm_pair_kernel<true>, grid, block, pair::kSmemBytes, s, chained, m[0], m[1], m[2], m[3],
+                       m[4], m[5], a);
+  else
+    le = launch_kernel(pair::gemm_pair_kernel<false>, grid, block, pair::kSmemBytes, s, chained, m[0], m[1], m[2], m[3],
+                       m[4], m[5], a);
   count_launch();
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 // N = 128 q = 384 a + 256 b with b in {0, 1, 2}: a wide column tiles, b narrow ones (q >= 2)
@@ -538,14 +545,14 @@ cudaError_t launch_wide(const GemmArgs& g0, const void* a0, const void* b0, cons
   a.n_tiles = a.n_tiles0 + (g1 ? (g1->M / 256) * a.p[1].tiles_n : 0);
   const int max_pairs = num_sms / 2;
   const int pairs = a.n_tiles < max_pairs ? a.n_tiles : max_pairs;
-  if (g0.mx)
-    wide::gemm_wide_kernel<true><<<2 * pairs, wide::kWThreads, wide::kWSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5],
-                                                                                        m[6], m[7], a);
-  else
-    wide::gemm_wide_kernel<false><<<2 * pairs, wide::kWThreads, wide::kWSmemBytes, s>>>(m[0], m[1], m[2], m[3], m[4], m[5],
-                                                                                         m[6], m[7], a);
+  const dim3 grid(2 * pairs), block(wide::kWThreads);
+  const cudaError_t le =
+      g0.mx ? launch_kernel(wide::gemm_wide_kernel<true>, grid, block, wide::kWSmemBytes, s, g0.chained != 0, m[0], m[1],
+                            m[2], m[3], m[4], m[5], m[6], m[7], a)
+            : launch_kernel(wide::gemm_wide_kernel<false>, grid, block, wide::kWSmemBytes, s, g0.chained != 0, m[0], m[1],
+                            m[2], m[3], m[4], m[5], m[6], m[7], a);
   count_launch();
-  return cudaGetLastError();
+  return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 cudaError_t sm_count(int* n) {

@@ -17,6 +17,7 @@ struct GemmArgs {
   int mx;                 // operands are MXFP4 (UE8M0 scale per 32 elements) instead of NVFP4
   const float* a_rows;    // per-row {amax, s_dec} pairs of A / B when their global scale is taken per row, else NULL
   const float* b_rows;    // (CTA-pair kernel with 256 x 256 tiles only)
+  int chained;            // the previous launch on the stream is a kernel of the same call (see launch_kernel)
 };
 
 // tile_n: 128 or 256 (one CTA per tile; 256 needs N % 256 == 0, otherwise 128 is used), 512 (CTA pairs, 256 x 256

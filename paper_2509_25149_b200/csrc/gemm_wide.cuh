@@ -176,6 +176,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
   cluster_sync_all();  // both CTAs' barriers are initialised before any remote signal
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // Launched behind the quantizer of the same call, the CTA reaches this point while that kernel still runs: from
+  // here on every role touches what it wrote (operands, scales, global scales), so all of them wait for it to end.
+  griddep_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer ----

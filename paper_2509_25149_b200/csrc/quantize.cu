@@ -31,6 +31,7 @@ __global__ void __launch_bounds__(256) amax_kernel(const uint16_t* __restrict__ 
   const int64_t r0 = tr * 128 + warp * 16;
   const int64_t c0 = tc * 256 + lane * 8;
   const bool in_range = (r0 < rows) && (c0 < cols);  // rows % 16 == 0, cols % 8 == 0
+  griddep_launch_dependents();  // pass 2 may set itself up while the last CTAs of this pass run
 
   uint4 raw[16];
   if (in_range) {
@@ -157,6 +158,7 @@ __global__ void __launch_bounds__(256) amax_rot_col_kernel(const uint16_t* __res
   const int g = lane >> 2, t = lane & 3;
   const int64_t tr = blockIdx.x / tiles_c, tc = blockIdx.x % tiles_c;
   const int64_t r0 = tr * 128 + warp * 16;
+  griddep_launch_dependents();  // pass 2 may set itself up while the last CTAs of this pass run
 
   uint32_t lo[4][8], hi[4][8];  // rows g and g + 8 of the slab, 16 columns each, four 64-column steps
 #pragma unroll
@@ -310,8 +312,9 @@ __device__ __forceinline__ float encode_scale_of_byte(uint32_t byte, float s_dec
   return (byte == 0u) ? 0.0f : fminf(__frcp_rn(d), kFltMax);
 }
 
-template <bool HAS_ROW, bool HAS_COL, bool BLOCK2D, bool RHT_ROW, bool RHT_COL, bool SR>
+template <bool HAS_ROW, bool HAS_COL, bool BLOCK2D, bool RHT_ROW, bool RHT_COL, bool SR, bool SIDE = false>
 __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant__ CUtensorMap src_map,
+                                                          const __grid_constant__ CUtensorMap side_map,
                                                           const QuantArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -326,11 +329,31 @@ __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant_
   const int total = a.tiles_r * a.tiles_c, stride = (int)gridDim.x;
   const int first = total - 1 - (int)blockIdx.x;         // this CTA's tiles: first, first - stride, ...
   const int n_mine = first >= 0 ? first / stride + 1 : 0;
-  auto issue_load = [&](int k) {  // tile k of this CTA into buffer k & 1 (one thread)
-    const int t = first - k * stride, tr = t / a.tiles_c, tc = t - tr * a.tiles_c;
-    const uint32_t bar = bar0 + 8 * (k & 1);
+  // SIDE: the CTA also streams its share of a second tensor's tiles through the same ring and takes their plain
+  // amax (pass 1 of that tensor, Appendix B.1): memory-bound work riding on an issue-bound kernel.  Side tiles go
+  // front to back (the tensor's own pass 2 starts from its end), interleaved in proportion with the CTA's own tiles.
+  const int side_total = SIDE ? a.side_tiles_r * a.side_tiles_c : 0;
+  const int m_mine = (int)blockIdx.x < side_total ? (side_total - 1 - (int)blockIdx.x) / stride + 1 : 0;
+  const int n_jobs = n_mine + m_mine;
+  // with k own tiles and sk side tiles behind it, the CTA's next job is a side tile iff ...
+  auto side_next = [&](int k, int sk) {
+    return SIDE && sk < m_mine && (k >= n_mine || (long long)sk * n_mine < (long long)k * m_mine);
+  };
+  auto issue_load = [&](int j, int k, int sk) {  // job j (own tile k or side tile sk) into buffer j & 1 (one thread)
+    const uint32_t bar = bar0 + 8 * (j & 1), dst = tile0 + (j & 1) * QuantSmem::kTileBytes;
     mbar_expect_tx(bar, QuantSmem::kTileBytes);
-    tma_load_2d(tile0 + (k & 1) * QuantSmem::kTileBytes, &src_map, tc * 128, tr * 128, bar);
+    if (side_next(k, sk)) {
+      const int t = (int)blockIdx.x + sk * stride, tr = t / a.side_tiles_c, tc = t - tr * a.side_tiles_c;
+      tma_load_2d(dst, &side_map, tc * 128, tr * 128, bar);
+    } else {
+      const int t = first - k * stride, tr = t / a.tiles_c, tc = t - tr * a.tiles_c;
+      tma_load_2d(dst, &src_map, tc * 128, tr * 128, bar);
+    }
+  };
+  int ahead_k = 0, ahead_sk = 0;  // thread 0: own / side tiles among the jobs already issued
+  auto issue_next = [&](int j) {
+    issue_load(j, ahead_k, ahead_sk);
+    if (side_next(ahead_k, ahead_sk)) ++ahead_sk; else ++ahead_k;
   };
 
   // ------------------------------------------------------------------ set-up ----
@@ -341,8 +364,11 @@ __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant_
     *abort_flag = 0u;
     fence_mbarrier_init();
     fence_proxy_async_smem();
-    if (n_mine > 0) issue_load(0);
-    if (n_mine > 1) issue_load(1);
+    if (n_jobs > 0) issue_next(0);
+    if (n_jobs > 1) issue_next(1);
+    // the source tiles above are nobody's output in this call; the tensor amax below is the previous kernel's.
+    // Every other thread passes the barrier below only after this wait, so no output is written before it either.
+    griddep_wait();
     // Eq. 1 (two IEEE divisions per copy)
     float re = 1.f, rd = 1.f, ce = 1.f, cd = 1.f;
     if (HAS_ROW || BLOCK2D) global_scales(HAS_ROW ? a.r_global[0] : a.c_global[0], re, rd);
@@ -361,6 +387,7 @@ __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant_
     }
   }
   __syncthreads();
+  griddep_launch_dependents();
   const float r_senc = g_sc[0], r_sdec = g_sc[1], c_senc = g_sc[2], c_sdec = g_sc[3];
   const float* enc_row = reinterpret_cast<const float*>(smem + QuantSmem::kEncRow);
   const float* enc_col = reinterpret_cast<const float*>(smem + QuantSmem::kEncCol);
@@ -397,20 +424,30 @@ __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant_
 
   const int step_r = stride / a.tiles_c, step_c = stride - step_r * a.tiles_c;  // tile coordinates move by these
   int tr = first >= 0 ? first / a.tiles_c : 0, tc = first >= 0 ? first - tr * a.tiles_c : 0;
-  int k = 0;
-  for (; k < n_mine; ++k, tr -= step_r, tc -= step_c) {
-    if (tc < 0) {
-      tc += a.tiles_c;
-      --tr;
+  int k = 0, sk = 0, j = 0;  // own tiles done, side tiles done, jobs done (the ring position)
+  uint32_t side_acc = 0;     // |.| maximum of the side tiles, two bf16 lanes
+  for (; j < n_jobs; ++j) {
+    const uint8_t* const tile_buf = smem + QuantSmem::kTile + (j & 1) * QuantSmem::kTileBytes;
+    quant_wait(bar0 + 8 * (j & 1), (uint32_t)(j >> 1) & 1u, abort_flag, a.status);  // the tile has landed
+    if (SIDE && side_next(k, sk)) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {  // zero fill outside the tensor leaves the maximum alone
+        const uint4 v = *reinterpret_cast<const uint4*>(tile_buf + i * 4096 + threadIdx.x * 16);
+        side_acc = absmax_bf16x2(absmax_bf16x2(side_acc, v.x), v.y);
+        side_acc = absmax_bf16x2(absmax_bf16x2(side_acc, v.z), v.w);
+      }
+      __syncthreads();
+      if (*abort_flag) break;
+      if (threadIdx.x == 0 && j + 2 < n_jobs) issue_next(j + 2);
+      ++sk;
+      continue;
     }
-    const int buf = k & 1;
+    const int buf = k & 1;  // staging buffers alternate with the CTA's own tiles
     const int64_t row0 = (int64_t)tr * 128, col0 = (int64_t)tc * 128;
     const bool full_tile = (row0 + 128 <= a.rows) && (col0 + 128 <= a.cols);
     uint8_t* const col_codes = smem + QuantSmem::kColCodes + buf * 8192;
     uint8_t* const sf_row = smem + QuantSmem::kSfRow + buf * 1024;
     uint8_t* const sf_col = smem + QuantSmem::kSfCol + buf * 1024;
-    const uint8_t* const tile_buf = smem + QuantSmem::kTile + buf * QuantSmem::kTileBytes;
-    quant_wait(bar0 + 8 * buf, (uint32_t)(k >> 1) & 1u, abort_flag, a.status);  // the tile has landed
 
     auto phases_1_2 = [&](auto full_c) {
       constexpr bool FULL = decltype(full_c)::value;
@@ -591,7 +628,7 @@ __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant_
       phases_1_2(std::false_type{});
     __syncthreads();
     if (*abort_flag) break;  // a wait expired (the word is read after the barrier: the same for every thread)
-    if (threadIdx.x == 0 && k + 2 < n_mine) issue_load(k + 2);  // every warp is done with this buffer
+    if (threadIdx.x == 0 && j + 2 < n_jobs) issue_next(j + 2);  // every warp is done with this buffer
 
     // ------------------------------------------------------------------ phase 3 ----
     if (HAS_COL) {
@@ -645,14 +682,38 @@ __global__ void __launch_bounds__(256, 2) quantize_kernel(const __grid_constant_
         }
       }
     }
+    ++k;  // on to the CTA's next own tile
+    tr -= step_r;
+    tc -= step_c;
+    if (tc < 0) {
+      tc += a.tiles_c;
+      --tr;
+    }
   }
-  if (k < n_mine && threadIdx.x == 0) {
-    // left early: tiles k and k + 1 may still be in flight; give each one more bounded wait so that no copy lands
+  if (j < n_jobs) {
+    // left early: jobs j and j + 1 may still be in flight; give each one more bounded wait so that no copy lands
     // in shared memory after the CTA has gone
-    for (int j = k; j < k + 2 && j < n_mine; ++j) {
-      const unsigned long long t0 = globaltimer_ns();
-      while (!mbar_try(bar0 + 8 * (j & 1), (uint32_t)(j >> 1) & 1u) && globaltimer_ns() - t0 < kWaitLimitNs) {
+    if (threadIdx.x == 0)
+      for (int i = j; i < j + 2 && i < n_jobs; ++i) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (!mbar_try(bar0 + 8 * (i & 1), (uint32_t)(i >> 1) & 1u) && globaltimer_ns() - t0 < kWaitLimitNs) {
+        }
       }
+    return;  // no maximum is published by a CTA that gave up
+  }
+  if (SIDE) {
+    float* red = reinterpret_cast<float*>(smem + QuantSmem::kBlkEnc);  // free in 1 x 16 mode
+    const float m = warp_max(fmaxf(bf16_lo(side_acc), bf16_hi(side_acc)));
+    __syncthreads();
+    if (lane == 0) red[warp] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float t = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) t = fmaxf(t, red[w]);
+      const uint32_t bits = __float_as_uint(t);  // non-negative floats order like their bit patterns
+      if (a.side_out0) atomicMax(reinterpret_cast<unsigned int*>(a.side_out0), bits);
+      if (a.side_out1) atomicMax(reinterpret_cast<unsigned int*>(a.side_out1), bits);
     }
   }
 }
@@ -790,9 +851,10 @@ cudaError_t launch_amax_rot_col_small(const QuantArgs& a, bool has_row, uint32_t
   return cudaGetLastError();
 }
 
-template <bool HR, bool HC, bool B2, bool RR, bool RC, bool SR>
-static cudaError_t launch_quant_t(const QuantArgs& a, cudaStream_t s) {
-  auto kern = quantize_kernel<HR, HC, B2, RR, RC, SR>;
+template <bool HR, bool HC, bool B2, bool RR, bool RC, bool SR, bool SIDE = false>
+static cudaError_t launch_quant_t(const QuantArgs& a_in, cudaStream_t s, const SideAmax* side = nullptr) {
+  auto kern = quantize_kernel<HR, HC, B2, RR, RC, SR, SIDE>;
+  QuantArgs a = a_in;
   constexpr bool kRowCodes = B2 && HR && HC;
   constexpr int smem = QuantSmem::bytes(SR && HC && !kRowCodes, kRowCodes);
   // the source as a 2-D tensor map: boxes of 128 x 128 bf16 (256-byte rows, no swizzle), zero fill outside
@@ -800,6 +862,19 @@ static cudaError_t launch_quant_t(const QuantArgs& a, cudaStream_t s) {
   if (!make_map_2d(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.x, (uint64_t)a.cols, (uint64_t)a.rows,
                    (uint64_t)a.ld * 2, 128, 128, false))
     return cudaErrorInvalidValue;
+  CUtensorMap side_map = map;
+  int64_t side_tiles = 0;
+  if (SIDE) {
+    if (!side || !make_map_2d(&side_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, side->x, (uint64_t)side->cols,
+                              (uint64_t)side->rows, (uint64_t)side->ld * 2, 128, 128, false))
+      return cudaErrorInvalidValue;
+    a.side_tiles_r = (int)((side->rows + 127) / 128);
+    a.side_tiles_c = (int)((side->cols + 127) / 128);
+    a.side_out0 = side->out0;
+    a.side_out1 = side->out1;
+    side_tiles = (int64_t)a.side_tiles_r * a.side_tiles_c;
+    if (side_tiles > 0x7fffffff) return cudaErrorInvalidValue;
+  }
   // per call site (template instantiation) and device: the dynamic shared-memory limit, and how many CTAs the device
   // keeps resident (the persistent grid)
   static std::atomic<uint64_t> configured{0};
@@ -815,11 +890,23 @@ static cudaError_t launch_quant_t(const QuantArgs& a, cudaStream_t s) {
     device_configured(configured, dev);
   }
   const int slots = (dev >= 0 && dev < 64) ? resident[dev].load(std::memory_order_relaxed) : 0;
-  const int64_t tiles = (int64_t)a.tiles_r * a.tiles_c;
+  const int64_t own = (int64_t)a.tiles_r * a.tiles_c, tiles = own > side_tiles ? own : side_tiles;
   const int64_t grid = (slots > 0 && tiles > slots) ? slots : tiles;
-  kern<<<(unsigned)grid, 256, smem, s>>>(map, a);
+  const cudaError_t e = launch_kernel(kern, dim3((unsigned)grid), dim3(256), smem, s, a.chained != 0, map, side_map, a);
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+cudaError_t zero_side_amax(const SideAmax& side, cudaStream_t s) {
+  cudaError_t e;
+  if (side.out0 && (e = cudaMemsetAsync(side.out0, 0, sizeof(float), s)) != cudaSuccess) return e;
+  if (side.out1 && (e = cudaMemsetAsync(side.out1, 0, sizeof(float), s)) != cudaSuccess) return e;
+  return cudaSuccess;
+}
+
+cudaError_t launch_quantize_with_amax_of(const QuantArgs& a, bool has_col, const SideAmax& side, cudaStream_t s) {
+  return has_col ? launch_quant_t<true, true, false, false, true, false, true>(a, s, &side)
+                 : launch_quant_t<true, false, false, false, false, false, true>(a, s, &side);
 }
 
 cudaError_t launch_quantize(const QuantArgs& a, bool has_row, bool has_col, bool block2d, bool rht_row,

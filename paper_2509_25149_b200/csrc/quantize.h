@@ -22,6 +22,19 @@ struct QuantArgs {
   uint32_t rk[20];       // Philox round keys (seed_lo + r * W0, seed_hi + r * W1), r = 0..9, filled by the host
   int tiles_r, tiles_c;  // 128 x 128 tiles of the source
   unsigned int* status;  // device status word: a bounded wait that expired leaves its code here (may be NULL)
+  int chained;  // host side: the previous launch on the stream is a kernel of the same call (see launch_kernel)
+  // side job of launch_quantize_with_amax_of: 128 x 128 tiles of the second tensor and where its amax goes
+  int side_tiles_r, side_tiles_c;
+  float* side_out0;
+  float* side_out1;
+};
+
+// A second bf16 tensor whose plain amax (pass 1 of its own quantization) a quantize launch takes on the side
+struct SideAmax {
+  const void* x;
+  int64_t rows, cols, ld;
+  float* out0;  // both receive the amax (the row-wise and the transposed copy's global[0]); either may be NULL
+  float* out1;
 };
 
 // Another transform size (quantize_rht.cu): d = 2, 4, 8 or 128 on the copies flagged rht_row / rht_col
@@ -41,6 +54,10 @@ cudaError_t launch_amax(const QuantArgs& a, bool has_row, bool has_col, bool rht
                         cudaStream_t s);
 cudaError_t launch_quantize(const QuantArgs& a, bool has_row, bool has_col, bool block2d, bool rht_row,
                             bool rht_col, bool sr, cudaStream_t s);
+// The row-wise copy (and, with has_col, the transformed transposed copy) of a, round-to-nearest, 1 x 16 blocks, and
+// on the side the plain amax of `side`: the memory-bound pass 1 of the next tensor rides on this issue-bound kernel.
+cudaError_t launch_quantize_with_amax_of(const QuantArgs& a, bool has_col, const SideAmax& side, cudaStream_t s);
+cudaError_t zero_side_amax(const SideAmax& side, cudaStream_t s);  // before the launches that lead up to it
 // MXFP4 outputs (quantize_mx.cu): one pass, no tensor-level scale
 cudaError_t launch_quantize_mx(const QuantArgs& a, bool has_row, bool has_col, bool block2d, bool rht_col, bool sr,
                                cudaStream_t s);

@@ -84,3 +84,40 @@ def test_cached_weight_and_skipped_outputs():
     B.nvfp4_linear_bwd(p.dY.cuda(), X_col, None, K, opts, None, dW2, True, ws_b)
     B.nvfp4_device_status()
     assert torch.allclose(dW2, 2 * dW, rtol=1e-6, atol=0)
+
+
+@pytest.mark.parametrize("M,N,K,with_col", [
+    (256, 5120, 1024, True),    # W has far more tiles than X: most CTAs only carry tiles of W
+    (4096, 256, 512, True),     # the reverse: few tiles of W among many of X
+    (1024, 2304, 768, False),   # forward only (no transposed copies): the row-wise variant of the kernel
+    (8192, 6144, 2560, True),   # more tiles of both than resident CTAs: every CTA interleaves the two kinds
+])
+def test_forward_call_quantizes_w_exactly_like_the_standalone_call(M, N, K, with_col):
+    """The forward call takes W's tensor amax (Appendix B.1) inside the kernel that quantizes X; the standalone call
+    runs its own amax pass.  Every byte of the W and X copies, the global scales and Y must agree."""
+    g = torch.Generator(device="cuda").manual_seed(M + N + K)
+    X = torch.randn((M, K), generator=g, device="cuda").to(torch.bfloat16)
+    W = (torch.randn((N, K), generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+    # the tensor amax sits in one corner tile each time (first, last, and a middle tile)
+    for pos in ((0, 0), (N - 1, K - 1), (N // 2 + 3, K // 2 + 5)):
+        Wp = W.clone()
+        Wp[pos] = -3.0
+        opts = B.quant_opts(rht_sign_mask=synth.DEFAULT_RHT_SIGN_MASK)
+        X_col = B.alloc_tensor(K, M) if with_col else None
+        W_row, W_col = B.alloc_tensor(N, K), (B.alloc_tensor(K, N) if with_col else None)
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        ws = torch.empty(B.nvfp4_linear_fwd_workspace_bytes(M, K), dtype=torch.uint8, device="cuda")
+        B.nvfp4_linear_fwd(X, Wp, opts, Y, X_col, W_row, W_col, False, ws)
+        W_row2, W_col2 = B.alloc_tensor(N, K), (B.alloc_tensor(K, N) if with_col else None)
+        B.nvfp4_quantize(Wp, B.quant_opts(block_rows=16), W_row2, W_col2)
+        X_row2, X_col2 = B.alloc_tensor(M, K), (B.alloc_tensor(K, M) if with_col else None)
+        B.nvfp4_quantize(X, B.quant_opts(rht_colwise=True, rht_sign_mask=synth.DEFAULT_RHT_SIGN_MASK), X_row2, X_col2)
+        Y2 = torch.empty_like(Y)
+        B.nvfp4_gemm(X_row2, W_row2, Y2)
+        B.nvfp4_device_status()
+        pairs = [(W_row, W_row2)] + ([(W_col, W_col2), (X_col, X_col2)] if with_col else [])
+        for a, b in pairs:
+            assert torch.equal(a.codes, b.codes) and torch.equal(a.scales, b.scales)
+            assert torch.equal(a.glob, b.glob)
+        assert float(W_row.glob[0]) == 3.0
+        assert torch.equal(Y, Y2)
