@@ -534,6 +534,8 @@ CASES = {
     "gemm_fprop_mx": ("gemm_mx", 4096, 5120, 5120), # MXFP4 operands, bf16 output
     "quant_w_f32": ("qw_f32", 20480, 5120, 0),      # 16x16 blocks, both copies, from a binary32 source (419 MB)
     "step": ("step", 8192, 20480, 5120),           # the whole cfg 3 fwd + bwd step, full size: ONE-PASS captures only
+    "fwd_half": ("fwd", 8192, 10240, 5120),         # forward call, half the output features (X 84 MB, W 105 MB): the
+                                                    # quantize kernel of X that carries the amax pass of W
     "gemm_bf16_fprop": ("bf16", 4096, 5120, 5120),  # BF16 layer (Section 4.1): Y = X W^T, both operands K-major
     "gemm_bf16_wgrad": ("bf16_wgrad", 5120, 5120, 4096),  # dW = dY^T X, both operands read transposed, fp32 output
     "step_bf16": ("step_bf16", 8192, 20480, 5120),  # the cfg 3 layer kept in BF16, fwd + bwd, full size
@@ -580,6 +582,15 @@ def run_case(args):
             B.nvfp4_linear_fwd(X, W, o, Y, X_col, W_row, W_col, False, ws_f)
             B.nvfp4_linear_bwd(dY, X_col, W_col, k, o, dX, dW, False, ws_b)
         work, unit = 3 * 2.0 * r * c * k / 1e12, "TFLOP/s"
+    elif kind == "fwd":
+        X = torch.randn((r, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        W = (torch.randn((c, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
+        Y = torch.empty((r, c), dtype=torch.bfloat16, device="cuda")
+        X_col, W_row, W_col = B.alloc_tensor(k, r), B.alloc_tensor(c, k), B.alloc_tensor(k, c)
+        ws_f = torch.empty(B.nvfp4_linear_fwd_workspace_bytes(r, k), dtype=torch.uint8, device="cuda")
+        o = B.quant_opts(rht_sign_mask=mask)
+        fn = lambda: B.nvfp4_linear_fwd(X, W, o, Y, X_col, W_row, W_col, False, ws_f)
+        work, unit = 2.0 * r * c * k / 1e12, "TFLOP/s"
     elif kind == "step_bf16":
         X = torch.randn((r, k), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
         W = (torch.randn((c, k), generator=g, device="cuda", dtype=torch.float32) * 0.02).to(torch.bfloat16)
