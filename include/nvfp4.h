@@ -234,6 +234,12 @@ NVFP4_API nvfp4_status nvfp4_sq_error(const void* ref, int32_t ref_is_fp32, int6
  *   for Wgrad.  dX or dW may be NULL to skip that GEMM.  accumulate_dw != 0 adds into dW.
  *   workspace: device scratch of nvfp4_linear_bwd_workspace_bytes(M, N) for the two copies of dY.
  *   When both GEMMs are requested they run in one launch of the CTA-pair kernel.
+ * Ordering: both calls are stream-ordered as a whole (everything enqueued before them on the stream has
+ *   finished before their first kernel starts, and their results are complete for whatever is enqueued after
+ *   them).  Inside a call the kernels overlap only their set-up with the tail of the kernel before them
+ *   (programmatic dependent launch) and never read each other's output early; in the NVFP4 bf16 path the tensor
+ *   amax of W (Appendix B.1) is taken inside the kernel that quantizes X.  Results are bit-identical to the
+ *   same steps issued one by one through nvfp4_quantize and nvfp4_gemm.
  * Format: the layer runs in the format of the copies it is given (W_row / W_col_saved / X_col_saved must
  *   agree).  With MXFP4 copies the same sequence uses 1x32 and 32x32 blocks and the 32-point transform
  *   (Section 5); opts->rht_sign_mask then supplies 32 sign bits.

@@ -339,8 +339,8 @@ nvfp4_status nvfp4_linear_fwd(const void* X, const void* W, int64_t M, int64_t N
   }
   if (!w_is_cached && (st = quantize_impl(W, N, K, K, &wo, W_row, W_col_saved, s)) != NVFP4_OK) return st;
   if ((st = quantize_impl(X, M, K, K, &xo, &x_row, X_col_saved, s)) != NVFP4_OK) return st;
-  // behind the bf16 NVFP4 quantizer the GEMM may set itself up while that kernel drains
-  return gemm_impl(&x_row, W_row, Y_bf16, 0, N, 0, s, side_amax_fits(fmt, xo));
+  // behind a quantizer of this call the GEMM may set itself up while that kernel drains
+  return gemm_impl(&x_row, W_row, Y_bf16, 0, N, 0, s, true);
 }
 
 nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, const nvfp4_tensor* W_col_saved,
@@ -390,7 +390,7 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, c
     GemmArgs gd, gw;
     if ((st = gemm_prepare(&g_row, W_col_saved, dX_bf16, 0, K, 0, gd)) != NVFP4_OK) return st;
     if ((st = gemm_prepare(&g_col, X_col_saved, dW_fp32, 1, K, accumulate_dw, gw)) != NVFP4_OK) return st;
-    gd.chained = gw.chained = side_amax_fits(fmt, go);  // behind the bf16 NVFP4 quantizer of dY
+    gd.chained = gw.chained = 1;  // behind the quantizer of dY
     const int td = gemm_tile(gd), tw = gemm_tile(gw);
     if ((td == 512 || td == 768) && (tw == 512 || tw == 768)) {
       const bool forced = g_tile_n.load(std::memory_order_relaxed) != 0;
@@ -402,8 +402,7 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, const nvfp4_tensor* X_col_saved, c
       return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
     }
   }
-  if (dX_bf16 && (st = gemm_impl(&g_row, W_col_saved, dX_bf16, 0, K, 0, s, side_amax_fits(fmt, go))) != NVFP4_OK)
-    return st;
+  if (dX_bf16 && (st = gemm_impl(&g_row, W_col_saved, dX_bf16, 0, K, 0, s, true)) != NVFP4_OK) return st;
   if (dW_fp32 && (st = gemm_impl(&g_col, X_col_saved, dW_fp32, 1, K, accumulate_dw, s)) != NVFP4_OK) return st;
   return NVFP4_OK;
 }

@@ -4,6 +4,7 @@
 // The recipe options are those of Section 4 at this format's block size: 1x32 blocks for activations and gradients,
 // 32x32 blocks for weights, a 32-point random Hadamard transform on the transposed (weight-gradient) copy, stochastic
 // rounding with the same Philox draws as the NVFP4 kernel.
+#include "async_ptx.cuh"
 #include "quantize.h"
 #include "quantize_common.cuh"
 
@@ -59,6 +60,7 @@ __global__ void __launch_bounds__(256, RHT_COL ? 2 : 3) quantize_mx_kernel(const
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = (int)blockIdx.x;
+  griddep_launch_dependents();  // the GEMM of a composed call may set itself up while the last CTAs run
   const int64_t row0 = (int64_t)(tile / a.tiles_c) * 128;
   const int64_t col0 = (int64_t)(tile % a.tiles_c) * 128;
   const int64_t n_cb = a.cols >> 4;  // 16-chunks per source row (index of the random draws)

@@ -15,6 +15,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include "async_ptx.cuh"
 #include "common.cuh"
 #include "quantize.h"
 #include "quantize_common.cuh"
@@ -63,6 +64,7 @@ __global__ void __launch_bounds__(256, 3) quantize_rht_kernel(const RhtArgs ra) 
   extern __shared__ __align__(128) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = MODE == 0 ? (int)blockIdx.x : (int)(gridDim.x - 1 - blockIdx.x);  // pass 2 walks backwards (L2)
+  griddep_launch_dependents();  // the GEMM of a composed call may set itself up while the last CTAs run
   const int64_t row0 = (int64_t)(tile / a.tiles_c) * 128;
   const int64_t col0 = (int64_t)(tile % a.tiles_c) * 128;
   const int64_t n_cb = a.cols >> 4, n_rb = a.rows >> 4;
