@@ -604,14 +604,16 @@ bool prefer_wide_tiles(const GemmArgs& g0, const GemmArgs* g1) {
   if (sm_count(&num_sms) != cudaSuccess) return false;
   // the estimate walks every tile of both schedules: remember the answers for the shapes seen (a training loop
   // repeats a handful of them)
-  struct Entry { int key[7]; bool wide; };
+  struct Entry { int key[8]; bool wide; };
   static std::mutex mu;
   static std::vector<Entry> seen;
-  const int key[7] = {g0.M, g0.N, g0.K, g1 ? g1->M : 0, g1 ? g1->N : 0, g1 ? g1->K : 0, num_sms};
+  // (the output type is part of the key: an fp32 output changes the hand-over cost and with it the choice)
+  const int key[8] = {g0.M, g0.N, g0.K, g1 ? g1->M : 0, g1 ? g1->N : 0, g1 ? g1->K : 0, num_sms,
+                      (g0.d_is_fp32 ? 1 : 0) | (g1 && g1->d_is_fp32 ? 2 : 0)};
   {
     std::lock_guard<std::mutex> lock(mu);
     for (const Entry& e : seen)
-      if (std::equal(key, key + 7, e.key)) return e.wide;
+      if (std::equal(key, key + 8, e.key)) return e.wide;
   }
   const GemmArgs* gs[2] = {&g0, g1};
   const int n = g1 ? 2 : 1, pairs = num_sms / 2;
@@ -619,7 +621,7 @@ bool prefer_wide_tiles(const GemmArgs& g0, const GemmArgs* g1) {
   std::lock_guard<std::mutex> lock(mu);
   if (seen.size() < 256) {
     Entry e{};
-    std::copy(key, key + 7, e.key);
+    std::copy(key, key + 8, e.key);
     e.wide = wide;
     seen.push_back(e);
   }
