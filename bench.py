@@ -711,7 +711,9 @@ def run_gemm_cycles(args, m, n, k):
     n_pairs = torch.cuda.get_device_properties(0).multi_processor_count // 2
     probe = torch.zeros(8 * n_pairs, dtype=torch.int64, device="cuda")
     variants = [("all on", 0), ("no MMAs (loads + scale path)", 1), ("no operand loads (MMAs + scale path)", 2),
-                ("no scale path (loads + MMAs)", 4), ("MMAs only", 6)]
+                ("no scale path (loads + MMAs)", 4), ("MMAs only", 6),
+                ("scale atoms through tcgen05.cp issued by the MMA issuer", 32),
+                ("the same, no MMAs", 33)]
     rows = {}
     for turn in range(4):
         for pairs in (n_pairs, n_pairs // 2):

@@ -170,6 +170,11 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
 }
+// one 512-byte scale atom (32 rows x 16 bytes) shared memory -> four columns of tensor memory, replicated to the four
+// lane quadrants, in both CTAs of the pair (each from its own shared memory at the same offset)
+__device__ __forceinline__ void tc2_cp_sf(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
 __device__ __forceinline__ void tc2_mma_nvf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                              uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
   asm volatile(
@@ -392,7 +397,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
         ok = mbar_wait(sfl_bar(stage), phase, abort_flag, 0x500u + stage);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) break;
-        if (g.exp & 4) {  // measurement aid: no scale copies
+        if (g.exp & (4 | 32)) {  // measurement aids: no scale copies / the issuer copies, this warp only relays
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(sff_leader + 8u * stage);
           if (++stage == kStages) {
@@ -465,6 +470,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
           const uint32_t a_lo = a_lo0 + stage * (kStageBytes >> 4);
           const uint32_t b_lo = b_lo0 + stage * (kStageBytes >> 4);
           const uint32_t sf_t = tmem + kSfCol + stage * kSfSlotCols;
+          if (g.exp & 32) {  // measurement aid: the scale atoms go through the copy engine, issued here
+            const uint32_t sf_lo = (((base + kABytes + kBBytes) >> 4) & 0x3fffu) + stage * (kStageBytes >> 4);
+            constexpr int kAtomsKb = MX ? 2 : 4;
+#pragma unroll
+            for (int j = 0; j < kAtomsKb; ++j) {
+              tc2_cp_sf(sf_t + j * 4, make_desc(sf_lo + j * 32, kDescHiSf));
+#pragma unroll
+              for (int grp = 0; grp < 2; ++grp)
+                tc2_cp_sf(sf_t + 16 + 8 * j + 4 * grp, make_desc(sf_lo + (kSfaBytes >> 4) + grp * 128 + j * 32, kDescHiSf));
+            }
+          }
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             if (g.exp & 1) break;  // measurement aid: no MMAs
