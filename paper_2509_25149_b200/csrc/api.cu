@@ -147,13 +147,14 @@ nvfp4_status quantize_impl(const void* x, int64_t rows, int64_t cols, int64_t ld
   }
   // pass 2 may become resident while the previous kernel of this call drains (its own pass 1, or the caller's launch)
   a.chained = chained;
+  // only the forward pass's activation quantize carries a side job (see side_amax_fits); checked before any launch
+  if (side && (!hr || b2 || sr || o->rht_rowwise || (hc && !o->rht_colwise))) return NVFP4_ERR_ARG;
   if (side && zero_side_amax(*side, s) != cudaSuccess) return NVFP4_ERR_CUDA;  // not between pass 1 and pass 2
   if (!(o->flags & NVFP4_AMAX_PROVIDED)) {
     if (launch_amax(a, hr, hc, o->rht_rowwise != 0, o->rht_colwise != 0, s) != cudaSuccess) return NVFP4_ERR_CUDA;
     a.chained = 1;
   }
-  if (side) {  // only the forward pass's activation quantize carries one (see side_amax_fits)
-    if (!hr || b2 || sr || o->rht_rowwise || (hc && !o->rht_colwise)) return NVFP4_ERR_ARG;
+  if (side) {
     return launch_quantize_with_amax_of(a, hc, *side, s) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
   }
   if (launch_quantize(a, hr, hc, b2, o->rht_rowwise != 0, o->rht_colwise != 0, sr, s) != cudaSuccess)
