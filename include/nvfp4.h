@@ -336,7 +336,8 @@ NVFP4_API int32_t nvfp4_set_gemm_tile_n(int32_t tile_n);
  *             bit 5: the scale atoms reach tensor memory through the copy engine (twelve tcgen05.cp per k-block,
  *             issued by the MMA issuer in front of the k-block's MMAs) instead of through the scale warps'
  *             registers; alone, this bit leaves the output CORRECT.
- *             With any of bits 0-4 set the OUTPUT IS MEANINGLESS (timing
+ *             bit 6: the epilogue converts but does not write its staging buffer; bit 7: it issues no TMA store.
+ *             With any of bits 0-4, 6, 7 set the OUTPUT IS MEANINGLESS (timing
  *             only); every barrier is still signalled, so the kernel runs to its end.
  *   max_pairs > 0: at most that many CTA pairs (SM pairs) take part.
  *   probe     device array of 8 x uint64 per pair; each pair's issuer writes five: SM cycles and nanoseconds of its

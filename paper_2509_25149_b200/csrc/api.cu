@@ -543,7 +543,7 @@ nvfp4_status nvfp4_test_wait_timeout(uint64_t limit_ns, void* cuda_stream) {
 }
 
 int32_t nvfp4_set_gemm_experiment(int32_t mode, int32_t max_pairs, void* probe) {
-  if (mode < 0 || mode > 63 || max_pairs < 0) return -1;
+  if (mode < 0 || mode > 255 || max_pairs < 0) return -1;
   set_gemm_experiment(mode, max_pairs, static_cast<unsigned long long*>(probe));
   return 0;
 }
