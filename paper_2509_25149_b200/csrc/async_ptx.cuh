@@ -86,8 +86,9 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn tensor_map_encoder();
-// 2-D map over a row-major [rows][row_bytes / elem] array; box = box_inner elements x box_rows
+// 2-D map over a row-major [rows][row_bytes / elem] array; box = box_inner elements x box_rows;
+// swizzle: 0 = none, 1 = 128-byte (box rows of 128 bytes), 2 = 64-byte (box rows of 64 bytes)
 bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dtype, int elem_bytes, const void* base, uint64_t inner_elems,
-                 uint64_t rows, uint64_t row_pitch_bytes, uint32_t box_inner, uint32_t box_rows, bool swizzle128);
+                 uint64_t rows, uint64_t row_pitch_bytes, uint32_t box_inner, uint32_t box_rows, int swizzle);
 
 }  // namespace nvfp4

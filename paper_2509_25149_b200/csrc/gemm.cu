@@ -47,7 +47,7 @@ EncodeTiledFn tensor_map_encoder() {
 // launch): the result depends only on the arguments, so a small per-thread cache keyed by them returns repeats (the
 // same buffers launch after launch, as in a training loop) without the call.
 bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dtype, int elem_bytes, const void* base, uint64_t inner_elems,
-                 uint64_t rows, uint64_t row_pitch_bytes, uint32_t box_inner, uint32_t box_rows, bool swizzle128) {
+                 uint64_t rows, uint64_t row_pitch_bytes, uint32_t box_inner, uint32_t box_rows, int swizzle) {
   (void)elem_bytes;
   struct Entry {
     uint64_t key[6];
@@ -57,7 +57,7 @@ bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dtype, int elem_bytes, co
   constexpr int kEntries = 64;
   static thread_local Entry cache[kEntries] = {};
   const uint64_t key[6] = {reinterpret_cast<uint64_t>(base), inner_elems, rows, row_pitch_bytes,
-                           ((uint64_t)box_inner << 32) | box_rows, ((uint64_t)dtype << 1) | (swizzle128 ? 1u : 0u)};
+                           ((uint64_t)box_inner << 32) | box_rows, ((uint64_t)dtype << 2) | (uint64_t)(swizzle & 3)};
   uint64_t h = 0x9E3779B97F4A7C15ull;
   for (uint64_t k : key) h = (h ^ k) * 0xFF51AFD7ED558CCDull + (h >> 29);
   Entry& e = cache[(h >> 20) % kEntries];
@@ -72,7 +72,8 @@ bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dtype, int elem_bytes, co
   cuuint32_t box[2] = {box_inner, box_rows};
   cuuint32_t estr[2] = {1, 1};
   if (fn(map, dtype, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-         swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+         swizzle == 1 ? CU_TENSOR_MAP_SWIZZLE_128B : swizzle == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE,
+         CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return false;
   std::copy(key, key + 6, e.key);
@@ -473,12 +474,13 @@ bool make_wide_maps(const GemmArgs& g, const void* a_codes, const void* b_codes,
   // m[0] A (128-row boxes), m[1] B (128-row boxes), m[2] B (64-row boxes), m[3] D
   bool ok = make_code_map(&m[0], a_codes, g.M, g.K / 2, 128) && make_code_map(&m[1], b_codes, g.N, g.K / 2, 128) &&
             make_code_map(&m[2], b_codes, g.N, g.K / 2, 64);
+  // D: the epilogue's store chunks, 128 rows x 64 bytes with the 64-byte swizzle (fp32) or x 128 bytes (bf16)
   if (g.d_is_fp32)
     ok = ok && make_map_2d(&m[3], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, g.d, (uint64_t)g.N, (uint64_t)g.M,
-                           (uint64_t)g.ldd * 4, 32, 128, true);
+                           (uint64_t)g.ldd * 4, 16, 128, 2);
   else
     ok = ok && make_map_2d(&m[3], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, g.d, (uint64_t)g.N, (uint64_t)g.M,
-                           (uint64_t)g.ldd * 2, 64, 128, true);
+                           (uint64_t)g.ldd * 2, 64, 128, 1);
   return ok;
 }
 
@@ -500,9 +502,9 @@ double pair_makespan(const GemmArgs* const* gs, int n_problems, bool wide_tiles,
       const int gm = tiles_m - m0 < kGroupM ? tiles_m - m0 : kGroupM;
       for (int n_idx = 0; n_idx < tiles_n; ++n_idx) {
         const bool w = n_idx < n_wide;
-        // hand-over per tile in k-block units, fitted to 24 layer shapes timed with both tile widths; the wide
-        // tile drains an fp32 output in six passes before it can release the accumulator
-        const double cost = w ? 1.5 * kb + (g.d_is_fp32 ? 5.3 : 3.3) : kb + (wide_tiles ? 2.9 : 2.5);
+        // hand-over per tile in k-block units, fitted to 24 layer shapes timed with both tile widths (the fp32 figure
+        // of the wide tile refitted after its store chunks stopped waiting for each other)
+        const double cost = w ? 1.5 * kb + (g.d_is_fp32 ? 3.8 : 3.3) : kb + (wide_tiles ? 2.9 : 2.5);
         for (int i = 0; i < gm; ++i, ++t) {
           const int64_t rnd = t / pairs, p = t % pairs;
           load[(size_t)((rnd & 1) ? pairs - 1 - p : p)] += cost;  // odd rounds run through the pairs in reverse

@@ -14,7 +14,8 @@
 //   - the scale slots in tensor memory are a ring of two, freed by the same event that frees the shared-memory
 //     stage of two k-blocks earlier (the scale warps wait on that stage's "empty" barrier);
 //   - the epilogue drains its half of the tile in passes of 64 columns (3 or 2), releasing the accumulator after
-//     the last read, and stores each pass through the swizzled staging buffer with TMA.
+//     the last read, and stores each pass through its staging buffer with TMA (fp32 outputs: in 64-byte-wide chunks
+//     through the two halves of the buffer in turn, so that no chunk waits for the store of the chunk before it).
 // Included by gemm.cu only.
 #pragma once
 
@@ -57,31 +58,57 @@ struct WArgs {
   int n_tiles;   // tiles of both problems
 };
 
-// 64 accumulator columns of one row per thread -> alpha, conversion -> swizzled staging -> TMA store / reduce-add
+// 64 accumulator columns of one row per thread -> alpha, conversion -> swizzled staging -> TMA store / reduce-add.
+// bf16: one chunk of 128-byte rows through the group's 16 KB buffer, converted once the store issued before it has
+// finished reading the buffer.
+// fp32: four chunks of 64-byte rows (16 columns) through the two 8 KB halves of the same buffer in turn: before a chunk
+// is written, the store issued from its half two chunks ago has finished reading it, while the latest store (from the
+// other half) may still be in flight, so the tensor-memory reads between the chunks do not wait for a store.  (The same
+// scheme for bf16 outputs, with 32-column chunks, was measured slower than the single buffer: twice the barriers and
+// stores of half the width.)  n_chunks counts the group's fp32 chunks; the caller drains all stores before a tile.
 template <bool FP32>
 __device__ __forceinline__ void store_cols64(const uint32_t (&r)[64], float alpha, int et, int bar_id, int row_in_tile,
-                                             uint32_t stage_buf, const CUtensorMap* map_d, int x0, int row0,
-                                             int accumulate) {
-  constexpr int kChunks = FP32 ? 2 : 1;
-  constexpr int kChunkCols = FP32 ? 32 : 64;
+                                             uint32_t stage_buf16k, uint32_t& n_chunks, const CUtensorMap* map_d, int x0,
+                                             int row0, int accumulate) {
+  if (FP32) {
 #pragma unroll
-  for (int c = 0; c < kChunks; ++c) {
+    for (int c = 0; c < 4; ++c, ++n_chunks) {
+      const uint32_t stage_buf = stage_buf16k + (n_chunks & 1u) * 8192u;
+      if (et == 0) bulk_wait_read<1>();
+      asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+      const uint32_t srow = stage_buf + row_in_tile * 64;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        uint32_t p[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) p[e] = __float_as_uint(__uint_as_float(r[c * 16 + 4 * j + e]) * alpha);
+        // 64-byte swizzle: the 16-byte unit index is XORed with bits 7-8 of the address, i.e. with (row >> 1) & 3
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(srow + ((j ^ ((row_in_tile >> 1) & 3)) << 4)),
+                     "r"(p[0]), "r"(p[1]), "r"(p[2]), "r"(p[3])
+                     : "memory");
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+      if (et == 0) {
+        if (accumulate)
+          tma_reduce_add_2d(map_d, x0 + c * 16, row0, stage_buf);
+        else
+          tma_store_2d(map_d, x0 + c * 16, row0, stage_buf);
+        bulk_commit();
+      }
+    }
+  } else {
     if (et == 0) bulk_wait_read<0>();  // the store issued from this buffer before has finished reading it
     asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-    const uint32_t srow = stage_buf + row_in_tile * 128;
+    const uint32_t srow = stage_buf16k + row_in_tile * 128;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       uint32_t p[4];
-      if (FP32) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) p[e] = __float_as_uint(__uint_as_float(r[c * 32 + 4 * j + e]) * alpha);
-      } else {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * j + 2 * e]) * alpha,
-                                                   __uint_as_float(r[8 * j + 2 * e + 1]) * alpha);
-          p[e] = *reinterpret_cast<uint32_t*>(&h);
-        }
+      for (int e = 0; e < 4; ++e) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * j + 2 * e]) * alpha,
+                                                 __uint_as_float(r[8 * j + 2 * e + 1]) * alpha);
+        p[e] = *reinterpret_cast<uint32_t*>(&h);
       }
       asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(srow + ((j ^ (row_in_tile & 7)) << 4)), "r"(p[0]),
                    "r"(p[1]), "r"(p[2]), "r"(p[3])
@@ -90,10 +117,7 @@ __device__ __forceinline__ void store_cols64(const uint32_t (&r)[64], float alph
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
     if (et == 0) {
-      if (accumulate)
-        tma_reduce_add_2d(map_d, x0 + c * kChunkCols, row0, stage_buf);
-      else
-        tma_store_2d(map_d, x0 + c * kChunkCols, row0, stage_buf);
+      tma_store_2d(map_d, x0, row0, stage_buf16k);
       bulk_commit();
     }
   }
@@ -348,7 +372,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
     const float alpha1 = __fmul_rn(g.p[1].a_global[1], g.p[1].b_global[1]);
     const uint32_t acce_leader = map_to_cta(acce_bar, 0);
     const int row_in_tile = quad * 32 + lane;
-    const uint32_t stage_buf = staging + half * 16384;
+    const uint32_t stage_bufs = staging + half * 16384;
+    uint32_t n_chunks = 0;  // chunks this group has stored so far (selects the buffer)
     for (int rnd = 0, tile = pair_id; tile < n_tiles; tile = next_tile(++rnd)) {
       int prob, m_blk, n0, width;
       tile_coords(tile, prob, m_blk, n0, width);
@@ -362,6 +387,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
       tc_fence_after();
       const int row0 = m_blk * 256 + (int)rank * 128;
       const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + half * cols_half;
+      // the previous tile's stores have long left the staging buffer; waiting for all of them here lets a tile with
+      // another output type (two problems in one launch) use the buffer its own way
+      if (et == 0) bulk_wait_read<0>();
       for (int p = 0; p < passes; ++p) {
         uint32_t r[64];
 #pragma unroll
@@ -374,9 +402,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kWThreads, 1)
         }
         const int x0 = n0 + half * cols_half + p * 64;
         if (d_is_fp32)
-          store_cols64<true>(r, alpha, et, bar_id, row_in_tile, stage_buf, map_d, x0, row0, accumulate);
+          store_cols64<true>(r, alpha, et, bar_id, row_in_tile, stage_bufs, n_chunks, map_d, x0, row0, accumulate);
         else
-          store_cols64<false>(r, alpha, et, bar_id, row_in_tile, stage_buf, map_d, x0, row0, accumulate);
+          store_cols64<false>(r, alpha, et, bar_id, row_in_tile, stage_bufs, n_chunks, map_d, x0, row0, accumulate);
       }
       acc_phase ^= 1u;
     }
